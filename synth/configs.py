@@ -1,0 +1,105 @@
+"""The five benchmark workloads: model shapes, request recipes and prune schedules.
+
+Model shapes follow the Qwen3 reranker family the paper evaluates (Table 1):
+decoder-only, GQA, RMSNorm, SwiGLU, RoPE, QK-norm.  The candidate counts,
+length distributions and probe schedules are the synthetic stand-ins for the
+paper's retrieval datasets (Sec. 6.1), which are not available offline.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field, replace
+from typing import List, Tuple
+
+MODE_NONE = 0        # no pruning: full forward, exact sort
+MODE_FIXED_KEEP = 1  # at probe j keep the keep_counts[j] best
+MODE_CLUSTER = 2     # progressive cluster pruning (Sec. 4.1)
+
+DTYPE_FP32 = 0
+DTYPE_BF16 = 1
+
+
+@dataclass(frozen=True)
+class ModelCfg:
+    n_layers: int
+    hidden: int
+    n_q_heads: int
+    n_kv_heads: int
+    head_dim: int
+    ffn: int
+    vocab: int
+    rope_theta: float
+    rms_eps: float = 1e-6
+    causal: int = 1
+    qk_norm: int = 1
+    dtype: int = DTYPE_BF16
+    yes_id: int = 0   # vocab rows the two-row score head is taken from
+    no_id: int = 1
+
+    @property
+    def qkv_rows(self) -> int:
+        return (self.n_q_heads + 2 * self.n_kv_heads) * self.head_dim
+
+    @property
+    def params_per_layer(self) -> int:
+        d = self.hidden
+        return d * self.qkv_rows + self.n_q_heads * self.head_dim * d + 3 * d * self.ffn
+
+
+@dataclass(frozen=True)
+class Schedule:
+    mode: int = MODE_NONE
+    probe_layers: Tuple[int, ...] = ()   # number of completed layers, 1-based, increasing, < n_layers
+    keep_counts: Tuple[int, ...] = ()    # MODE_FIXED_KEEP only, one per probe
+    cv_threshold: float = 0.0            # MODE_CLUSTER: prune only if CV > threshold
+    n_clusters: int = 3
+    std_ddof: int = 0
+    select_winners: int = 1              # 1: three-way routing, 0: drop-only variant (Sec. 7)
+
+    def unpruned(self) -> "Schedule":
+        return Schedule(mode=MODE_NONE)
+
+
+@dataclass(frozen=True)
+class Workload:
+    name: str
+    model: ModelCfg
+    n_candidates: int
+    top_k: int
+    query_len: int
+    doc_len: Tuple[str, float, float, float, float]  # (kind, a, b, lo, hi)
+    schedule: Schedule
+    dup_fraction: float = 0.0
+    activation_budget_bytes: int = 0
+    stream_weights: int = 0
+    weight_seed: int = 0
+    cfg_index: int = 0
+
+
+_QWEN3_06B = ModelCfg(n_layers=28, hidden=1024, n_q_heads=16, n_kv_heads=8, head_dim=128,
+                      ffn=3072, vocab=151669, rope_theta=1e6, yes_id=9693, no_id=2152)
+_QWEN3_4B = replace(_QWEN3_06B, n_layers=36, hidden=2560, n_q_heads=32, ffn=9728)
+_QWEN3_8B = replace(_QWEN3_06B, n_layers=36, hidden=4096, n_q_heads=32, ffn=12288)
+_TINY = ModelCfg(n_layers=2, hidden=256, n_q_heads=4, n_kv_heads=2, head_dim=64, ffn=768,
+                 vocab=4096, rope_theta=1e4, qk_norm=0, dtype=DTYPE_FP32, yes_id=7, no_id=11)
+
+# Dispersion thresholds: the paper only shows "low"/"high" settings in figures.  Random-init
+# score means sit near zero, so CV is usually well above 1; 0.5 makes the rule fire at most
+# probes, which is the regime the method is designed for.
+WORKLOADS: List[Workload] = [
+    Workload("cfg0_tiny_fp32", _TINY, 16, 3, 16, ("uniform", 16, 48, 16, 48),
+             Schedule(MODE_FIXED_KEEP, (1,), (8,)), cfg_index=0),
+    Workload("cfg1_qwen3_0p6b", _QWEN3_06B, 100, 10, 32, ("uniform", 128, 512, 128, 512),
+             Schedule(MODE_CLUSTER, (8, 12, 16, 20, 24), cv_threshold=0.5), cfg_index=1),
+    Workload("cfg2_qwen3_4b", _QWEN3_4B, 200, 10, 48, ("uniform", 256, 1024, 256, 1024),
+             Schedule(MODE_CLUSTER, (8, 12, 16, 20, 24, 28, 32), cv_threshold=0.5), cfg_index=2),
+    Workload("cfg3_qwen3_8b_streamed", _QWEN3_8B, 100, 5, 64, ("uniform", 512, 2048, 512, 2048),
+             Schedule(MODE_CLUSTER, (8, 12, 16, 20, 24, 28, 32), cv_threshold=0.5),
+             activation_budget_bytes=16 << 30, stream_weights=1, cfg_index=3),
+    Workload("cfg4_stress_0p6b", _QWEN3_06B, 1000, 20, 32, ("lognormal", 256, 0.6, 32, 1024),
+             Schedule(MODE_CLUSTER, tuple(range(4, 28, 2)), cv_threshold=0.5),
+             dup_fraction=0.3, cfg_index=4),
+]
+
+
+def workload(i: int) -> Workload:
+    return WORKLOADS[i]
