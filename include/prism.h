@@ -1,0 +1,210 @@
+/*
+ * prism.h -- C ABI of the PRISM hot path on one NVIDIA B200 (sm_100a).
+ *
+ * The library computes semantic top-K selection the way the paper's "monolithic forwarding"
+ * does (Sec. 3.3): all N query||candidate sequences of one request advance through the layers
+ * of a decoder cross-encoder reranker together, as ONE padding-free packed batch.  After the
+ * designated layers a relevance score is probed per candidate with the model's own classifier
+ * (Sec. 3.1, 4.1); the dispersion CV = |std/mean| of the scores decides whether clustering runs;
+ * clusters above the one holding the K-th ranked candidate are *selected*, clusters below it are
+ * *dropped*, the boundary cluster is *deferred* and is the only part that keeps computing
+ * (Sec. 4.1, Fig. 4); the survivors are stream-compacted before the next layer; the forward
+ * stops when #deferred equals the remaining top-K slots (Sec. 4.1, 4.5).  Chunked execution
+ * (Sec. 4.3) and overlapped layer streaming (Sec. 4.2) are options of the handle.
+ *
+ * Conventions
+ *   - plain C, no exceptions, nothing printed; every call returns a prism_status (0 = OK).
+ *   - "device pointer" = CUDA global memory of the current device; "host pointer" = CPU memory.
+ *   - matrices are row-major [out_features, in_features] (both GEMM operands are K-major).
+ *   - element type of every weight tensor is cfg.dtype (PRISM_FP32: float, PRISM_BF16: bfloat16).
+ *   - a handle serves one request at a time (not re-entrant); different handles are independent.
+ *   - the library never takes ownership of caller memory and never frees it.
+ */
+#ifndef PRISM_H_
+#define PRISM_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define PRISM_API __attribute__((visibility("default")))
+#else
+#define PRISM_API
+#endif
+
+#define PRISM_MAX_CLUSTERS 8      /* upper bound for prism_prune_schedule.n_clusters          */
+#define PRISM_MAX_CANDIDATES 4096 /* upper bound for prism_model_cfg.max_candidates           */
+#define PRISM_MAX_LAYERS 128
+
+typedef enum {
+  PRISM_OK = 0,
+  PRISM_ERR_INVALID_ARG = -1, /* null pointer, negative size, K < 1, malformed schedule/config          */
+  PRISM_ERR_SHAPE_LIMIT = -2, /* N, a sequence length or the token total exceeds the handle's maxima    */
+  PRISM_ERR_BAD_INPUT = -3,   /* token id outside [0, vocab) or non-monotone offsets (found on device)  */
+  PRISM_ERR_BUDGET = -4,      /* activation budget cannot hold the hidden states plus one sequence      */
+  PRISM_ERR_CUDA = -5,        /* a CUDA call failed; text via prism_last_error                          */
+  PRISM_ERR_TIMEOUT = -6,     /* a bounded device-side wait expired (kernel returned, context usable)   */
+  PRISM_ERR_NOMEM = -7,       /* device or host allocation failed                                       */
+  PRISM_ERR_UNSUPPORTED = -8  /* shape not supported by the kernels (e.g. head_dim, alignment)          */
+} prism_status;
+
+enum { PRISM_FP32 = 0, PRISM_BF16 = 1 };
+enum { PRISM_WEIGHTS_DEVICE = 0, PRISM_WEIGHTS_HOST_STREAMED = 1 };
+enum { PRISM_PRUNE_NONE = 0, PRISM_PRUNE_FIXED_KEEP = 1, PRISM_PRUNE_CLUSTER = 2 };
+/* Implementation selectors (debug/validation): AUTO picks the tensor-core kernels in bf16 mode. */
+enum { PRISM_IMPL_AUTO = 0, PRISM_IMPL_SIMT = 1 };
+
+typedef struct prism_handle prism_handle;
+
+/* Model description: a pre-norm decoder block stack (RMSNorm -> GQA attention with optional
+ * per-head QK-norm and rotary embedding -> residual -> RMSNorm -> SwiGLU -> residual), the
+ * architecture of the rerankers the paper evaluates (Sec. 6.1, Table 1). */
+typedef struct {
+  int32_t n_layers;   /* 1..PRISM_MAX_LAYERS */
+  int32_t hidden;     /* D; multiple of 64 in bf16 mode, of 4 in fp32 mode */
+  int32_t n_q_heads;  /* Hq, multiple of n_kv_heads */
+  int32_t n_kv_heads; /* Hkv */
+  int32_t head_dim;   /* dh: 128 in bf16 mode; even, <= 256 in fp32 mode */
+  int32_t ffn;        /* F; multiple of 128 in bf16 mode */
+  int32_t vocab;
+  float rope_theta;
+  float rms_eps;
+  int32_t causal;  /* 1 = decoder (causal) attention, 0 = bidirectional */
+  int32_t qk_norm; /* 1 = RMSNorm over head_dim on q and k before the rotary embedding */
+  int32_t dtype;   /* PRISM_FP32 or PRISM_BF16: weights, activations and GEMM inputs; the residual
+                      stream, accumulators, norms, softmax and scores are always fp32 */
+  int32_t max_seq_len;      /* max query_len + doc length of one sequence */
+  int32_t max_candidates;   /* max N (<= PRISM_MAX_CANDIDATES) */
+  int32_t max_total_tokens; /* max sum over candidates of (query_len + doc length) */
+  int64_t activation_budget_bytes; /* 0 = unlimited.  Otherwise chunked execution (Sec. 4.3): the
+                      hidden states of all sequences plus the intermediates of ONE chunk stay
+                      within this many bytes; chunks are cut on sequence boundaries */
+  int32_t weight_residency; /* PRISM_WEIGHTS_DEVICE, or PRISM_WEIGHTS_HOST_STREAMED: layer tensors
+                      are pinned host memory, two device slots, layer l+1 is copied on a side
+                      stream while layer l computes (overlapped layer streaming, Sec. 4.2) */
+  int32_t gemm_impl;      /* PRISM_IMPL_* */
+  int32_t attention_impl; /* PRISM_IMPL_* */
+} prism_model_cfg;
+
+typedef struct {
+  const void* g_attn; /* [D] */
+  const void* w_qkv;  /* [(Hq+2Hkv)*dh, D]: all q heads, then k heads, then v heads */
+  const void* g_q;    /* [dh], used when qk_norm */
+  const void* g_k;    /* [dh], used when qk_norm */
+  const void* w_o;    /* [D, Hq*dh] */
+  const void* g_ffn;  /* [D] */
+  const void* w_gate; /* [F, D] */
+  const void* w_up;   /* [F, D] */
+  const void* w_down; /* [D, F] */
+} prism_layer_weights;
+
+/* Pointers only.  embed/g_final/score_head are device pointers.  The layer tensors are device
+ * pointers (PRISM_WEIGHTS_DEVICE) or pinned host pointers (PRISM_WEIGHTS_HOST_STREAMED); each
+ * must be 16-byte aligned.  The caller keeps all of them alive and unchanged until
+ * prism_destroy.  `layers` itself is a host array of n_layers structs, read during
+ * prism_create only. */
+typedef struct {
+  const void* embed;      /* [vocab, D] */
+  const void* g_final;    /* [D] final RMSNorm gain */
+  const void* score_head; /* [2, D]: row 0 = "yes" logit row, row 1 = "no"; score = yes - no */
+  const prism_layer_weights* layers;
+} prism_weights;
+
+/* When and how to prune (Sec. 4.1).  probe_layers[j] counts completed layers (1-based),
+ * strictly increasing, each < n_layers; the last layer is always scored and never prunes.
+ *   NONE        no probes; the result is the exact top-K by final score.
+ *   FIXED_KEEP  at probe j keep the keep_counts[j] best (each >= K).
+ *   CLUSTER     if CV > cv_threshold: split the ranked scores into n_clusters contiguous groups of
+ *               minimum within-group variance, route selected / deferred / dropped around the
+ *               group that holds rank K_rem.  select_winners = 0 is the drop-only variant (Sec. 7):
+ *               contenders above the boundary keep computing, so every returned score is a
+ *               final-layer score. */
+typedef struct {
+  int32_t mode;
+  int32_t n_probes;
+  const int32_t* probe_layers; /* host */
+  const int32_t* keep_counts;  /* host, FIXED_KEEP only */
+  double cv_threshold;
+  int32_t n_clusters;     /* 2..PRISM_MAX_CLUSTERS (0 = default 3) */
+  int32_t std_ddof;       /* 0 population std (default), 1 sample std */
+  int32_t select_winners; /* 1 three-way routing, 0 drop-only */
+} prism_prune_schedule;
+
+typedef struct {
+  int32_t layer;           /* completed layers when the scores were probed */
+  int32_t n_active_before; /* candidates scored */
+  int32_t fired;           /* 1 if candidates were removed at this probe */
+  int32_t n_selected, n_dropped, n_deferred;
+  int32_t k_rem_after; /* top-K slots still open after the probe */
+  int32_t n_cuts;
+  int32_t cuts[PRISM_MAX_CLUSTERS]; /* cluster boundaries in rank space */
+  int32_t tokens_before;            /* live tokens entering the probe */
+  double cv;
+} prism_probe_record;
+
+/* Optional per-request record, all host memory owned by the caller.  Scored layers are written in
+ * order: every probe layer reached, then the final layer if it was reached (fired = 0 there). */
+typedef struct {
+  int32_t capacity;            /* in: records available in `records` (and rows in scores/ids) */
+  int32_t n_records;           /* out */
+  prism_probe_record* records; /* out [capacity] */
+  float* scores;               /* out, nullable: [capacity, N] probe scores, batch order */
+  int32_t* ids;                /* out, nullable: [capacity, N] original candidate index per score */
+  int32_t layers_run;          /* out: layers executed before the forward stopped */
+  int32_t* tokens_per_layer;   /* out, nullable: [n_layers] live tokens forwarded through each layer */
+  int32_t n_chunks_max;        /* out: largest number of chunks used for one layer */
+  int64_t workspace_bytes;     /* out: device bytes held by the handle */
+} prism_trace;
+
+/* Validate cfg, take the weight pointers, allocate every workspace the handle will ever need
+ * (no allocation happens later), build TMA descriptors and the rotary table.
+ * Errors: INVALID_ARG, UNSUPPORTED, BUDGET (budget below hidden states + one max_seq_len sequence),
+ * NOMEM, CUDA.  On error *out = NULL. */
+PRISM_API int prism_create(const prism_model_cfg* cfg, const prism_weights* w, prism_handle** out);
+
+/* Top-K selection for one request (problem statement Sec. 2.1; method Sec. 3.3-4.3).
+ *   query_tokens  device int32[query_len]
+ *   cand_tokens   device int32[cand_offsets[N]]   document token ids, concatenated
+ *   cand_offsets  device int32[N+1], cand_offsets[0] = 0, non-decreasing
+ *   topk_idx      device int32[K]   original candidate indices
+ *   topk_scores   device float[K]   score each had when it left the computation
+ *   n_out         host   int32      min(K, N) on success, 0 on error
+ *   trace         host, nullable
+ *   cuda_stream   a cudaStream_t (NULL = default stream); work is enqueued there and the call
+ *                 returns after the stream has drained.
+ * Sequence i is query_tokens followed by document i, positions restart at 0.  Output order:
+ * candidates selected at earlier probes first (within a probe: score descending, index
+ * ascending), then the final fill in the same order.  K > N is not an error.
+ * Errors: INVALID_ARG, SHAPE_LIMIT, BAD_INPUT, BUDGET, CUDA, TIMEOUT; outputs are then unspecified. */
+PRISM_API int prism_select(prism_handle* h, const int32_t* query_tokens, int32_t query_len,
+                 const int32_t* cand_tokens, const int32_t* cand_offsets, int32_t N, int32_t K,
+                 const prism_prune_schedule* sched, int32_t* topk_idx, float* topk_scores,
+                 int32_t* n_out, prism_trace* trace, void* cuda_stream);
+
+/* Same request with HOST buffers: copies the three inputs to the device, runs prism_select's path
+ * and copies topk_idx / topk_scores back (all on cuda_stream, inside the call).  Pinned buffers
+ * make the copies asynchronous; pageable ones work too. */
+PRISM_API int prism_select_host(prism_handle* h, const int32_t* query_tokens, int32_t query_len,
+                      const int32_t* cand_tokens, const int32_t* cand_offsets, int32_t N, int32_t K,
+                      const prism_prune_schedule* sched, int32_t* topk_idx, float* topk_scores,
+                      int32_t* n_out, prism_trace* trace, void* cuda_stream);
+
+/* Free the handle and its workspaces (NULL is allowed).  Caller memory is untouched. */
+PRISM_API void prism_destroy(prism_handle* h);
+
+/* Text of the last error on this handle ("" if none); valid until the next call on the handle. */
+PRISM_API const char* prism_last_error(const prism_handle* h);
+
+/* Static name of a status code. */
+PRISM_API const char* prism_status_str(int status);
+
+/* Number of kernels this library launched since the handle was created (for launch accounting). */
+PRISM_API int64_t prism_launch_count(const prism_handle* h);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PRISM_H_ */

@@ -1,0 +1,90 @@
+/*
+ * prism_ops.h -- the individual steps of the PRISM hot path as C entry points.
+ *
+ * prism_select (prism.h) chains these steps; they are exported one by one so that every kernel can be
+ * checked against the CPU oracle and timed in isolation.  All pointers are DEVICE pointers unless
+ * marked host; every call only enqueues work on `stream` (a cudaStream_t, NULL = default stream)
+ * and returns a prism_status; nothing is copied to the host and nothing synchronises, except where a
+ * call says it allocates temporary device scratch (cudaMalloc/cudaFree synchronise implicitly).
+ * `dtype` is PRISM_FP32 or PRISM_BF16 and names the element type of weights and activations; the
+ * residual stream x and all scores are float.  The caller owns every buffer.
+ */
+#ifndef PRISM_OPS_H_
+#define PRISM_OPS_H_
+
+#include "prism.h"
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Packing (Sec. 4.5 "consolidate all candidates into one monolithic batch", padding-free):
+ * cu[N+1] = exclusive scan of (query_len + doc_len_i); seq2orig[i] = i; tokens[total] = query in front
+ * of every document; pos[t] = position of row t inside its sequence.  err_word (int, zeroed by the
+ * caller) receives bit 1 for a token id outside [0, vocab) and bit 2 for bad offsets.
+ * `total` = sum of all sequence lengths (the caller knows the offsets). */
+PRISM_API int prism_op_pack(const int32_t* query, int32_t query_len, const int32_t* cand_tokens, const int32_t* cand_offsets,
+                  int32_t N, int32_t total, int32_t vocab, int32_t* tokens, int32_t* pos, int32_t* cu,
+                  int32_t* seq2orig, int32_t* err_word, void* stream);
+
+/* Embedding lookup into the fp32 residual stream: x[t,:] = table[tokens[t],:]. */
+PRISM_API int prism_op_embed(const void* table, int32_t dtype, const int32_t* tokens, int32_t total, int32_t d, float* x,
+                   void* stream);
+
+/* RMSNorm: out[r,:] = x[r,:] / sqrt(mean(x[r,:]^2) + eps) * gain; out has element type `dtype`. */
+PRISM_API int prism_op_rmsnorm(const float* x, const void* gain, int32_t dtype, int32_t rows, int32_t d, float eps, void* out,
+                     void* stream);
+
+/* Optional per-head RMSNorm over head_dim (gains g_q / g_k), then the rotary embedding with half-split
+ * pairing (j, j + head_dim/2) and angle pos * theta^(-2j/head_dim); in place on the q and k heads of
+ * qkv [rows, (Hq+2Hkv)*head_dim].  Allocates and frees a temporary rotary table of max_pos rows. */
+PRISM_API int prism_op_qknorm_rope(void* qkv, int32_t dtype, const int32_t* pos, int32_t rows, int32_t n_q_heads,
+                         int32_t n_kv_heads, int32_t head_dim, int32_t qk_norm, const void* g_q, const void* g_k,
+                         float eps, float theta, int32_t max_pos, void* stream);
+
+/* Projection GEMM C = A[m,k] * B[n,k]^T with a fused epilogue:
+ *   epilogue 0: out[m,n] = C                      (dtype elements)
+ *   epilogue 1: resid[m,n] += C                   (float residual stream; out unused)
+ *   epilogue 2: out[m,n] = silu(A*B^T) * (A*B2^T) (SwiGLU; B = gate rows, B2 = up rows)
+ * impl PRISM_IMPL_AUTO uses the tcgen05 tensor-core kernel in bf16 mode (k, n multiples of 8; n a
+ * multiple of 128 for epilogue 2), PRISM_IMPL_SIMT the CUDA-core kernel.  The tensor-core kernel
+ * reports an expired bounded wait in err_word bit 4 (nullable for SIMT). */
+PRISM_API int prism_op_gemm(const void* a, const void* b, const void* b2, void* out, float* resid, int32_t m, int32_t n,
+                  int32_t k, int32_t dtype, int32_t epilogue, int32_t impl, int32_t* err_word, void* stream);
+
+/* Attention over packed sequences: for sequence s (rows cu[s]..cu[s+1]) and query head h (kv head
+ * h / (Hq/Hkv)): out = softmax(q k^T / sqrt(head_dim) [+ causal mask]) v.  qkv [total, (Hq+2Hkv)*dh],
+ * out [total, Hq*dh].  max_len >= the longest sequence. */
+PRISM_API int prism_op_attention(const void* qkv, void* out, const int32_t* cu, int32_t n_seq, int32_t max_len,
+                       int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim, int32_t causal, int32_t dtype,
+                       int32_t impl, void* stream);
+
+/* Score probe (Sec. 4.1: the model's classifier on an intermediate hidden state): for each sequence,
+ * final RMSNorm of its last row, then logit(score_head row 0) - logit(score_head row 1).
+ * Allocates and frees a temporary [d] float vector. */
+PRISM_API int prism_op_probe(const float* x, const int32_t* cu, int32_t n, int32_t d, const void* g_final,
+                   const void* score_head, int32_t dtype, float eps, float* scores, void* stream);
+
+/* One pruning decision (Sec. 4.1): rank, CV, clustering, routing, survivor offsets.
+ *   in : scores[n], cu_old[n+1], seq2orig_old[n]; state[8] = {n_active, n_tokens, k_rem, n_result,
+ *        done, err, 0, 0} (only k_rem and n_result are read); sched fields as in prism_prune_schedule
+ *        (keep_count applies to FIXED_KEEP); is_final = 1 scores the last layer; layer is recorded.
+ *   out: cu_new[n_new+1], seq2orig_new[n_new], old_of_new[n_new] (old batch position of each
+ *        survivor), state (updated), res_idx/res_score (leavers appended at n_result), rec (one
+ *        prism_probe_record in device memory, nullable).
+ * n <= PRISM_MAX_CANDIDATES.  Allocates and frees temporary device scratch. */
+PRISM_API int prism_op_route(const float* scores, const int32_t* cu_old, const int32_t* seq2orig_old, int32_t n, int32_t mode,
+                   int32_t keep_count, double cv_threshold, int32_t n_clusters, int32_t std_ddof,
+                   int32_t select_winners, int32_t is_final, int32_t layer, int32_t* cu_new, int32_t* seq2orig_new,
+                   int32_t* old_of_new, int32_t* state, int32_t* res_idx, float* res_score, prism_probe_record* rec,
+                   void* stream);
+
+/* Survivor gather (Fig. 4: only the deferred candidates are retained): row t of the new batch, owned
+ * by new sequence s, is copied from x_old[cu_old[old_of_new[s]] + (t - cu_new[s])]. */
+PRISM_API int prism_op_compact(const float* x_old, float* x_new, const int32_t* cu_old, const int32_t* cu_new,
+                     const int32_t* old_of_new, int32_t n_new, int32_t total_new, int32_t d, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PRISM_OPS_H_ */

@@ -1,0 +1,115 @@
+// Shared declarations of the PRISM CUDA path (internal; the public surface is include/*.h).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace prism {
+
+constexpr int kMaxCandidates = 4096;
+constexpr int kMaxClusters = 8;
+
+// Device error word bits (written by kernels instead of trapping).
+constexpr int kErrBadToken = 1;    // token id outside [0, vocab)
+constexpr int kErrBadOffsets = 2;  // non-monotone candidate offsets
+constexpr int kErrTimeout = 4;     // a bounded mbarrier wait gave up
+constexpr int kErrInternal = 8;
+
+// Epilogues of the projection GEMMs (C = A[M,K] * B[N,K]^T).
+enum Epilogue : int {
+  kEpiStore = 0,     // out[M,N] = acc                               (QKV projection)
+  kEpiResidual = 1,  // x[M,N] += acc, x fp32 residual stream        (O-proj, down-proj)
+  kEpiSwiGLU = 2,    // out[M,N] = silu(acc_gate) * acc_up           (gate/up projection)
+};
+
+struct RouteParams {
+  int mode;  // PRISM_PRUNE_*
+  int keep_count;
+  double cv_threshold;
+  int n_clusters;
+  int ddof;
+  int select_winners;
+  int is_final;  // 1: last layer, append the best k_rem and stop
+  int layer;
+};
+
+// Request state that lives on the device and is mirrored to the host after every scored layer.
+struct RouteState {
+  int n_active;
+  int n_tokens;
+  int k_rem;
+  int n_result;
+  int done;
+  int err;
+  int pad0, pad1;
+};
+
+struct ProbeRecordDev {  // layout mirrors prism_probe_record
+  int layer, n_active_before, fired, n_selected, n_dropped, n_deferred, k_rem_after, n_cuts;
+  int cuts[kMaxClusters];
+  int tokens_before;
+  int pad;
+  double cv;
+};
+
+// Bytes of global scratch the routing kernel needs for n candidates.
+inline size_t route_scratch_bytes(int n) {
+  size_t np1 = (size_t)n + 1;
+  return np1 * sizeof(double) * 4            // P1, P2, D[2]
+         + np1 * sizeof(int) * kMaxClusters  // argmin table
+         + np1 * sizeof(int) * 2             // valid flags, sorted positions
+         + 256;
+}
+
+// Opaque 128-byte TMA tensor map (mirrors CUtensorMap so that headers need not include cuda.h).
+struct alignas(64) TmaDesc {
+  unsigned char bytes[128];
+};
+
+// ---- launchers (each returns the CUDA error of the launch; none synchronises) -----------------
+cudaError_t launch_pack_offsets(const int* cand_offsets, int n, int query_len, int* cu, int* seq2orig,
+                                int* err, cudaStream_t st);
+cudaError_t launch_pack_tokens(const int* query, int query_len, const int* cand_tokens,
+                               const int* cand_offsets, const int* cu, int n, int total, int vocab,
+                               int* tokens, int* pos, int* err, cudaStream_t st);
+cudaError_t launch_positions(const int* cu, int n, int total, int* pos, cudaStream_t st);
+cudaError_t launch_embed(const void* table, int dtype, const int* tokens, int total, int d, float* x,
+                         cudaStream_t st);
+cudaError_t launch_rmsnorm(const float* x, const void* gain, int dtype, int rows, int d, float eps,
+                           void* out, cudaStream_t st);
+cudaError_t launch_rope_table(float* cos_t, float* sin_t, int max_pos, int head_dim, float theta,
+                              cudaStream_t st);
+cudaError_t launch_qknorm_rope(void* qkv, int dtype, const int* pos, int rows, int n_q_heads,
+                               int n_kv_heads, int head_dim, int qk_norm, const void* g_q,
+                               const void* g_k, float eps, const float* cos_t, const float* sin_t,
+                               cudaStream_t st);
+cudaError_t launch_probe(const float* x, const int* cu, int n, int d, const void* g_final, int dtype,
+                         const float* w_diff, float eps, float* scores, cudaStream_t st);
+cudaError_t launch_score_diff(const void* score_head, int dtype, int d, float* w_diff, cudaStream_t st);
+cudaError_t launch_compact_rows(const float* x_old, float* x_new, const int* cu_old, const int* cu_new,
+                                const int* old_of_new, int n_new, int total_new, int d, cudaStream_t st);
+
+cudaError_t launch_gemm_simt(const void* a, const void* b, const void* b2, void* out, float* resid, int m,
+                             int n, int k, int dtype, int epilogue, cudaStream_t st);
+cudaError_t launch_attention_simt(const void* qkv, void* out, const int* cu, int seq0, int nseq, int row0,
+                                  int max_len, int n_q_heads, int n_kv_heads, int head_dim, int causal,
+                                  int dtype, cudaStream_t st);
+
+// Tensor-core path (bf16).  make_tma_2d_bf16 describes a row-major [rows, cols] bf16 matrix that is
+// fetched in boxes of box_rows x 64 columns with the 128-byte swizzle the MMA descriptors expect.
+cudaError_t make_tma_2d_bf16(TmaDesc* out, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows,
+                             uint32_t box_cols);
+// b0/b1 describe the first and second 128 weight rows of a tile: the same matrix for plain
+// projections, the gate and the up matrix for kEpiSwiGLU.
+cudaError_t launch_gemm_tc(const TmaDesc& a, const TmaDesc& b0, const TmaDesc& b1, void* out, float* resid, int m,
+                           int n, int k, int epilogue, int* err, cudaStream_t st);
+cudaError_t launch_attention_mma(const void* qkv, void* out, const int* cu, int seq0, int nseq, int row0,
+                                 int max_len, int n_q_heads, int n_kv_heads, int causal, cudaStream_t st);
+
+cudaError_t launch_route(const float* scores, const int* cu_old, const int* seq2orig_old, int n,
+                         const RouteParams& p, int* cu_new, int* seq2orig_new, int* old_of_new,
+                         RouteState* state, int* res_idx, float* res_score, ProbeRecordDev* rec,
+                         float* trace_scores, int* trace_ids, void* scratch, cudaStream_t st);
+
+}  // namespace prism

@@ -1,0 +1,404 @@
+// HBM-bound kernels of the PRISM hot path: packing, embedding gather, RMSNorm, QK-norm + rotary
+// embedding, the score probe and the survivor row gather.  All accesses are 16-byte vectorised
+// and coalesced along the hidden dimension; reductions are fp32.
+#include "common.cuh"
+
+namespace prism {
+
+namespace {
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// Sum over the block; every thread gets the result.  red must hold 32 floats.
+__device__ __forceinline__ float block_sum(float v, float* red) {
+  v = warp_sum(v);
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
+  __syncthreads();
+  if (lane == 0) red[w] = v;
+  __syncthreads();
+  float t = (lane < nw) ? red[lane] : 0.f;
+  t = warp_sum(t);
+  return t;
+}
+
+__device__ __forceinline__ float to_f(float v) { return v; }
+__device__ __forceinline__ float to_f(__nv_bfloat16 v) { return __bfloat162float(v); }
+__device__ __forceinline__ void from_f(float& o, float v) { o = v; }
+__device__ __forceinline__ void from_f(__nv_bfloat16& o, float v) { o = __float2bfloat16_rn(v); }
+
+// upper_bound(cu[0..n], t) - 1: the sequence that owns packed row t.
+__device__ __forceinline__ int seq_of_row(const int* __restrict__ cu, int n, int t) {
+  int lo = 0, hi = n;  // invariant: cu[lo] <= t < cu[hi]
+  while (hi - lo > 1) {
+    int mid = (lo + hi) >> 1;
+    if (cu[mid] <= t) lo = mid; else hi = mid;
+  }
+  return lo;
+}
+
+// ------------------------------------------------------------------------------------------------
+// S0 pack: cu = exclusive scan of (query_len + doc_len_i), seq2orig = identity.  One block.
+__global__ void __launch_bounds__(1024) k_pack_offsets(const int* __restrict__ off, int n, int lq,
+                                                       int* __restrict__ cu, int* __restrict__ seq2orig,
+                                                       int* __restrict__ err) {
+  __shared__ int warp_tot[32];
+  __shared__ int carry;
+  if (threadIdx.x == 0) {
+    carry = 0;
+    if (n > 0 && off[0] != 0) atomicOr(err, kErrBadOffsets);
+  }
+  __syncthreads();
+  for (int base = 0; base < n; base += blockDim.x) {
+    int i = base + threadIdx.x;
+    int len = 0;
+    if (i < n) {
+      int dl = off[i + 1] - off[i];
+      if (dl < 0) { atomicOr(err, kErrBadOffsets); dl = 0; }
+      len = lq + dl;
+      seq2orig[i] = i;
+    }
+    int v = len;
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      int u = __shfl_up_sync(0xffffffffu, v, o);
+      if (lane >= o) v += u;
+    }
+    if (lane == 31) warp_tot[w] = v;
+    __syncthreads();
+    if (w == 0) {
+      int t = warp_tot[lane];
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        int u = __shfl_up_sync(0xffffffffu, t, o);
+        if (lane >= o) t += u;
+      }
+      warp_tot[lane] = t;
+    }
+    __syncthreads();
+    int excl = carry + (w ? warp_tot[w - 1] : 0) + v - len;
+    if (i < n) cu[i] = excl;
+    __syncthreads();
+    if (threadIdx.x == blockDim.x - 1) carry += warp_tot[31];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) cu[n] = carry;
+}
+
+// Packed token ids (query in front of every document) and per-token positions.
+__global__ void k_pack_tokens(const int* __restrict__ query, int lq, const int* __restrict__ cand,
+                              const int* __restrict__ off, const int* __restrict__ cu, int n, int total,
+                              int vocab, int* __restrict__ tokens, int* __restrict__ pos,
+                              int* __restrict__ err) {
+  for (int t = blockIdx.x * blockDim.x + threadIdx.x; t < total; t += gridDim.x * blockDim.x) {
+    int s = seq_of_row(cu, n, t);
+    int p = t - cu[s];
+    int tok = (p < lq) ? query[p] : cand[off[s] + (p - lq)];
+    if (tok < 0 || tok >= vocab) { atomicOr(err, kErrBadToken); tok = 0; }
+    tokens[t] = tok;
+    pos[t] = p;
+  }
+}
+
+__global__ void k_positions(const int* __restrict__ cu, int n, int total, int* __restrict__ pos) {
+  for (int t = blockIdx.x * blockDim.x + threadIdx.x; t < total; t += gridDim.x * blockDim.x) {
+    int s = seq_of_row(cu, n, t);
+    pos[t] = t - cu[s];
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// S1 embedding gather into the fp32 residual stream.  One block per token row.
+template <typename WT>
+__global__ void __launch_bounds__(128) k_embed(const WT* __restrict__ table, const int* __restrict__ tokens,
+                                               int d, float* __restrict__ x) {
+  const int t = blockIdx.x;
+  const WT* src = table + (size_t)tokens[t] * d;
+  float* dst = x + (size_t)t * d;
+  if constexpr (sizeof(WT) == 2) {
+    for (int c = threadIdx.x * 8; c < d; c += blockDim.x * 8) {
+      uint4 raw = *reinterpret_cast<const uint4*>(src + c);
+      const __nv_bfloat16* b = reinterpret_cast<const __nv_bfloat16*>(&raw);
+      float4 lo = make_float4(to_f(b[0]), to_f(b[1]), to_f(b[2]), to_f(b[3]));
+      float4 hi = make_float4(to_f(b[4]), to_f(b[5]), to_f(b[6]), to_f(b[7]));
+      *reinterpret_cast<float4*>(dst + c) = lo;
+      *reinterpret_cast<float4*>(dst + c + 4) = hi;
+    }
+  } else {
+    for (int c = threadIdx.x * 4; c < d; c += blockDim.x * 4)
+      *reinterpret_cast<float4*>(dst + c) = *reinterpret_cast<const float4*>(src + c);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// S2/S7 RMSNorm: y = x * rsqrt(mean(x^2) + eps) * g.  One block per row; the row stays in registers.
+template <typename OT, int kVec>
+__global__ void __launch_bounds__(256) k_rmsnorm(const float* __restrict__ x, const OT* __restrict__ gain, int d,
+                                                 float eps, OT* __restrict__ out) {
+  __shared__ float red[32];
+  const size_t row = blockIdx.x;
+  const float4* xr = reinterpret_cast<const float4*>(x + row * d);
+  const int nv = d >> 2;
+  float4 v[kVec];
+  float ss = 0.f;
+#pragma unroll
+  for (int i = 0; i < kVec; ++i) {
+    int c = threadIdx.x + i * 256;
+    if (c < nv) {
+      v[i] = xr[c];
+      ss += v[i].x * v[i].x + v[i].y * v[i].y + v[i].z * v[i].z + v[i].w * v[i].w;
+    }
+  }
+  ss = block_sum(ss, red);
+  const float r = 1.0f / sqrtf(ss / (float)d + eps);
+  OT* orow = out + row * d;
+#pragma unroll
+  for (int i = 0; i < kVec; ++i) {
+    int c = threadIdx.x + i * 256;
+    if (c < nv) {
+      const OT* g = gain + 4 * c;
+      float o0 = v[i].x * r * to_f(g[0]), o1 = v[i].y * r * to_f(g[1]);
+      float o2 = v[i].z * r * to_f(g[2]), o3 = v[i].w * r * to_f(g[3]);
+      if constexpr (sizeof(OT) == 2) {
+        __nv_bfloat162 a = __floats2bfloat162_rn(o0, o1), b = __floats2bfloat162_rn(o2, o3);
+        uint2 pk = make_uint2(*reinterpret_cast<uint32_t*>(&a), *reinterpret_cast<uint32_t*>(&b));
+        *reinterpret_cast<uint2*>(orow + 4 * c) = pk;
+      } else {
+        *reinterpret_cast<float4*>(orow + 4 * c) = make_float4(o0, o1, o2, o3);
+      }
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Rotary table in fp64, stored fp32: cos/sin(pos * theta^(-2j/dh)), j < dh/2.
+__global__ void k_rope_table(float* __restrict__ cos_t, float* __restrict__ sin_t, int max_pos, int half,
+                             double theta) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= max_pos * half) return;
+  int p = i / half, j = i % half;
+  double inv = pow(theta, -(double)j / (double)half);
+  double a = (double)p * inv;
+  cos_t[i] = (float)cos(a);
+  sin_t[i] = (float)sin(a);
+}
+
+// S4 optional per-head RMSNorm over dh, then rotation of pairs (j, j + dh/2).  In place on the q and
+// k heads of the packed qkv rows.  One warp per (row, head).
+template <typename T>
+__global__ void __launch_bounds__(256) k_qknorm_rope(T* __restrict__ qkv, const int* __restrict__ pos, int rows,
+                                                     int hq, int hkv, int dh, int qk_norm,
+                                                     const T* __restrict__ g_q, const T* __restrict__ g_k,
+                                                     float eps, const float* __restrict__ cos_t,
+                                                     const float* __restrict__ sin_t) {
+  const int heads = hq + hkv;
+  const long long wid = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (wid >= (long long)rows * heads) return;
+  const int row = (int)(wid / heads), h = (int)(wid % heads);
+  const int half = dh >> 1;
+  T* u = qkv + (size_t)row * (size_t)((hq + 2 * hkv) * dh) + (size_t)h * dh;
+  const T* g = (h < hq) ? g_q : g_k;
+  float a[4], b[4];  // dh <= 256 -> at most 4 pairs per lane
+  float ss = 0.f;
+  int cnt = 0;
+  for (int j = lane; j < half; j += 32, ++cnt) {
+    a[cnt] = to_f(u[j]);
+    b[cnt] = to_f(u[j + half]);
+    ss += a[cnt] * a[cnt] + b[cnt] * b[cnt];
+  }
+  float r = 1.f;
+  if (qk_norm) {
+    ss = warp_sum(ss);
+    r = 1.0f / sqrtf(ss / (float)dh + eps);
+  }
+  const float* ct = cos_t + (size_t)pos[row] * half;
+  const float* st = sin_t + (size_t)pos[row] * half;
+  cnt = 0;
+  for (int j = lane; j < half; j += 32, ++cnt) {
+    float x0 = a[cnt], x1 = b[cnt];
+    if (qk_norm) {
+      x0 = x0 * r * to_f(g[j]);
+      x1 = x1 * r * to_f(g[j + half]);
+    }
+    const float c = ct[j], s = st[j];
+    from_f(u[j], x0 * c - x1 * s);
+    from_f(u[j + half], x1 * c + x0 * s);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// S10 score probe: final RMSNorm of each sequence's last row, dotted with (w_yes - w_no).
+template <typename WT>
+__global__ void __launch_bounds__(256) k_probe(const float* __restrict__ x, const int* __restrict__ cu, int d,
+                                               const WT* __restrict__ g_final, const float* __restrict__ w_diff,
+                                               float eps, float* __restrict__ scores) {
+  __shared__ float red[32];
+  const int i = blockIdx.x;
+  const float* row = x + (size_t)(cu[i + 1] - 1) * d;
+  float ss = 0.f, dot = 0.f;
+  for (int c = threadIdx.x * 4; c < d; c += blockDim.x * 4) {
+    float4 v = *reinterpret_cast<const float4*>(row + c);
+    float4 w = *reinterpret_cast<const float4*>(w_diff + c);
+    ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+    dot += v.x * to_f(g_final[c]) * w.x + v.y * to_f(g_final[c + 1]) * w.y +
+           v.z * to_f(g_final[c + 2]) * w.z + v.w * to_f(g_final[c + 3]) * w.w;
+  }
+  ss = block_sum(ss, red);
+  dot = block_sum(dot, red);
+  if (threadIdx.x == 0) scores[i] = dot / sqrtf(ss / (float)d + eps);
+}
+
+template <typename WT>
+__global__ void k_score_diff(const WT* __restrict__ head, int d, float* __restrict__ w_diff) {
+  int c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (c < d) w_diff[c] = to_f(head[c]) - to_f(head[d + c]);
+}
+
+// ------------------------------------------------------------------------------------------------
+// S12 survivor gather: rows of the kept sequences move to their new packed position, order kept.
+__global__ void __launch_bounds__(256) k_compact_rows(const float* __restrict__ x_old, float* __restrict__ x_new,
+                                                      const int* __restrict__ cu_old,
+                                                      const int* __restrict__ cu_new,
+                                                      const int* __restrict__ old_of_new, int n_new,
+                                                      int total_new, int d) {
+  const int nv = d >> 2;
+  for (int t = blockIdx.x; t < total_new; t += gridDim.x) {
+    const int s = seq_of_row(cu_new, n_new, t);
+    const int src = cu_old[old_of_new[s]] + (t - cu_new[s]);
+    const float4* a = reinterpret_cast<const float4*>(x_old + (size_t)src * d);
+    float4* b = reinterpret_cast<float4*>(x_new + (size_t)t * d);
+    for (int c = threadIdx.x; c < nv; c += 4 * 256) {
+      float4 r0 = a[c], r1, r2, r3;
+      const bool h1 = c + 256 < nv, h2 = c + 512 < nv, h3 = c + 768 < nv;
+      if (h1) r1 = a[c + 256];
+      if (h2) r2 = a[c + 512];
+      if (h3) r3 = a[c + 768];
+      b[c] = r0;
+      if (h1) b[c + 256] = r1;
+      if (h2) b[c + 512] = r2;
+      if (h3) b[c + 768] = r3;
+    }
+  }
+}
+
+inline int grid_for(long long work, int block, int cap = 148 * 16) {
+  long long g = (work + block - 1) / block;
+  if (g < 1) g = 1;
+  if (g > cap) g = cap;
+  return (int)g;
+}
+
+}  // namespace
+
+cudaError_t launch_pack_offsets(const int* cand_offsets, int n, int query_len, int* cu, int* seq2orig,
+                                int* err, cudaStream_t st) {
+  k_pack_offsets<<<1, 1024, 0, st>>>(cand_offsets, n, query_len, cu, seq2orig, err);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_pack_tokens(const int* query, int query_len, const int* cand_tokens,
+                               const int* cand_offsets, const int* cu, int n, int total, int vocab,
+                               int* tokens, int* pos, int* err, cudaStream_t st) {
+  if (total <= 0) return cudaSuccess;
+  k_pack_tokens<<<grid_for(total, 256), 256, 0, st>>>(query, query_len, cand_tokens, cand_offsets, cu, n,
+                                                      total, vocab, tokens, pos, err);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_positions(const int* cu, int n, int total, int* pos, cudaStream_t st) {
+  if (total <= 0) return cudaSuccess;
+  k_positions<<<grid_for(total, 256), 256, 0, st>>>(cu, n, total, pos);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_embed(const void* table, int dtype, const int* tokens, int total, int d, float* x,
+                         cudaStream_t st) {
+  if (total <= 0) return cudaSuccess;
+  if (dtype == 1)
+    k_embed<__nv_bfloat16><<<total, 128, 0, st>>>((const __nv_bfloat16*)table, tokens, d, x);
+  else
+    k_embed<float><<<total, 128, 0, st>>>((const float*)table, tokens, d, x);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_rmsnorm(const float* x, const void* gain, int dtype, int rows, int d, float eps,
+                           void* out, cudaStream_t st) {
+  if (rows <= 0) return cudaSuccess;
+  const int nv = d >> 2;
+  if (nv > 8 * 256) return cudaErrorInvalidValue;
+#define PRISM_NORM(OT, V) \
+  k_rmsnorm<OT, V><<<rows, 256, 0, st>>>(x, (const OT*)gain, d, eps, (OT*)out)
+  if (dtype == 1) {
+    if (nv <= 256) PRISM_NORM(__nv_bfloat16, 1);
+    else if (nv <= 512) PRISM_NORM(__nv_bfloat16, 2);
+    else if (nv <= 1024) PRISM_NORM(__nv_bfloat16, 4);
+    else PRISM_NORM(__nv_bfloat16, 8);
+  } else {
+    if (nv <= 256) PRISM_NORM(float, 1);
+    else if (nv <= 512) PRISM_NORM(float, 2);
+    else if (nv <= 1024) PRISM_NORM(float, 4);
+    else PRISM_NORM(float, 8);
+  }
+#undef PRISM_NORM
+  return cudaGetLastError();
+}
+
+cudaError_t launch_rope_table(float* cos_t, float* sin_t, int max_pos, int head_dim, float theta,
+                              cudaStream_t st) {
+  const int half = head_dim / 2;
+  const long long n = (long long)max_pos * half;
+  if (n <= 0) return cudaSuccess;
+  k_rope_table<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(cos_t, sin_t, max_pos, half, (double)theta);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_qknorm_rope(void* qkv, int dtype, const int* pos, int rows, int n_q_heads,
+                               int n_kv_heads, int head_dim, int qk_norm, const void* g_q,
+                               const void* g_k, float eps, const float* cos_t, const float* sin_t,
+                               cudaStream_t st) {
+  if (rows <= 0) return cudaSuccess;
+  const long long warps = (long long)rows * (n_q_heads + n_kv_heads);
+  const unsigned grid = (unsigned)((warps + 7) / 8);
+  if (dtype == 1)
+    k_qknorm_rope<__nv_bfloat16><<<grid, 256, 0, st>>>((__nv_bfloat16*)qkv, pos, rows, n_q_heads, n_kv_heads,
+                                                       head_dim, qk_norm, (const __nv_bfloat16*)g_q,
+                                                       (const __nv_bfloat16*)g_k, eps, cos_t, sin_t);
+  else
+    k_qknorm_rope<float><<<grid, 256, 0, st>>>((float*)qkv, pos, rows, n_q_heads, n_kv_heads, head_dim,
+                                               qk_norm, (const float*)g_q, (const float*)g_k, eps, cos_t,
+                                               sin_t);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_probe(const float* x, const int* cu, int n, int d, const void* g_final, int dtype,
+                         const float* w_diff, float eps, float* scores, cudaStream_t st) {
+  if (n <= 0) return cudaSuccess;
+  if (dtype == 1)
+    k_probe<__nv_bfloat16><<<n, 256, 0, st>>>(x, cu, d, (const __nv_bfloat16*)g_final, w_diff, eps, scores);
+  else
+    k_probe<float><<<n, 256, 0, st>>>(x, cu, d, (const float*)g_final, w_diff, eps, scores);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_score_diff(const void* score_head, int dtype, int d, float* w_diff, cudaStream_t st) {
+  if (dtype == 1)
+    k_score_diff<__nv_bfloat16><<<(d + 255) / 256, 256, 0, st>>>((const __nv_bfloat16*)score_head, d, w_diff);
+  else
+    k_score_diff<float><<<(d + 255) / 256, 256, 0, st>>>((const float*)score_head, d, w_diff);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_compact_rows(const float* x_old, float* x_new, const int* cu_old, const int* cu_new,
+                                const int* old_of_new, int n_new, int total_new, int d, cudaStream_t st) {
+  if (total_new <= 0) return cudaSuccess;
+  int grid = total_new < 148 * 8 ? total_new : 148 * 8;
+  k_compact_rows<<<grid, 256, 0, st>>>(x_old, x_new, cu_old, cu_new, old_of_new, n_new, total_new, d);
+  return cudaGetLastError();
+}
+
+}  // namespace prism

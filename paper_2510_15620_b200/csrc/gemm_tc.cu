@@ -1,0 +1,393 @@
+// Projection GEMMs of the decoder block on the 5th-generation tensor cores (sm_100a):
+//   C[M,N] = A[M,K] * B[N,K]^T, bf16 operands (both K-major), fp32 accumulation in tensor memory.
+//
+// One persistent CTA per SM, warp-specialised:
+//   warp 0      TMA producer: 128x64 A tile + 256x64 B tile per stage, 128-byte swizzle, 4 stages
+//   warp 1      MMA issuer: one elected lane issues tcgen05.mma (M=128, N=256, K=16) into one of two
+//               256-column TMEM accumulators, commits stage-release and accumulator-ready barriers
+//   warps 2..5  epilogue: tcgen05.ld the accumulator (one row per thread), apply the fused epilogue
+//               (bf16 store | fp32 residual add | SwiGLU), while the MMA warp fills the other buffer
+// Every tile uses the same shape and the same K order whatever M is, so a row's result does not
+// depend on where it sits in the batch (duplicated candidates give bit-identical scores).
+//
+// Every mbarrier wait is bounded: on expiry the kernel records kErrTimeout and all roles drain to
+// the common exit, which frees the tensor memory.  No cluster multicast is used anywhere.
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace prism {
+
+namespace {
+
+constexpr int BM = 128, BN = 256, BK = 64, UMMA_K = 16;
+constexpr int kStages = 4;
+constexpr int kABytes = BM * BK * 2;           // 16 KB
+constexpr int kBBytes = BN * BK * 2;           // 32 KB
+constexpr int kStageBytes = kABytes + kBBytes; // 48 KB
+constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int kThreads = 192;
+constexpr unsigned long long kWaitCycles = 4000000000ull;  // ~2 s at boost clock
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return (uint32_t)__cvta_generic_to_shared(p);
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false (and records the timeout) instead of spinning forever.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* err, volatile int* abort_flag) {
+  if (mbar_try(bar, parity)) return true;
+  const unsigned long long t0 = clock64();
+  uint32_t it = 0;
+  while (!mbar_try(bar, parity)) {
+    if ((++it & 0x3ff) == 0) {
+      if (*abort_flag || clock64() - t0 > kWaitCycles) {
+        *abort_flag = 1;
+        atomicOr(err, kErrTimeout);
+        return false;
+      }
+    }
+  }
+  return true;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar)
+      : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// K-major operand tile, 128-byte swizzle: rows are 128 B apart, 8-row groups 1024 B apart.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr >> 4) & 0x3fff);
+  d |= (uint64_t)1 << 16;             // leading byte offset (unused for swizzled K-major)
+  d |= (uint64_t)(1024 >> 4) << 32;   // stride byte offset between 8-row groups
+  d |= (uint64_t)1 << 46;             // descriptor version of this architecture
+  d |= (uint64_t)2 << 61;             // SWIZZLE_128B
+  return d;
+}
+
+// kind::f16 instruction descriptor: D fp32, A/B bf16, both K-major, M=128, N=256.
+constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+
+__device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+template <int kEpi>
+__global__ void __launch_bounds__(kThreads, 1)
+k_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b0,
+          const __grid_constant__ CUtensorMap map_b1, __nv_bfloat16* __restrict__ out, float* __restrict__ resid,
+          int m, int n, int k, int* __restrict__ err) {
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t tiles = (raw + 1023u) & ~1023u;  // swizzled tiles need 1024-byte alignment
+  unsigned char* gen_tiles = smem_raw + (tiles - raw);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(gen_tiles + kStages * kStageBytes);
+  // bars: full[kStages], empty[kStages], acc_full[2], acc_empty[2]; then tmem base and abort flag
+  const uint32_t bar_full = smem_u32(bars), bar_empty = smem_u32(bars + kStages);
+  const uint32_t bar_acc_full = smem_u32(bars + 2 * kStages), bar_acc_empty = smem_u32(bars + 2 * kStages + 2);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 4);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  // Output tile width: SwiGLU tiles hold 128 gate + 128 up columns and produce 128 outputs.
+  constexpr int kOutCols = (kEpi == kEpiSwiGLU) ? 128 : 256;
+  const int m_tiles = (m + BM - 1) / BM, n_tiles = (n + kOutCols - 1) / kOutCols;
+  const int num_tiles = m_tiles * n_tiles, num_kb = (k + BK - 1) / BK;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(bar_full + 8 * s, 1);
+      mbar_init(bar_empty + 8 * s, 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(bar_acc_full + 8 * a, 1);
+      mbar_init(bar_acc_empty + 8 * a, 4);
+    }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {  // allocate all 512 tensor-memory columns (two 256-column accumulators)
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512));
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::);
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      uint32_t stage = 0, phase = 0, armed = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+        const int mt = tile / n_tiles, nt = tile % n_tiles;
+        const int row_a = mt * BM;
+        const int row_b0 = (kEpi == kEpiSwiGLU) ? nt * 128 : nt * BN;
+        const int row_b1 = (kEpi == kEpiSwiGLU) ? nt * 128 : nt * BN + 128;
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1, err, abort_flag)) { ok = false; break; }
+          const uint32_t sa = tiles + stage * kStageBytes, sb = sa + kABytes;
+          mbar_expect_tx(bar_full + 8 * stage, kStageBytes);
+          tma_load_2d(sa, &map_a, kb * BK, row_a, bar_full + 8 * stage);
+          tma_load_2d(sb, &map_b0, kb * BK, row_b0, bar_full + 8 * stage);
+          tma_load_2d(sb + kBBytes / 2, &map_b1, kb * BK, row_b1, bar_full + 8 * stage);
+          armed |= 1u << stage;
+          if (++stage == kStages) { stage = 0; phase ^= 1; }
+        }
+      }
+      if (!ok) {
+        // Let copies already in flight land before shared memory is released (bounded).
+        for (int s = 0; s < kStages; ++s) {
+          if (!(armed & (1u << s))) continue;
+          const uint32_t par = (s < (int)stage) ? phase : (phase ^ 1);
+          const unsigned long long t0 = clock64();
+          while (!mbar_try(bar_full + 8 * s, par) && clock64() - t0 < kWaitCycles / 8) {}
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      uint32_t stage = 0, phase = 0;
+      bool ok = true;
+      int it = 0;
+      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++it) {
+        const uint32_t acc = it & 1, acc_phase = (it >> 1) & 1;
+        if (!mbar_wait(bar_acc_empty + 8 * acc, acc_phase ^ 1, err, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + acc * BN;
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!mbar_wait(bar_full + 8 * stage, phase, err, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = tiles + stage * kStageBytes, sb = sa + kABytes;
+          const uint64_t da = smem_desc_sw128(sa), db = smem_desc_sw128(sb);
+#pragma unroll
+          for (int kk = 0; kk < BK / UMMA_K; ++kk) {
+            // advancing K by 16 bf16 = 32 bytes inside the swizzle atom: +2 in 16-byte units
+            umma_bf16(d_tmem, da + 2 * kk, db + 2 * kk, kIdesc, (kb | kk) != 0);
+          }
+          umma_commit(bar_empty + 8 * stage);  // stage is free once these MMAs have read it
+          if (++stage == kStages) { stage = 0; phase ^= 1; }
+        }
+        if (ok) umma_commit(bar_acc_full + 8 * acc);  // accumulator complete
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue (4 warps, 128 rows)
+    const int quarter = warp & 3;  // TMEM lane quarter this warp may read
+    bool ok = true;
+    int it = 0;
+    for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++it) {
+      const uint32_t acc = it & 1, acc_phase = (it >> 1) & 1;
+      const int mt = tile / n_tiles, nt = tile % n_tiles;
+      if (!mbar_wait(bar_acc_full + 8 * acc, acc_phase, err, abort_flag)) { ok = false; break; }
+      tc_fence_after();
+      const int row = mt * BM + quarter * 32 + lane;
+      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN;
+      const int col0 = nt * kOutCols;
+      if constexpr (kEpi == kEpiSwiGLU) {
+#pragma unroll 1
+        for (int c = 0; c < 4; ++c) {
+          uint32_t g[32], u[32];
+          tmem_ld32(taddr + c * 32, g);
+          tmem_ld32(taddr + 128 + c * 32, u);
+          tmem_ld_wait();
+          if (row < m) {
+            __nv_bfloat16* o = out + (size_t)row * n + col0 + c * 32;
+#pragma unroll
+            for (int v = 0; v < 4; ++v) {
+              if (col0 + c * 32 + v * 8 < n) {
+                uint32_t pk[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                  const float g0 = __uint_as_float(g[v * 8 + 2 * e]), g1 = __uint_as_float(g[v * 8 + 2 * e + 1]);
+                  const float u0 = __uint_as_float(u[v * 8 + 2 * e]), u1 = __uint_as_float(u[v * 8 + 2 * e + 1]);
+                  pk[e] = pack_bf16(g0 / (1.f + __expf(-g0)) * u0, g1 / (1.f + __expf(-g1)) * u1);
+                }
+                *reinterpret_cast<uint4*>(o + v * 8) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+              }
+            }
+          }
+        }
+      } else {
+#pragma unroll 1
+        for (int c = 0; c < 8; ++c) {
+          uint32_t r[32];
+          tmem_ld32(taddr + c * 32, r);
+          tmem_ld_wait();
+          if (row < m) {
+            if constexpr (kEpi == kEpiStore) {
+              __nv_bfloat16* o = out + (size_t)row * n + col0 + c * 32;
+#pragma unroll
+              for (int v = 0; v < 4; ++v) {
+                if (col0 + c * 32 + v * 8 < n) {
+                  uint4 pk;
+                  pk.x = pack_bf16(__uint_as_float(r[v * 8 + 0]), __uint_as_float(r[v * 8 + 1]));
+                  pk.y = pack_bf16(__uint_as_float(r[v * 8 + 2]), __uint_as_float(r[v * 8 + 3]));
+                  pk.z = pack_bf16(__uint_as_float(r[v * 8 + 4]), __uint_as_float(r[v * 8 + 5]));
+                  pk.w = pack_bf16(__uint_as_float(r[v * 8 + 6]), __uint_as_float(r[v * 8 + 7]));
+                  *reinterpret_cast<uint4*>(o + v * 8) = pk;
+                }
+              }
+            } else {
+              float* o = resid + (size_t)row * n + col0 + c * 32;
+#pragma unroll
+              for (int v = 0; v < 8; ++v) {
+                if (col0 + c * 32 + v * 4 < n) {
+                  float4 x = *reinterpret_cast<float4*>(o + v * 4);
+                  x.x += __uint_as_float(r[v * 4 + 0]);
+                  x.y += __uint_as_float(r[v * 4 + 1]);
+                  x.z += __uint_as_float(r[v * 4 + 2]);
+                  x.w += __uint_as_float(r[v * 4 + 3]);
+                  *reinterpret_cast<float4*>(o + v * 4) = x;
+                }
+              }
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_acc_empty + 8 * acc);
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512));
+  }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+}  // namespace
+
+static_assert(sizeof(CUtensorMap) == sizeof(TmaDesc), "TmaDesc must mirror CUtensorMap");
+
+cudaError_t make_tma_2d_bf16(TmaDesc* out, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows,
+                             uint32_t box_cols) {
+  EncodeTiledFn enc = get_encode();
+  if (!enc) return cudaErrorNotSupported;
+  if ((reinterpret_cast<uintptr_t>(base) & 15) || (cols * 2) % 16 || box_cols * 2 != 128 || box_rows > 256)
+    return cudaErrorInvalidValue;
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {cols * 2};
+  cuuint32_t box[2] = {box_cols, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = enc(reinterpret_cast<CUtensorMap*>(out), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base),
+                   dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
+int gemm_tc_sm_count() {
+  static int sms = 0;
+  if (!sms) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (sms <= 0) sms = 148;
+  }
+  return sms;
+}
+
+cudaError_t launch_gemm_tc(const TmaDesc& a, const TmaDesc& b0, const TmaDesc& b1, void* out, float* resid, int m,
+                           int n, int k, int epilogue, int* err, cudaStream_t st) {
+  if (m <= 0 || n <= 0) return cudaSuccess;
+  if (k <= 0 || (k % 8) || (n % 8)) return cudaErrorInvalidValue;
+  static bool attr = false;
+  if (!attr) {
+    cudaError_t e;
+    if ((e = cudaFuncSetAttribute(k_gemm_tc<kEpiStore>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes)) ||
+        (e = cudaFuncSetAttribute(k_gemm_tc<kEpiResidual>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes)) ||
+        (e = cudaFuncSetAttribute(k_gemm_tc<kEpiSwiGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes)))
+      return e;
+    attr = true;
+  }
+  const int out_cols = epilogue == kEpiSwiGLU ? 128 : 256;
+  const long long tiles = (long long)((m + BM - 1) / BM) * ((n + out_cols - 1) / out_cols);
+  const int sms = gemm_tc_sm_count();
+  const int grid = (int)(tiles < sms ? tiles : sms);
+  const CUtensorMap& ma = reinterpret_cast<const CUtensorMap&>(a);
+  const CUtensorMap& mb0 = reinterpret_cast<const CUtensorMap&>(b0);
+  const CUtensorMap& mb1 = reinterpret_cast<const CUtensorMap&>(b1);
+  if (epilogue == kEpiStore)
+    k_gemm_tc<kEpiStore><<<grid, kThreads, kSmemBytes, st>>>(ma, mb0, mb1, (__nv_bfloat16*)out, resid, m, n, k, err);
+  else if (epilogue == kEpiResidual)
+    k_gemm_tc<kEpiResidual><<<grid, kThreads, kSmemBytes, st>>>(ma, mb0, mb1, (__nv_bfloat16*)out, resid, m, n, k, err);
+  else
+    k_gemm_tc<kEpiSwiGLU><<<grid, kThreads, kSmemBytes, st>>>(ma, mb0, mb1, (__nv_bfloat16*)out, resid, m, n, k, err);
+  return cudaGetLastError();
+}
+
+}  // namespace prism

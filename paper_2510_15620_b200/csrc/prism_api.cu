@@ -1,0 +1,668 @@
+// Host side of the C ABI: handle, workspaces, the layer-major request driver with chunked execution
+// (Sec. 4.3) and overlapped layer streaming (Sec. 4.2), probe -> route -> compact after the
+// designated layers (Sec. 4.1), final top-K.  All arithmetic of the method runs in the kernels.
+#include <algorithm>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "../../include/prism.h"
+#include "common.cuh"
+
+using namespace prism;
+
+static_assert(sizeof(prism_probe_record) == sizeof(ProbeRecordDev), "probe record layouts must match");
+static_assert(PRISM_MAX_CLUSTERS == kMaxClusters && PRISM_MAX_CANDIDATES == kMaxCandidates, "limits must match");
+
+namespace {
+
+struct LayerDev {  // device pointers of one layer's tensors (resident, or inside a streaming slot)
+  const void *g_attn, *w_qkv, *g_q, *g_k, *w_o, *g_ffn, *w_gate, *w_up, *w_down;
+};
+
+struct LayerMaps {  // TMA descriptors of the B operands
+  TmaDesc qkv, o, gate, up, down;
+};
+
+}  // namespace
+
+struct prism_handle {
+  prism_model_cfg cfg{};
+  std::vector<prism_layer_weights> layers;  // caller's pointers (device, or pinned host when streamed)
+  const void *embed = nullptr, *g_final = nullptr, *score_head = nullptr;
+  int esz = 4;
+  int chunk_tokens = 0;
+  bool tc = false;  // tensor-core GEMM path
+  bool fa = false;  // tensor-core attention path
+
+  std::vector<void*> dev_allocs;
+  std::vector<void*> host_allocs;
+  int64_t workspace_bytes = 0;
+  int64_t launches = 0;
+  std::string err;
+
+  float* x[2] = {nullptr, nullptr};
+  int *tokens = nullptr, *pos = nullptr, *cu[2] = {nullptr, nullptr}, *seq2orig[2] = {nullptr, nullptr};
+  int* old_of_new = nullptr;
+  void *a_norm = nullptr, *qkv = nullptr, *attn = nullptr, *hbuf = nullptr;
+  float *scores = nullptr, *res_score = nullptr, *w_diff = nullptr, *rope_cos = nullptr, *rope_sin = nullptr;
+  int *res_idx = nullptr, *errword = nullptr;
+  RouteState* state = nullptr;
+  ProbeRecordDev* recs = nullptr;
+  float* trace_scores = nullptr;
+  int* trace_ids = nullptr;
+  void* route_scratch = nullptr;
+  int *in_query = nullptr, *in_cand = nullptr, *in_off = nullptr, *out_idx = nullptr;
+  float* out_score = nullptr;
+
+  // pinned host mirrors
+  int* h_cu = nullptr;       // offsets of the live batch
+  int* h_cu_next = nullptr;  // offsets after the pending prune decision
+  int* h_off = nullptr;
+  RouteState* h_state = nullptr;
+  int* h_err = nullptr;
+
+  // streaming
+  unsigned char* slot[2] = {nullptr, nullptr};
+  size_t slot_bytes = 0;
+  size_t off_g_attn = 0, off_qkv = 0, off_gq = 0, off_gk = 0, off_o = 0, off_g_ffn = 0, off_gate = 0, off_up = 0,
+         off_down = 0;
+  cudaStream_t copy_stream = nullptr;
+  cudaEvent_t ev_copied[2] = {nullptr, nullptr}, ev_freed[2] = {nullptr, nullptr};
+
+  // TMA descriptors
+  TmaDesc map_a_norm{}, map_attn{}, map_hbuf{};
+  std::vector<LayerMaps> maps;  // per layer (resident) or per slot (streamed)
+};
+
+namespace {
+
+int fail(prism_handle* h, int code, const std::string& msg) {
+  if (h) h->err = msg;
+  return code;
+}
+
+int cuda_fail(prism_handle* h, cudaError_t e, const char* what) {
+  return fail(h, e == cudaErrorMemoryAllocation ? PRISM_ERR_NOMEM : PRISM_ERR_CUDA,
+              std::string(what) + ": " + cudaGetErrorString(e));
+}
+
+#define PRISM_CUDA(h, call)                                    \
+  do {                                                         \
+    cudaError_t e__ = (call);                                  \
+    if (e__ != cudaSuccess) return cuda_fail((h), e__, #call); \
+  } while (0)
+
+#define PRISM_LAUNCH(h, call)                                  \
+  do {                                                         \
+    cudaError_t e__ = (call);                                  \
+    (h)->launches++;                                           \
+    if (e__ != cudaSuccess) return cuda_fail((h), e__, #call); \
+  } while (0)
+
+template <typename T>
+cudaError_t dev_alloc(prism_handle* h, T** p, size_t count) {
+  size_t bytes = std::max<size_t>(count * sizeof(T), 256);
+  void* q = nullptr;
+  cudaError_t e = cudaMalloc(&q, bytes);
+  if (e != cudaSuccess) return e;
+  h->dev_allocs.push_back(q);
+  h->workspace_bytes += (int64_t)bytes;
+  *p = reinterpret_cast<T*>(q);
+  return cudaSuccess;
+}
+
+template <typename T>
+cudaError_t host_alloc(prism_handle* h, T** p, size_t count) {
+  void* q = nullptr;
+  cudaError_t e = cudaMallocHost(&q, std::max<size_t>(count * sizeof(T), 64));
+  if (e != cudaSuccess) return e;
+  h->host_allocs.push_back(q);
+  *p = reinterpret_cast<T*>(q);
+  return cudaSuccess;
+}
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// Bytes of per-token chunk intermediates: normed input, qkv, attention output, SwiGLU output.
+size_t per_token_bytes(const prism_model_cfg& c, int esz) {
+  const size_t nqkv = (size_t)(c.n_q_heads + 2 * c.n_kv_heads) * c.head_dim;
+  return ((size_t)c.hidden + nqkv + (size_t)c.n_q_heads * c.head_dim + (size_t)c.ffn) * esz;
+}
+
+LayerDev layer_in_slot(const prism_handle* h, int s) {
+  const unsigned char* b = h->slot[s];
+  LayerDev d;
+  d.g_attn = b + h->off_g_attn;
+  d.w_qkv = b + h->off_qkv;
+  d.g_q = b + h->off_gq;
+  d.g_k = b + h->off_gk;
+  d.w_o = b + h->off_o;
+  d.g_ffn = b + h->off_g_ffn;
+  d.w_gate = b + h->off_gate;
+  d.w_up = b + h->off_up;
+  d.w_down = b + h->off_down;
+  return d;
+}
+
+LayerDev layer_resident(const prism_handle* h, int l) {
+  const prism_layer_weights& w = h->layers[l];
+  return LayerDev{w.g_attn, w.w_qkv, w.g_q, w.g_k, w.w_o, w.g_ffn, w.w_gate, w.w_up, w.w_down};
+}
+
+cudaError_t build_maps(const prism_handle* h, const LayerDev& d, LayerMaps* m) {
+  const prism_model_cfg& c = h->cfg;
+  const uint64_t nqkv = (uint64_t)(c.n_q_heads + 2 * c.n_kv_heads) * c.head_dim;
+  const uint64_t hd = (uint64_t)c.n_q_heads * c.head_dim;
+  cudaError_t e;
+  if ((e = make_tma_2d_bf16(&m->qkv, d.w_qkv, nqkv, c.hidden, 128, 64))) return e;
+  if ((e = make_tma_2d_bf16(&m->o, d.w_o, c.hidden, hd, 128, 64))) return e;
+  if ((e = make_tma_2d_bf16(&m->gate, d.w_gate, c.ffn, c.hidden, 128, 64))) return e;
+  if ((e = make_tma_2d_bf16(&m->up, d.w_up, c.ffn, c.hidden, 128, 64))) return e;
+  if ((e = make_tma_2d_bf16(&m->down, d.w_down, c.hidden, c.ffn, 128, 64))) return e;
+  return cudaSuccess;
+}
+
+// Enqueue the host->device copy of layer l into slot s on the copy stream.
+int enqueue_layer_copy(prism_handle* h, int l, int s) {
+  const prism_model_cfg& c = h->cfg;
+  const prism_layer_weights& w = h->layers[l];
+  const size_t e = h->esz, d = c.hidden, dh = c.head_dim;
+  const size_t nqkv = (size_t)(c.n_q_heads + 2 * c.n_kv_heads) * dh, hd = (size_t)c.n_q_heads * dh;
+  unsigned char* b = h->slot[s];
+  cudaStream_t cs = h->copy_stream;
+  PRISM_CUDA(h, cudaMemcpyAsync(b + h->off_g_attn, w.g_attn, d * e, cudaMemcpyHostToDevice, cs));
+  PRISM_CUDA(h, cudaMemcpyAsync(b + h->off_qkv, w.w_qkv, nqkv * d * e, cudaMemcpyHostToDevice, cs));
+  if (c.qk_norm) {
+    PRISM_CUDA(h, cudaMemcpyAsync(b + h->off_gq, w.g_q, dh * e, cudaMemcpyHostToDevice, cs));
+    PRISM_CUDA(h, cudaMemcpyAsync(b + h->off_gk, w.g_k, dh * e, cudaMemcpyHostToDevice, cs));
+  }
+  PRISM_CUDA(h, cudaMemcpyAsync(b + h->off_o, w.w_o, d * hd * e, cudaMemcpyHostToDevice, cs));
+  PRISM_CUDA(h, cudaMemcpyAsync(b + h->off_g_ffn, w.g_ffn, d * e, cudaMemcpyHostToDevice, cs));
+  PRISM_CUDA(h, cudaMemcpyAsync(b + h->off_gate, w.w_gate, (size_t)c.ffn * d * e, cudaMemcpyHostToDevice, cs));
+  PRISM_CUDA(h, cudaMemcpyAsync(b + h->off_up, w.w_up, (size_t)c.ffn * d * e, cudaMemcpyHostToDevice, cs));
+  PRISM_CUDA(h, cudaMemcpyAsync(b + h->off_down, w.w_down, d * (size_t)c.ffn * e, cudaMemcpyHostToDevice, cs));
+  PRISM_CUDA(h, cudaEventRecord(h->ev_copied[s], cs));
+  return PRISM_OK;
+}
+
+int validate_cfg(const prism_model_cfg& c, std::string* why) {
+  auto bad = [&](const char* m) { *why = m; return PRISM_ERR_INVALID_ARG; };
+  if (c.n_layers < 1 || c.n_layers > PRISM_MAX_LAYERS) return bad("n_layers out of range");
+  if (c.hidden < 4 || c.n_q_heads < 1 || c.n_kv_heads < 1 || c.head_dim < 2 || c.ffn < 1 || c.vocab < 2)
+    return bad("non-positive model dimension");
+  if (c.n_q_heads % c.n_kv_heads) return bad("n_q_heads must be a multiple of n_kv_heads");
+  if (c.dtype != PRISM_FP32 && c.dtype != PRISM_BF16) return bad("dtype must be PRISM_FP32 or PRISM_BF16");
+  if (c.max_seq_len < 1 || c.max_candidates < 1 || c.max_total_tokens < 1) return bad("maxima must be positive");
+  if (c.max_candidates > PRISM_MAX_CANDIDATES) return bad("max_candidates exceeds PRISM_MAX_CANDIDATES");
+  if (c.activation_budget_bytes < 0) return bad("negative activation budget");
+  if (c.weight_residency != PRISM_WEIGHTS_DEVICE && c.weight_residency != PRISM_WEIGHTS_HOST_STREAMED)
+    return bad("unknown weight_residency");
+  if (!(c.rope_theta > 0.f) || !(c.rms_eps >= 0.f)) return bad("rope_theta must be > 0 and rms_eps >= 0");
+  auto unsup = [&](const char* m) { *why = m; return PRISM_ERR_UNSUPPORTED; };
+  if (c.head_dim % 2 || c.head_dim > 256) return unsup("head_dim must be even and <= 256");
+  if (c.hidden % 4 || c.hidden > 8192) return unsup("hidden must be a multiple of 4 and <= 8192");
+  if (c.dtype == PRISM_BF16) {
+    if (c.hidden % 8 || c.ffn % 8 || c.head_dim % 8) return unsup("bf16 mode needs hidden, ffn, head_dim multiples of 8");
+    if (c.gemm_impl == PRISM_IMPL_AUTO && (c.ffn % 128)) return unsup("tensor-core SwiGLU needs ffn multiple of 128");
+    if (c.attention_impl == PRISM_IMPL_AUTO && c.head_dim != 128) return unsup("tensor-core attention needs head_dim 128");
+  }
+  return PRISM_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* prism_status_str(int s) {
+  switch (s) {
+    case PRISM_OK: return "PRISM_OK";
+    case PRISM_ERR_INVALID_ARG: return "PRISM_ERR_INVALID_ARG";
+    case PRISM_ERR_SHAPE_LIMIT: return "PRISM_ERR_SHAPE_LIMIT";
+    case PRISM_ERR_BAD_INPUT: return "PRISM_ERR_BAD_INPUT";
+    case PRISM_ERR_BUDGET: return "PRISM_ERR_BUDGET";
+    case PRISM_ERR_CUDA: return "PRISM_ERR_CUDA";
+    case PRISM_ERR_TIMEOUT: return "PRISM_ERR_TIMEOUT";
+    case PRISM_ERR_NOMEM: return "PRISM_ERR_NOMEM";
+    case PRISM_ERR_UNSUPPORTED: return "PRISM_ERR_UNSUPPORTED";
+    default: return "PRISM_ERR_UNKNOWN";
+  }
+}
+
+const char* prism_last_error(const prism_handle* h) { return h ? h->err.c_str() : ""; }
+
+int64_t prism_launch_count(const prism_handle* h) { return h ? h->launches : 0; }
+
+void prism_destroy(prism_handle* h) {
+  if (!h) return;
+  cudaDeviceSynchronize();
+  for (void* p : h->dev_allocs) cudaFree(p);
+  for (void* p : h->host_allocs) cudaFreeHost(p);
+  for (int s = 0; s < 2; ++s) {
+    if (h->ev_copied[s]) cudaEventDestroy(h->ev_copied[s]);
+    if (h->ev_freed[s]) cudaEventDestroy(h->ev_freed[s]);
+  }
+  if (h->copy_stream) cudaStreamDestroy(h->copy_stream);
+  delete h;
+}
+
+static int create_impl(prism_handle* h, const prism_model_cfg* cfg, const prism_weights* w) {
+  const prism_model_cfg& c = *cfg;
+  h->cfg = c;
+  h->esz = c.dtype == PRISM_BF16 ? 2 : 4;
+  h->tc = c.dtype == PRISM_BF16 && c.gemm_impl == PRISM_IMPL_AUTO;
+  h->fa = c.dtype == PRISM_BF16 && c.attention_impl == PRISM_IMPL_AUTO;
+  const bool streamed = c.weight_residency == PRISM_WEIGHTS_HOST_STREAMED;
+  if (!w->embed || !w->g_final || !w->score_head || !w->layers) return fail(h, PRISM_ERR_INVALID_ARG, "null weight pointer");
+  h->embed = w->embed;
+  h->g_final = w->g_final;
+  h->score_head = w->score_head;
+  h->layers.assign(w->layers, w->layers + c.n_layers);
+  for (int l = 0; l < c.n_layers; ++l) {
+    const prism_layer_weights& lw = h->layers[l];
+    const void* req[] = {lw.g_attn, lw.w_qkv, lw.w_o, lw.g_ffn, lw.w_gate, lw.w_up, lw.w_down};
+    for (const void* p : req)
+      if (!p || (reinterpret_cast<uintptr_t>(p) & 15)) return fail(h, PRISM_ERR_INVALID_ARG, "layer tensor null or not 16-byte aligned");
+    if (c.qk_norm && (!lw.g_q || !lw.g_k)) return fail(h, PRISM_ERR_INVALID_ARG, "qk_norm set but g_q/g_k null");
+  }
+
+  const size_t D = c.hidden, T = c.max_total_tokens, N = c.max_candidates;
+  const size_t nqkv = (size_t)(c.n_q_heads + 2 * c.n_kv_heads) * c.head_dim, hd = (size_t)c.n_q_heads * c.head_dim;
+  // Chunked execution: hidden states of all sequences (both ping-pong buffers) + one chunk's
+  // intermediates must fit the activation budget.
+  const size_t hidden_bytes = 2 * T * D * sizeof(float);
+  const size_t ptb = per_token_bytes(c, h->esz);
+  size_t chunk = T;
+  if (c.activation_budget_bytes > 0) {
+    const size_t budget = (size_t)c.activation_budget_bytes;
+    if (budget <= hidden_bytes || (budget - hidden_bytes) / ptb < (size_t)c.max_seq_len)
+      return fail(h, PRISM_ERR_BUDGET, "activation budget cannot hold the hidden states plus one max_seq_len sequence");
+    chunk = std::min(T, (budget - hidden_bytes) / ptb);
+  }
+  h->chunk_tokens = (int)chunk;
+
+  PRISM_CUDA(h, dev_alloc(h, &h->x[0], T * D));
+  PRISM_CUDA(h, dev_alloc(h, &h->x[1], T * D));
+  PRISM_CUDA(h, dev_alloc(h, &h->tokens, T));
+  PRISM_CUDA(h, dev_alloc(h, &h->pos, T));
+  for (int i = 0; i < 2; ++i) {
+    PRISM_CUDA(h, dev_alloc(h, &h->cu[i], N + 1));
+    PRISM_CUDA(h, dev_alloc(h, &h->seq2orig[i], N));
+  }
+  PRISM_CUDA(h, dev_alloc(h, &h->old_of_new, N));
+  PRISM_CUDA(h, dev_alloc(h, (unsigned char**)&h->a_norm, chunk * D * h->esz));
+  PRISM_CUDA(h, dev_alloc(h, (unsigned char**)&h->qkv, chunk * nqkv * h->esz));
+  PRISM_CUDA(h, dev_alloc(h, (unsigned char**)&h->attn, chunk * hd * h->esz));
+  PRISM_CUDA(h, dev_alloc(h, (unsigned char**)&h->hbuf, chunk * (size_t)c.ffn * h->esz));
+  PRISM_CUDA(h, dev_alloc(h, &h->scores, N));
+  PRISM_CUDA(h, dev_alloc(h, &h->res_idx, N));
+  PRISM_CUDA(h, dev_alloc(h, &h->res_score, N));
+  PRISM_CUDA(h, dev_alloc(h, &h->w_diff, D));
+  PRISM_CUDA(h, dev_alloc(h, &h->rope_cos, (size_t)c.max_seq_len * (c.head_dim / 2)));
+  PRISM_CUDA(h, dev_alloc(h, &h->rope_sin, (size_t)c.max_seq_len * (c.head_dim / 2)));
+  PRISM_CUDA(h, dev_alloc(h, &h->errword, 1));
+  PRISM_CUDA(h, dev_alloc(h, &h->state, 1));
+  PRISM_CUDA(h, dev_alloc(h, &h->recs, (size_t)c.n_layers));
+  PRISM_CUDA(h, dev_alloc(h, &h->trace_scores, (size_t)c.n_layers * N));
+  PRISM_CUDA(h, dev_alloc(h, &h->trace_ids, (size_t)c.n_layers * N));
+  PRISM_CUDA(h, dev_alloc(h, (unsigned char**)&h->route_scratch, route_scratch_bytes((int)N)));
+  PRISM_CUDA(h, dev_alloc(h, &h->in_query, (size_t)c.max_seq_len));
+  PRISM_CUDA(h, dev_alloc(h, &h->in_cand, T));
+  PRISM_CUDA(h, dev_alloc(h, &h->in_off, N + 1));
+  PRISM_CUDA(h, dev_alloc(h, &h->out_idx, N));
+  PRISM_CUDA(h, dev_alloc(h, &h->out_score, N));
+  PRISM_CUDA(h, host_alloc(h, &h->h_cu, N + 1));
+  PRISM_CUDA(h, host_alloc(h, &h->h_cu_next, N + 1));
+  PRISM_CUDA(h, host_alloc(h, &h->h_off, N + 1));
+  PRISM_CUDA(h, host_alloc(h, &h->h_state, 1));
+  PRISM_CUDA(h, host_alloc(h, &h->h_err, 1));
+  PRISM_CUDA(h, cudaMemset(h->errword, 0, sizeof(int)));
+
+  if (streamed) {
+    const size_t e = h->esz, dh = c.head_dim;
+    size_t off = 0;
+    auto place = [&](size_t* o, size_t elems) { *o = off; off = align_up(off + elems * e, 256); };
+    place(&h->off_g_attn, D);
+    place(&h->off_qkv, nqkv * D);
+    place(&h->off_gq, dh);
+    place(&h->off_gk, dh);
+    place(&h->off_o, D * hd);
+    place(&h->off_g_ffn, D);
+    place(&h->off_gate, (size_t)c.ffn * D);
+    place(&h->off_up, (size_t)c.ffn * D);
+    place(&h->off_down, D * (size_t)c.ffn);
+    h->slot_bytes = off;
+    for (int s = 0; s < 2; ++s) PRISM_CUDA(h, dev_alloc(h, &h->slot[s], off));
+    PRISM_CUDA(h, cudaStreamCreateWithFlags(&h->copy_stream, cudaStreamNonBlocking));
+    for (int s = 0; s < 2; ++s) {
+      PRISM_CUDA(h, cudaEventCreateWithFlags(&h->ev_copied[s], cudaEventDisableTiming));
+      PRISM_CUDA(h, cudaEventCreateWithFlags(&h->ev_freed[s], cudaEventDisableTiming));
+    }
+  }
+
+  if (h->tc) {
+    PRISM_CUDA(h, make_tma_2d_bf16(&h->map_a_norm, h->a_norm, chunk, D, 128, 64));
+    PRISM_CUDA(h, make_tma_2d_bf16(&h->map_attn, h->attn, chunk, hd, 128, 64));
+    PRISM_CUDA(h, make_tma_2d_bf16(&h->map_hbuf, h->hbuf, chunk, c.ffn, 128, 64));
+    if (streamed) {
+      h->maps.resize(2);
+      for (int s = 0; s < 2; ++s) PRISM_CUDA(h, build_maps(h, layer_in_slot(h, s), &h->maps[s]));
+    } else {
+      h->maps.resize(c.n_layers);
+      for (int l = 0; l < c.n_layers; ++l) PRISM_CUDA(h, build_maps(h, layer_resident(h, l), &h->maps[l]));
+    }
+  }
+
+  PRISM_LAUNCH(h, launch_rope_table(h->rope_cos, h->rope_sin, c.max_seq_len, c.head_dim, c.rope_theta, 0));
+  PRISM_LAUNCH(h, launch_score_diff(h->score_head, c.dtype, c.hidden, h->w_diff, 0));
+  PRISM_CUDA(h, cudaDeviceSynchronize());
+  return PRISM_OK;
+}
+
+int prism_create(const prism_model_cfg* cfg, const prism_weights* w, prism_handle** out) {
+  if (out) *out = nullptr;
+  if (!cfg || !w || !out) return PRISM_ERR_INVALID_ARG;
+  std::string why;
+  int rc = validate_cfg(*cfg, &why);
+  if (rc != PRISM_OK) return rc;
+  prism_handle* h = new (std::nothrow) prism_handle();
+  if (!h) return PRISM_ERR_NOMEM;
+  rc = create_impl(h, cfg, w);
+  if (rc != PRISM_OK) {
+    prism_destroy(h);
+    return rc;
+  }
+  *out = h;
+  return PRISM_OK;
+}
+
+}  // extern "C"
+
+namespace {
+
+int validate_schedule(const prism_handle* h, const prism_prune_schedule* s, int k_eff, std::string* why) {
+  auto bad = [&](const char* m) { *why = m; return PRISM_ERR_INVALID_ARG; };
+  if (!s) return PRISM_OK;
+  if (s->mode != PRISM_PRUNE_NONE && s->mode != PRISM_PRUNE_FIXED_KEEP && s->mode != PRISM_PRUNE_CLUSTER)
+    return bad("unknown prune mode");
+  if (s->mode == PRISM_PRUNE_NONE) return PRISM_OK;
+  if (s->n_probes < 0 || (s->n_probes > 0 && !s->probe_layers)) return bad("probe_layers missing");
+  int prev = 0;
+  for (int j = 0; j < s->n_probes; ++j) {
+    const int l = s->probe_layers[j];
+    if (l <= prev || l >= h->cfg.n_layers) return bad("probe_layers must be strictly increasing in [1, n_layers)");
+    prev = l;
+  }
+  if (s->mode == PRISM_PRUNE_FIXED_KEEP) {
+    if (s->n_probes > 0 && !s->keep_counts) return bad("keep_counts missing");
+    for (int j = 0; j < s->n_probes; ++j)
+      if (s->keep_counts[j] < k_eff || s->keep_counts[j] < 1) return bad("keep_counts must be >= K");
+  } else {
+    const int k = s->n_clusters == 0 ? 3 : s->n_clusters;
+    if (k < 2 || k > PRISM_MAX_CLUSTERS) return bad("n_clusters must be in [2, PRISM_MAX_CLUSTERS]");
+    if (s->std_ddof != 0 && s->std_ddof != 1) return bad("std_ddof must be 0 or 1");
+    if (s->cv_threshold != s->cv_threshold) return bad("cv_threshold is NaN");
+  }
+  return PRISM_OK;
+}
+
+// One decoder block over rows [r0, r0+rows) (sequences [s0, s1)) of the live batch.
+int run_layer_chunk(prism_handle* h, const LayerDev& W, const LayerMaps* maps, float* x, const int* cu_dev, int s0, int s1,
+                    int r0, int rows, int max_len, cudaStream_t st) {
+  const prism_model_cfg& c = h->cfg;
+  const int D = c.hidden, dh = c.head_dim;
+  const int nqkv = (c.n_q_heads + 2 * c.n_kv_heads) * dh, hd = c.n_q_heads * dh;
+  float* xr = x + (size_t)r0 * D;
+  PRISM_LAUNCH(h, launch_rmsnorm(xr, W.g_attn, c.dtype, rows, D, c.rms_eps, h->a_norm, st));
+  if (h->tc)
+    PRISM_LAUNCH(h, launch_gemm_tc(h->map_a_norm, maps->qkv, maps->qkv, h->qkv, nullptr, rows, nqkv, D, kEpiStore, h->errword, st));
+  else
+    PRISM_LAUNCH(h, launch_gemm_simt(h->a_norm, W.w_qkv, nullptr, h->qkv, nullptr, rows, nqkv, D, c.dtype, kEpiStore, st));
+  PRISM_LAUNCH(h, launch_qknorm_rope(h->qkv, c.dtype, h->pos + r0, rows, c.n_q_heads, c.n_kv_heads, dh, c.qk_norm, W.g_q,
+                                     W.g_k, c.rms_eps, h->rope_cos, h->rope_sin, st));
+  if (h->fa)
+    PRISM_LAUNCH(h, launch_attention_mma(h->qkv, h->attn, cu_dev, s0, s1 - s0, r0, max_len, c.n_q_heads, c.n_kv_heads,
+                                         c.causal, st));
+  else
+    PRISM_LAUNCH(h, launch_attention_simt(h->qkv, h->attn, cu_dev, s0, s1 - s0, r0, max_len, c.n_q_heads, c.n_kv_heads, dh,
+                                          c.causal, c.dtype, st));
+  if (h->tc)
+    PRISM_LAUNCH(h, launch_gemm_tc(h->map_attn, maps->o, maps->o, nullptr, xr, rows, D, hd, kEpiResidual, h->errword, st));
+  else
+    PRISM_LAUNCH(h, launch_gemm_simt(h->attn, W.w_o, nullptr, nullptr, xr, rows, D, hd, c.dtype, kEpiResidual, st));
+  PRISM_LAUNCH(h, launch_rmsnorm(xr, W.g_ffn, c.dtype, rows, D, c.rms_eps, h->a_norm, st));
+  if (h->tc)
+    PRISM_LAUNCH(h, launch_gemm_tc(h->map_a_norm, maps->gate, maps->up, h->hbuf, nullptr, rows, c.ffn, D, kEpiSwiGLU, h->errword, st));
+  else
+    PRISM_LAUNCH(h, launch_gemm_simt(h->a_norm, W.w_gate, W.w_up, h->hbuf, nullptr, rows, c.ffn, D, c.dtype, kEpiSwiGLU, st));
+  if (h->tc)
+    PRISM_LAUNCH(h, launch_gemm_tc(h->map_hbuf, maps->down, maps->down, nullptr, xr, rows, D, c.ffn, kEpiResidual, h->errword, st));
+  else
+    PRISM_LAUNCH(h, launch_gemm_simt(h->hbuf, W.w_down, nullptr, nullptr, xr, rows, D, c.ffn, c.dtype, kEpiResidual, st));
+  return PRISM_OK;
+}
+
+int select_impl(prism_handle* h, const int32_t* query, int32_t lq, const int32_t* cand, const int32_t* off, int32_t N,
+                int32_t K, const prism_prune_schedule* sched, int32_t* topk_idx, float* topk_scores, int32_t* n_out,
+                prism_trace* trace, cudaStream_t st) {
+  const prism_model_cfg& c = h->cfg;
+  h->err.clear();
+  if (trace) {
+    trace->n_records = 0;
+    trace->layers_run = 0;
+    trace->n_chunks_max = 0;
+    trace->workspace_bytes = h->workspace_bytes;
+  }
+  const int k_eff = std::min(K, N);
+  std::string why;
+  int rc = validate_schedule(h, sched, k_eff, &why);
+  if (rc != PRISM_OK) return fail(h, rc, why);
+  if (N > c.max_candidates) return fail(h, PRISM_ERR_SHAPE_LIMIT, "N exceeds max_candidates");
+  if (N == 0) {
+    *n_out = 0;
+    return PRISM_OK;
+  }
+  const bool streamed = c.weight_residency == PRISM_WEIGHTS_HOST_STREAMED;
+  const int mode = sched ? sched->mode : PRISM_PRUNE_NONE;
+  const int n_probes = mode == PRISM_PRUNE_NONE ? 0 : sched->n_probes;
+
+  // Offsets to the host: launch geometry, limits and chunk planning need them.
+  PRISM_CUDA(h, cudaMemcpyAsync(h->h_off, off, (size_t)(N + 1) * sizeof(int), cudaMemcpyDeviceToHost, st));
+  PRISM_CUDA(h, cudaStreamSynchronize(st));
+  if (h->h_off[0] != 0) return fail(h, PRISM_ERR_BAD_INPUT, "cand_offsets[0] != 0");
+  long long total = 0;
+  h->h_cu[0] = 0;
+  for (int i = 0; i < N; ++i) {
+    const long long dl = (long long)h->h_off[i + 1] - h->h_off[i];
+    if (dl < 0) return fail(h, PRISM_ERR_BAD_INPUT, "cand_offsets not monotone");
+    if (dl + lq > c.max_seq_len) return fail(h, PRISM_ERR_SHAPE_LIMIT, "a sequence exceeds max_seq_len");
+    if (dl + lq > h->chunk_tokens) return fail(h, PRISM_ERR_BUDGET, "a sequence exceeds the chunk the activation budget allows");
+    if (dl + lq < 1) return fail(h, PRISM_ERR_INVALID_ARG, "empty sequence (query_len = 0 and an empty document)");
+    total += dl + lq;
+    if (total > c.max_total_tokens) return fail(h, PRISM_ERR_SHAPE_LIMIT, "token total exceeds max_total_tokens");
+    h->h_cu[i + 1] = (int)total;
+  }
+
+  RouteState init{};
+  init.n_active = N;
+  init.n_tokens = (int)total;
+  init.k_rem = k_eff;
+  *h->h_state = init;
+  PRISM_CUDA(h, cudaMemcpyAsync(h->state, h->h_state, sizeof(RouteState), cudaMemcpyHostToDevice, st));
+  PRISM_CUDA(h, cudaMemsetAsync(h->errword, 0, sizeof(int), st));
+
+  int cur = 0;  // ping-pong index of x / cu / seq2orig
+  PRISM_LAUNCH(h, launch_pack_offsets(off, N, lq, h->cu[cur], h->seq2orig[cur], h->errword, st));
+  PRISM_LAUNCH(h, launch_pack_tokens(query, lq, cand, off, h->cu[cur], N, (int)total, c.vocab, h->tokens, h->pos, h->errword, st));
+  PRISM_LAUNCH(h, launch_embed(h->embed, c.dtype, h->tokens, (int)total, c.hidden, h->x[cur], st));
+
+  if (streamed) {
+    // The previous request drained both streams before returning, so both slots are free.
+    for (int l = 0; l < std::min(2, c.n_layers); ++l)
+      if ((rc = enqueue_layer_copy(h, l, l)) != PRISM_OK) return rc;
+  }
+
+  int n = N, T = (int)total, n_rec = 0, probe_j = 0, layers_run = 0, chunks_max = 0;
+  bool done = false;
+  for (int l = 0; l < c.n_layers && !done; ++l) {
+    const int s = l & 1;
+    LayerDev W = streamed ? layer_in_slot(h, s) : layer_resident(h, l);
+    const LayerMaps* maps = h->tc ? &h->maps[streamed ? s : l] : nullptr;
+    if (streamed) PRISM_CUDA(h, cudaStreamWaitEvent(st, h->ev_copied[s], 0));
+    // chunks on sequence boundaries: the longest prefix of the remaining sequences that fits
+    int s0 = 0, chunks = 0;
+    while (s0 < n) {
+      int s1 = s0 + 1, max_len = h->h_cu[s1] - h->h_cu[s0];
+      while (s1 < n && h->h_cu[s1 + 1] - h->h_cu[s0] <= h->chunk_tokens) {
+        max_len = std::max(max_len, h->h_cu[s1 + 1] - h->h_cu[s1]);
+        ++s1;
+      }
+      const int r0 = h->h_cu[s0], rows = h->h_cu[s1] - r0;
+      if ((rc = run_layer_chunk(h, W, maps, h->x[cur], h->cu[cur], s0, s1, r0, rows, max_len, st)) != PRISM_OK) return rc;
+      s0 = s1;
+      ++chunks;
+    }
+    chunks_max = std::max(chunks_max, chunks);
+    if (trace && trace->tokens_per_layer) trace->tokens_per_layer[l] = T;
+    layers_run = l + 1;
+    if (streamed) {
+      PRISM_CUDA(h, cudaEventRecord(h->ev_freed[s], st));
+    }
+
+    const bool is_final = (layers_run == c.n_layers);
+    const bool is_probe = probe_j < n_probes && sched->probe_layers[probe_j] == layers_run;
+    if (is_final || is_probe) {
+      RouteParams p{};
+      p.mode = mode;
+      p.keep_count = (mode == PRISM_PRUNE_FIXED_KEEP && is_probe) ? sched->keep_counts[probe_j] : 0;
+      p.cv_threshold = sched ? sched->cv_threshold : 0.0;
+      p.n_clusters = (sched && sched->n_clusters) ? sched->n_clusters : 3;
+      p.ddof = sched ? sched->std_ddof : 0;
+      p.select_winners = sched ? sched->select_winners : 1;
+      p.is_final = is_final ? 1 : 0;
+      p.layer = layers_run;
+      const int nxt = cur ^ 1;
+      PRISM_LAUNCH(h, launch_probe(h->x[cur], h->cu[cur], n, c.hidden, h->g_final, c.dtype, h->w_diff, c.rms_eps, h->scores, st));
+      PRISM_LAUNCH(h, launch_route(h->scores, h->cu[cur], h->seq2orig[cur], n, p, h->cu[nxt], h->seq2orig[nxt], h->old_of_new,
+                                   h->state, h->res_idx, h->res_score, h->recs + n_rec,
+                                   h->trace_scores + (size_t)n_rec * c.max_candidates,
+                                   h->trace_ids + (size_t)n_rec * c.max_candidates, h->route_scratch, st));
+      ++n_rec;
+      if (is_probe) ++probe_j;
+      PRISM_CUDA(h, cudaMemcpyAsync(h->h_state, h->state, sizeof(RouteState), cudaMemcpyDeviceToHost, st));
+      PRISM_CUDA(h, cudaMemcpyAsync(h->h_err, h->errword, sizeof(int), cudaMemcpyDeviceToHost, st));
+      if (!is_final)
+        PRISM_CUDA(h, cudaMemcpyAsync(h->h_cu_next, h->cu[nxt], (size_t)(n + 1) * sizeof(int), cudaMemcpyDeviceToHost, st));
+      PRISM_CUDA(h, cudaStreamSynchronize(st));  // the one host round trip per scored layer
+      if (*h->h_err & kErrTimeout) return fail(h, PRISM_ERR_TIMEOUT, "a bounded device-side wait expired");
+      if (*h->h_err & (kErrBadToken | kErrBadOffsets)) return fail(h, PRISM_ERR_BAD_INPUT, "token id outside [0, vocab) or bad offsets");
+      const RouteState stt = *h->h_state;
+      done = stt.done != 0;
+      if (!done && stt.n_active < n) {
+        // survivors move to the other buffer, order kept; offsets and positions follow
+        std::swap(h->h_cu, h->h_cu_next);
+        PRISM_LAUNCH(h, launch_compact_rows(h->x[cur], h->x[nxt], h->cu[cur], h->cu[nxt], h->old_of_new, stt.n_active,
+                                            stt.n_tokens, c.hidden, st));
+        PRISM_LAUNCH(h, launch_positions(h->cu[nxt], stt.n_active, stt.n_tokens, h->pos, st));
+        cur = nxt;
+        n = stt.n_active;
+        T = stt.n_tokens;
+      }
+    }
+    if (streamed && !done && l + 2 < c.n_layers) {
+      PRISM_CUDA(h, cudaStreamWaitEvent(h->copy_stream, h->ev_freed[s], 0));
+      if ((rc = enqueue_layer_copy(h, l + 2, s)) != PRISM_OK) return rc;
+    }
+  }
+
+  PRISM_CUDA(h, cudaMemcpyAsync(topk_idx, h->res_idx, (size_t)k_eff * sizeof(int), cudaMemcpyDeviceToDevice, st));
+  PRISM_CUDA(h, cudaMemcpyAsync(topk_scores, h->res_score, (size_t)k_eff * sizeof(float), cudaMemcpyDeviceToDevice, st));
+  if (trace) {
+    const int take = std::min(n_rec, trace->capacity);
+    if (take > 0 && trace->records)
+      PRISM_CUDA(h, cudaMemcpyAsync(trace->records, h->recs, (size_t)take * sizeof(prism_probe_record), cudaMemcpyDeviceToHost, st));
+    for (int r = 0; r < take; ++r) {
+      if (trace->scores)
+        PRISM_CUDA(h, cudaMemcpyAsync(trace->scores + (size_t)r * N, h->trace_scores + (size_t)r * c.max_candidates,
+                                      (size_t)N * sizeof(float), cudaMemcpyDeviceToHost, st));
+      if (trace->ids)
+        PRISM_CUDA(h, cudaMemcpyAsync(trace->ids + (size_t)r * N, h->trace_ids + (size_t)r * c.max_candidates,
+                                      (size_t)N * sizeof(int), cudaMemcpyDeviceToHost, st));
+    }
+    trace->n_records = take;
+    trace->layers_run = layers_run;
+    trace->n_chunks_max = chunks_max;
+  }
+  PRISM_CUDA(h, cudaStreamSynchronize(st));
+  if (streamed) PRISM_CUDA(h, cudaStreamSynchronize(h->copy_stream));
+  if (h->h_state->n_result != k_eff) return fail(h, PRISM_ERR_CUDA, "internal: result count mismatch");
+  *n_out = k_eff;
+  return PRISM_OK;
+}
+
+int check_args(prism_handle* h, const void* q, int lq, const void* cand, const void* off, int N, int K, const void* oi,
+               const void* os, const void* n_out) {
+  if (!h) return PRISM_ERR_INVALID_ARG;
+  if (!n_out) return fail(h, PRISM_ERR_INVALID_ARG, "n_out is null");
+  if (N < 0 || K < 1 || lq < 0) return fail(h, PRISM_ERR_INVALID_ARG, "N < 0, K < 1 or query_len < 0");
+  if (!off || !oi || !os || (lq > 0 && !q)) return fail(h, PRISM_ERR_INVALID_ARG, "null pointer argument");
+  if (lq > h->cfg.max_seq_len) return fail(h, PRISM_ERR_SHAPE_LIMIT, "query_len exceeds max_seq_len");
+  (void)cand;
+  return PRISM_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int prism_select(prism_handle* h, const int32_t* query_tokens, int32_t query_len, const int32_t* cand_tokens,
+                 const int32_t* cand_offsets, int32_t N, int32_t K, const prism_prune_schedule* sched, int32_t* topk_idx,
+                 float* topk_scores, int32_t* n_out, prism_trace* trace, void* cuda_stream) {
+  int rc = check_args(h, query_tokens, query_len, cand_tokens, cand_offsets, N, K, topk_idx, topk_scores, n_out);
+  if (rc != PRISM_OK) return rc;
+  *n_out = 0;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  rc = select_impl(h, query_tokens, query_len, cand_tokens, cand_offsets, N, K, sched, topk_idx, topk_scores, n_out, trace, st);
+  if (rc != PRISM_OK) {
+    *n_out = 0;
+    cudaStreamSynchronize(st);
+    if (h->copy_stream) cudaStreamSynchronize(h->copy_stream);
+  }
+  return rc;
+}
+
+int prism_select_host(prism_handle* h, const int32_t* query_tokens, int32_t query_len, const int32_t* cand_tokens,
+                      const int32_t* cand_offsets, int32_t N, int32_t K, const prism_prune_schedule* sched,
+                      int32_t* topk_idx, float* topk_scores, int32_t* n_out, prism_trace* trace, void* cuda_stream) {
+  int rc = check_args(h, query_tokens, query_len, cand_tokens, cand_offsets, N, K, topk_idx, topk_scores, n_out);
+  if (rc != PRISM_OK) return rc;
+  *n_out = 0;
+  if (N > h->cfg.max_candidates) return fail(h, PRISM_ERR_SHAPE_LIMIT, "N exceeds max_candidates");
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  const long long n_cand = N > 0 ? cand_offsets[N] : 0;  // host buffer: readable here
+  if (n_cand < 0) return fail(h, PRISM_ERR_BAD_INPUT, "cand_offsets[N] negative");
+  if (n_cand > h->cfg.max_total_tokens) return fail(h, PRISM_ERR_SHAPE_LIMIT, "token total exceeds max_total_tokens");
+  if (n_cand > 0 && !cand_tokens) return fail(h, PRISM_ERR_INVALID_ARG, "cand_tokens is null");
+  if (query_len > 0)
+    PRISM_CUDA(h, cudaMemcpyAsync(h->in_query, query_tokens, (size_t)query_len * sizeof(int), cudaMemcpyHostToDevice, st));
+  if (n_cand > 0)
+    PRISM_CUDA(h, cudaMemcpyAsync(h->in_cand, cand_tokens, (size_t)n_cand * sizeof(int), cudaMemcpyHostToDevice, st));
+  PRISM_CUDA(h, cudaMemcpyAsync(h->in_off, cand_offsets, (size_t)(N + 1) * sizeof(int), cudaMemcpyHostToDevice, st));
+  rc = select_impl(h, h->in_query, query_len, h->in_cand, h->in_off, N, K, sched, h->out_idx, h->out_score, n_out, trace, st);
+  if (rc == PRISM_OK && *n_out > 0) {
+    cudaError_t e = cudaMemcpyAsync(topk_idx, h->out_idx, (size_t)*n_out * sizeof(int), cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(topk_scores, h->out_score, (size_t)*n_out * sizeof(float), cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) rc = cuda_fail(h, e, "copy of the result to the host");
+  }
+  if (rc != PRISM_OK) {
+    *n_out = 0;
+    cudaStreamSynchronize(st);
+    if (h->copy_stream) cudaStreamSynchronize(h->copy_stream);
+  }
+  return rc;
+}
+
+}  // extern "C"

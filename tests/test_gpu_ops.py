@@ -1,0 +1,333 @@
+"""-m gpu: every kernel of the hot path against the CPU oracle, through the C ABI (prism_op_*)."""
+import numpy as np
+import pytest
+
+import oracle
+from oracle.prune_rule import MODE_CLUSTER, MODE_FIXED_KEEP, replay_select
+from synth.configs import Schedule
+from synth.weights import round_to_bf16
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+FP32, BF16 = 0, 1
+AUTO, SIMT = 0, 1
+
+
+@pytest.fixture(scope="module")
+def P():
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    import paper_2510_15620_b200 as pkg
+    return pkg
+
+
+def dev(a, dtype=None):
+    t = torch.from_numpy(np.ascontiguousarray(a))
+    if dtype is not None:
+        t = t.to(dtype)
+    return t.cuda()
+
+
+def bf(a):
+    return dev(np.asarray(a, np.float32), torch.bfloat16)
+
+
+# ------------------------------------------------------------------------------------------ pack
+@pytest.mark.parametrize("n,lq,lo,hi", [(1, 4, 0, 1), (16, 16, 16, 48), (257, 3, 0, 9), (1500, 32, 1, 40)])
+def test_pack_bit_exact(P, n, lq, lo, hi):
+    rng = np.random.default_rng(n)
+    vocab = 1000
+    lens = rng.integers(lo, hi + 1, size=n)
+    off = np.zeros(n + 1, np.int32)
+    off[1:] = np.cumsum(lens)
+    cand = rng.integers(0, vocab, size=int(off[-1])).astype(np.int32)
+    query = rng.integers(0, vocab, size=lq).astype(np.int32)
+    total = int(off[-1]) + n * lq
+    tokens = torch.empty(total, dtype=torch.int32, device="cuda")
+    pos = torch.empty_like(tokens)
+    cu = torch.empty(n + 1, dtype=torch.int32, device="cuda")
+    s2o = torch.empty(n, dtype=torch.int32, device="cuda")
+    err = torch.zeros(1, dtype=torch.int32, device="cuda")
+    P.ops.prism_op_pack(dev(query), dev(cand) if cand.size else torch.zeros(1, dtype=torch.int32, device="cuda"),
+                        dev(off), total, vocab, tokens, pos, cu, s2o, err)
+    exp_cu = np.zeros(n + 1, np.int64)
+    exp_cu[1:] = np.cumsum(lens + lq)
+    exp_tok = np.concatenate([np.concatenate([query, cand[off[i]:off[i + 1]]]) for i in range(n)])
+    exp_pos = np.concatenate([np.arange(lq + lens[i]) for i in range(n)])
+    assert np.array_equal(cu.cpu().numpy(), exp_cu)
+    assert np.array_equal(tokens.cpu().numpy(), exp_tok)
+    assert np.array_equal(pos.cpu().numpy(), exp_pos)
+    assert np.array_equal(s2o.cpu().numpy(), np.arange(n))
+    assert int(err.item()) == 0
+
+
+def test_pack_flags_bad_tokens_without_trapping(P):
+    off = np.array([0, 3, 5], np.int32)
+    cand = np.array([1, 2, 99, 4, -1], np.int32)
+    query = np.array([0, 1], np.int32)
+    total = 9
+    tokens = torch.empty(total, dtype=torch.int32, device="cuda")
+    pos = torch.empty_like(tokens)
+    cu = torch.empty(3, dtype=torch.int32, device="cuda")
+    s2o = torch.empty(2, dtype=torch.int32, device="cuda")
+    err = torch.zeros(1, dtype=torch.int32, device="cuda")
+    P.ops.prism_op_pack(dev(query), dev(cand), dev(off), total, 50, tokens, pos, cu, s2o, err)
+    assert int(err.item()) & 1
+    assert tokens.cpu().numpy().max() < 50 and tokens.cpu().numpy().min() >= 0
+
+
+# ------------------------------------------------------------------------------------------ embed / norm / rope / probe
+@pytest.mark.parametrize("dtype", [FP32, BF16])
+def test_embed_rmsnorm_probe(P, dtype):
+    rng = np.random.default_rng(5)
+    v, d, t = 300, 1024 if dtype == BF16 else 256, 777
+    table = (rng.normal(size=(v, d)) * 0.02).astype(np.float32)
+    gain = (1 + 0.1 * rng.normal(size=d)).astype(np.float32)
+    head = (rng.normal(size=(2, d)) * 0.02).astype(np.float32)
+    if dtype == BF16:
+        table, gain, head = round_to_bf16(table), round_to_bf16(gain), round_to_bf16(head)
+    tdt = torch.bfloat16 if dtype == BF16 else torch.float32
+    toks = rng.integers(0, v, size=t).astype(np.int32)
+    x = torch.empty(t, d, dtype=torch.float32, device="cuda")
+    P.ops.prism_op_embed(dev(table, tdt), dtype, dev(toks), x)
+    assert np.array_equal(x.cpu().numpy(), table[toks])                     # a copy: exact
+    xs = (rng.normal(size=(t, d)) * 3).astype(np.float32)
+    out = torch.empty(t, d, dtype=tdt, device="cuda")
+    P.ops.prism_op_rmsnorm(dev(xs), dev(gain, tdt), dtype, 1e-6, out)
+    ref = oracle.rmsnorm(xs.astype(np.float64), gain.astype(np.float64), 1e-6)
+    got = out.float().cpu().numpy()
+    tol = 2.0 ** -8 if dtype == BF16 else 2e-6
+    assert np.max(np.abs(got - ref) / (np.abs(ref) + 1e-3)) < tol
+    lens = rng.integers(1, 40, size=30)
+    cu = np.zeros(31, np.int32)
+    cu[1:] = np.cumsum(lens)
+    xs = xs[: cu[-1]]
+    sc = torch.empty(30, dtype=torch.float32, device="cuda")
+    P.ops.prism_op_probe(dev(xs), dev(cu), 30, dev(gain, tdt), dev(head, tdt), dtype, 1e-6, sc)
+    ref = np.array([oracle.reranker.probe_score(xs[cu[i + 1] - 1], gain, head, 1e-6) for i in range(30)])
+    assert np.max(np.abs(sc.cpu().numpy() - ref)) < 2e-5
+
+
+@pytest.mark.parametrize("dtype,dh,qk_norm", [(FP32, 64, 0), (FP32, 64, 1), (BF16, 128, 1), (FP32, 20, 1)])
+def test_qknorm_rope(P, dtype, dh, qk_norm):
+    rng = np.random.default_rng(dh + qk_norm)
+    hq, hkv, rows, theta = 4, 2, 333, 1e4
+    qkv = rng.normal(size=(rows, (hq + 2 * hkv) * dh)).astype(np.float32)
+    gq = (1 + 0.1 * rng.normal(size=dh)).astype(np.float32)
+    gk = (1 + 0.1 * rng.normal(size=dh)).astype(np.float32)
+    if dtype == BF16:
+        qkv, gq, gk = round_to_bf16(qkv), round_to_bf16(gq), round_to_bf16(gk)
+    pos = rng.integers(0, 600, size=rows).astype(np.int32)
+    tdt = torch.bfloat16 if dtype == BF16 else torch.float32
+    t = dev(qkv, tdt)
+    P.ops.prism_op_qknorm_rope(t, dtype, dev(pos), hq, hkv, dh, qk_norm, dev(gq, tdt), dev(gk, tdt), 1e-6, theta, 600)
+    got = t.float().cpu().numpy()
+    q = qkv[:, : hq * dh].reshape(rows, hq, dh).astype(np.float64)
+    k = qkv[:, hq * dh:(hq + hkv) * dh].reshape(rows, hkv, dh).astype(np.float64)
+    if qk_norm:
+        q, k = oracle.rmsnorm(q, gq.astype(np.float64), 1e-6), oracle.rmsnorm(k, gk.astype(np.float64), 1e-6)
+    q, k = oracle.rope_rotate(q, pos, theta), oracle.rope_rotate(k, pos, theta)
+    ref = np.concatenate([q.reshape(rows, -1), k.reshape(rows, -1), qkv[:, (hq + hkv) * dh:]], axis=1)
+    tol = 2.0 ** -7 if dtype == BF16 else 3e-6
+    assert np.max(np.abs(got - ref)) < tol * max(1.0, np.max(np.abs(ref)))
+    assert np.array_equal(got[:, (hq + hkv) * dh:], qkv[:, (hq + hkv) * dh:])       # v untouched
+
+
+# ------------------------------------------------------------------------------------------ GEMM
+def _gemm_ref(a, b, b2, resid, epi):
+    c = a.astype(np.float64) @ b.astype(np.float64).T
+    if epi == 0:
+        return c
+    if epi == 1:
+        return resid.astype(np.float64) + c
+    u = a.astype(np.float64) @ b2.astype(np.float64).T
+    return c / (1 + np.exp(-c)) * u
+
+
+@pytest.mark.parametrize("m,n,k", [(5, 64, 32), (130, 192, 100), (300, 512, 768)])
+@pytest.mark.parametrize("epi", [0, 1, 2])
+def test_gemm_fp32_simt(P, m, n, k, epi):
+    rng = np.random.default_rng(m + n + k + epi)
+    a = rng.normal(size=(m, k)).astype(np.float32)
+    b = (rng.normal(size=(n, k)) * 0.05).astype(np.float32)
+    b2 = (rng.normal(size=(n, k)) * 0.05).astype(np.float32)
+    resid = rng.normal(size=(m, n)).astype(np.float32)
+    out = torch.zeros(m, n, device="cuda")
+    rs = dev(resid)
+    P.ops.prism_op_gemm(dev(a), dev(b), dev(b2), out, rs, m, n, k, FP32, epi, SIMT, None)
+    got = (rs if epi == 1 else out).cpu().numpy()
+    assert np.max(np.abs(got - _gemm_ref(a, b, b2, resid, epi))) < 2e-5
+
+
+@pytest.mark.parametrize("impl", [AUTO, SIMT])
+@pytest.mark.parametrize("epi", [0, 1, 2])
+@pytest.mark.parametrize("m,n,k", [(1, 256, 64), (300, 512, 320), (1000, 1024, 1024), (777, 384, 200), (4100, 2560, 512)])
+def test_gemm_bf16(P, m, n, k, epi, impl):
+    """tcgen05 kernel (AUTO) and the CUDA-core kernel on the same bf16 inputs vs an fp64 matmul.
+    Shapes span several 128x256 tiles, ragged M/N/K tails and more tiles than SMs."""
+    rng = np.random.default_rng(m * 7 + n + k + epi)
+    a = round_to_bf16(rng.normal(size=(m, k)).astype(np.float32))
+    b = round_to_bf16((rng.normal(size=(n, k)) * 0.05).astype(np.float32))
+    b2 = round_to_bf16((rng.normal(size=(n, k)) * 0.05).astype(np.float32))
+    resid = rng.normal(size=(m, n)).astype(np.float32)
+    out = torch.zeros(m, n, dtype=torch.bfloat16, device="cuda")
+    rs = dev(resid)
+    err = torch.zeros(1, dtype=torch.int32, device="cuda")
+    P.ops.prism_op_gemm(bf(a), bf(b), bf(b2), out, rs, m, n, k, BF16, epi, impl, err)
+    torch.cuda.synchronize()
+    assert int(err.item()) == 0
+    ref = _gemm_ref(a, b, b2, resid, epi)
+    got = (rs if epi == 1 else out.float()).cpu().numpy()
+    scale = np.max(np.abs(ref))
+    tol = (2.0 ** -8) * scale + 1e-3 if epi != 1 else 1e-4 * scale + 1e-4    # bf16 store vs fp32 residual add
+    assert np.max(np.abs(got - ref)) < tol, np.max(np.abs(got - ref))
+
+
+def test_gemm_tc_rows_do_not_depend_on_their_position(P):
+    """Duplicate rows anywhere in the batch, and the same row in a smaller batch, give identical bits
+    (exact score ties between duplicated candidates rely on this)."""
+    rng = np.random.default_rng(0)
+    m, n, k = 700, 512, 1024
+    a = round_to_bf16(rng.normal(size=(m, k)).astype(np.float32))
+    a[650] = a[3]
+    a[129] = a[3]
+    b = round_to_bf16((rng.normal(size=(n, k)) * 0.05).astype(np.float32))
+    err = torch.zeros(1, dtype=torch.int32, device="cuda")
+    out = torch.zeros(m, n, dtype=torch.bfloat16, device="cuda")
+    P.ops.prism_op_gemm(bf(a), bf(b), None, out, None, m, n, k, BF16, 0, AUTO, err)
+    o = out.view(torch.int16).cpu().numpy()
+    assert np.array_equal(o[3], o[650]) and np.array_equal(o[3], o[129])
+    out2 = torch.zeros(5, n, dtype=torch.bfloat16, device="cuda")
+    P.ops.prism_op_gemm(bf(a[:5]), bf(b), None, out2, None, 5, n, k, BF16, 0, AUTO, err)
+    assert np.array_equal(out2.view(torch.int16).cpu().numpy()[3], o[3])
+    assert int(err.item()) == 0
+
+
+# ------------------------------------------------------------------------------------------ attention
+def _attn_ref(qkv, cu, hq, hkv, dh, causal):
+    out = np.zeros((qkv.shape[0], hq * dh))
+    for s in range(len(cu) - 1):
+        x = qkv[cu[s]:cu[s + 1]].astype(np.float64)
+        L = x.shape[0]
+        q = x[:, : hq * dh].reshape(L, hq, dh)
+        k = x[:, hq * dh:(hq + hkv) * dh].reshape(L, hkv, dh)
+        v = x[:, (hq + hkv) * dh:].reshape(L, hkv, dh)
+        out[cu[s]:cu[s + 1]] = oracle.attention(q, k, v, causal).reshape(L, hq * dh)
+    return out
+
+
+@pytest.mark.parametrize("causal", [1, 0])
+@pytest.mark.parametrize("dtype,impl,dh", [(FP32, SIMT, 64), (BF16, SIMT, 128), (BF16, AUTO, 128)])
+def test_attention(P, dtype, impl, dh, causal):
+    rng = np.random.default_rng(dh + causal)
+    hq, hkv = 4, 2
+    lens = np.array([1, 7, 64, 65, 130, 200, 63, 128])      # below, at and across the 64-row tiles
+    cu = np.zeros(len(lens) + 1, np.int32)
+    cu[1:] = np.cumsum(lens)
+    qkv = rng.normal(size=(cu[-1], (hq + 2 * hkv) * dh)).astype(np.float32)
+    if dtype == BF16:
+        qkv = round_to_bf16(qkv)
+    tdt = torch.bfloat16 if dtype == BF16 else torch.float32
+    out = torch.zeros(int(cu[-1]), hq * dh, dtype=tdt, device="cuda")
+    P.ops.prism_op_attention(dev(qkv, tdt), out, dev(cu), len(lens), int(lens.max()), hq, hkv, dh, causal, dtype, impl)
+    ref = _attn_ref(qkv, cu, hq, hkv, dh, bool(causal))
+    got = out.float().cpu().numpy()
+    tol = 2e-2 if dtype == BF16 else 2e-5
+    assert np.max(np.abs(got - ref)) < tol, np.max(np.abs(got - ref))
+
+
+# ------------------------------------------------------------------------------------------ route / compact
+def _run_route(P, scores, ids, lens, k_rem, n_result, sched_kw, is_final=0, layer=3):
+    n = len(scores)
+    cu = np.zeros(n + 1, np.int32)
+    cu[1:] = np.cumsum(lens)
+    state = np.array([n, cu[-1], k_rem, n_result, 0, 0, 0, 0], np.int32)
+    d = dict(mode=MODE_CLUSTER, keep_count=0, cv_threshold=0.0, n_clusters=3, std_ddof=0, select_winners=1)
+    d.update(sched_kw)
+    cu_new = torch.full((n + 1,), -1, dtype=torch.int32, device="cuda")
+    s2o_new = torch.full((max(n, 1),), -1, dtype=torch.int32, device="cuda")
+    oon = torch.full((max(n, 1),), -1, dtype=torch.int32, device="cuda")
+    st = dev(state)
+    ridx = torch.full((n + n_result + 1,), -1, dtype=torch.int32, device="cuda")
+    rsc = torch.zeros(n + n_result + 1, dtype=torch.float32, device="cuda")
+    rec = torch.zeros(P.ops.RECORD_BYTES, dtype=torch.uint8, device="cuda")
+    P.ops.prism_op_route(dev(np.asarray(scores, np.float32)), dev(cu), dev(np.asarray(ids, np.int32)), n, d["mode"],
+                         d["keep_count"], d["cv_threshold"], d["n_clusters"], d["std_ddof"], d["select_winners"],
+                         is_final, layer, cu_new, s2o_new, oon, st, ridx, rsc, rec)
+    torch.cuda.synchronize()
+    return (st.cpu().numpy(), cu_new.cpu().numpy(), s2o_new.cpu().numpy(), oon.cpu().numpy(), ridx.cpu().numpy(),
+            rsc.cpu().numpy(), P.ops.decode_record(rec), cu)
+
+
+@pytest.mark.parametrize("n_clusters", [2, 3, 5, 8])
+@pytest.mark.parametrize("winners", [1, 0])
+def test_route_matches_oracle_rule_bit_exact(P, n_clusters, winners):
+    rng = np.random.default_rng(n_clusters * 2 + winners)
+    for trial in range(25):
+        n = int(rng.choice([1, 2, 3, 17, 100, 333, 1000, 1500]))
+        k = int(rng.integers(1, 25))
+        base = rng.normal(size=n) * (3 if trial % 2 else 0.3) + (0 if trial % 3 else 2.0)
+        sc = base.astype(np.float32)
+        if trial % 4 == 0 and n > 4:
+            sc[rng.integers(0, n, size=n // 3)] = sc[0]                  # exact ties
+        ids = np.sort(rng.choice(5000, size=n, replace=False)).astype(np.int32)
+        lens = rng.integers(1, 50, size=n)
+        thr = float(rng.choice([0.0, 0.3, 5.0]))
+        st, cu_new, s2o_new, oon, ridx, rsc, rec, cu = _run_route(
+            P, sc, ids, lens, k, 2, dict(cv_threshold=thr, n_clusters=n_clusters, select_winners=winners))
+        # the oracle's rule on the same scores: a one-probe schedule over a two-layer "model"
+        sched = Schedule(MODE_CLUSTER, (1,), cv_threshold=thr, n_clusters=n_clusters, select_winners=winners)
+        table = {1: dict(zip(range(n), sc)), 2: dict(zip(range(n), sc))}
+        ref = replay_select(lambda l, a: np.asarray([table[l][i] for i in a], np.float32), n, k, 2, sched)
+        t = ref.trace[0]
+        assert (rec.fired, rec.n_selected, rec.n_dropped, rec.n_deferred, rec.k_rem_after) == \
+               (t.fired, t.n_selected, t.n_dropped, t.n_deferred, t.k_rem_after), (n, k, thr)
+        assert [rec.cuts[i] for i in range(rec.n_cuts)] == t.cuts
+        assert rec.cv == t.cv
+        survivors = ref.active_per_layer[1] if len(ref.active_per_layer) > 1 else []
+        n_new = int(st[0])
+        assert n_new == len(survivors)
+        assert list(oon[:n_new]) == survivors                          # positions in the old batch, order kept
+        assert list(s2o_new[:n_new]) == [int(ids[p]) for p in survivors]
+        exp_cu = np.concatenate([[0], np.cumsum(lens[survivors])]) if survivors else np.array([0])
+        assert list(cu_new[: n_new + 1]) == list(exp_cu)
+        assert int(st[1]) == int(exp_cu[-1]) and int(st[2]) == t.k_rem_after
+        done = ref.layers_run == 1
+        assert int(st[4]) == int(done)
+        left = len(ref.topk_idx) if done else t.n_selected
+        assert int(st[3]) == 2 + left
+        assert list(ridx[2:2 + left]) == [int(ids[p]) for p in ref.topk_idx[:left]]
+        assert list(rsc[2:2 + left]) == [np.float32(x) for x in ref.topk_scores[:left]]
+
+
+def test_route_fixed_keep_and_final(P):
+    rng = np.random.default_rng(9)
+    n = 40
+    sc = rng.normal(size=n).astype(np.float32)
+    sc[5] = sc[9]
+    ids = np.arange(n, dtype=np.int32)
+    lens = rng.integers(1, 9, size=n)
+    st, cu_new, s2o_new, oon, ridx, rsc, rec, cu = _run_route(P, sc, ids, lens, 4, 0, dict(mode=MODE_FIXED_KEEP, keep_count=10))
+    order = sorted(range(n), key=lambda i: (-sc[i], i))
+    assert list(oon[:10]) == sorted(order[:10]) and int(st[0]) == 10 and rec.n_dropped == 30 and int(st[4]) == 0
+    st, *_, ridx, rsc, rec, cu = _run_route(P, sc, ids, lens, 4, 0, dict(), is_final=1)
+    assert int(st[4]) == 1 and list(ridx[:4]) == order[:4] and list(rsc[:4]) == [sc[i] for i in order[:4]]
+    st, *_, ridx, rsc, rec, cu = _run_route(P, sc[:3], ids[:3], lens[:3], 5, 0, dict())          # n <= k_rem: all leave
+    assert int(st[4]) == 1 and int(st[3]) == 3 and int(st[2]) == 2
+
+
+def test_compact_rows_exact(P):
+    rng = np.random.default_rng(3)
+    n, d = 37, 1024
+    lens = rng.integers(1, 30, size=n)
+    cu = np.zeros(n + 1, np.int32)
+    cu[1:] = np.cumsum(lens)
+    x = rng.normal(size=(cu[-1], d)).astype(np.float32)
+    keep = np.sort(rng.choice(n, size=11, replace=False)).astype(np.int32)
+    cu_new = np.zeros(12, np.int32)
+    cu_new[1:] = np.cumsum(lens[keep])
+    out = torch.zeros(int(cu_new[-1]), d, device="cuda")
+    P.ops.prism_op_compact(dev(x), out, dev(cu), dev(cu_new), dev(keep), 11, int(cu_new[-1]))
+    exp = np.concatenate([x[cu[i]:cu[i + 1]] for i in keep])
+    assert np.array_equal(out.cpu().numpy(), exp)
