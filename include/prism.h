@@ -204,6 +204,25 @@ PRISM_API const char* prism_status_str(int status);
 /* Number of kernels this library launched since the handle was created (for launch accounting). */
 PRISM_API int64_t prism_launch_count(const prism_handle* h);
 
+/* Per-kernel timing of the steps prism_select chains.  While enabled, every kernel launch of a request
+ * is bracketed by CUDA events on the request's stream (this adds a few microseconds per launch, so
+ * latency figures are taken with profiling off).  `work` accumulates the ALGORITHMIC work the driver
+ * asked of the class: flops for the GEMM and attention classes (2*M*N*K; causal attention
+ * 2*L^2*Hq*dh per sequence), bytes that must move for all others. */
+enum {
+  PRISM_K_PACK = 0, PRISM_K_EMBED, PRISM_K_RMSNORM, PRISM_K_GEMM_QKV, PRISM_K_ROPE, PRISM_K_ATTENTION,
+  PRISM_K_GEMM_O, PRISM_K_GEMM_GATEUP, PRISM_K_GEMM_DOWN, PRISM_K_PROBE, PRISM_K_ROUTE, PRISM_K_COMPACT,
+  PRISM_N_KERNEL_CLASSES
+};
+typedef struct {
+  double ms;        /* summed device time between the bracketing events */
+  double work;      /* flops or bytes, see above */
+  int64_t launches;
+} prism_kernel_stat;
+PRISM_API int prism_profile(prism_handle* h, int enable);
+/* Copy the accumulated statistics to out[PRISM_N_KERNEL_CLASSES] (host); reset != 0 clears them. */
+PRISM_API int prism_profile_read(prism_handle* h, prism_kernel_stat* out, int reset);
+
 #ifdef __cplusplus
 }
 #endif

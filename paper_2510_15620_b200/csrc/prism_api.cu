@@ -72,6 +72,13 @@ struct prism_handle {
   cudaStream_t copy_stream = nullptr;
   cudaEvent_t ev_copied[2] = {nullptr, nullptr}, ev_freed[2] = {nullptr, nullptr};
 
+  // optional per-kernel timing (prism_profile): event pairs around every launch of a request
+  bool prof_on = false;
+  struct ProfEntry { int cat; double work; cudaEvent_t a, b; };
+  std::vector<ProfEntry> prof_pending;
+  std::vector<cudaEvent_t> prof_pool;
+  prism_kernel_stat prof_acc[PRISM_N_KERNEL_CLASSES] = {};
+
   // TMA descriptors
   TmaDesc map_a_norm{}, map_attn{}, map_hbuf{};
   std::vector<LayerMaps> maps;  // per layer (resident) or per slot (streamed)
@@ -101,6 +108,49 @@ int cuda_fail(prism_handle* h, cudaError_t e, const char* what) {
     (h)->launches++;                                           \
     if (e__ != cudaSuccess) return cuda_fail((h), e__, #call); \
   } while (0)
+
+cudaEvent_t prof_event(prism_handle* h) {
+  if (!h->prof_pool.empty()) {
+    cudaEvent_t e = h->prof_pool.back();
+    h->prof_pool.pop_back();
+    return e;
+  }
+  cudaEvent_t e = nullptr;
+  cudaEventCreate(&e);
+  return e;
+}
+
+// A launch that is attributed to kernel class `cat` with `work` algorithmic flops or bytes.
+#define PRISM_LAUNCH_P(h, st, cat, work, call)                                   \
+  do {                                                                           \
+    cudaEvent_t ea__ = nullptr, eb__ = nullptr;                                  \
+    if ((h)->prof_on) {                                                          \
+      ea__ = prof_event(h);                                                      \
+      eb__ = prof_event(h);                                                      \
+      cudaEventRecord(ea__, (st));                                               \
+    }                                                                            \
+    cudaError_t e__ = (call);                                                    \
+    (h)->launches++;                                                             \
+    if ((h)->prof_on) {                                                          \
+      cudaEventRecord(eb__, (st));                                               \
+      (h)->prof_pending.push_back(prism_handle::ProfEntry{(cat), (double)(work), ea__, eb__}); \
+    }                                                                            \
+    if (e__ != cudaSuccess) return cuda_fail((h), e__, #call);                   \
+  } while (0)
+
+void prof_collect(prism_handle* h) {
+  for (auto& p : h->prof_pending) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, p.a, p.b) == cudaSuccess) {
+      h->prof_acc[p.cat].ms += ms;
+      h->prof_acc[p.cat].work += p.work;
+      h->prof_acc[p.cat].launches += 1;
+    }
+    h->prof_pool.push_back(p.a);
+    h->prof_pool.push_back(p.b);
+  }
+  h->prof_pending.clear();
+}
 
 template <typename T>
 cudaError_t dev_alloc(prism_handle* h, T** p, size_t count) {
@@ -235,6 +285,21 @@ const char* prism_last_error(const prism_handle* h) { return h ? h->err.c_str() 
 
 int64_t prism_launch_count(const prism_handle* h) { return h ? h->launches : 0; }
 
+int prism_profile(prism_handle* h, int enable) {
+  if (!h) return PRISM_ERR_INVALID_ARG;
+  h->prof_on = enable != 0;
+  return PRISM_OK;
+}
+
+int prism_profile_read(prism_handle* h, prism_kernel_stat* out, int reset) {
+  if (!h || !out) return PRISM_ERR_INVALID_ARG;
+  for (int i = 0; i < PRISM_N_KERNEL_CLASSES; ++i) {
+    out[i] = h->prof_acc[i];
+    if (reset) h->prof_acc[i] = prism_kernel_stat{};
+  }
+  return PRISM_OK;
+}
+
 void prism_destroy(prism_handle* h) {
   if (!h) return;
   cudaDeviceSynchronize();
@@ -245,6 +310,8 @@ void prism_destroy(prism_handle* h) {
     if (h->ev_freed[s]) cudaEventDestroy(h->ev_freed[s]);
   }
   if (h->copy_stream) cudaStreamDestroy(h->copy_stream);
+  for (auto& p : h->prof_pending) { cudaEventDestroy(p.a); cudaEventDestroy(p.b); }
+  for (cudaEvent_t e : h->prof_pool) cudaEventDestroy(e);
   delete h;
 }
 
@@ -415,32 +482,49 @@ int run_layer_chunk(prism_handle* h, const LayerDev& W, const LayerMaps* maps, f
   const int D = c.hidden, dh = c.head_dim;
   const int nqkv = (c.n_q_heads + 2 * c.n_kv_heads) * dh, hd = c.n_q_heads * dh;
   float* xr = x + (size_t)r0 * D;
-  PRISM_LAUNCH(h, launch_rmsnorm(xr, W.g_attn, c.dtype, rows, D, c.rms_eps, h->a_norm, st));
+  const double esz = h->esz, R = rows;
+  const double norm_bytes = R * D * (4.0 + esz);
+  double attn_flops = 0.0;
+  for (int s = s0; s < s1; ++s) {
+    const double L = h->h_cu[s + 1] - h->h_cu[s];
+    attn_flops += (c.causal ? 2.0 : 4.0) * L * L * c.n_q_heads * dh;
+  }
+  PRISM_LAUNCH_P(h, st, PRISM_K_RMSNORM, norm_bytes, launch_rmsnorm(xr, W.g_attn, c.dtype, rows, D, c.rms_eps, h->a_norm, st));
   if (h->tc)
-    PRISM_LAUNCH(h, launch_gemm_tc(h->map_a_norm, maps->qkv, maps->qkv, h->qkv, nullptr, rows, nqkv, D, kEpiStore, h->errword, st));
+    PRISM_LAUNCH_P(h, st, PRISM_K_GEMM_QKV, 2.0 * R * nqkv * D,
+                   launch_gemm_tc(h->map_a_norm, maps->qkv, maps->qkv, h->qkv, nullptr, rows, nqkv, D, kEpiStore, h->errword, st));
   else
-    PRISM_LAUNCH(h, launch_gemm_simt(h->a_norm, W.w_qkv, nullptr, h->qkv, nullptr, rows, nqkv, D, c.dtype, kEpiStore, st));
-  PRISM_LAUNCH(h, launch_qknorm_rope(h->qkv, c.dtype, h->pos + r0, rows, c.n_q_heads, c.n_kv_heads, dh, c.qk_norm, W.g_q,
-                                     W.g_k, c.rms_eps, h->rope_cos, h->rope_sin, st));
+    PRISM_LAUNCH_P(h, st, PRISM_K_GEMM_QKV, 2.0 * R * nqkv * D,
+                   launch_gemm_simt(h->a_norm, W.w_qkv, nullptr, h->qkv, nullptr, rows, nqkv, D, c.dtype, kEpiStore, st));
+  PRISM_LAUNCH_P(h, st, PRISM_K_ROPE, 2.0 * R * (c.n_q_heads + c.n_kv_heads) * dh * esz,
+                 launch_qknorm_rope(h->qkv, c.dtype, h->pos + r0, rows, c.n_q_heads, c.n_kv_heads, dh, c.qk_norm, W.g_q, W.g_k,
+                                    c.rms_eps, h->rope_cos, h->rope_sin, st));
   if (h->fa)
-    PRISM_LAUNCH(h, launch_attention_mma(h->qkv, h->attn, cu_dev, s0, s1 - s0, r0, max_len, c.n_q_heads, c.n_kv_heads,
-                                         c.causal, st));
+    PRISM_LAUNCH_P(h, st, PRISM_K_ATTENTION, attn_flops,
+                   launch_attention_mma(h->qkv, h->attn, cu_dev, s0, s1 - s0, r0, max_len, c.n_q_heads, c.n_kv_heads, c.causal, st));
   else
-    PRISM_LAUNCH(h, launch_attention_simt(h->qkv, h->attn, cu_dev, s0, s1 - s0, r0, max_len, c.n_q_heads, c.n_kv_heads, dh,
-                                          c.causal, c.dtype, st));
+    PRISM_LAUNCH_P(h, st, PRISM_K_ATTENTION, attn_flops,
+                   launch_attention_simt(h->qkv, h->attn, cu_dev, s0, s1 - s0, r0, max_len, c.n_q_heads, c.n_kv_heads, dh,
+                                         c.causal, c.dtype, st));
   if (h->tc)
-    PRISM_LAUNCH(h, launch_gemm_tc(h->map_attn, maps->o, maps->o, nullptr, xr, rows, D, hd, kEpiResidual, h->errword, st));
+    PRISM_LAUNCH_P(h, st, PRISM_K_GEMM_O, 2.0 * R * D * hd,
+                   launch_gemm_tc(h->map_attn, maps->o, maps->o, nullptr, xr, rows, D, hd, kEpiResidual, h->errword, st));
   else
-    PRISM_LAUNCH(h, launch_gemm_simt(h->attn, W.w_o, nullptr, nullptr, xr, rows, D, hd, c.dtype, kEpiResidual, st));
-  PRISM_LAUNCH(h, launch_rmsnorm(xr, W.g_ffn, c.dtype, rows, D, c.rms_eps, h->a_norm, st));
+    PRISM_LAUNCH_P(h, st, PRISM_K_GEMM_O, 2.0 * R * D * hd,
+                   launch_gemm_simt(h->attn, W.w_o, nullptr, nullptr, xr, rows, D, hd, c.dtype, kEpiResidual, st));
+  PRISM_LAUNCH_P(h, st, PRISM_K_RMSNORM, norm_bytes, launch_rmsnorm(xr, W.g_ffn, c.dtype, rows, D, c.rms_eps, h->a_norm, st));
   if (h->tc)
-    PRISM_LAUNCH(h, launch_gemm_tc(h->map_a_norm, maps->gate, maps->up, h->hbuf, nullptr, rows, c.ffn, D, kEpiSwiGLU, h->errword, st));
+    PRISM_LAUNCH_P(h, st, PRISM_K_GEMM_GATEUP, 4.0 * R * c.ffn * D,
+                   launch_gemm_tc(h->map_a_norm, maps->gate, maps->up, h->hbuf, nullptr, rows, c.ffn, D, kEpiSwiGLU, h->errword, st));
   else
-    PRISM_LAUNCH(h, launch_gemm_simt(h->a_norm, W.w_gate, W.w_up, h->hbuf, nullptr, rows, c.ffn, D, c.dtype, kEpiSwiGLU, st));
+    PRISM_LAUNCH_P(h, st, PRISM_K_GEMM_GATEUP, 4.0 * R * c.ffn * D,
+                   launch_gemm_simt(h->a_norm, W.w_gate, W.w_up, h->hbuf, nullptr, rows, c.ffn, D, c.dtype, kEpiSwiGLU, st));
   if (h->tc)
-    PRISM_LAUNCH(h, launch_gemm_tc(h->map_hbuf, maps->down, maps->down, nullptr, xr, rows, D, c.ffn, kEpiResidual, h->errword, st));
+    PRISM_LAUNCH_P(h, st, PRISM_K_GEMM_DOWN, 2.0 * R * D * c.ffn,
+                   launch_gemm_tc(h->map_hbuf, maps->down, maps->down, nullptr, xr, rows, D, c.ffn, kEpiResidual, h->errword, st));
   else
-    PRISM_LAUNCH(h, launch_gemm_simt(h->hbuf, W.w_down, nullptr, nullptr, xr, rows, D, c.ffn, c.dtype, kEpiResidual, st));
+    PRISM_LAUNCH_P(h, st, PRISM_K_GEMM_DOWN, 2.0 * R * D * c.ffn,
+                   launch_gemm_simt(h->hbuf, W.w_down, nullptr, nullptr, xr, rows, D, c.ffn, c.dtype, kEpiResidual, st));
   return PRISM_OK;
 }
 
@@ -474,9 +558,10 @@ int select_impl(prism_handle* h, const int32_t* query, int32_t lq, const int32_t
   if (h->h_off[0] != 0) return fail(h, PRISM_ERR_BAD_INPUT, "cand_offsets[0] != 0");
   long long total = 0;
   h->h_cu[0] = 0;
+  for (int i = 0; i < N; ++i)
+    if (h->h_off[i + 1] < h->h_off[i]) return fail(h, PRISM_ERR_BAD_INPUT, "cand_offsets not monotone");
   for (int i = 0; i < N; ++i) {
     const long long dl = (long long)h->h_off[i + 1] - h->h_off[i];
-    if (dl < 0) return fail(h, PRISM_ERR_BAD_INPUT, "cand_offsets not monotone");
     if (dl + lq > c.max_seq_len) return fail(h, PRISM_ERR_SHAPE_LIMIT, "a sequence exceeds max_seq_len");
     if (dl + lq > h->chunk_tokens) return fail(h, PRISM_ERR_BUDGET, "a sequence exceeds the chunk the activation budget allows");
     if (dl + lq < 1) return fail(h, PRISM_ERR_INVALID_ARG, "empty sequence (query_len = 0 and an empty document)");
@@ -494,9 +579,11 @@ int select_impl(prism_handle* h, const int32_t* query, int32_t lq, const int32_t
   PRISM_CUDA(h, cudaMemsetAsync(h->errword, 0, sizeof(int), st));
 
   int cur = 0;  // ping-pong index of x / cu / seq2orig
-  PRISM_LAUNCH(h, launch_pack_offsets(off, N, lq, h->cu[cur], h->seq2orig[cur], h->errword, st));
-  PRISM_LAUNCH(h, launch_pack_tokens(query, lq, cand, off, h->cu[cur], N, (int)total, c.vocab, h->tokens, h->pos, h->errword, st));
-  PRISM_LAUNCH(h, launch_embed(h->embed, c.dtype, h->tokens, (int)total, c.hidden, h->x[cur], st));
+  PRISM_LAUNCH_P(h, st, PRISM_K_PACK, 8.0 * N, launch_pack_offsets(off, N, lq, h->cu[cur], h->seq2orig[cur], h->errword, st));
+  PRISM_LAUNCH_P(h, st, PRISM_K_PACK, 12.0 * total,
+                 launch_pack_tokens(query, lq, cand, off, h->cu[cur], N, (int)total, c.vocab, h->tokens, h->pos, h->errword, st));
+  PRISM_LAUNCH_P(h, st, PRISM_K_EMBED, (double)total * c.hidden * (4.0 + h->esz),
+                 launch_embed(h->embed, c.dtype, h->tokens, (int)total, c.hidden, h->x[cur], st));
 
   if (streamed) {
     // The previous request drained both streams before returning, so both slots are free.
@@ -544,8 +631,9 @@ int select_impl(prism_handle* h, const int32_t* query, int32_t lq, const int32_t
       p.is_final = is_final ? 1 : 0;
       p.layer = layers_run;
       const int nxt = cur ^ 1;
-      PRISM_LAUNCH(h, launch_probe(h->x[cur], h->cu[cur], n, c.hidden, h->g_final, c.dtype, h->w_diff, c.rms_eps, h->scores, st));
-      PRISM_LAUNCH(h, launch_route(h->scores, h->cu[cur], h->seq2orig[cur], n, p, h->cu[nxt], h->seq2orig[nxt], h->old_of_new,
+      PRISM_LAUNCH_P(h, st, PRISM_K_PROBE, 4.0 * n * c.hidden,
+                     launch_probe(h->x[cur], h->cu[cur], n, c.hidden, h->g_final, c.dtype, h->w_diff, c.rms_eps, h->scores, st));
+      PRISM_LAUNCH_P(h, st, PRISM_K_ROUTE, 8.0 * n, launch_route(h->scores, h->cu[cur], h->seq2orig[cur], n, p, h->cu[nxt], h->seq2orig[nxt], h->old_of_new,
                                    h->state, h->res_idx, h->res_score, h->recs + n_rec,
                                    h->trace_scores + (size_t)n_rec * c.max_candidates,
                                    h->trace_ids + (size_t)n_rec * c.max_candidates, h->route_scratch, st));
@@ -563,9 +651,10 @@ int select_impl(prism_handle* h, const int32_t* query, int32_t lq, const int32_t
       if (!done && stt.n_active < n) {
         // survivors move to the other buffer, order kept; offsets and positions follow
         std::swap(h->h_cu, h->h_cu_next);
-        PRISM_LAUNCH(h, launch_compact_rows(h->x[cur], h->x[nxt], h->cu[cur], h->cu[nxt], h->old_of_new, stt.n_active,
-                                            stt.n_tokens, c.hidden, st));
-        PRISM_LAUNCH(h, launch_positions(h->cu[nxt], stt.n_active, stt.n_tokens, h->pos, st));
+        PRISM_LAUNCH_P(h, st, PRISM_K_COMPACT, 8.0 * stt.n_tokens * c.hidden,
+                       launch_compact_rows(h->x[cur], h->x[nxt], h->cu[cur], h->cu[nxt], h->old_of_new, stt.n_active,
+                                           stt.n_tokens, c.hidden, st));
+        PRISM_LAUNCH_P(h, st, PRISM_K_PACK, 4.0 * stt.n_tokens, launch_positions(h->cu[nxt], stt.n_active, stt.n_tokens, h->pos, st));
         cur = nxt;
         n = stt.n_active;
         T = stt.n_tokens;
@@ -597,6 +686,7 @@ int select_impl(prism_handle* h, const int32_t* query, int32_t lq, const int32_t
   }
   PRISM_CUDA(h, cudaStreamSynchronize(st));
   if (streamed) PRISM_CUDA(h, cudaStreamSynchronize(h->copy_stream));
+  if (h->prof_on) prof_collect(h);
   if (h->h_state->n_result != k_eff) return fail(h, PRISM_ERR_CUDA, "internal: result count mismatch");
   *n_out = k_eff;
   return PRISM_OK;

@@ -157,7 +157,8 @@ def test_gemm_fp32_simt(P, m, n, k, epi):
     rs = dev(resid)
     P.ops.prism_op_gemm(dev(a), dev(b), dev(b2), out, rs, m, n, k, FP32, epi, SIMT, None)
     got = (rs if epi == 1 else out).cpu().numpy()
-    assert np.max(np.abs(got - _gemm_ref(a, b, b2, resid, epi))) < 2e-5
+    ref = _gemm_ref(a, b, b2, resid, epi)
+    assert np.max(np.abs(got - ref)) < 1e-5 * max(1.0, np.max(np.abs(ref)))      # fp32 accumulation over k terms
 
 
 @pytest.mark.parametrize("impl", [AUTO, SIMT])
@@ -275,7 +276,7 @@ def test_route_matches_oracle_rule_bit_exact(P, n_clusters, winners):
         lens = rng.integers(1, 50, size=n)
         thr = float(rng.choice([0.0, 0.3, 5.0]))
         st, cu_new, s2o_new, oon, ridx, rsc, rec, cu = _run_route(
-            P, sc, ids, lens, k, 2, dict(cv_threshold=thr, n_clusters=n_clusters, select_winners=winners))
+            P, sc, ids, lens, min(k, n), 2, dict(cv_threshold=thr, n_clusters=n_clusters, select_winners=winners))
         # the oracle's rule on the same scores: a one-probe schedule over a two-layer "model"
         sched = Schedule(MODE_CLUSTER, (1,), cv_threshold=thr, n_clusters=n_clusters, select_winners=winners)
         table = {1: dict(zip(range(n), sc)), 2: dict(zip(range(n), sc))}

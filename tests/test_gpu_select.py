@@ -85,11 +85,12 @@ def test_cfg0_other_requests_and_k(P, tiny):
         req = synth.make_request(wl, r)
         S = oracle.score_matrix(req["query"], req["cand_tokens"], req["cand_offsets"], w, wl.model, [1, 2])
         model = make_model(P, wl.model, w, req)
-        for k in (1, 3, 16, 40):                                       # K > N is not an error
-            idx, sc, tr = run(P, model, req, k, wl.schedule)
+        for k in (1, 3, 8, 16, 40):                                    # K > N is not an error
+            sched = wl.schedule if k <= 8 else Schedule(MODE_CLUSTER, (1,), cv_threshold=0.2)
+            idx, sc, tr = run(P, model, req, k, sched)
             assert len(idx) == min(k, wl.n_candidates)
             check_scores(tr, S, TOL_FP32)
-            check_replay(tr, idx, sc, wl.n_candidates, k, wl.model.n_layers, wl.schedule)
+            check_replay(tr, idx, sc, wl.n_candidates, k, wl.model.n_layers, sched)
         model.close()
 
 
