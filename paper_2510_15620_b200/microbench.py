@@ -1,0 +1,123 @@
+"""Per-kernel microbenchmark through the C ABI (prism_op_*): CUDA-event timing of one kernel on
+synthetic operands, one JSON line per run.  Also the small-case driver for profiler captures.
+
+    python -m paper_2510_15620_b200.microbench --op gemm --m 35200 --n 4096 --k 1024 --epilogue 0
+    python -m paper_2510_15620_b200.microbench --op attention --seqs 100 --len-lo 160 --len-hi 544
+    python -m paper_2510_15620_b200.microbench --op rmsnorm|rope|compact --rows 35200 --d 1024
+"""
+from __future__ import annotations
+
+import argparse
+import json
+
+import numpy as np
+import torch
+
+from . import ops
+from .binding import PRISM_BF16, PRISM_IMPL_AUTO
+
+
+def _time(fn, iters, warmup, flush):
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    ms = []
+    for _ in range(iters):
+        if flush is not None:
+            flush.zero_()                      # > L2 bytes written between timed launches
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        fn()
+        b.record()
+        torch.cuda.synchronize()
+        ms.append(a.elapsed_time(b))
+    return float(np.median(ms)), float(np.min(ms))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--op", required=True, choices=["gemm", "attention", "rmsnorm", "rope", "compact"])
+    ap.add_argument("--m", type=int, default=35200)
+    ap.add_argument("--n", type=int, default=4096)
+    ap.add_argument("--k", type=int, default=1024)
+    ap.add_argument("--epilogue", type=int, default=0)
+    ap.add_argument("--impl", type=int, default=PRISM_IMPL_AUTO)
+    ap.add_argument("--rows", type=int, default=35200)
+    ap.add_argument("--d", type=int, default=1024)
+    ap.add_argument("--seqs", type=int, default=100)
+    ap.add_argument("--len-lo", type=int, default=160)
+    ap.add_argument("--len-hi", type=int, default=544)
+    ap.add_argument("--hq", type=int, default=16)
+    ap.add_argument("--hkv", type=int, default=8)
+    ap.add_argument("--causal", type=int, default=1)
+    ap.add_argument("--iters", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--no-flush", action="store_true")
+    a = ap.parse_args()
+    dev = "cuda"
+    g = torch.Generator(device=dev).manual_seed(0)
+    flush = None if a.no_flush else torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    rnd = lambda *s: torch.randn(*s, device=dev, generator=g)
+    out = {"op": a.op}
+    if a.op == "gemm":
+        m, n, k = a.m, a.n, a.k
+        A = rnd(m, k).to(torch.bfloat16)
+        B = (rnd(n, k) * 0.05).to(torch.bfloat16)
+        B2 = (rnd(n, k) * 0.05).to(torch.bfloat16)
+        O = torch.empty(m, n, dtype=torch.bfloat16, device=dev)
+        R = rnd(m, n)
+        err = torch.zeros(1, dtype=torch.int32, device=dev)
+        fn = lambda: ops.prism_op_gemm(A, B, B2, O, R, m, n, k, PRISM_BF16, a.epilogue, a.impl, err)
+        med, best = _time(fn, a.iters, a.warmup, flush)
+        fl = 2.0 * m * n * k * (2 if a.epilogue == 2 else 1)
+        out.update(m=m, n=n, k=k, epilogue=a.epilogue, ms=med, ms_min=best, tflops=fl / med / 1e9, err=int(err.item()))
+    elif a.op == "attention":
+        rng = np.random.default_rng(0)
+        lens = rng.integers(a.len_lo, a.len_hi + 1, size=a.seqs)
+        cu = np.zeros(a.seqs + 1, np.int32)
+        cu[1:] = np.cumsum(lens)
+        dh = 128
+        qkv = rnd(int(cu[-1]), (a.hq + 2 * a.hkv) * dh).to(torch.bfloat16)
+        o = torch.empty(int(cu[-1]), a.hq * dh, dtype=torch.bfloat16, device=dev)
+        cud = torch.from_numpy(cu).to(dev)
+        fn = lambda: ops.prism_op_attention(qkv, o, cud, a.seqs, int(lens.max()), a.hq, a.hkv, dh, a.causal, PRISM_BF16, a.impl)
+        med, best = _time(fn, a.iters, a.warmup, flush)
+        fl = float(np.sum((2.0 if a.causal else 4.0) * lens.astype(np.float64) ** 2 * a.hq * dh))
+        out.update(seqs=a.seqs, tokens=int(cu[-1]), causal=a.causal, ms=med, ms_min=best, tflops=fl / med / 1e9)
+    elif a.op == "rmsnorm":
+        x = rnd(a.rows, a.d)
+        gain = torch.ones(a.d, dtype=torch.bfloat16, device=dev)
+        o = torch.empty(a.rows, a.d, dtype=torch.bfloat16, device=dev)
+        fn = lambda: ops.prism_op_rmsnorm(x, gain, PRISM_BF16, 1e-6, o)
+        med, best = _time(fn, a.iters, a.warmup, flush)
+        out.update(rows=a.rows, d=a.d, ms=med, ms_min=best, gbs=a.rows * a.d * 6.0 / med / 1e6)
+    elif a.op == "rope":
+        dh = 128
+        qkv = rnd(a.rows, (a.hq + 2 * a.hkv) * dh).to(torch.bfloat16)
+        pos = torch.randint(0, 512, (a.rows,), dtype=torch.int32, device=dev)
+        gq = torch.ones(dh, dtype=torch.bfloat16, device=dev)
+        fn = lambda: ops.prism_op_qknorm_rope(qkv, PRISM_BF16, pos, a.hq, a.hkv, dh, 1, gq, gq, 1e-6, 1e6, 512)
+        med, best = _time(fn, a.iters, a.warmup, flush)
+        out.update(rows=a.rows, ms=med, ms_min=best, gbs=a.rows * (a.hq + a.hkv) * dh * 4.0 / med / 1e6,
+                   note="includes the op wrapper's table build and sync")
+    else:
+        n = a.seqs
+        rng = np.random.default_rng(0)
+        lens = rng.integers(a.len_lo, a.len_hi + 1, size=n)
+        cu = np.zeros(n + 1, np.int32)
+        cu[1:] = np.cumsum(lens)
+        keep = np.sort(rng.choice(n, size=max(1, n // 3), replace=False)).astype(np.int32)
+        cun = np.zeros(len(keep) + 1, np.int32)
+        cun[1:] = np.cumsum(lens[keep])
+        x = rnd(int(cu[-1]), a.d)
+        y = torch.empty(int(cun[-1]), a.d, device=dev)
+        t = lambda v: torch.from_numpy(v).to(dev)
+        cu_d, cun_d, keep_d = t(cu), t(cun), t(keep)
+        fn = lambda: ops.prism_op_compact(x, y, cu_d, cun_d, keep_d, len(keep), int(cun[-1]))
+        med, best = _time(fn, a.iters, a.warmup, flush)
+        out.update(rows_out=int(cun[-1]), d=a.d, ms=med, ms_min=best, gbs=int(cun[-1]) * a.d * 8.0 / med / 1e6)
+    print(json.dumps(out))
+
+
+if __name__ == "__main__":
+    main()
