@@ -79,6 +79,34 @@ PRISM_API int prism_op_route(const float* scores, const int32_t* cu_old, const i
                    int32_t* old_of_new, int32_t* state, int32_t* res_idx, float* res_score, prism_probe_record* rec,
                    void* stream);
 
+/* The same pruning decision as prism_op_route for callers that cannot allocate device memory.  (The
+ * paper has no counterpart: this is a property of the library, not of the method.)
+ *
+ * Who needs it: a host program whose own memory pool has already claimed the whole GPU, so that a
+ * cudaMalloc made on its behalf fails; or a serving loop that must not stall, because cudaMalloc and
+ * cudaFree wait for the device to go idle.  prism_op_route allocates and frees its clustering scratch
+ * on every call; this entry point calls no cudaMalloc, cudaFree or any other allocating routine.  Its
+ * scratch is an array of about 74 KB built into the library image, which every GPU that loads the
+ * library keeps until the process ends.
+ *
+ * Limits and rules:
+ *   - n <= PRISM_ROUTE_STATIC_MAX_CANDIDATES; a larger n returns PRISM_ERR_SHAPE_LIMIT and nothing runs.
+ *   - The first call on each device looks up the array's address on that device (the device must be
+ *     current).  Make that first call outside any stream capture.
+ *   - All calls share the one array, and it keeps what the previous call left there.  The kernel
+ *     writes every scratch word before it reads it, so nothing has to be cleared between calls; but
+ *     two calls that overlap on the GPU (different streams, no ordering between them) race on it.
+ *     Calls on one stream are safe.
+ *   - Arguments, outputs and the result are exactly those of prism_op_route; the call only enqueues
+ *     the kernel on `stream` and does not synchronise. */
+#define PRISM_ROUTE_STATIC_MAX_CANDIDATES 1024
+PRISM_API int prism_op_route_static(const float* scores, const int32_t* cu_old, const int32_t* seq2orig_old,
+                                    int32_t n, int32_t mode, int32_t keep_count, double cv_threshold,
+                                    int32_t n_clusters, int32_t std_ddof, int32_t select_winners,
+                                    int32_t is_final, int32_t layer, int32_t* cu_new, int32_t* seq2orig_new,
+                                    int32_t* old_of_new, int32_t* state, int32_t* res_idx, float* res_score,
+                                    prism_probe_record* rec, void* stream);
+
 /* Survivor gather (Fig. 4: only the deferred candidates are retained): row t of the new batch, owned
  * by new sequence s, is copied from x_old[cu_old[old_of_new[s]] + (t - cu_new[s])]. */
 PRISM_API int prism_op_compact(const float* x_old, float* x_new, const int32_t* cu_old, const int32_t* cu_new,

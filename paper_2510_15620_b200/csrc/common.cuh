@@ -54,11 +54,10 @@ struct ProbeRecordDev {  // layout mirrors prism_probe_record
 };
 
 // Bytes of global scratch the routing kernel needs for n candidates.
-inline size_t route_scratch_bytes(int n) {
-  size_t np1 = (size_t)n + 1;
-  return np1 * sizeof(double) * 4            // P1, P2, D[2]
-         + np1 * sizeof(int) * kMaxClusters  // argmin table
-         + np1 * sizeof(int) * 2             // valid flags, sorted positions
+constexpr size_t route_scratch_bytes(int n) {
+  return ((size_t)n + 1) * sizeof(double) * 4            // P1, P2, D[2]
+         + ((size_t)n + 1) * sizeof(int) * kMaxClusters  // argmin table
+         + ((size_t)n + 1) * sizeof(int) * 2             // valid flags, sorted positions
          + 256;
 }
 

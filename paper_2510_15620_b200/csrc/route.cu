@@ -4,6 +4,7 @@
 // The decision arithmetic is fp64 on fp32 scores in a fixed left-to-right order with explicitly
 // rounded operations (no FMA contraction), so that the integer outcome (cuts, survivor set, new
 // offsets, top-K order) is a pure function of the scores.
+#include "../../include/prism_ops.h"
 #include "common.cuh"
 
 namespace prism {
@@ -333,3 +334,56 @@ cudaError_t launch_route(const float* scores, const int* cu_old, const int* seq2
 }
 
 }  // namespace prism
+
+// ------------------------------------------------------------------------------------------------
+// prism_op_route_static: the pruning decision for callers that cannot allocate device memory.
+//
+// The scratch the kernel needs (prefix sums, the two cost rows and the argmin table of the
+// clustering) lives in a fixed array inside the library image instead of a cudaMalloc'd buffer.
+// Every GPU that loads the library holds these bytes until the process exits.
+namespace {
+
+constexpr int kStaticRouteMaxN = PRISM_ROUTE_STATIC_MAX_CANDIDATES;
+constexpr size_t kStaticRouteBytes = (prism::route_scratch_bytes(kStaticRouteMaxN) + 255) / 256 * 256;
+
+static __device__ __align__(256) unsigned char g_route_static_scratch[kStaticRouteBytes];
+
+constexpr int kMaxDevices = 64;
+void* g_route_static_ptr[kMaxDevices] = {};  // device address of the array, per device, filled on first use
+
+}  // namespace
+
+extern "C" int prism_op_route_static(const float* scores, const int32_t* cu_old, const int32_t* seq2orig_old,
+                                     int32_t n, int32_t mode, int32_t keep_count, double cv_threshold,
+                                     int32_t n_clusters, int32_t std_ddof, int32_t select_winners, int32_t is_final,
+                                     int32_t layer, int32_t* cu_new, int32_t* seq2orig_new, int32_t* old_of_new,
+                                     int32_t* state, int32_t* res_idx, float* res_score, prism_probe_record* rec,
+                                     void* stream) {
+  using namespace prism;
+  if (!scores || !cu_old || !seq2orig_old || !cu_new || !seq2orig_new || !old_of_new || !state || !res_idx || !res_score)
+    return PRISM_ERR_INVALID_ARG;
+  if (n < 0 || n_clusters < 2 || n_clusters > kMaxClusters) return PRISM_ERR_INVALID_ARG;
+  if (n > kStaticRouteMaxN) return PRISM_ERR_SHAPE_LIMIT;  // the built-in scratch is sized for this many candidates
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return PRISM_ERR_CUDA;
+  if (!g_route_static_ptr[dev]) {
+    // In host code the array's name is only a handle; the kernel needs the address it has on THIS device.
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_route_static_scratch) != cudaSuccess || !p) return PRISM_ERR_CUDA;
+    g_route_static_ptr[dev] = p;
+  }
+  RouteParams prm{};
+  prm.mode = mode;
+  prm.keep_count = keep_count;
+  prm.cv_threshold = cv_threshold;
+  prm.n_clusters = n_clusters;
+  prm.ddof = std_ddof;
+  prm.select_winners = select_winners;
+  prm.is_final = is_final;
+  prm.layer = layer;
+  cudaError_t e = launch_route(scores, cu_old, seq2orig_old, n, prm, cu_new, seq2orig_new, old_of_new,
+                               reinterpret_cast<RouteState*>(state), res_idx, res_score,
+                               reinterpret_cast<ProbeRecordDev*>(rec), nullptr, nullptr, g_route_static_ptr[dev],
+                               reinterpret_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? PRISM_OK : PRISM_ERR_CUDA;
+}

@@ -24,6 +24,8 @@ def _L():
         L.prism_op_attention.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, i32, vp]
         L.prism_op_probe.argtypes = [vp, vp, i32, i32, vp, vp, i32, f32, vp, vp]
         L.prism_op_route.argtypes = [vp, vp, vp, i32, i32, i32, f64, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
+        L.prism_op_route_static.argtypes = L.prism_op_route.argtypes
+        L.prism_op_route_static.restype = C.c_int
         L.prism_op_compact.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, vp]
         for n in ("pack", "embed", "rmsnorm", "qknorm_rope", "gemm", "attention", "probe", "route", "compact"):
             getattr(L, "prism_op_" + n).restype = C.c_int
@@ -82,6 +84,15 @@ def prism_op_route(scores, cu_old, seq2orig_old, n, mode, keep_count, cv_thresho
     _check(_L().prism_op_route(_p(scores), _p(cu_old), _p(seq2orig_old), n, mode, keep_count, cv_threshold, n_clusters,
                                std_ddof, select_winners, is_final, layer, _p(cu_new), _p(seq2orig_new), _p(old_of_new),
                                _p(state), _p(res_idx), _p(res_score), _p(rec), _stream()), "route")
+
+
+def prism_op_route_static(scores, cu_old, seq2orig_old, n, mode, keep_count, cv_threshold, n_clusters, std_ddof,
+                          select_winners, is_final, layer, cu_new, seq2orig_new, old_of_new, state, res_idx, res_score, rec):
+    """prism_op_route without any device allocation (scratch built into the library; n <= 1024)."""
+    _check(_L().prism_op_route_static(_p(scores), _p(cu_old), _p(seq2orig_old), n, mode, keep_count, cv_threshold,
+                                      n_clusters, std_ddof, select_winners, is_final, layer, _p(cu_new), _p(seq2orig_new),
+                                      _p(old_of_new), _p(state), _p(res_idx), _p(res_score), _p(rec), _stream()),
+           "route_static")
 
 
 def prism_op_compact(x_old, x_new, cu_old, cu_new, old_of_new, n_new, total_new):
