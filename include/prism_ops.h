@@ -52,6 +52,16 @@ PRISM_API int prism_op_qknorm_rope(void* qkv, int32_t dtype, const int32_t* pos,
 PRISM_API int prism_op_gemm(const void* a, const void* b, const void* b2, void* out, float* resid, int32_t m, int32_t n,
                   int32_t k, int32_t dtype, int32_t epilogue, int32_t impl, int32_t* err_word, void* stream);
 
+/* The QKV projection with QK-norm and the rotary embedding fused into its epilogue (tensor-core path,
+ * bf16, head_dim 128): out[m, (Hq+2Hkv)*128] = rope(qknorm(a[m,k] * w_qkv^T)) on the q and k heads, plain
+ * projection on the v heads.  Equals prism_op_gemm(epilogue 0) followed by prism_op_qknorm_rope, except
+ * that norm and rotation act on the fp32 accumulator (one rounding to bf16 instead of two).
+ * Allocates and frees a temporary rotary table of max_pos rows. */
+PRISM_API int prism_op_gemm_qkv_rope(const void* a, const void* w_qkv, void* out, int32_t m, int32_t k,
+                                     int32_t n_q_heads, int32_t n_kv_heads, int32_t qk_norm, const void* g_q,
+                                     const void* g_k, float eps, const int32_t* pos, float theta, int32_t max_pos,
+                                     int32_t* err_word, void* stream);
+
 /* Attention over packed sequences: for sequence s (rows cu[s]..cu[s+1]) and query head h (kv head
  * h / (Hq/Hkv)): out = softmax(q k^T / sqrt(head_dim) [+ causal mask]) v.  qkv [total, (Hq+2Hkv)*dh],
  * out [total, Hq*dh].  max_len >= the longest sequence. */

@@ -21,6 +21,18 @@ enum Epilogue : int {
   kEpiStore = 0,     // out[M,N] = acc                               (QKV projection)
   kEpiResidual = 1,  // x[M,N] += acc, x fp32 residual stream        (O-proj, down-proj)
   kEpiSwiGLU = 2,    // out[M,N] = silu(acc_gate) * acc_up           (gate/up projection)
+  kEpiQkvRope = 3,   // QKV projection with QK-norm + rotary embedding applied to the q and k heads
+};
+
+// Inputs of the fused QK-norm + RoPE epilogue (head_dim 128; rotary table rows of 64 floats).
+struct QkvRopeArgs {
+  const int* pos;        // [m] position of each row inside its sequence
+  const float* cos_t;    // [max_pos, 64]
+  const float* sin_t;    // [max_pos, 64]
+  const __nv_bfloat16* g_q;  // [128] (used when qk_norm)
+  const __nv_bfloat16* g_k;  // [128]
+  int hq, hkv, qk_norm;
+  float eps;
 };
 
 struct RouteParams {
@@ -102,7 +114,7 @@ cudaError_t make_tma_2d_bf16(TmaDesc* out, const void* base, uint64_t rows, uint
 // b0/b1 describe the first and second 128 weight rows of a tile: the same matrix for plain
 // projections, the gate and the up matrix for kEpiSwiGLU.
 cudaError_t launch_gemm_tc(const TmaDesc& a, const TmaDesc& b0, const TmaDesc& b1, void* out, float* resid, int m,
-                           int n, int k, int epilogue, int* err, cudaStream_t st);
+                           int n, int k, int epilogue, const QkvRopeArgs* qa, int* err, cudaStream_t st);
 cudaError_t launch_attention_mma(const void* qkv, void* out, const int* cu, int seq0, int nseq, int row0,
                                  int max_len, int n_q_heads, int n_kv_heads, int causal, cudaStream_t st);
 

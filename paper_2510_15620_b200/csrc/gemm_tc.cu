@@ -6,7 +6,13 @@
 //   warp 1      MMA issuer: one elected lane issues tcgen05.mma (M=128, N=256, K=16) into one of two
 //               256-column TMEM accumulators, commits stage-release and accumulator-ready barriers
 //   warps 2..5  epilogue: tcgen05.ld the accumulator (one row per thread), apply the fused epilogue
-//               (bf16 store | fp32 residual add | SwiGLU), while the MMA warp fills the other buffer
+//               while the MMA warp fills the other buffer:
+//                 store     bf16 store
+//                 residual  x += acc through shared memory and a TMA reduce-add (asynchronous, no read of
+//                           x by the SM, one add per element so the result is deterministic)
+//                 SwiGLU    silu(gate) * up
+//                 QKV       per-head RMSNorm (QK-norm) and rotary embedding on the q and k heads before
+//                           the bf16 store (a 256-column tile is exactly two heads of 128)
 // Every tile uses the same shape and the same K order whatever M is, so a row's result does not
 // depend on where it sits in the batch (duplicated candidates give bit-identical scores).
 //
@@ -25,7 +31,9 @@ constexpr int kStages = 4;
 constexpr int kABytes = BM * BK * 2;           // 16 KB
 constexpr int kBBytes = BN * BK * 2;           // 32 KB
 constexpr int kStageBytes = kABytes + kBBytes; // 48 KB
-constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int kEpiBufBytes = 32 * 32 * 4;      // one 32x32 fp32 sub-tile staged for a TMA reduce-add
+constexpr int kEpiStageBytes = 4 * 2 * kEpiBufBytes;  // 4 epilogue warps x 2 buffers
+constexpr int kSmemBytes = kStages * kStageBytes + kEpiStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
 constexpr int kThreads = 192;
 constexpr unsigned long long kWaitCycles = 4000000000ull;  // ~2 s at boost clock
 
@@ -76,6 +84,19 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar)
       : "memory");
 }
+
+// x[tile] += smem tile (fp32), performed by the TMA unit / L2; rows and columns outside the tensor are clipped.
+__device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap* map, uint32_t src, int c0, int c1) {
+  asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3}], [%1];"
+               ::"l"(map), "r"(src), "r"(c0), "r"(c1)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait() { asm volatile("cp.async.bulk.wait_group %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -128,13 +149,14 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
 template <int kEpi>
 __global__ void __launch_bounds__(kThreads, 1)
 k_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b0,
-          const __grid_constant__ CUtensorMap map_b1, __nv_bfloat16* __restrict__ out, float* __restrict__ resid,
-          int m, int n, int k, int* __restrict__ err) {
+          const __grid_constant__ CUtensorMap map_b1, const __grid_constant__ CUtensorMap map_r,
+          __nv_bfloat16* __restrict__ out, int m, int n, int k, const QkvRopeArgs qa, int* __restrict__ err) {
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t tiles = (raw + 1023u) & ~1023u;  // swizzled tiles need 1024-byte alignment
   unsigned char* gen_tiles = smem_raw + (tiles - raw);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(gen_tiles + kStages * kStageBytes);
+  const uint32_t epi_stage = tiles + kStages * kStageBytes;  // 1024-byte aligned
+  uint64_t* bars = reinterpret_cast<uint64_t*>(gen_tiles + kStages * kStageBytes + kEpiStageBytes);
   // bars: full[kStages], empty[kStages], acc_full[2], acc_empty[2]; then tmem base and abort flag
   const uint32_t bar_full = smem_u32(bars), bar_empty = smem_u32(bars + kStages);
   const uint32_t bar_acc_full = smem_u32(bars + 2 * kStages), bar_acc_empty = smem_u32(bars + 2 * kStages + 2);
@@ -144,6 +166,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // Output tile width: SwiGLU tiles hold 128 gate + 128 up columns and produce 128 outputs.
   constexpr int kOutCols = (kEpi == kEpiSwiGLU) ? 128 : 256;
+  (void)epi_stage;
   const int m_tiles = (m + BM - 1) / BM, n_tiles = (n + kOutCols - 1) / kOutCols;
   const int num_tiles = m_tiles * n_tiles, num_kb = (k + BK - 1) / BK;
 
@@ -263,6 +286,127 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
             }
           }
         }
+      } else if constexpr (kEpi == kEpiResidual) {
+        // 32x32 fp32 sub-tiles go through shared memory (128-byte swizzle) into a TMA reduce-add.
+        const uint32_t my_bufs = epi_stage + (uint32_t)(warp - 2) * 2 * kEpiBufBytes;
+#pragma unroll 1
+        for (int c = 0; c < 8; ++c) {
+          // Sub-tiles outside the matrix are skipped entirely (warp-uniform): a staging buffer is only
+          // rewritten after a later commit has made the wait below cover its previous reduce.
+          if (col0 + c * 32 >= n || mt * BM + quarter * 32 >= m) break;
+          const uint32_t buf = my_bufs + (c & 1) * kEpiBufBytes;
+          uint32_t r[32];
+          tmem_ld32(taddr + c * 32, r);
+          if (lane == 0) bulk_wait_read<1>();  // the reduce that last read this buffer has finished with it
+          __syncwarp();
+          tmem_ld_wait();
+#pragma unroll
+          for (int v = 0; v < 8; ++v) {
+            const uint32_t dst = buf + lane * 128 + ((v ^ (lane & 7)) << 4);
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(r[4 * v]), "r"(r[4 * v + 1]),
+                         "r"(r[4 * v + 2]), "r"(r[4 * v + 3]) : "memory");
+          }
+          fence_async_smem();
+          __syncwarp();
+          if (lane == 0) {
+            tma_reduce_add_2d(&map_r, buf, col0 + c * 32, mt * BM + quarter * 32);
+            bulk_commit();
+          }
+        }
+      } else if constexpr (kEpi == kEpiQkvRope) {
+        // A 256-column tile is two heads.  q and k heads: optional RMSNorm over the head, then the
+        // rotation of pairs (j, j+64); v heads are stored as they are.
+        const int prow = row < m ? row : 0;
+        const float* ct = qa.cos_t + (size_t)qa.pos[prow] * 64;
+        const float* st = qa.sin_t + (size_t)qa.pos[prow] * 64;
+#pragma unroll 1
+        for (int hh = 0; hh < 2; ++hh) {
+          const int head = nt * 2 + hh;
+          if (head * 128 >= n) break;
+          __nv_bfloat16* o = out + (size_t)row * n + (size_t)head * 128;
+          const uint32_t th = taddr + hh * 128;
+          if (head >= qa.hq + qa.hkv) {
+#pragma unroll 1
+            for (int c = 0; c < 4; ++c) {
+              uint32_t r[32];
+              tmem_ld32(th + c * 32, r);
+              tmem_ld_wait();
+              if (row < m) {
+#pragma unroll
+                for (int v = 0; v < 4; ++v) {
+                  uint4 pk;
+                  pk.x = pack_bf16(__uint_as_float(r[v * 8 + 0]), __uint_as_float(r[v * 8 + 1]));
+                  pk.y = pack_bf16(__uint_as_float(r[v * 8 + 2]), __uint_as_float(r[v * 8 + 3]));
+                  pk.z = pack_bf16(__uint_as_float(r[v * 8 + 4]), __uint_as_float(r[v * 8 + 5]));
+                  pk.w = pack_bf16(__uint_as_float(r[v * 8 + 6]), __uint_as_float(r[v * 8 + 7]));
+                  *reinterpret_cast<uint4*>(o + c * 32 + v * 8) = pk;
+                }
+              }
+            }
+            continue;
+          }
+          float rn = 1.f;
+          if (qa.qk_norm) {
+            float ss = 0.f;
+#pragma unroll 1
+            for (int c = 0; c < 4; ++c) {
+              uint32_t r[32];
+              tmem_ld32(th + c * 32, r);
+              tmem_ld_wait();
+#pragma unroll
+              for (int e = 0; e < 32; ++e) ss = fmaf(__uint_as_float(r[e]), __uint_as_float(r[e]), ss);
+            }
+            rn = 1.0f / sqrtf(ss * (1.f / 128.f) + qa.eps);
+          }
+          const __nv_bfloat16* gain = head < qa.hq ? qa.g_q : qa.g_k;
+#pragma unroll 1
+          for (int j = 0; j < 2; ++j) {
+            uint32_t a[32], b[32];
+            tmem_ld32(th + j * 32, a);
+            tmem_ld32(th + 64 + j * 32, b);
+            tmem_ld_wait();
+            if (row < m) {
+#pragma unroll
+              for (int v = 0; v < 4; ++v) {
+                float x0[8], x1[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                  x0[e] = __uint_as_float(a[v * 8 + e]);
+                  x1[e] = __uint_as_float(b[v * 8 + e]);
+                }
+                if (qa.qk_norm) {
+                  const uint4 g0 = __ldg(reinterpret_cast<const uint4*>(gain + j * 32 + v * 8));
+                  const uint4 g1 = __ldg(reinterpret_cast<const uint4*>(gain + 64 + j * 32 + v * 8));
+                  const __nv_bfloat16* p0 = reinterpret_cast<const __nv_bfloat16*>(&g0);
+                  const __nv_bfloat16* p1 = reinterpret_cast<const __nv_bfloat16*>(&g1);
+#pragma unroll
+                  for (int e = 0; e < 8; ++e) {
+                    x0[e] = x0[e] * rn * __bfloat162float(p0[e]);
+                    x1[e] = x1[e] * rn * __bfloat162float(p1[e]);
+                  }
+                }
+                const float4 c0 = __ldg(reinterpret_cast<const float4*>(ct + j * 32 + v * 8));
+                const float4 c1 = __ldg(reinterpret_cast<const float4*>(ct + j * 32 + v * 8 + 4));
+                const float4 s0 = __ldg(reinterpret_cast<const float4*>(st + j * 32 + v * 8));
+                const float4 s1 = __ldg(reinterpret_cast<const float4*>(st + j * 32 + v * 8 + 4));
+                const float cs[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
+                const float sn[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
+                uint32_t lo[4], hi[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                  const float y0 = x0[2 * e] * cs[2 * e] - x1[2 * e] * sn[2 * e];
+                  const float y1 = x0[2 * e + 1] * cs[2 * e + 1] - x1[2 * e + 1] * sn[2 * e + 1];
+                  const float z0 = x1[2 * e] * cs[2 * e] + x0[2 * e] * sn[2 * e];
+                  const float z1 = x1[2 * e + 1] * cs[2 * e + 1] + x0[2 * e + 1] * sn[2 * e + 1];
+                  lo[e] = pack_bf16(y0, y1);
+                  hi[e] = pack_bf16(z0, z1);
+                }
+                *reinterpret_cast<uint4*>(o + j * 32 + v * 8) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+                *reinterpret_cast<uint4*>(o + 64 + j * 32 + v * 8) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+              }
+            }
+          }
+        }
       } else {
 #pragma unroll 1
         for (int c = 0; c < 8; ++c) {
@@ -270,31 +414,16 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
           tmem_ld32(taddr + c * 32, r);
           tmem_ld_wait();
           if (row < m) {
-            if constexpr (kEpi == kEpiStore) {
-              __nv_bfloat16* o = out + (size_t)row * n + col0 + c * 32;
+            __nv_bfloat16* o = out + (size_t)row * n + col0 + c * 32;
 #pragma unroll
-              for (int v = 0; v < 4; ++v) {
-                if (col0 + c * 32 + v * 8 < n) {
-                  uint4 pk;
-                  pk.x = pack_bf16(__uint_as_float(r[v * 8 + 0]), __uint_as_float(r[v * 8 + 1]));
-                  pk.y = pack_bf16(__uint_as_float(r[v * 8 + 2]), __uint_as_float(r[v * 8 + 3]));
-                  pk.z = pack_bf16(__uint_as_float(r[v * 8 + 4]), __uint_as_float(r[v * 8 + 5]));
-                  pk.w = pack_bf16(__uint_as_float(r[v * 8 + 6]), __uint_as_float(r[v * 8 + 7]));
-                  *reinterpret_cast<uint4*>(o + v * 8) = pk;
-                }
-              }
-            } else {
-              float* o = resid + (size_t)row * n + col0 + c * 32;
-#pragma unroll
-              for (int v = 0; v < 8; ++v) {
-                if (col0 + c * 32 + v * 4 < n) {
-                  float4 x = *reinterpret_cast<float4*>(o + v * 4);
-                  x.x += __uint_as_float(r[v * 4 + 0]);
-                  x.y += __uint_as_float(r[v * 4 + 1]);
-                  x.z += __uint_as_float(r[v * 4 + 2]);
-                  x.w += __uint_as_float(r[v * 4 + 3]);
-                  *reinterpret_cast<float4*>(o + v * 4) = x;
-                }
+            for (int v = 0; v < 4; ++v) {
+              if (col0 + c * 32 + v * 8 < n) {
+                uint4 pk;
+                pk.x = pack_bf16(__uint_as_float(r[v * 8 + 0]), __uint_as_float(r[v * 8 + 1]));
+                pk.y = pack_bf16(__uint_as_float(r[v * 8 + 2]), __uint_as_float(r[v * 8 + 3]));
+                pk.z = pack_bf16(__uint_as_float(r[v * 8 + 4]), __uint_as_float(r[v * 8 + 5]));
+                pk.w = pack_bf16(__uint_as_float(r[v * 8 + 6]), __uint_as_float(r[v * 8 + 7]));
+                *reinterpret_cast<uint4*>(o + v * 8) = pk;
               }
             }
           }
@@ -303,6 +432,9 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_acc_empty + 8 * acc);
+    }
+    if constexpr (kEpi == kEpiResidual) {
+      if (lane == 0) bulk_wait<0>();  // all reduce-adds of this warp have completed
     }
   }
 
@@ -361,8 +493,22 @@ int gemm_tc_sm_count() {
   return sms;
 }
 
+cudaError_t make_tma_2d_f32_box32(TmaDesc* out, const void* base, uint64_t rows, uint64_t cols) {
+  EncodeTiledFn enc = get_encode();
+  if (!enc) return cudaErrorNotSupported;
+  if ((reinterpret_cast<uintptr_t>(base) & 15) || (cols * 4) % 16) return cudaErrorInvalidValue;
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {cols * 4};
+  cuuint32_t box[2] = {32, 32};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = enc(reinterpret_cast<CUtensorMap*>(out), CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base),
+                   dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                   CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
 cudaError_t launch_gemm_tc(const TmaDesc& a, const TmaDesc& b0, const TmaDesc& b1, void* out, float* resid, int m,
-                           int n, int k, int epilogue, int* err, cudaStream_t st) {
+                           int n, int k, int epilogue, const QkvRopeArgs* qa, int* err, cudaStream_t st) {
   if (m <= 0 || n <= 0) return cudaSuccess;
   if (k <= 0 || (k % 8) || (n % 8)) return cudaErrorInvalidValue;
   static bool attr = false;
@@ -370,7 +516,8 @@ cudaError_t launch_gemm_tc(const TmaDesc& a, const TmaDesc& b0, const TmaDesc& b
     cudaError_t e;
     if ((e = cudaFuncSetAttribute(k_gemm_tc<kEpiStore>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes)) ||
         (e = cudaFuncSetAttribute(k_gemm_tc<kEpiResidual>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes)) ||
-        (e = cudaFuncSetAttribute(k_gemm_tc<kEpiSwiGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes)))
+        (e = cudaFuncSetAttribute(k_gemm_tc<kEpiSwiGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes)) ||
+        (e = cudaFuncSetAttribute(k_gemm_tc<kEpiQkvRope>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes)))
       return e;
     attr = true;
   }
@@ -381,12 +528,29 @@ cudaError_t launch_gemm_tc(const TmaDesc& a, const TmaDesc& b0, const TmaDesc& b
   const CUtensorMap& ma = reinterpret_cast<const CUtensorMap&>(a);
   const CUtensorMap& mb0 = reinterpret_cast<const CUtensorMap&>(b0);
   const CUtensorMap& mb1 = reinterpret_cast<const CUtensorMap&>(b1);
+  TmaDesc rdesc = a;  // placeholder for the epilogues that do not use it
+  QkvRopeArgs q{};
+  if (epilogue == kEpiResidual) {
+    // the residual rows of this launch, exactly m of them, so that the TMA unit clips the ragged last tile
+    cudaError_t e = make_tma_2d_f32_box32(&rdesc, resid, (uint64_t)m, (uint64_t)n);
+    if (e != cudaSuccess) return e;
+  }
+  if (epilogue == kEpiQkvRope) {
+    if (!qa || n % 128) return cudaErrorInvalidValue;
+    q = *qa;
+  }
+  const CUtensorMap& mr = reinterpret_cast<const CUtensorMap&>(rdesc);
+  __nv_bfloat16* o = (__nv_bfloat16*)out;
   if (epilogue == kEpiStore)
-    k_gemm_tc<kEpiStore><<<grid, kThreads, kSmemBytes, st>>>(ma, mb0, mb1, (__nv_bfloat16*)out, resid, m, n, k, err);
+    k_gemm_tc<kEpiStore><<<grid, kThreads, kSmemBytes, st>>>(ma, mb0, mb1, mr, o, m, n, k, q, err);
   else if (epilogue == kEpiResidual)
-    k_gemm_tc<kEpiResidual><<<grid, kThreads, kSmemBytes, st>>>(ma, mb0, mb1, (__nv_bfloat16*)out, resid, m, n, k, err);
+    k_gemm_tc<kEpiResidual><<<grid, kThreads, kSmemBytes, st>>>(ma, mb0, mb1, mr, o, m, n, k, q, err);
+  else if (epilogue == kEpiSwiGLU)
+    k_gemm_tc<kEpiSwiGLU><<<grid, kThreads, kSmemBytes, st>>>(ma, mb0, mb1, mr, o, m, n, k, q, err);
+  else if (epilogue == kEpiQkvRope)
+    k_gemm_tc<kEpiQkvRope><<<grid, kThreads, kSmemBytes, st>>>(ma, mb0, mb1, mr, o, m, n, k, q, err);
   else
-    k_gemm_tc<kEpiSwiGLU><<<grid, kThreads, kSmemBytes, st>>>(ma, mb0, mb1, (__nv_bfloat16*)out, resid, m, n, k, err);
+    return cudaErrorInvalidValue;
   return cudaGetLastError();
 }
 

@@ -66,10 +66,31 @@ int prism_op_gemm(const void* a, const void* b, const void* b2, void* out, float
     cudaError_t e = make_tma_2d_bf16(&ma, a, (uint64_t)m, (uint64_t)k, 128, 64);
     if (e == cudaSuccess) e = make_tma_2d_bf16(&mb0, b, (uint64_t)n, (uint64_t)k, 128, 64);
     if (e == cudaSuccess) e = make_tma_2d_bf16(&mb1, epilogue == kEpiSwiGLU ? b2 : b, (uint64_t)n, (uint64_t)k, 128, 64);
-    if (e == cudaSuccess) e = launch_gemm_tc(ma, mb0, mb1, out, resid, m, n, k, epilogue, err_word, S(stream));
+    if (e == cudaSuccess) e = launch_gemm_tc(ma, mb0, mb1, out, resid, m, n, k, epilogue, nullptr, err_word, S(stream));
     return st_of(e);
   }
   return st_of(launch_gemm_simt(a, b, b2, out, resid, m, n, k, dtype, epilogue, S(stream)));
+}
+
+int prism_op_gemm_qkv_rope(const void* a, const void* w_qkv, void* out, int32_t m, int32_t k, int32_t n_q_heads,
+                           int32_t n_kv_heads, int32_t qk_norm, const void* g_q, const void* g_k, float eps,
+                           const int32_t* pos, float theta, int32_t max_pos, int32_t* err_word, void* stream) {
+  if (!a || !w_qkv || !out || !pos || !err_word || m < 0 || k < 1 || (k % 8) || max_pos < 1) return PRISM_ERR_INVALID_ARG;
+  if (qk_norm && (!g_q || !g_k)) return PRISM_ERR_INVALID_ARG;
+  const int n = (n_q_heads + 2 * n_kv_heads) * 128;
+  float* tab = nullptr;
+  cudaError_t e = cudaMalloc(&tab, 2 * (size_t)max_pos * 64 * sizeof(float));
+  if (e != cudaSuccess) return st_of(e);
+  e = launch_rope_table(tab, tab + (size_t)max_pos * 64, max_pos, 128, theta, S(stream));
+  TmaDesc ma, mb;
+  if (e == cudaSuccess) e = make_tma_2d_bf16(&ma, a, (uint64_t)m, (uint64_t)k, 128, 64);
+  if (e == cudaSuccess) e = make_tma_2d_bf16(&mb, w_qkv, (uint64_t)n, (uint64_t)k, 128, 64);
+  QkvRopeArgs qa{pos, tab, tab + (size_t)max_pos * 64, (const __nv_bfloat16*)g_q, (const __nv_bfloat16*)g_k,
+                 n_q_heads, n_kv_heads, qk_norm, eps};
+  if (e == cudaSuccess) e = launch_gemm_tc(ma, mb, mb, out, nullptr, m, n, k, kEpiQkvRope, &qa, err_word, S(stream));
+  cudaStreamSynchronize(S(stream));
+  cudaFree(tab);
+  return st_of(e);
 }
 
 int prism_op_attention(const void* qkv, void* out, const int32_t* cu, int32_t n_seq, int32_t max_len,

@@ -490,12 +490,19 @@ int run_layer_chunk(prism_handle* h, const LayerDev& W, const LayerMaps* maps, f
     attn_flops += (c.causal ? 2.0 : 4.0) * L * L * c.n_q_heads * dh;
   }
   PRISM_LAUNCH_P(h, st, PRISM_K_RMSNORM, norm_bytes, launch_rmsnorm(xr, W.g_attn, c.dtype, rows, D, c.rms_eps, h->a_norm, st));
-  if (h->tc)
+  const bool fused_rope = h->tc && dh == 128;  // QK-norm + RoPE inside the QKV GEMM's epilogue
+  if (fused_rope) {
+    QkvRopeArgs qa{h->pos + r0, h->rope_cos, h->rope_sin, (const __nv_bfloat16*)W.g_q, (const __nv_bfloat16*)W.g_k,
+                   c.n_q_heads, c.n_kv_heads, c.qk_norm, c.rms_eps};
     PRISM_LAUNCH_P(h, st, PRISM_K_GEMM_QKV, 2.0 * R * nqkv * D,
-                   launch_gemm_tc(h->map_a_norm, maps->qkv, maps->qkv, h->qkv, nullptr, rows, nqkv, D, kEpiStore, h->errword, st));
+                   launch_gemm_tc(h->map_a_norm, maps->qkv, maps->qkv, h->qkv, nullptr, rows, nqkv, D, kEpiQkvRope, &qa, h->errword, st));
+  } else if (h->tc)
+    PRISM_LAUNCH_P(h, st, PRISM_K_GEMM_QKV, 2.0 * R * nqkv * D,
+                   launch_gemm_tc(h->map_a_norm, maps->qkv, maps->qkv, h->qkv, nullptr, rows, nqkv, D, kEpiStore, nullptr, h->errword, st));
   else
     PRISM_LAUNCH_P(h, st, PRISM_K_GEMM_QKV, 2.0 * R * nqkv * D,
                    launch_gemm_simt(h->a_norm, W.w_qkv, nullptr, h->qkv, nullptr, rows, nqkv, D, c.dtype, kEpiStore, st));
+  if (!fused_rope)
   PRISM_LAUNCH_P(h, st, PRISM_K_ROPE, 2.0 * R * (c.n_q_heads + c.n_kv_heads) * dh * esz,
                  launch_qknorm_rope(h->qkv, c.dtype, h->pos + r0, rows, c.n_q_heads, c.n_kv_heads, dh, c.qk_norm, W.g_q, W.g_k,
                                     c.rms_eps, h->rope_cos, h->rope_sin, st));
@@ -508,20 +515,20 @@ int run_layer_chunk(prism_handle* h, const LayerDev& W, const LayerMaps* maps, f
                                          c.causal, c.dtype, st));
   if (h->tc)
     PRISM_LAUNCH_P(h, st, PRISM_K_GEMM_O, 2.0 * R * D * hd,
-                   launch_gemm_tc(h->map_attn, maps->o, maps->o, nullptr, xr, rows, D, hd, kEpiResidual, h->errword, st));
+                   launch_gemm_tc(h->map_attn, maps->o, maps->o, nullptr, xr, rows, D, hd, kEpiResidual, nullptr, h->errword, st));
   else
     PRISM_LAUNCH_P(h, st, PRISM_K_GEMM_O, 2.0 * R * D * hd,
                    launch_gemm_simt(h->attn, W.w_o, nullptr, nullptr, xr, rows, D, hd, c.dtype, kEpiResidual, st));
   PRISM_LAUNCH_P(h, st, PRISM_K_RMSNORM, norm_bytes, launch_rmsnorm(xr, W.g_ffn, c.dtype, rows, D, c.rms_eps, h->a_norm, st));
   if (h->tc)
     PRISM_LAUNCH_P(h, st, PRISM_K_GEMM_GATEUP, 4.0 * R * c.ffn * D,
-                   launch_gemm_tc(h->map_a_norm, maps->gate, maps->up, h->hbuf, nullptr, rows, c.ffn, D, kEpiSwiGLU, h->errword, st));
+                   launch_gemm_tc(h->map_a_norm, maps->gate, maps->up, h->hbuf, nullptr, rows, c.ffn, D, kEpiSwiGLU, nullptr, h->errword, st));
   else
     PRISM_LAUNCH_P(h, st, PRISM_K_GEMM_GATEUP, 4.0 * R * c.ffn * D,
                    launch_gemm_simt(h->a_norm, W.w_gate, W.w_up, h->hbuf, nullptr, rows, c.ffn, D, c.dtype, kEpiSwiGLU, st));
   if (h->tc)
     PRISM_LAUNCH_P(h, st, PRISM_K_GEMM_DOWN, 2.0 * R * D * c.ffn,
-                   launch_gemm_tc(h->map_hbuf, maps->down, maps->down, nullptr, xr, rows, D, c.ffn, kEpiResidual, h->errword, st));
+                   launch_gemm_tc(h->map_hbuf, maps->down, maps->down, nullptr, xr, rows, D, c.ffn, kEpiResidual, nullptr, h->errword, st));
   else
     PRISM_LAUNCH_P(h, st, PRISM_K_GEMM_DOWN, 2.0 * R * D * c.ffn,
                    launch_gemm_simt(h->hbuf, W.w_down, nullptr, nullptr, xr, rows, D, c.ffn, c.dtype, kEpiResidual, st));

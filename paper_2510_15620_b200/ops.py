@@ -21,6 +21,8 @@ def _L():
         L.prism_op_rmsnorm.argtypes = [vp, vp, i32, i32, i32, f32, vp, vp]
         L.prism_op_qknorm_rope.argtypes = [vp, i32, vp, i32, i32, i32, i32, i32, vp, vp, f32, f32, i32, vp]
         L.prism_op_gemm.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, vp, vp]
+        L.prism_op_gemm_qkv_rope.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, vp, vp, f32, vp, f32, i32, vp, vp]
+        L.prism_op_gemm_qkv_rope.restype = C.c_int
         L.prism_op_attention.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, i32, vp]
         L.prism_op_probe.argtypes = [vp, vp, i32, i32, vp, vp, i32, f32, vp, vp]
         L.prism_op_route.argtypes = [vp, vp, vp, i32, i32, i32, f64, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
@@ -67,6 +69,11 @@ def prism_op_qknorm_rope(qkv, dtype, pos, n_q_heads, n_kv_heads, head_dim, qk_no
 def prism_op_gemm(a, b, b2, out, resid, m, n, k, dtype, epilogue, impl, err_word):
     _check(_L().prism_op_gemm(_p(a), _p(b), _p(b2), _p(out), _p(resid), m, n, k, dtype, epilogue, impl, _p(err_word),
                               _stream()), "gemm")
+
+
+def prism_op_gemm_qkv_rope(a, w_qkv, out, m, k, n_q_heads, n_kv_heads, qk_norm, g_q, g_k, eps, pos, theta, max_pos, err_word):
+    _check(_L().prism_op_gemm_qkv_rope(_p(a), _p(w_qkv), _p(out), m, k, n_q_heads, n_kv_heads, qk_norm, _p(g_q), _p(g_k),
+                                       eps, _p(pos), theta, max_pos, _p(err_word), _stream()), "gemm_qkv_rope")
 
 
 def prism_op_attention(qkv, out, cu, n_seq, max_len, n_q_heads, n_kv_heads, head_dim, causal, dtype, impl):

@@ -185,6 +185,35 @@ def test_gemm_bf16(P, m, n, k, epi, impl):
     assert np.max(np.abs(got - ref)) < tol, np.max(np.abs(got - ref))
 
 
+@pytest.mark.parametrize("qk_norm", [1, 0])
+@pytest.mark.parametrize("m,k,hq,hkv", [(300, 320, 2, 1), (1000, 1024, 16, 8), (4100, 256, 3, 1)])
+def test_gemm_qkv_with_fused_qknorm_rope(P, m, k, hq, hkv, qk_norm):
+    """QKV projection whose epilogue applies QK-norm and the rotary embedding, vs the oracle's
+    rmsnorm/rope_rotate on an fp64 product."""
+    rng = np.random.default_rng(m + k + qk_norm)
+    dh, theta = 128, 1e6
+    n = (hq + 2 * hkv) * dh
+    a = round_to_bf16(rng.normal(size=(m, k)).astype(np.float32))
+    w = round_to_bf16((rng.normal(size=(n, k)) * 0.05).astype(np.float32))
+    gq = round_to_bf16((1 + 0.1 * rng.normal(size=dh)).astype(np.float32))
+    gk = round_to_bf16((1 + 0.1 * rng.normal(size=dh)).astype(np.float32))
+    pos = rng.integers(0, 700, size=m).astype(np.int32)
+    out = torch.zeros(m, n, dtype=torch.bfloat16, device="cuda")
+    err = torch.zeros(1, dtype=torch.int32, device="cuda")
+    P.ops.prism_op_gemm_qkv_rope(bf(a), bf(w), out, m, k, hq, hkv, qk_norm, bf(gq), bf(gk), 1e-6, dev(pos), theta, 700, err)
+    torch.cuda.synchronize()
+    assert int(err.item()) == 0
+    c = a.astype(np.float64) @ w.astype(np.float64).T
+    q = c[:, : hq * dh].reshape(m, hq, dh)
+    kk = c[:, hq * dh:(hq + hkv) * dh].reshape(m, hkv, dh)
+    if qk_norm:
+        q, kk = oracle.rmsnorm(q, gq.astype(np.float64), 1e-6), oracle.rmsnorm(kk, gk.astype(np.float64), 1e-6)
+    q, kk = oracle.rope_rotate(q, pos, theta), oracle.rope_rotate(kk, pos, theta)
+    ref = np.concatenate([q.reshape(m, -1), kk.reshape(m, -1), c[:, (hq + hkv) * dh:]], axis=1)
+    got = out.float().cpu().numpy()
+    assert np.max(np.abs(got - ref)) < (2.0 ** -8) * np.max(np.abs(ref)) + 1e-3
+
+
 def test_gemm_tc_rows_do_not_depend_on_their_position(P):
     """Duplicate rows anywhere in the batch, and the same row in a smaller batch, give identical bits
     (exact score ties between duplicated candidates rely on this)."""
