@@ -54,8 +54,9 @@ typedef enum {
 enum { PRISM_FP32 = 0, PRISM_BF16 = 1 };
 enum { PRISM_WEIGHTS_DEVICE = 0, PRISM_WEIGHTS_HOST_STREAMED = 1 };
 enum { PRISM_PRUNE_NONE = 0, PRISM_PRUNE_FIXED_KEEP = 1, PRISM_PRUNE_CLUSTER = 2 };
-/* Implementation selectors (debug/validation): AUTO picks the tensor-core kernels in bf16 mode. */
-enum { PRISM_IMPL_AUTO = 0, PRISM_IMPL_SIMT = 1 };
+/* Implementation selectors (validation): AUTO picks the tcgen05 tensor-core kernels in bf16 mode,
+ * SIMT the CUDA-core kernels, MMA (attention only) the warp-level mma.sync flash-attention kernel. */
+enum { PRISM_IMPL_AUTO = 0, PRISM_IMPL_SIMT = 1, PRISM_IMPL_MMA = 2 };
 
 typedef struct prism_handle prism_handle;
 

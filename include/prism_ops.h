@@ -64,10 +64,12 @@ PRISM_API int prism_op_gemm_qkv_rope(const void* a, const void* w_qkv, void* out
 
 /* Attention over packed sequences: for sequence s (rows cu[s]..cu[s+1]) and query head h (kv head
  * h / (Hq/Hkv)): out = softmax(q k^T / sqrt(head_dim) [+ causal mask]) v.  qkv [total, (Hq+2Hkv)*dh],
- * out [total, Hq*dh].  max_len >= the longest sequence. */
-PRISM_API int prism_op_attention(const void* qkv, void* out, const int32_t* cu, int32_t n_seq, int32_t max_len,
-                       int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim, int32_t causal, int32_t dtype,
-                       int32_t impl, void* stream);
+ * out [total, Hq*dh].  total = cu[n_seq] rows; max_len >= the longest sequence.  impl: PRISM_IMPL_AUTO =
+ * tcgen05 kernel (bf16, head_dim 128; reports an expired bounded wait in err_word bit 4),
+ * PRISM_IMPL_MMA = warp-level MMA kernel (bf16, head_dim 128), PRISM_IMPL_SIMT = CUDA cores. */
+PRISM_API int prism_op_attention(const void* qkv, void* out, const int32_t* cu, int32_t n_seq, int32_t total,
+                                 int32_t max_len, int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim,
+                                 int32_t causal, int32_t dtype, int32_t impl, int32_t* err_word, void* stream);
 
 /* Score probe (Sec. 4.1: the model's classifier on an intermediate hidden state): for each sequence,
  * final RMSNorm of its last row, then logit(score_head row 0) - logit(score_head row 1).

@@ -10,7 +10,7 @@ import numpy as np
 import torch
 
 PRISM_FP32, PRISM_BF16 = 0, 1
-PRISM_IMPL_AUTO, PRISM_IMPL_SIMT = 0, 1
+PRISM_IMPL_AUTO, PRISM_IMPL_SIMT, PRISM_IMPL_MMA = 0, 1, 2
 PRISM_MAX_CLUSTERS = 8
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "lib", "libprism.so")

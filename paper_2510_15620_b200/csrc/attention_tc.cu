@@ -1,0 +1,373 @@
+// S5 on the 5th-generation tensor cores: varlen flash attention over packed sequences, bf16,
+// head_dim 128, GQA, causal or bidirectional.
+//
+// One CTA = 128 query rows of one (sequence, head); two CTAs fit on an SM.  Warp-specialised:
+//   warp 0      TMA producer: Q once, then (K_j, V_j) tiles of 64 keys into a 2-stage ring
+//   warp 1      MMA issuer:   S_j = Q K_j^T (tcgen05.mma M128 N64 K16 x 8) into one of two TMEM buffers,
+//                             O += P_j V_j  (M128 N128 K16 x 4, V as an MN-major operand) into TMEM
+//   warps 2..5  softmax: one query row per thread; read S_j from TMEM, exponentiate against a running
+//               reference maximum, write P_j (bf16, 128-byte swizzle) over the K_j tile, which the
+//               tensor core has finished with; O stays in TMEM and is rescaled (TMEM read-modify-write)
+//               only when a row's maximum outgrows the reference by more than 2^8.
+// S_{j+1} is issued before P_j is awaited, so the tensor core computes the next scores while the
+// softmax warps work.  Every mbarrier wait is bounded; on expiry the kernel records kErrTimeout, all
+// roles drain to the common exit and the tensor memory is freed.  No cluster multicast.
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace prism {
+
+namespace {
+
+constexpr int BM = 128, BN = 64, DH = 128;
+constexpr int kQBytes = BM * DH * 2;          // 32 KB: two [128 x 64] swizzled sub-tiles
+constexpr int kKBytes = BN * DH * 2;          // 16 KB: two [64 x 64] sub-tiles; later holds P_j [128 x 64]
+constexpr int kVBytes = BN * DH * 2;          // 16 KB: two [64 keys x 64 dh] sub-tiles
+constexpr int kStageBytes = kKBytes + kVBytes;
+constexpr int kSmemBytes = kQBytes + 2 * kStageBytes + 1024 + 128;
+constexpr int kThreads = 192;
+constexpr int kTmemCols = 256;                // S: 2 x 64, O: 128
+constexpr unsigned long long kWaitCycles = 4000000000ull;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* err, volatile int* abort_flag) {
+  if (mbar_try(bar, parity)) return true;
+  const unsigned long long t0 = clock64();
+  uint32_t it = 0;
+  while (!mbar_try(bar, parity)) {
+    if ((++it & 0x3ff) == 0) {
+      if (*abort_flag || clock64() - t0 > kWaitCycles) {
+        *abort_flag = 1;
+        atomicOr(err, kErrTimeout);
+        return false;
+      }
+    }
+  }
+  return true;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(acc) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+        "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+        "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor, 128-byte swizzle.  lbo/sbo in bytes.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint32_t sbo) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr >> 4) & 0x3fff);
+  d |= (uint64_t)((lbo >> 4) & 0x3fff) << 16;
+  d |= (uint64_t)((sbo >> 4) & 0x3fff) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
+}
+// kind::f16 instruction descriptors: D fp32, A/B bf16, M = 128.
+__host__ __device__ constexpr uint32_t idesc(int n, int b_mn_major) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)b_mn_major << 16) | ((uint32_t)(n >> 3) << 17) |
+         ((uint32_t)(BM >> 4) << 24);
+}
+__device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+__global__ void __launch_bounds__(kThreads, 2)
+k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_kv,
+               __nv_bfloat16* __restrict__ out, const int* __restrict__ cu, int seq0, int row0, int hq, int hkv,
+               int causal, float scale_log2, int* __restrict__ err) {
+  extern __shared__ unsigned char smem_raw[];
+  const int s = seq0 + blockIdx.z;
+  const int beg = cu[s] - row0, len = cu[s + 1] - cu[s];
+  const int qb = (int)gridDim.x - 1 - (int)blockIdx.x;  // heaviest query blocks first
+  if (qb * BM >= len) return;
+  const int h = blockIdx.y, kvh = h / (hq / hkv);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  unsigned char* gen = smem_raw + (base - raw);
+  const uint32_t s_q = base, s_stage = base + kQBytes;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(gen + kQBytes + 2 * kStageBytes);
+  const uint32_t b_q = smem_u32(bars), b_kv_full = smem_u32(bars + 1), b_kv_empty = smem_u32(bars + 3);
+  const uint32_t b_s_full = smem_u32(bars + 5), b_s_empty = smem_u32(bars + 7);
+  const uint32_t b_p_full = smem_u32(bars + 9), b_o_full = smem_u32(bars + 10);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 11);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int kv_end = causal ? min(len, (qb + 1) * BM) : len;
+  const int n_blocks = (kv_end + BN - 1) / BN;
+
+  if (threadIdx.x == 0) {
+    mbar_init(b_q, 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(b_kv_full + 8 * i, 1);
+      mbar_init(b_kv_empty + 8 * i, 1);
+      mbar_init(b_s_full + 8 * i, 1);
+      mbar_init(b_s_empty + 8 * i, 128);
+    }
+    mbar_init(b_p_full, 128);
+    mbar_init(b_o_full, 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols));
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::);
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+  const uint32_t t_s = tmem, t_o = tmem + 2 * BN;  // columns [0,128): S buffers, [128,256): O
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      mbar_expect_tx(b_q, kQBytes);
+      tma_load_2d(s_q, &map_q, h * DH, beg + qb * BM, b_q);
+      tma_load_2d(s_q + kQBytes / 2, &map_q, h * DH + 64, beg + qb * BM, b_q);
+      const int kcol = (hq + kvh) * DH, vcol = (hq + hkv + kvh) * DH;
+      for (int j = 0; j < n_blocks; ++j) {
+        const int st = j & 1, u = j >> 1;
+        if (!mbar_wait(b_kv_empty + 8 * st, (u & 1) ^ 1, err, abort_flag)) break;
+        const uint32_t sk = s_stage + st * kStageBytes, sv = sk + kKBytes;
+        mbar_expect_tx(b_kv_full + 8 * st, kStageBytes);
+        tma_load_2d(sk, &map_kv, kcol, beg + j * BN, b_kv_full + 8 * st);
+        tma_load_2d(sk + kKBytes / 2, &map_kv, kcol + 64, beg + j * BN, b_kv_full + 8 * st);
+        tma_load_2d(sv, &map_kv, vcol, beg + j * BN, b_kv_full + 8 * st);
+        tma_load_2d(sv + kVBytes / 2, &map_kv, vcol + 64, beg + j * BN, b_kv_full + 8 * st);
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t kIdescS = idesc(BN, 0), kIdescO = idesc(DH, 1);
+      bool ok = mbar_wait(b_q, 0, err, abort_flag);
+      auto issue_qk = [&](int j) {
+        const int st = j & 1;
+        const uint32_t sk = s_stage + st * kStageBytes;
+        tc_fence_after();
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk) {  // 16 head-dim elements per step; sub-tile switches at kk = 4
+          const uint64_t da = smem_desc(s_q + (kk >> 2) * (kQBytes / 2) + (kk & 3) * 32, 16, 1024);
+          const uint64_t db = smem_desc(sk + (kk >> 2) * (kKBytes / 2) + (kk & 3) * 32, 16, 1024);
+          umma_bf16(t_s + st * BN, da, db, kIdescS, kk != 0);
+        }
+        umma_commit(b_s_full + 8 * st);
+      };
+      if (ok) ok = mbar_wait(b_kv_full, 0, err, abort_flag);
+      if (ok) issue_qk(0);
+      for (int j = 0; j < n_blocks && ok; ++j) {
+        if (j + 1 < n_blocks) {
+          const int b = (j + 1) & 1, u = (j + 1) >> 1;
+          if (!mbar_wait(b_kv_full + 8 * b, u & 1, err, abort_flag)) { ok = false; break; }
+          if (!mbar_wait(b_s_empty + 8 * b, (u & 1) ^ 1, err, abort_flag)) { ok = false; break; }
+          issue_qk(j + 1);
+        }
+        if (!mbar_wait(b_p_full, j & 1, err, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const int st = j & 1;
+        const uint32_t sp = s_stage + st * kStageBytes, sv = sp + kKBytes;
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk) {  // 16 keys per step
+          const uint64_t da = smem_desc(sp + kk * 32, 16, 1024);               // P: K-major, one 64-key atom
+          const uint64_t db = smem_desc(sv + kk * 2048, kVBytes / 2, 1024);    // V: MN-major, two 64-wide dh atoms
+          umma_bf16(t_o, da, db, kIdescO, (j | kk) != 0);
+        }
+        umma_commit(b_o_full);
+        umma_commit(b_kv_empty + 8 * st);
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ softmax + output (128 rows)
+    const int quarter = warp & 3;
+    const int r = quarter * 32 + lane;             // row inside the tile = TMEM lane
+    const int qrow = qb * BM + r;                  // row inside the sequence
+    const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
+    float m_ref = 0.f, l = 0.f;                    // reference maximum (raw score units), running sum
+    bool ok = true;
+    for (int j = 0; j < n_blocks; ++j) {
+      const int b = j & 1, u = j >> 1;
+      // Parity waits are only meaningful one phase at a time: observe every completion of O += P V in
+      // order (PV(j-2) finished long ago, so this costs nothing) before a later wait may target PV(j-1).
+      if (j >= 2 && !mbar_wait(b_o_full, (j - 2) & 1, err, abort_flag)) { ok = false; break; }
+      if (!mbar_wait(b_s_full + 8 * b, u & 1, err, abort_flag)) { ok = false; break; }
+      tc_fence_after();
+      uint32_t sr[64];
+      tmem_ld32(t_s + lane_base + b * BN, sr);
+      tmem_ld32(t_s + lane_base + b * BN + 32, sr + 32);
+      tmem_ld_wait();
+      tc_fence_before();
+      mbar_arrive(b_s_empty + 8 * b);
+      const int key0 = j * BN;
+      if ((causal && key0 + BN - 1 > qb * BM) || key0 + BN > len) {
+#pragma unroll
+        for (int c = 0; c < 64; ++c) {
+          const int key = key0 + c;
+          if (key >= len || (causal && key > qrow)) sr[c] = 0xff800000u;  // -inf
+        }
+      }
+      float bm = -INFINITY;
+#pragma unroll
+      for (int c = 0; c < 64; ++c) bm = fmaxf(bm, __uint_as_float(sr[c]));
+      if (j == 0) {
+        m_ref = (bm == -INFINITY) ? 0.f : bm;
+      } else {
+        // Rescale O only when this row's maximum outgrew the reference by more than 2^8 (rare).
+        const bool need = (bm - m_ref) * scale_log2 > 8.f;
+        if (__any_sync(0xffffffffu, need)) {
+          if (!mbar_wait(b_o_full, (j - 1) & 1, err, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const float m_new = need ? bm : m_ref;
+          const float f = exp2f((m_ref - m_new) * scale_log2);
+#pragma unroll 1
+          for (int c = 0; c < 4; ++c) {
+            uint32_t o[32];
+            tmem_ld32(t_o + lane_base + c * 32, o);
+            tmem_ld_wait();
+#pragma unroll
+            for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * f);
+            tmem_st32(t_o + lane_base + c * 32, o);
+          }
+          tmem_st_wait();
+          l *= f;
+          m_ref = m_new;
+        }
+      }
+      const float ms = m_ref * scale_log2;
+      const uint32_t sp = s_stage + b * kStageBytes;  // P_j overwrites K_j (its MMAs have completed)
+      float rs = 0.f;
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        float p[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          p[e] = exp2f(__uint_as_float(sr[c * 8 + e]) * scale_log2 - ms);
+          rs += p[e];
+        }
+        const uint32_t dst = sp + r * 128 + ((c ^ (r & 7)) << 4);
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(pack_bf16(p[0], p[1])),
+                     "r"(pack_bf16(p[2], p[3])), "r"(pack_bf16(p[4], p[5])), "r"(pack_bf16(p[6], p[7])) : "memory");
+      }
+      l += rs;
+      fence_async_smem();
+      tc_fence_before();
+      // A warp that runs ahead must not let its arrival for block j be counted in block j-1's phase.
+      if (j > 0 && !mbar_wait(b_p_full, (j - 1) & 1, err, abort_flag)) { ok = false; break; }
+      mbar_arrive(b_p_full);
+    }
+    if (ok && n_blocks >= 2) ok = mbar_wait(b_o_full, (n_blocks - 2) & 1, err, abort_flag);
+    if (ok && mbar_wait(b_o_full, (n_blocks - 1) & 1, err, abort_flag)) {
+      tc_fence_after();
+      const float inv = 1.f / l;
+      __nv_bfloat16* orow = out + (size_t)(beg + qrow) * ((size_t)hq * DH) + (size_t)h * DH;
+#pragma unroll 1
+      for (int c = 0; c < 4; ++c) {
+        uint32_t o[32];
+        tmem_ld32(t_o + lane_base + c * 32, o);
+        tmem_ld_wait();
+        if (qrow < len) {
+#pragma unroll
+          for (int v = 0; v < 4; ++v) {
+            uint4 pk;
+            pk.x = pack_bf16(__uint_as_float(o[v * 8 + 0]) * inv, __uint_as_float(o[v * 8 + 1]) * inv);
+            pk.y = pack_bf16(__uint_as_float(o[v * 8 + 2]) * inv, __uint_as_float(o[v * 8 + 3]) * inv);
+            pk.z = pack_bf16(__uint_as_float(o[v * 8 + 4]) * inv, __uint_as_float(o[v * 8 + 5]) * inv);
+            pk.w = pack_bf16(__uint_as_float(o[v * 8 + 6]) * inv, __uint_as_float(o[v * 8 + 7]) * inv);
+            *reinterpret_cast<uint4*>(orow + c * 32 + v * 8) = pk;
+          }
+        }
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols));
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_attention_tc(const void* qkv, void* out, const int* cu, int seq0, int nseq, int row0, int rows,
+                                int max_len, int n_q_heads, int n_kv_heads, int causal, int* err, cudaStream_t st) {
+  if (nseq <= 0 || max_len <= 0 || rows <= 0) return cudaSuccess;
+  static bool attr = false;
+  if (!attr) {
+    cudaError_t e = cudaFuncSetAttribute(k_attention_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (e != cudaSuccess) return e;
+    attr = true;
+  }
+  // Exactly `rows` rows are described, so tiles that run past the batch read zeros, never stale memory.
+  const uint64_t ld = (uint64_t)(n_q_heads + 2 * n_kv_heads) * DH;
+  TmaDesc mq, mkv;
+  cudaError_t e = make_tma_2d_bf16(&mq, qkv, (uint64_t)rows, ld, BM, 64);
+  if (e == cudaSuccess) e = make_tma_2d_bf16(&mkv, qkv, (uint64_t)rows, ld, BN, 64);
+  if (e != cudaSuccess) return e;
+  dim3 grid((max_len + BM - 1) / BM, n_q_heads, nseq);
+  const float scale_log2 = 1.4426950408889634f / sqrtf((float)DH);
+  k_attention_tc<<<grid, kThreads, kSmemBytes, st>>>(reinterpret_cast<const CUtensorMap&>(mq),
+                                                     reinterpret_cast<const CUtensorMap&>(mkv), (__nv_bfloat16*)out, cu,
+                                                     seq0, row0, n_q_heads, n_kv_heads, causal, scale_log2, err);
+  return cudaGetLastError();
+}
+
+}  // namespace prism

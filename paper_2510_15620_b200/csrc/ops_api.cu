@@ -93,12 +93,17 @@ int prism_op_gemm_qkv_rope(const void* a, const void* w_qkv, void* out, int32_t 
   return st_of(e);
 }
 
-int prism_op_attention(const void* qkv, void* out, const int32_t* cu, int32_t n_seq, int32_t max_len,
+int prism_op_attention(const void* qkv, void* out, const int32_t* cu, int32_t n_seq, int32_t total, int32_t max_len,
                        int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim, int32_t causal, int32_t dtype,
-                       int32_t impl, void* stream) {
-  if (!qkv || !out || !cu || n_seq < 0 || n_kv_heads < 1 || n_q_heads % n_kv_heads) return PRISM_ERR_INVALID_ARG;
-  if (dtype == PRISM_BF16 && impl == PRISM_IMPL_AUTO) {
+                       int32_t impl, int32_t* err_word, void* stream) {
+  if (!qkv || !out || !cu || n_seq < 0 || total < 0 || n_kv_heads < 1 || n_q_heads % n_kv_heads) return PRISM_ERR_INVALID_ARG;
+  if (dtype == PRISM_BF16 && impl != PRISM_IMPL_SIMT) {
     if (head_dim != 128) return PRISM_ERR_UNSUPPORTED;
+    if (impl == PRISM_IMPL_AUTO) {
+      if (!err_word) return PRISM_ERR_INVALID_ARG;
+      return st_of(launch_attention_tc(qkv, out, cu, 0, n_seq, 0, total, max_len, n_q_heads, n_kv_heads, causal, err_word,
+                                       S(stream)));
+    }
     return st_of(launch_attention_mma(qkv, out, cu, 0, n_seq, 0, max_len, n_q_heads, n_kv_heads, causal, S(stream)));
   }
   if (head_dim > 256) return PRISM_ERR_UNSUPPORTED;

@@ -35,7 +35,7 @@ struct prism_handle {
   int esz = 4;
   int chunk_tokens = 0;
   bool tc = false;  // tensor-core GEMM path
-  bool fa = false;  // tensor-core attention path
+  int fa = 0;       // attention path: 0 SIMT, 1 tcgen05, 2 warp-level MMA
 
   std::vector<void*> dev_allocs;
   std::vector<void*> host_allocs;
@@ -257,7 +257,7 @@ int validate_cfg(const prism_model_cfg& c, std::string* why) {
   if (c.dtype == PRISM_BF16) {
     if (c.hidden % 8 || c.ffn % 8 || c.head_dim % 8) return unsup("bf16 mode needs hidden, ffn, head_dim multiples of 8");
     if (c.gemm_impl == PRISM_IMPL_AUTO && (c.ffn % 128)) return unsup("tensor-core SwiGLU needs ffn multiple of 128");
-    if (c.attention_impl == PRISM_IMPL_AUTO && c.head_dim != 128) return unsup("tensor-core attention needs head_dim 128");
+    if (c.attention_impl != PRISM_IMPL_SIMT && c.head_dim != 128) return unsup("tensor-core attention needs head_dim 128");
   }
   return PRISM_OK;
 }
@@ -320,7 +320,7 @@ static int create_impl(prism_handle* h, const prism_model_cfg* cfg, const prism_
   h->cfg = c;
   h->esz = c.dtype == PRISM_BF16 ? 2 : 4;
   h->tc = c.dtype == PRISM_BF16 && c.gemm_impl == PRISM_IMPL_AUTO;
-  h->fa = c.dtype == PRISM_BF16 && c.attention_impl == PRISM_IMPL_AUTO;
+  h->fa = c.dtype != PRISM_BF16 ? 0 : (c.attention_impl == PRISM_IMPL_AUTO ? 1 : (c.attention_impl == PRISM_IMPL_MMA ? 2 : 0));
   const bool streamed = c.weight_residency == PRISM_WEIGHTS_HOST_STREAMED;
   if (!w->embed || !w->g_final || !w->score_head || !w->layers) return fail(h, PRISM_ERR_INVALID_ARG, "null weight pointer");
   h->embed = w->embed;
@@ -506,7 +506,11 @@ int run_layer_chunk(prism_handle* h, const LayerDev& W, const LayerMaps* maps, f
   PRISM_LAUNCH_P(h, st, PRISM_K_ROPE, 2.0 * R * (c.n_q_heads + c.n_kv_heads) * dh * esz,
                  launch_qknorm_rope(h->qkv, c.dtype, h->pos + r0, rows, c.n_q_heads, c.n_kv_heads, dh, c.qk_norm, W.g_q, W.g_k,
                                     c.rms_eps, h->rope_cos, h->rope_sin, st));
-  if (h->fa)
+  if (h->fa == 1)
+    PRISM_LAUNCH_P(h, st, PRISM_K_ATTENTION, attn_flops,
+                   launch_attention_tc(h->qkv, h->attn, cu_dev, s0, s1 - s0, r0, rows, max_len, c.n_q_heads, c.n_kv_heads, c.causal,
+                                       h->errword, st));
+  else if (h->fa == 2)
     PRISM_LAUNCH_P(h, st, PRISM_K_ATTENTION, attn_flops,
                    launch_attention_mma(h->qkv, h->attn, cu_dev, s0, s1 - s0, r0, max_len, c.n_q_heads, c.n_kv_heads, c.causal, st));
   else

@@ -80,7 +80,8 @@ def main():
         qkv = rnd(int(cu[-1]), (a.hq + 2 * a.hkv) * dh).to(torch.bfloat16)
         o = torch.empty(int(cu[-1]), a.hq * dh, dtype=torch.bfloat16, device=dev)
         cud = torch.from_numpy(cu).to(dev)
-        fn = lambda: ops.prism_op_attention(qkv, o, cud, a.seqs, int(lens.max()), a.hq, a.hkv, dh, a.causal, PRISM_BF16, a.impl)
+        err = torch.zeros(1, dtype=torch.int32, device=dev)
+        fn = lambda: ops.prism_op_attention(qkv, o, cud, a.seqs, int(lens.max()), a.hq, a.hkv, dh, a.causal, PRISM_BF16, a.impl, err)
         med, best = _time(fn, a.iters, a.warmup, flush)
         fl = float(np.sum((2.0 if a.causal else 4.0) * lens.astype(np.float64) ** 2 * a.hq * dh))
         out.update(seqs=a.seqs, tokens=int(cu[-1]), causal=a.causal, ms=med, ms_min=best, tflops=fl / med / 1e9)

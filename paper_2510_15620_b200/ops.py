@@ -23,7 +23,7 @@ def _L():
         L.prism_op_gemm.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, vp, vp]
         L.prism_op_gemm_qkv_rope.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, vp, vp, f32, vp, f32, i32, vp, vp]
         L.prism_op_gemm_qkv_rope.restype = C.c_int
-        L.prism_op_attention.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, i32, vp]
+        L.prism_op_attention.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, i32, i32, vp, vp]
         L.prism_op_probe.argtypes = [vp, vp, i32, i32, vp, vp, i32, f32, vp, vp]
         L.prism_op_route.argtypes = [vp, vp, vp, i32, i32, i32, f64, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
         L.prism_op_route_static.argtypes = L.prism_op_route.argtypes
@@ -76,9 +76,9 @@ def prism_op_gemm_qkv_rope(a, w_qkv, out, m, k, n_q_heads, n_kv_heads, qk_norm, 
                                        eps, _p(pos), theta, max_pos, _p(err_word), _stream()), "gemm_qkv_rope")
 
 
-def prism_op_attention(qkv, out, cu, n_seq, max_len, n_q_heads, n_kv_heads, head_dim, causal, dtype, impl):
-    _check(_L().prism_op_attention(_p(qkv), _p(out), _p(cu), n_seq, max_len, n_q_heads, n_kv_heads, head_dim, causal,
-                                   dtype, impl, _stream()), "attention")
+def prism_op_attention(qkv, out, cu, n_seq, max_len, n_q_heads, n_kv_heads, head_dim, causal, dtype, impl, err_word=None):
+    _check(_L().prism_op_attention(_p(qkv), _p(out), _p(cu), n_seq, qkv.shape[0], max_len, n_q_heads, n_kv_heads, head_dim,
+                                   causal, dtype, impl, _p(err_word), _stream()), "attention")
 
 
 def prism_op_probe(x, cu, n, g_final, score_head, dtype, eps, scores):

@@ -248,11 +248,11 @@ def _attn_ref(qkv, cu, hq, hkv, dh, causal):
 
 
 @pytest.mark.parametrize("causal", [1, 0])
-@pytest.mark.parametrize("dtype,impl,dh", [(FP32, SIMT, 64), (BF16, SIMT, 128), (BF16, AUTO, 128)])
+@pytest.mark.parametrize("dtype,impl,dh", [(FP32, SIMT, 64), (BF16, SIMT, 128), (BF16, AUTO, 128), (BF16, 2, 128)])
 def test_attention(P, dtype, impl, dh, causal):
     rng = np.random.default_rng(dh + causal)
     hq, hkv = 4, 2
-    lens = np.array([1, 7, 64, 65, 130, 200, 63, 128])      # below, at and across the 64-row tiles
+    lens = np.array([1, 7, 64, 65, 130, 200, 63, 128, 129, 300, 513])      # below, at and across the 64/128-row tiles
     cu = np.zeros(len(lens) + 1, np.int32)
     cu[1:] = np.cumsum(lens)
     qkv = rng.normal(size=(cu[-1], (hq + 2 * hkv) * dh)).astype(np.float32)
@@ -260,11 +260,38 @@ def test_attention(P, dtype, impl, dh, causal):
         qkv = round_to_bf16(qkv)
     tdt = torch.bfloat16 if dtype == BF16 else torch.float32
     out = torch.zeros(int(cu[-1]), hq * dh, dtype=tdt, device="cuda")
-    P.ops.prism_op_attention(dev(qkv, tdt), out, dev(cu), len(lens), int(lens.max()), hq, hkv, dh, causal, dtype, impl)
+    err = torch.zeros(1, dtype=torch.int32, device="cuda")
+    P.ops.prism_op_attention(dev(qkv, tdt), out, dev(cu), len(lens), int(lens.max()), hq, hkv, dh, causal, dtype, impl, err)
+    torch.cuda.synchronize()
+    assert int(err.item()) == 0
     ref = _attn_ref(qkv, cu, hq, hkv, dh, bool(causal))
     got = out.float().cpu().numpy()
     tol = 2e-2 if dtype == BF16 else 2e-5
     assert np.max(np.abs(got - ref)) < tol, np.max(np.abs(got - ref))
+
+
+def test_attention_tc_rescales_when_the_maximum_grows(P):
+    """Scores that keep growing along the keys force the running reference maximum to move by far more
+    than 2^8 between key blocks, so the in-TMEM rescale of O must run (and be right)."""
+    rng = np.random.default_rng(4)
+    hq, hkv, dh = 2, 1, 128
+    lens = np.array([400, 150])
+    cu = np.zeros(3, np.int32)
+    cu[1:] = np.cumsum(lens)
+    qkv = (rng.normal(size=(cu[-1], (hq + 2 * hkv) * dh)) * 0.5).astype(np.float32)
+    ramp = np.concatenate([np.arange(l) for l in lens])[:, None] * 0.02           # key norm grows with position
+    qkv[:, hq * dh:(hq + hkv) * dh] *= (1 + ramp * 3)
+    qkv[:, : hq * dh] = np.abs(qkv[:, : hq * dh]) * 2
+    qkv[:, hq * dh:(hq + hkv) * dh] = np.abs(qkv[:, hq * dh:(hq + hkv) * dh])
+    qkv = round_to_bf16(qkv)
+    out = torch.zeros(int(cu[-1]), hq * dh, dtype=torch.bfloat16, device="cuda")
+    err = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for causal in (1, 0):
+        P.ops.prism_op_attention(dev(qkv, torch.bfloat16), out, dev(cu), 2, 400, hq, hkv, dh, causal, BF16, AUTO, err)
+        torch.cuda.synchronize()
+        assert int(err.item()) == 0
+        ref = _attn_ref(qkv, cu, hq, hkv, dh, bool(causal))
+        assert np.max(np.abs(out.float().cpu().numpy() - ref)) < 2e-2 * max(1.0, np.max(np.abs(ref)))
 
 
 # ------------------------------------------------------------------------------------------ route / compact

