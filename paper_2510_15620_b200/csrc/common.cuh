@@ -27,8 +27,7 @@ enum Epilogue : int {
 // Inputs of the fused QK-norm + RoPE epilogue (head_dim 128; rotary table rows of 64 floats).
 struct QkvRopeArgs {
   const int* pos;        // [m] position of each row inside its sequence
-  const float* cos_t;    // [max_pos, 64]
-  const float* sin_t;    // [max_pos, 64]
+  const float* tab;      // [max_pos, 2, 64]: for half h, cos(32h + 0..31) then sin(32h + 0..31) of pos * theta^(-i/64)
   const __nv_bfloat16* g_q;  // [128] (used when qk_norm)
   const __nv_bfloat16* g_k;  // [128]
   int hq, hkv, qk_norm;
@@ -91,6 +90,7 @@ cudaError_t launch_rmsnorm(const float* x, const void* gain, int dtype, int rows
                            void* out, cudaStream_t st);
 cudaError_t launch_rope_table(float* cos_t, float* sin_t, int max_pos, int head_dim, float theta,
                               cudaStream_t st);
+cudaError_t launch_rope_table_fused(float* tab, int max_pos, float theta, cudaStream_t st);
 cudaError_t launch_qknorm_rope(void* qkv, int dtype, const int* pos, int rows, int n_q_heads,
                                int n_kv_heads, int head_dim, int qk_norm, const void* g_q,
                                const void* g_k, float eps, const float* cos_t, const float* sin_t,

@@ -174,6 +174,49 @@ __global__ void __launch_bounds__(256) k_rmsnorm(const float* __restrict__ x, co
   }
 }
 
+// The same norm with one WARP per row (8 rows per block): every lane keeps kPer float4 of the row in
+// flight, which hides HBM latency better than one block per row when the row is only a few KB.
+template <typename OT, int kPer>
+__global__ void __launch_bounds__(256) k_rmsnorm_warp(const float* __restrict__ x, const OT* __restrict__ gain,
+                                                      int rows, int d, float eps, OT* __restrict__ out) {
+  const int lane = threadIdx.x & 31;
+  const long long row = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (row >= rows) return;
+  const float4* xr = reinterpret_cast<const float4*>(x + (size_t)row * d);
+  const int nv = d >> 2;
+  float4 v[kPer];
+  float ss = 0.f;
+#pragma unroll
+  for (int i = 0; i < kPer; ++i) {
+    const int c = lane + i * 32;
+    if (c < nv) v[i] = xr[c];
+  }
+#pragma unroll
+  for (int i = 0; i < kPer; ++i) {
+    const int c = lane + i * 32;
+    if (c < nv) ss += v[i].x * v[i].x + v[i].y * v[i].y + v[i].z * v[i].z + v[i].w * v[i].w;
+  }
+  ss = warp_sum(ss);
+  const float r = 1.0f / sqrtf(ss / (float)d + eps);
+  OT* orow = out + (size_t)row * d;
+#pragma unroll
+  for (int i = 0; i < kPer; ++i) {
+    const int c = lane + i * 32;
+    if (c < nv) {
+      const OT* g = gain + 4 * c;
+      float o0 = v[i].x * r * to_f(g[0]), o1 = v[i].y * r * to_f(g[1]);
+      float o2 = v[i].z * r * to_f(g[2]), o3 = v[i].w * r * to_f(g[3]);
+      if constexpr (sizeof(OT) == 2) {
+        __nv_bfloat162 a = __floats2bfloat162_rn(o0, o1), b = __floats2bfloat162_rn(o2, o3);
+        uint2 pk = make_uint2(*reinterpret_cast<uint32_t*>(&a), *reinterpret_cast<uint32_t*>(&b));
+        *reinterpret_cast<uint2*>(orow + 4 * c) = pk;
+      } else {
+        *reinterpret_cast<float4*>(orow + 4 * c) = make_float4(o0, o1, o2, o3);
+      }
+    }
+  }
+}
+
 // ------------------------------------------------------------------------------------------------
 // Rotary table in fp64, stored fp32: cos/sin(pos * theta^(-2j/dh)), j < dh/2.
 __global__ void k_rope_table(float* __restrict__ cos_t, float* __restrict__ sin_t, int max_pos, int half,
@@ -185,6 +228,17 @@ __global__ void k_rope_table(float* __restrict__ cos_t, float* __restrict__ sin_
   double a = (double)p * inv;
   cos_t[i] = (float)cos(a);
   sin_t[i] = (float)sin(a);
+}
+
+// The same angles for head_dim 128, laid out for the fused QKV epilogue: [pos][half][cos 32 | sin 32].
+__global__ void k_rope_table_fused(float* __restrict__ tab, int max_pos, double theta) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= max_pos * 64) return;
+  int p = i / 64, f = i % 64;  // f = frequency index 0..63
+  double a = (double)p * pow(theta, -(double)f / 64.0);
+  float* row = tab + (size_t)p * 128 + (f / 32) * 64;
+  row[f % 32] = (float)cos(a);
+  row[32 + f % 32] = (float)sin(a);
 }
 
 // S4 optional per-head RMSNorm over dh, then rotation of pairs (j, j + dh/2).  In place on the q and
@@ -331,6 +385,21 @@ cudaError_t launch_rmsnorm(const float* x, const void* gain, int dtype, int rows
   if (rows <= 0) return cudaSuccess;
   const int nv = d >> 2;
   if (nv > 8 * 256) return cudaErrorInvalidValue;
+  if (nv <= 16 * 32) {  // rows of up to 8 KB: one warp per row
+    const unsigned grid = (unsigned)((rows + 7) / 8);
+#define PRISM_NORMW(OT, V) k_rmsnorm_warp<OT, V><<<grid, 256, 0, st>>>(x, (const OT*)gain, rows, d, eps, (OT*)out)
+    if (dtype == 1) {
+      if (nv <= 128) PRISM_NORMW(__nv_bfloat16, 4);
+      else if (nv <= 256) PRISM_NORMW(__nv_bfloat16, 8);
+      else PRISM_NORMW(__nv_bfloat16, 16);
+    } else {
+      if (nv <= 128) PRISM_NORMW(float, 4);
+      else if (nv <= 256) PRISM_NORMW(float, 8);
+      else PRISM_NORMW(float, 16);
+    }
+#undef PRISM_NORMW
+    return cudaGetLastError();
+  }
 #define PRISM_NORM(OT, V) \
   k_rmsnorm<OT, V><<<rows, 256, 0, st>>>(x, (const OT*)gain, d, eps, (OT*)out)
   if (dtype == 1) {
@@ -354,6 +423,13 @@ cudaError_t launch_rope_table(float* cos_t, float* sin_t, int max_pos, int head_
   const long long n = (long long)max_pos * half;
   if (n <= 0) return cudaSuccess;
   k_rope_table<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(cos_t, sin_t, max_pos, half, (double)theta);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_rope_table_fused(float* tab, int max_pos, float theta, cudaStream_t st) {
+  const long long n = (long long)max_pos * 64;
+  if (n <= 0) return cudaSuccess;
+  k_rope_table_fused<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(tab, max_pos, (double)theta);
   return cudaGetLastError();
 }
 

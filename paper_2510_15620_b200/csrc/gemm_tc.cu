@@ -5,7 +5,8 @@
 //   warp 0      TMA producer: 128x64 A tile + 256x64 B tile per stage, 128-byte swizzle, 4 stages
 //   warp 1      MMA issuer: one elected lane issues tcgen05.mma (M=128, N=256, K=16) into one of two
 //               256-column TMEM accumulators, commits stage-release and accumulator-ready barriers
-//   warps 2..5  epilogue: tcgen05.ld the accumulator (one row per thread), apply the fused epilogue
+//   warps 2..9  epilogue: two warps per 32-row TMEM lane quarter, each taking one half of the tile's
+//               columns; tcgen05.ld the accumulator (one row per thread), apply the fused epilogue
 //               while the MMA warp fills the other buffer:
 //                 store     bf16 store
 //                 residual  x += acc through shared memory and a TMA reduce-add (asynchronous, no read of
@@ -34,7 +35,7 @@ constexpr int kStageBytes = kABytes + kBBytes; // 48 KB
 constexpr int kEpiBufBytes = 32 * 32 * 4;      // one 32x32 fp32 sub-tile staged for a TMA reduce-add
 constexpr int kEpiStageBytes = 4 * 2 * kEpiBufBytes;  // 4 epilogue warps x 2 buffers
 constexpr int kSmemBytes = kStages * kStageBytes + kEpiStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
-constexpr int kThreads = 192;
+constexpr int kThreads = 320;  // TMA warp, MMA warp, 8 epilogue warps
 constexpr unsigned long long kWaitCycles = 4000000000ull;  // ~2 s at boost clock
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -177,7 +178,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(bar_acc_full + 8 * a, 1);
-      mbar_init(bar_acc_empty + 8 * a, 4);
+      mbar_init(bar_acc_empty + 8 * a, 8);
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -250,8 +251,9 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
       }
     }
   } else {
-    // ------------------------------------------------------------------ epilogue (4 warps, 128 rows)
-    const int quarter = warp & 3;  // TMEM lane quarter this warp may read
+    // ------------------------------------------------------------------ epilogue (8 warps, 128 rows x 2 column halves)
+    const int quarter = warp & 3;        // TMEM lane quarter this warp may read
+    const int colhalf = (warp - 2) >> 2;  // 0: first half of the tile's columns, 1: second half
     bool ok = true;
     int it = 0;
     for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++it) {
@@ -264,7 +266,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
       const int col0 = nt * kOutCols;
       if constexpr (kEpi == kEpiSwiGLU) {
 #pragma unroll 1
-        for (int c = 0; c < 4; ++c) {
+        for (int cc = 0; cc < 2; ++cc) {
+          const int c = colhalf * 2 + cc;  // 32 of the tile's 128 outputs: gate columns c*32.., up columns 128 + c*32..
           uint32_t g[32], u[32];
           tmem_ld32(taddr + c * 32, g);
           tmem_ld32(taddr + 128 + c * 32, u);
@@ -279,7 +282,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
                 for (int e = 0; e < 4; ++e) {
                   const float g0 = __uint_as_float(g[v * 8 + 2 * e]), g1 = __uint_as_float(g[v * 8 + 2 * e + 1]);
                   const float u0 = __uint_as_float(u[v * 8 + 2 * e]), u1 = __uint_as_float(u[v * 8 + 2 * e + 1]);
-                  pk[e] = pack_bf16(g0 / (1.f + __expf(-g0)) * u0, g1 / (1.f + __expf(-g1)) * u1);
+                  pk[e] = pack_bf16(__fdividef(g0, 1.f + __expf(-g0)) * u0, __fdividef(g1, 1.f + __expf(-g1)) * u1);
                 }
                 *reinterpret_cast<uint4*>(o + v * 8) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
               }
@@ -287,17 +290,16 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
           }
         }
       } else if constexpr (kEpi == kEpiResidual) {
-        // 32x32 fp32 sub-tiles go through shared memory (128-byte swizzle) into a TMA reduce-add.
-        const uint32_t my_bufs = epi_stage + (uint32_t)(warp - 2) * 2 * kEpiBufBytes;
+        // 32x32 fp32 sub-tiles go through this warp's staging buffer (128-byte swizzle) into a TMA reduce-add.
+        const uint32_t buf = epi_stage + (uint32_t)(warp - 2) * kEpiBufBytes;
 #pragma unroll 1
-        for (int c = 0; c < 8; ++c) {
-          // Sub-tiles outside the matrix are skipped entirely (warp-uniform): a staging buffer is only
-          // rewritten after a later commit has made the wait below cover its previous reduce.
+        for (int cc = 0; cc < 4; ++cc) {
+          const int c = colhalf * 4 + cc;
+          // sub-tiles outside the matrix are skipped (warp-uniform)
           if (col0 + c * 32 >= n || mt * BM + quarter * 32 >= m) break;
-          const uint32_t buf = my_bufs + (c & 1) * kEpiBufBytes;
           uint32_t r[32];
           tmem_ld32(taddr + c * 32, r);
-          if (lane == 0) bulk_wait_read<1>();  // the reduce that last read this buffer has finished with it
+          if (lane == 0) bulk_wait_read<0>();  // the previous reduce has finished reading the buffer
           __syncwarp();
           tmem_ld_wait();
 #pragma unroll
@@ -314,102 +316,124 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
           }
         }
       } else if constexpr (kEpi == kEpiQkvRope) {
-        // A 256-column tile is two heads.  q and k heads: optional RMSNorm over the head, then the
-        // rotation of pairs (j, j+64); v heads are stored as they are.
+        // A 256-column tile is two heads; this warp owns head `colhalf` of the tile.  q and k heads:
+        // optional RMSNorm over the head, then the rotation of pairs (i, i+64); v heads are stored as
+        // they are.  The rotary table rows of the quarter's 32 rows are fetched coalesced (256 bytes per
+        // row and half) into a staging buffer shared by the two warps of the quarter, 16-byte chunks
+        // XOR-swizzled by row so that every thread reads its own row without bank conflicts.
         const int prow = row < m ? row : 0;
-        const float* ct = qa.cos_t + (size_t)qa.pos[prow] * 64;
-        const float* st = qa.sin_t + (size_t)qa.pos[prow] * 64;
+        const int my_pos = qa.pos[prow];
+        const uint32_t stage = epi_stage + (uint32_t)quarter * 2 * kEpiBufBytes;  // 8 KB = 32 rows x 256 B
+        const int pair_bar = 1 + quarter;                                         // named barrier of the two warps
+        const int head = nt * 2 + colhalf;
+        const bool live = head * 128 < n;
+        const bool rot = live && head < qa.hq + qa.hkv;
+        const bool any_rot = nt * 2 < qa.hq + qa.hkv;  // same for both warps of the pair
+        const uint32_t th = taddr + colhalf * 128;
+        float rnh = 1.f;
+        if (rot && qa.qk_norm) {
+          float ss = 0.f;
 #pragma unroll 1
-        for (int hh = 0; hh < 2; ++hh) {
-          const int head = nt * 2 + hh;
-          if (head * 128 >= n) break;
-          __nv_bfloat16* o = out + (size_t)row * n + (size_t)head * 128;
-          const uint32_t th = taddr + hh * 128;
-          if (head >= qa.hq + qa.hkv) {
-#pragma unroll 1
-            for (int c = 0; c < 4; ++c) {
-              uint32_t r[32];
-              tmem_ld32(th + c * 32, r);
-              tmem_ld_wait();
-              if (row < m) {
+          for (int c = 0; c < 4; ++c) {
+            uint32_t r[32];
+            tmem_ld32(th + c * 32, r);
+            tmem_ld_wait();
 #pragma unroll
-                for (int v = 0; v < 4; ++v) {
-                  uint4 pk;
-                  pk.x = pack_bf16(__uint_as_float(r[v * 8 + 0]), __uint_as_float(r[v * 8 + 1]));
-                  pk.y = pack_bf16(__uint_as_float(r[v * 8 + 2]), __uint_as_float(r[v * 8 + 3]));
-                  pk.z = pack_bf16(__uint_as_float(r[v * 8 + 4]), __uint_as_float(r[v * 8 + 5]));
-                  pk.w = pack_bf16(__uint_as_float(r[v * 8 + 6]), __uint_as_float(r[v * 8 + 7]));
-                  *reinterpret_cast<uint4*>(o + c * 32 + v * 8) = pk;
-                }
+            for (int e = 0; e < 32; ++e) ss = fmaf(__uint_as_float(r[e]), __uint_as_float(r[e]), ss);
+          }
+          rnh = 1.0f / sqrtf(ss * (1.f / 128.f) + qa.eps);
+        }
+        __nv_bfloat16* o = out + (size_t)row * n + (size_t)head * 128;
+        const __nv_bfloat16* gain = head < qa.hq ? qa.g_q : qa.g_k;
+#pragma unroll 1
+        for (int half = 0; half < 2; ++half) {
+          if (any_rot) {
+            // both warps are done reading the previous half before it is overwritten
+            asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
+#pragma unroll
+            for (int i8 = 0; i8 < 8; ++i8) {
+              const int rr = (colhalf * 8 + i8) * 2 + (lane >> 4), ch = lane & 15;  // this warp fetches 16 of the 32 rows
+              const int p = __shfl_sync(0xffffffffu, my_pos, rr);
+              const float4 v = __ldg(reinterpret_cast<const float4*>(qa.tab + (size_t)p * 128 + half * 64) + ch);
+              const uint32_t dst = stage + rr * 256 + ((ch ^ (rr & 7)) << 4);
+              asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
+            }
+            asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
+          }
+          if (!live) continue;
+          uint32_t a[32], b[32];
+          tmem_ld32(th + half * 32, a);
+          tmem_ld32(th + 64 + half * 32, b);
+          tmem_ld_wait();
+          if (!rot) {  // v head: plain store of the two 32-column pieces
+            if (row < m) {
+#pragma unroll
+              for (int v = 0; v < 4; ++v) {
+                uint4 pa, pb;
+                pa.x = pack_bf16(__uint_as_float(a[v * 8 + 0]), __uint_as_float(a[v * 8 + 1]));
+                pa.y = pack_bf16(__uint_as_float(a[v * 8 + 2]), __uint_as_float(a[v * 8 + 3]));
+                pa.z = pack_bf16(__uint_as_float(a[v * 8 + 4]), __uint_as_float(a[v * 8 + 5]));
+                pa.w = pack_bf16(__uint_as_float(a[v * 8 + 6]), __uint_as_float(a[v * 8 + 7]));
+                pb.x = pack_bf16(__uint_as_float(b[v * 8 + 0]), __uint_as_float(b[v * 8 + 1]));
+                pb.y = pack_bf16(__uint_as_float(b[v * 8 + 2]), __uint_as_float(b[v * 8 + 3]));
+                pb.z = pack_bf16(__uint_as_float(b[v * 8 + 4]), __uint_as_float(b[v * 8 + 5]));
+                pb.w = pack_bf16(__uint_as_float(b[v * 8 + 6]), __uint_as_float(b[v * 8 + 7]));
+                *reinterpret_cast<uint4*>(o + half * 32 + v * 8) = pa;
+                *reinterpret_cast<uint4*>(o + 64 + half * 32 + v * 8) = pb;
               }
             }
             continue;
           }
-          float rn = 1.f;
-          if (qa.qk_norm) {
-            float ss = 0.f;
-#pragma unroll 1
-            for (int c = 0; c < 4; ++c) {
-              uint32_t r[32];
-              tmem_ld32(th + c * 32, r);
-              tmem_ld_wait();
 #pragma unroll
-              for (int e = 0; e < 32; ++e) ss = fmaf(__uint_as_float(r[e]), __uint_as_float(r[e]), ss);
+          for (int v = 0; v < 4; ++v) {
+            float x0[8], x1[8], cs[8], sn[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+              x0[e] = __uint_as_float(a[v * 8 + e]);
+              x1[e] = __uint_as_float(b[v * 8 + e]);
             }
-            rn = 1.0f / sqrtf(ss * (1.f / 128.f) + qa.eps);
-          }
-          const __nv_bfloat16* gain = head < qa.hq ? qa.g_q : qa.g_k;
-#pragma unroll 1
-          for (int j = 0; j < 2; ++j) {
-            uint32_t a[32], b[32];
-            tmem_ld32(th + j * 32, a);
-            tmem_ld32(th + 64 + j * 32, b);
-            tmem_ld_wait();
-            if (row < m) {
+            if (qa.qk_norm) {
+              const uint4 g0 = __ldg(reinterpret_cast<const uint4*>(gain + half * 32 + v * 8));
+              const uint4 g1 = __ldg(reinterpret_cast<const uint4*>(gain + 64 + half * 32 + v * 8));
+              const __nv_bfloat16* p0 = reinterpret_cast<const __nv_bfloat16*>(&g0);
+              const __nv_bfloat16* p1 = reinterpret_cast<const __nv_bfloat16*>(&g1);
 #pragma unroll
-              for (int v = 0; v < 4; ++v) {
-                float x0[8], x1[8];
-#pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                  x0[e] = __uint_as_float(a[v * 8 + e]);
-                  x1[e] = __uint_as_float(b[v * 8 + e]);
-                }
-                if (qa.qk_norm) {
-                  const uint4 g0 = __ldg(reinterpret_cast<const uint4*>(gain + j * 32 + v * 8));
-                  const uint4 g1 = __ldg(reinterpret_cast<const uint4*>(gain + 64 + j * 32 + v * 8));
-                  const __nv_bfloat16* p0 = reinterpret_cast<const __nv_bfloat16*>(&g0);
-                  const __nv_bfloat16* p1 = reinterpret_cast<const __nv_bfloat16*>(&g1);
-#pragma unroll
-                  for (int e = 0; e < 8; ++e) {
-                    x0[e] = x0[e] * rn * __bfloat162float(p0[e]);
-                    x1[e] = x1[e] * rn * __bfloat162float(p1[e]);
-                  }
-                }
-                const float4 c0 = __ldg(reinterpret_cast<const float4*>(ct + j * 32 + v * 8));
-                const float4 c1 = __ldg(reinterpret_cast<const float4*>(ct + j * 32 + v * 8 + 4));
-                const float4 s0 = __ldg(reinterpret_cast<const float4*>(st + j * 32 + v * 8));
-                const float4 s1 = __ldg(reinterpret_cast<const float4*>(st + j * 32 + v * 8 + 4));
-                const float cs[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
-                const float sn[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
-                uint32_t lo[4], hi[4];
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                  const float y0 = x0[2 * e] * cs[2 * e] - x1[2 * e] * sn[2 * e];
-                  const float y1 = x0[2 * e + 1] * cs[2 * e + 1] - x1[2 * e + 1] * sn[2 * e + 1];
-                  const float z0 = x1[2 * e] * cs[2 * e] + x0[2 * e] * sn[2 * e];
-                  const float z1 = x1[2 * e + 1] * cs[2 * e + 1] + x0[2 * e + 1] * sn[2 * e + 1];
-                  lo[e] = pack_bf16(y0, y1);
-                  hi[e] = pack_bf16(z0, z1);
-                }
-                *reinterpret_cast<uint4*>(o + j * 32 + v * 8) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
-                *reinterpret_cast<uint4*>(o + 64 + j * 32 + v * 8) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+              for (int e = 0; e < 8; ++e) {
+                x0[e] = x0[e] * rnh * __bfloat162float(p0[e]);
+                x1[e] = x1[e] * rnh * __bfloat162float(p1[e]);
               }
+            }
+            // staged row: chunks 0..7 = cos(32*half + 0..31), chunks 8..15 = sin
+#pragma unroll
+            for (int q4 = 0; q4 < 2; ++q4) {
+              const int cc = v * 2 + q4;
+              const uint32_t ca = stage + lane * 256 + ((cc ^ (lane & 7)) << 4);
+              const uint32_t sa = stage + lane * 256 + (((cc + 8) ^ (lane & 7)) << 4);
+              asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                           : "=f"(cs[q4 * 4]), "=f"(cs[q4 * 4 + 1]), "=f"(cs[q4 * 4 + 2]), "=f"(cs[q4 * 4 + 3]) : "r"(ca));
+              asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                           : "=f"(sn[q4 * 4]), "=f"(sn[q4 * 4 + 1]), "=f"(sn[q4 * 4 + 2]), "=f"(sn[q4 * 4 + 3]) : "r"(sa));
+            }
+            uint32_t lo[4], hi[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const float y0 = x0[2 * e] * cs[2 * e] - x1[2 * e] * sn[2 * e];
+              const float y1 = x0[2 * e + 1] * cs[2 * e + 1] - x1[2 * e + 1] * sn[2 * e + 1];
+              const float z0 = x1[2 * e] * cs[2 * e] + x0[2 * e] * sn[2 * e];
+              const float z1 = x1[2 * e + 1] * cs[2 * e + 1] + x0[2 * e + 1] * sn[2 * e + 1];
+              lo[e] = pack_bf16(y0, y1);
+              hi[e] = pack_bf16(z0, z1);
+            }
+            if (row < m) {
+              *reinterpret_cast<uint4*>(o + half * 32 + v * 8) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+              *reinterpret_cast<uint4*>(o + 64 + half * 32 + v * 8) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
             }
           }
         }
       } else {
 #pragma unroll 1
-        for (int c = 0; c < 8; ++c) {
+        for (int cc = 0; cc < 4; ++cc) {
+          const int c = colhalf * 4 + cc;
           uint32_t r[32];
           tmem_ld32(taddr + c * 32, r);
           tmem_ld_wait();

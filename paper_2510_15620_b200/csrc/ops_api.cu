@@ -81,11 +81,11 @@ int prism_op_gemm_qkv_rope(const void* a, const void* w_qkv, void* out, int32_t 
   float* tab = nullptr;
   cudaError_t e = cudaMalloc(&tab, 2 * (size_t)max_pos * 64 * sizeof(float));
   if (e != cudaSuccess) return st_of(e);
-  e = launch_rope_table(tab, tab + (size_t)max_pos * 64, max_pos, 128, theta, S(stream));
+  e = launch_rope_table_fused(tab, max_pos, theta, S(stream));
   TmaDesc ma, mb;
   if (e == cudaSuccess) e = make_tma_2d_bf16(&ma, a, (uint64_t)m, (uint64_t)k, 128, 64);
   if (e == cudaSuccess) e = make_tma_2d_bf16(&mb, w_qkv, (uint64_t)n, (uint64_t)k, 128, 64);
-  QkvRopeArgs qa{pos, tab, tab + (size_t)max_pos * 64, (const __nv_bfloat16*)g_q, (const __nv_bfloat16*)g_k,
+  QkvRopeArgs qa{pos, tab, (const __nv_bfloat16*)g_q, (const __nv_bfloat16*)g_k,
                  n_q_heads, n_kv_heads, qk_norm, eps};
   if (e == cudaSuccess) e = launch_gemm_tc(ma, mb, mb, out, nullptr, m, n, k, kEpiQkvRope, &qa, err_word, S(stream));
   cudaStreamSynchronize(S(stream));

@@ -47,7 +47,7 @@ struct prism_handle {
   int *tokens = nullptr, *pos = nullptr, *cu[2] = {nullptr, nullptr}, *seq2orig[2] = {nullptr, nullptr};
   int* old_of_new = nullptr;
   void *a_norm = nullptr, *qkv = nullptr, *attn = nullptr, *hbuf = nullptr;
-  float *scores = nullptr, *res_score = nullptr, *w_diff = nullptr, *rope_cos = nullptr, *rope_sin = nullptr;
+  float *scores = nullptr, *res_score = nullptr, *w_diff = nullptr, *rope_cos = nullptr, *rope_sin = nullptr, *rope_fused = nullptr;
   int *res_idx = nullptr, *errword = nullptr;
   RouteState* state = nullptr;
   ProbeRecordDev* recs = nullptr;
@@ -369,6 +369,7 @@ static int create_impl(prism_handle* h, const prism_model_cfg* cfg, const prism_
   PRISM_CUDA(h, dev_alloc(h, &h->w_diff, D));
   PRISM_CUDA(h, dev_alloc(h, &h->rope_cos, (size_t)c.max_seq_len * (c.head_dim / 2)));
   PRISM_CUDA(h, dev_alloc(h, &h->rope_sin, (size_t)c.max_seq_len * (c.head_dim / 2)));
+  if (c.head_dim == 128) PRISM_CUDA(h, dev_alloc(h, &h->rope_fused, (size_t)c.max_seq_len * 128));
   PRISM_CUDA(h, dev_alloc(h, &h->errword, 1));
   PRISM_CUDA(h, dev_alloc(h, &h->state, 1));
   PRISM_CUDA(h, dev_alloc(h, &h->recs, (size_t)c.n_layers));
@@ -423,6 +424,7 @@ static int create_impl(prism_handle* h, const prism_model_cfg* cfg, const prism_
   }
 
   PRISM_LAUNCH(h, launch_rope_table(h->rope_cos, h->rope_sin, c.max_seq_len, c.head_dim, c.rope_theta, 0));
+  if (h->rope_fused) PRISM_LAUNCH(h, launch_rope_table_fused(h->rope_fused, c.max_seq_len, c.rope_theta, 0));
   PRISM_LAUNCH(h, launch_score_diff(h->score_head, c.dtype, c.hidden, h->w_diff, 0));
   PRISM_CUDA(h, cudaDeviceSynchronize());
   return PRISM_OK;
@@ -492,7 +494,7 @@ int run_layer_chunk(prism_handle* h, const LayerDev& W, const LayerMaps* maps, f
   PRISM_LAUNCH_P(h, st, PRISM_K_RMSNORM, norm_bytes, launch_rmsnorm(xr, W.g_attn, c.dtype, rows, D, c.rms_eps, h->a_norm, st));
   const bool fused_rope = h->tc && dh == 128;  // QK-norm + RoPE inside the QKV GEMM's epilogue
   if (fused_rope) {
-    QkvRopeArgs qa{h->pos + r0, h->rope_cos, h->rope_sin, (const __nv_bfloat16*)W.g_q, (const __nv_bfloat16*)W.g_k,
+    QkvRopeArgs qa{h->pos + r0, h->rope_fused, (const __nv_bfloat16*)W.g_q, (const __nv_bfloat16*)W.g_k,
                    c.n_q_heads, c.n_kv_heads, c.qk_norm, c.rms_eps};
     PRISM_LAUNCH_P(h, st, PRISM_K_GEMM_QKV, 2.0 * R * nqkv * D,
                    launch_gemm_tc(h->map_a_norm, maps->qkv, maps->qkv, h->qkv, nullptr, rows, nqkv, D, kEpiQkvRope, &qa, h->errword, st));
