@@ -31,6 +31,11 @@ UNIT = "candidate-tokens/s"
 KERNEL_CLASSES = ["pack", "embed", "rmsnorm", "gemm_qkv", "rope", "attention", "gemm_o", "gemm_gateup", "gemm_down",
                   "probe", "route", "compact"]
 GEMM_CLASSES = ("gemm_qkv", "gemm_o", "gemm_gateup", "gemm_down")
+# dram__bytes_read.sum + dram__bytes_write.sum of one k_gemm_tc launch at M = 8192 with the cfg1 weight
+# shapes, from the ncu captures summarised under profiles/ (down-proj: A + W + residual, not captured).
+# Reads grow in proportion to M; writes are mostly absorbed by the 126 MB L2 inside the kernel's window.
+NCU_TRAFFIC_M8192 = {"gemm_qkv": 41.7e6, "gemm_o": 71.6e6, "gemm_gateup": 31.7e6, "gemm_down": 90.2e6}
+CFG1_NK = {"gemm_qkv": (4096, 1024), "gemm_o": (1024, 2048), "gemm_gateup": (6144, 1024), "gemm_down": (1024, 3072)}
 
 
 # ----------------------------------------------------------------------------------------------- helpers
@@ -299,12 +304,23 @@ def run_prism(args):
         peak = peaks["bf16_tflops_sustained"]
         ach = g_fl / (g_ms * 1e-3) / 1e12 if g_ms > 0 else 0.0
         tot_ms = sum(v["ms_per_step"] for v in per.values())
+        traffic = None
+        if args.workload in (1, 4) and g_n:      # the captures are for the 0.6B weight shapes
+            tb = 0.0
+            for n in GEMM_CLASSES:
+                nn, kk = CFG1_NK[n]
+                rows_total = per[n]["work_per_step"] / (2.0 * nn * kk)          # sum of M over the class's launches
+                tb += NCU_TRAFFIC_M8192[n] * rows_total / 8192.0
+            traffic = tb / g_n
         line["roofline"] = {"kernel": "k_gemm_tc (tcgen05 projection GEMMs: qkv, o, gate/up, down)", "bound": "tensor",
                             "achieved": ach, "peak": peak, "unit": "TFLOP/s", "frac": ach / peak if peak else None,
                             "peak_source": f"bf16_tflops_sustained of {peaks['source']} (kernel timed inside a long step)",
                             "frac_of_burst_peak": ach / peaks["bf16_tflops"],
                             "flops_per_launch": g_fl / g_n if g_n else 0, "avg_launch_ms": g_ms / g_n if g_n else 0,
-                            "traffic": None, "share_of_kernel_time": g_ms / tot_ms if tot_ms else None}
+                            "traffic": traffic,
+                            "traffic_note": "bytes per launch: ncu dram read+write of each GEMM shape at M = 8192 "
+                                            "(profiles/gemm_tc_*.md) scaled by the rows each launch processed",
+                            "share_of_kernel_time": g_ms / tot_ms if tot_ms else None}
         line["kernels"] = {n: {"ms_per_step": round(v["ms_per_step"], 4), "share": round(v["ms_per_step"] / tot_ms, 4),
                                "launches_per_step": v["launches_per_step"],
                                ("tflops" if n in GEMM_CLASSES or n == "attention" else "gbs"):

@@ -36,7 +36,7 @@ def _time(fn, iters, warmup, flush):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--op", required=True, choices=["gemm", "attention", "rmsnorm", "rope", "compact"])
+    ap.add_argument("--op", required=True, choices=["gemm", "qkv_rope", "attention", "rmsnorm", "rope", "compact"])
     ap.add_argument("--m", type=int, default=35200)
     ap.add_argument("--n", type=int, default=4096)
     ap.add_argument("--k", type=int, default=1024)
@@ -71,6 +71,19 @@ def main():
         med, best = _time(fn, a.iters, a.warmup, flush)
         fl = 2.0 * m * n * k * (2 if a.epilogue == 2 else 1)
         out.update(m=m, n=n, k=k, epilogue=a.epilogue, ms=med, ms_min=best, tflops=fl / med / 1e9, err=int(err.item()))
+    elif a.op == "qkv_rope":
+        m, k = a.m, a.k
+        n = (a.hq + 2 * a.hkv) * 128
+        A = rnd(m, k).to(torch.bfloat16)
+        B = (rnd(n, k) * 0.05).to(torch.bfloat16)
+        O = torch.empty(m, n, dtype=torch.bfloat16, device=dev)
+        gq = torch.ones(128, dtype=torch.bfloat16, device=dev)
+        pos = (torch.arange(m, dtype=torch.int32, device=dev) % 512).contiguous()
+        err = torch.zeros(1, dtype=torch.int32, device=dev)
+        fn = lambda: ops.prism_op_gemm_qkv_rope(A, B, O, m, k, a.hq, a.hkv, 1, gq, gq, 1e-6, pos, 1e6, 512, err)
+        med, best = _time(fn, a.iters, a.warmup, flush)
+        out.update(m=m, n=n, k=k, ms=med, ms_min=best, tflops=2.0 * m * n * k / med / 1e9, err=int(err.item()),
+                   note="includes the op wrapper's table build and sync")
     elif a.op == "attention":
         rng = np.random.default_rng(0)
         lens = rng.integers(a.len_lo, a.len_hi + 1, size=a.seqs)
