@@ -56,7 +56,8 @@ PRISM_API int prism_op_gemm(const void* a, const void* b, const void* b2, void* 
  * bf16, head_dim 128): out[m, (Hq+2Hkv)*128] = rope(qknorm(a[m,k] * w_qkv^T)) on the q and k heads, plain
  * projection on the v heads.  Equals prism_op_gemm(epilogue 0) followed by prism_op_qknorm_rope, except
  * that norm and rotation act on the fp32 accumulator (one rounding to bf16 instead of two).
- * Allocates and frees a temporary rotary table of max_pos rows. */
+ * The first call for a (device, theta, max_pos) builds a rotary table of max_pos rows (cudaMalloc) and
+ * keeps it until the process exits or the parameters change; later calls only enqueue the kernel. */
 PRISM_API int prism_op_gemm_qkv_rope(const void* a, const void* w_qkv, void* out, int32_t m, int32_t k,
                                      int32_t n_q_heads, int32_t n_kv_heads, int32_t qk_norm, const void* g_q,
                                      const void* g_k, float eps, const int32_t* pos, float theta, int32_t max_pos,

@@ -330,6 +330,27 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
         const bool rot = live && head < qa.hq + qa.hkv;
         const bool any_rot = nt * 2 < qa.hq + qa.hkv;  // same for both warps of the pair
         const uint32_t th = taddr + colhalf * 128;
+        // Table rows are requested one half ahead of their use, so that the L2 round trip overlaps the
+        // TMEM passes and the arithmetic.  This warp fetches 16 of the quarter's 32 rows.
+        float4 tv[8];
+        auto fetch_table = [&](int half) {
+#pragma unroll
+          for (int i8 = 0; i8 < 8; ++i8) {
+            const int rr = (colhalf * 8 + i8) * 2 + (lane >> 4);
+            const int p = __shfl_sync(0xffffffffu, my_pos, rr);
+            tv[i8] = __ldg(reinterpret_cast<const float4*>(qa.tab + (size_t)p * 128 + half * 64) + (lane & 15));
+          }
+        };
+        auto stage_table = [&]() {
+#pragma unroll
+          for (int i8 = 0; i8 < 8; ++i8) {
+            const int rr = (colhalf * 8 + i8) * 2 + (lane >> 4), ch = lane & 15;
+            const uint32_t dst = stage + rr * 256 + ((ch ^ (rr & 7)) << 4);
+            asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "f"(tv[i8].x), "f"(tv[i8].y), "f"(tv[i8].z),
+                         "f"(tv[i8].w) : "memory");
+          }
+        };
+        if (any_rot) fetch_table(0);
         float rnh = 1.f;
         if (rot && qa.qk_norm) {
           float ss = 0.f;
@@ -350,15 +371,9 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
           if (any_rot) {
             // both warps are done reading the previous half before it is overwritten
             asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
-#pragma unroll
-            for (int i8 = 0; i8 < 8; ++i8) {
-              const int rr = (colhalf * 8 + i8) * 2 + (lane >> 4), ch = lane & 15;  // this warp fetches 16 of the 32 rows
-              const int p = __shfl_sync(0xffffffffu, my_pos, rr);
-              const float4 v = __ldg(reinterpret_cast<const float4*>(qa.tab + (size_t)p * 128 + half * 64) + ch);
-              const uint32_t dst = stage + rr * 256 + ((ch ^ (rr & 7)) << 4);
-              asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
-            }
+            stage_table();
             asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
+            if (half == 0) fetch_table(1);
           }
           if (!live) continue;
           uint32_t a[32], b[32];

@@ -78,18 +78,32 @@ int prism_op_gemm_qkv_rope(const void* a, const void* w_qkv, void* out, int32_t 
   if (!a || !w_qkv || !out || !pos || !err_word || m < 0 || k < 1 || (k % 8) || max_pos < 1) return PRISM_ERR_INVALID_ARG;
   if (qk_norm && (!g_q || !g_k)) return PRISM_ERR_INVALID_ARG;
   const int n = (n_q_heads + 2 * n_kv_heads) * 128;
-  float* tab = nullptr;
-  cudaError_t e = cudaMalloc(&tab, 2 * (size_t)max_pos * 64 * sizeof(float));
-  if (e != cudaSuccess) return st_of(e);
-  e = launch_rope_table_fused(tab, max_pos, theta, S(stream));
+  // The rotary table is built once per (device, theta, max_pos) and kept until the process exits.
+  static float* tab = nullptr;
+  static int tab_dev = -1, tab_pos = 0;
+  static float tab_theta = 0.f;
+  int dev = 0;
+  cudaGetDevice(&dev);
+  cudaError_t e = cudaSuccess;
+  if (!tab || tab_dev != dev || tab_pos != max_pos || tab_theta != theta) {
+    if (tab) {
+      cudaDeviceSynchronize();
+      cudaFree(tab);
+      tab = nullptr;
+    }
+    e = cudaMalloc(&tab, (size_t)max_pos * 128 * sizeof(float));
+    if (e != cudaSuccess) return st_of(e);
+    e = launch_rope_table_fused(tab, max_pos, theta, S(stream));
+    if (e == cudaSuccess) e = cudaStreamSynchronize(S(stream));
+    tab_dev = dev;
+    tab_pos = max_pos;
+    tab_theta = theta;
+  }
   TmaDesc ma, mb;
   if (e == cudaSuccess) e = make_tma_2d_bf16(&ma, a, (uint64_t)m, (uint64_t)k, 128, 64);
   if (e == cudaSuccess) e = make_tma_2d_bf16(&mb, w_qkv, (uint64_t)n, (uint64_t)k, 128, 64);
-  QkvRopeArgs qa{pos, tab, (const __nv_bfloat16*)g_q, (const __nv_bfloat16*)g_k,
-                 n_q_heads, n_kv_heads, qk_norm, eps};
+  QkvRopeArgs qa{pos, tab, (const __nv_bfloat16*)g_q, (const __nv_bfloat16*)g_k, n_q_heads, n_kv_heads, qk_norm, eps};
   if (e == cudaSuccess) e = launch_gemm_tc(ma, mb, mb, out, nullptr, m, n, k, kEpiQkvRope, &qa, err_word, S(stream));
-  cudaStreamSynchronize(S(stream));
-  cudaFree(tab);
   return st_of(e);
 }
 

@@ -50,6 +50,7 @@ def main():
     ap.add_argument("--hq", type=int, default=16)
     ap.add_argument("--hkv", type=int, default=8)
     ap.add_argument("--causal", type=int, default=1)
+    ap.add_argument("--qk-norm", type=int, default=1)
     ap.add_argument("--iters", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--no-flush", action="store_true")
@@ -80,10 +81,9 @@ def main():
         gq = torch.ones(128, dtype=torch.bfloat16, device=dev)
         pos = (torch.arange(m, dtype=torch.int32, device=dev) % 512).contiguous()
         err = torch.zeros(1, dtype=torch.int32, device=dev)
-        fn = lambda: ops.prism_op_gemm_qkv_rope(A, B, O, m, k, a.hq, a.hkv, 1, gq, gq, 1e-6, pos, 1e6, 512, err)
+        fn = lambda: ops.prism_op_gemm_qkv_rope(A, B, O, m, k, a.hq, a.hkv, a.qk_norm, gq, gq, 1e-6, pos, 1e6, 512, err)
         med, best = _time(fn, a.iters, a.warmup, flush)
-        out.update(m=m, n=n, k=k, ms=med, ms_min=best, tflops=2.0 * m * n * k / med / 1e9, err=int(err.item()),
-                   note="includes the op wrapper's table build and sync")
+        out.update(m=m, n=n, k=k, qk_norm=a.qk_norm, ms=med, ms_min=best, tflops=2.0 * m * n * k / med / 1e9, err=int(err.item()))
     elif a.op == "attention":
         rng = np.random.default_rng(0)
         lens = rng.integers(a.len_lo, a.len_hi + 1, size=a.seqs)

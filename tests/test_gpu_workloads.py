@@ -114,9 +114,10 @@ def test_cfg3_qwen3_8b_streamed_and_chunked(P):
     per_tok = (4096 + 6144 + 4096 + 12288) * 2
     tight = hidden + per_tok * 30000
     # The stored candidate is the longest of the request (2048 document tokens) and its scores are large
-    # (|s| = 3.3 .. 4.0).  bf16 rounding of the GEMM inputs is relative, and at this depth and width the
-    # measured deviation is 0.3 % .. 1.9 % of the score (0.014 .. 0.075 absolute, CUDA-core and tensor-core
-    # paths alike), so this one check bounds the error relative to the score: 2 % instead of 3e-2 absolute.
+    # (|s| = 3.3 .. 4.0).  bf16 rounding of the GEMM inputs is relative; at this depth and width the four
+    # kernel-path combinations (CUDA-core / tensor-core GEMM x attention) land 0.0008 .. 0.075 from the
+    # oracle at layer 8 and the tensor-core path 0.040 at layer 12, up to 1.9 % of the score.  They differ
+    # only in rounding order, so this one check bounds the error relative to the score: 2 %, not 3e-2.
     _, _, res = _run_workload(P, 3, "cfg3_qwen3_8b_streamed_scores_r0_c0_1.txt", budgets=(None, tight), rel=2e-2)
     a, b = res
     assert b[2].n_chunks_max >= 4 and a[2].n_chunks_max < b[2].n_chunks_max
