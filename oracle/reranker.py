@@ -21,6 +21,15 @@ from typing import Dict, Iterable, List, Sequence
 import numpy as np
 
 
+def to_bf16(x: np.ndarray) -> np.ndarray:
+    """Round to the nearest bfloat16 (ties to even), returned as float64.  Used only by the optional
+    "bf16 activations" mode below, which places one rounding wherever the precision contract of the
+    bf16 path stores an activation as bfloat16."""
+    b = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32)
+    r = (b + (np.uint32(0x7FFF) + ((b >> np.uint32(16)) & np.uint32(1)))) & np.uint32(0xFFFF0000)
+    return r.view(np.float32).astype(np.float64)
+
+
 def rmsnorm(x: np.ndarray, g: np.ndarray, eps: float) -> np.ndarray:
     """y = x / sqrt(mean(x^2) + eps) * g over the last axis."""
     ms = np.mean(x * x, axis=-1, keepdims=True)
@@ -43,9 +52,11 @@ def rope_rotate(u: np.ndarray, pos: np.ndarray, theta: float) -> np.ndarray:
     return np.concatenate([a * c - b * s, b * c + a * s], axis=-1)
 
 
-def attention(q: np.ndarray, k: np.ndarray, v: np.ndarray, causal: bool) -> np.ndarray:
+def attention(q: np.ndarray, k: np.ndarray, v: np.ndarray, causal: bool, round_p=None) -> np.ndarray:
     """q: [L, Hq, dh], k/v: [L, Hkv, dh] -> [L, Hq, dh].  Query head h reads kv head
-    h // (Hq/Hkv).  softmax(q k^T / sqrt(dh)) over keys u <= t (causal) or all keys."""
+    h // (Hq/Hkv).  softmax(q k^T / sqrt(dh)) over keys u <= t (causal) or all keys.
+    round_p (optional) rounds the unnormalised probabilities that multiply v; the normaliser is
+    the sum of the unrounded ones."""
     L, hq, dh = q.shape
     hkv = k.shape[1]
     grp = hq // hkv
@@ -57,17 +68,25 @@ def attention(q: np.ndarray, k: np.ndarray, v: np.ndarray, causal: bool) -> np.n
         s = np.where(mask, s, -np.inf)
         s = s - s.max(axis=-1, keepdims=True)
         p = np.exp(s)
-        p = p / p.sum(axis=-1, keepdims=True)
-        out[:, h, :] = p @ v[:, kh, :]
+        den = p.sum(axis=-1, keepdims=True)
+        if round_p is not None:
+            p = round_p(p)
+        out[:, h, :] = (p @ v[:, kh, :]) / den
     return out
 
 
-def layer_forward(x: np.ndarray, w: Dict[str, np.ndarray], cfg) -> np.ndarray:
-    """One pre-norm decoder block on one sequence.  x: [L, D] fp64 -> [L, D]."""
+def layer_forward(x: np.ndarray, w: Dict[str, np.ndarray], cfg, act: str = "exact") -> np.ndarray:
+    """One pre-norm decoder block on one sequence.  x: [L, D] fp64 -> [L, D].
+
+    act = "exact": no rounding anywhere (the definition).  act = "bf16": the same steps with every
+    stored activation rounded to bfloat16 where the bf16 precision contract stores it (normed inputs,
+    q/k after the rotary embedding, v, attention probabilities, attention output, SwiGLU output); the
+    residual stream, norms, softmax and all sums stay exact."""
+    rnd = to_bf16 if act == "bf16" else (lambda t: t)
     L = x.shape[0]
     hq, hkv, dh = cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim
     W = {k: np.asarray(t, dtype=np.float64) for k, t in w.items()}
-    a = rmsnorm(x, W["g_attn"], cfg.rms_eps)
+    a = rnd(rmsnorm(x, W["g_attn"], cfg.rms_eps))
     qkv = a @ W["w_qkv"].T
     q = qkv[:, : hq * dh].reshape(L, hq, dh)
     k = qkv[:, hq * dh: (hq + hkv) * dh].reshape(L, hkv, dh)
@@ -76,14 +95,15 @@ def layer_forward(x: np.ndarray, w: Dict[str, np.ndarray], cfg) -> np.ndarray:
         q = rmsnorm(q, W["g_q"], cfg.rms_eps)
         k = rmsnorm(k, W["g_k"], cfg.rms_eps)
     pos = np.arange(L)
-    q = rope_rotate(q, pos, cfg.rope_theta)
-    k = rope_rotate(k, pos, cfg.rope_theta)
-    o = attention(q, k, v, bool(cfg.causal)).reshape(L, hq * dh)
+    q = rnd(rope_rotate(q, pos, cfg.rope_theta))
+    k = rnd(rope_rotate(k, pos, cfg.rope_theta))
+    v = rnd(v)
+    o = rnd(attention(q, k, v, bool(cfg.causal), round_p=rnd if act == "bf16" else None)).reshape(L, hq * dh)
     x = x + o @ W["w_o"].T
-    b = rmsnorm(x, W["g_ffn"], cfg.rms_eps)
+    b = rnd(rmsnorm(x, W["g_ffn"], cfg.rms_eps))
     gate = b @ W["w_gate"].T
     up = b @ W["w_up"].T
-    h = gate / (1.0 + np.exp(-gate)) * up          # silu(gate) * up
+    h = rnd(gate / (1.0 + np.exp(-gate)) * up)     # silu(gate) * up
     return x + h @ W["w_down"].T
 
 
@@ -96,7 +116,7 @@ def probe_score(x_last: np.ndarray, g_final: np.ndarray, score_head: np.ndarray,
 
 
 def candidate_scores(tokens: np.ndarray, weights: Dict[str, object], cfg,
-                     score_layers: Iterable[int], return_hidden: bool = False):
+                     score_layers: Iterable[int], return_hidden: bool = False, act: str = "exact"):
     """Forward one sequence (query||doc token ids) through all layers needed and return
     {layer: score} for every layer count in score_layers (1-based: after that many blocks).
     `weights['layers']` may be a list or any iterable yielding per-layer dicts in order."""
@@ -109,7 +129,7 @@ def candidate_scores(tokens: np.ndarray, weights: Dict[str, object], cfg,
     for l, w in enumerate(weights["layers"], start=1):
         if l > last:
             break
-        x = layer_forward(x, w, cfg)
+        x = layer_forward(x, w, cfg, act)
         if l in want:
             out[l] = probe_score(x[-1], weights["g_final"], weights["score_head"], cfg.rms_eps)
             if return_hidden:
@@ -119,7 +139,7 @@ def candidate_scores(tokens: np.ndarray, weights: Dict[str, object], cfg,
 
 def score_matrix(query: np.ndarray, cand_tokens: np.ndarray, cand_offsets: np.ndarray,
                  weights: Dict[str, object], cfg, score_layers: Sequence[int],
-                 candidates: Sequence[int] | None = None) -> Dict[int, np.ndarray]:
+                 candidates: Sequence[int] | None = None, act: str = "exact") -> Dict[int, np.ndarray]:
     """S[layer][i] for the requested candidates (default all): each candidate is forwarded
     alone as query||doc_i.  Returns {layer: float64 array indexed like `candidates`}.
 
@@ -142,7 +162,7 @@ def score_matrix(query: np.ndarray, cand_tokens: np.ndarray, cand_offsets: np.nd
             break
         w = {k: np.asarray(t, dtype=np.float64) for k, t in w.items()}   # widen once per layer
         for c in range(len(ids)):
-            xs[c] = layer_forward(xs[c], w, cfg)
+            xs[c] = layer_forward(xs[c], w, cfg, act)
         if l in S:
             for c in range(len(ids)):
                 S[l][c] = probe_score(xs[c][-1], weights["g_final"], weights["score_head"], cfg.rms_eps)

@@ -2,13 +2,17 @@
 // head_dim 128, GQA, causal or bidirectional.
 //
 // One CTA = 128 query rows of one (sequence, head); two CTAs fit on an SM.  Warp-specialised:
-//   warp 0      TMA producer: Q once, then (K_j, V_j) tiles of 64 keys into a 2-stage ring
+//   warp 0      TMA producer: Q once, then K_j tiles (64 keys) into a 3-deep ring and V_j tiles into a
+//               2-deep ring; a K slot is released as soon as its Q K^T has run, a V slot after P V
 //   warp 1      MMA issuer:   S_j = Q K_j^T (tcgen05.mma M128 N64 K16 x 8) into one of two TMEM buffers,
-//                             O += P_j V_j  (M128 N128 K16 x 4, V as an MN-major operand) into TMEM
-//   warps 2..5  softmax: one query row per thread; read S_j from TMEM, exponentiate against a running
-//               reference maximum, write P_j (bf16, 128-byte swizzle) over the K_j tile, which the
-//               tensor core has finished with; O stays in TMEM and is rescaled (TMEM read-modify-write)
-//               only when a row's maximum outgrows the reference by more than 2^8.
+//                             O += P_j V_j  (M128 N128 K16 x 4; P read from TENSOR MEMORY, V as an
+//                             MN-major shared-memory operand) into TMEM
+//   warps 2..9  softmax: two threads per query row (warps w and w+4 share a 32-row TMEM lane quarter and
+//               take 32 of the 64 key columns each); read S_j from TMEM, exchange the row maximum,
+//               exponentiate against a running reference maximum and store P_j as packed bf16 back
+//               into the first 32 columns of the S_j buffer (tcgen05.st); O stays in TMEM and is
+//               rescaled (TMEM read-modify-write) only when a row's maximum outgrows the reference by
+//               more than 2^8.
 // S_{j+1} is issued before P_j is awaited, so the tensor core computes the next scores while the
 // softmax warps work.  Every mbarrier wait is bounded; on expiry the kernel records kErrTimeout, all
 // roles drain to the common exit and the tensor memory is freed.  No cluster multicast.
@@ -22,11 +26,16 @@ namespace {
 
 constexpr int BM = 128, BN = 64, DH = 128;
 constexpr int kQBytes = BM * DH * 2;          // 32 KB: two [128 x 64] swizzled sub-tiles
-constexpr int kKBytes = BN * DH * 2;          // 16 KB: two [64 x 64] sub-tiles; later holds P_j [128 x 64]
+constexpr int kKBytes = BN * DH * 2;          // 16 KB: two [64 x 64] sub-tiles
 constexpr int kVBytes = BN * DH * 2;          // 16 KB: two [64 keys x 64 dh] sub-tiles
-constexpr int kStageBytes = kKBytes + kVBytes;
-constexpr int kSmemBytes = kQBytes + 2 * kStageBytes + 1024 + 128;
-constexpr int kThreads = 192;
+constexpr int NK = 3, NV = 2;                 // ring depths
+constexpr int kXchBytes = 2 * 128 * 2;        // per-row exchange of the block maximum (bf16) between the two threads of a row
+constexpr int kTileBytes = kQBytes + NK * kKBytes + NV * kVBytes;  // 112 KB
+// No alignment slack: two CTAs per SM only fit if nothing is wasted.  The kernel checks that its
+// shared window starts on a 1024-byte boundary (the swizzled tiles need it) and reports if not.
+constexpr int kSmemBytes = kTileBytes + 256 + kXchBytes;
+static_assert(2 * (kSmemBytes + 1024) <= 233472, "two CTAs per SM must fit in 228 KB of shared memory");
+constexpr int kThreads = 320;                 // TMA warp, MMA warp, 8 softmax warps
 constexpr int kTmemCols = 256;                // S: 2 x 64, O: 128
 constexpr unsigned long long kWaitCycles = 4000000000ull;
 
@@ -55,7 +64,8 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* er
   uint32_t it = 0;
   while (!mbar_try(bar, parity)) {
     if ((++it & 0x3ff) == 0) {
-      if (*abort_flag || clock64() - t0 > kWaitCycles) {
+      // a timeout anywhere on the device (recorded in the error word) ends every other wait quickly
+      if (*abort_flag || (*reinterpret_cast<volatile int*>(err) & kErrTimeout) || clock64() - t0 > kWaitCycles) {
         *abort_flag = 1;
         atomicOr(err, kErrTimeout);
         return false;
@@ -71,7 +81,6 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t acc) {
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
@@ -104,6 +113,23 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
         "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
       : "memory");
 }
+// 16 registers = 32 packed bf16 per lane
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+      : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem]: the A operand (P, packed bf16) is read from tensor memory.
+__device__ __forceinline__ void umma_bf16_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t db, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "r"(tmem_a), "l"(db), "r"(idesc), "r"(acc) : "memory");
+}
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
@@ -122,6 +148,11 @@ __host__ __device__ constexpr uint32_t idesc(int n, int b_mn_major) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)b_mn_major << 16) | ((uint32_t)(n >> 3) << 17) |
          ((uint32_t)(BM >> 4) << 24);
 }
+__device__ __forceinline__ float ex2(float x) {  // 2^x on the special-function unit; -inf -> 0
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
   __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
   return *reinterpret_cast<uint32_t*>(&v);
@@ -139,29 +170,40 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   const int h = blockIdx.y, kvh = h / (hq / hkv);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
-  const uint32_t raw = smem_u32(smem_raw);
-  const uint32_t base = (raw + 1023u) & ~1023u;
-  unsigned char* gen = smem_raw + (base - raw);
-  const uint32_t s_q = base, s_stage = base + kQBytes;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(gen + kQBytes + 2 * kStageBytes);
-  const uint32_t b_q = smem_u32(bars), b_kv_full = smem_u32(bars + 1), b_kv_empty = smem_u32(bars + 3);
-  const uint32_t b_s_full = smem_u32(bars + 5), b_s_empty = smem_u32(bars + 7);
-  const uint32_t b_p_full = smem_u32(bars + 9), b_o_full = smem_u32(bars + 10);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 11);
+  const uint32_t base = smem_u32(smem_raw);
+  unsigned char* gen = smem_raw;
+  const uint32_t s_q = base, s_k = base + kQBytes, s_v = s_k + NK * kKBytes;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(gen + kTileBytes);
+  // q, k_full[3], k_empty[3], v_full[2], v_empty[2], s_full[2], s_empty[2], p_full, o_full
+  const uint32_t b_q = smem_u32(bars), b_k_full = smem_u32(bars + 1), b_k_empty = smem_u32(bars + 4);
+  const uint32_t b_v_full = smem_u32(bars + 7), b_v_empty = smem_u32(bars + 9);
+  const uint32_t b_s_full = smem_u32(bars + 11), b_s_empty = smem_u32(bars + 13);
+  const uint32_t b_p_full = smem_u32(bars + 15), b_o_full = smem_u32(bars + 16);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 17);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  __nv_bfloat16* xch = reinterpret_cast<__nv_bfloat16*>(gen + kTileBytes + 256);  // [2][128]
+  float* xch_l = reinterpret_cast<float*>(gen);  // [2][128] over the Q tile, used once all MMAs are done
+  if (base & 1023u) {  // cannot run correctly: say so instead of computing garbage
+    if (threadIdx.x == 0) atomicOr(err, kErrInternal);
+    return;
+  }
 
   const int kv_end = causal ? min(len, (qb + 1) * BM) : len;
   const int n_blocks = (kv_end + BN - 1) / BN;
 
   if (threadIdx.x == 0) {
     mbar_init(b_q, 1);
-    for (int i = 0; i < 2; ++i) {
-      mbar_init(b_kv_full + 8 * i, 1);
-      mbar_init(b_kv_empty + 8 * i, 1);
-      mbar_init(b_s_full + 8 * i, 1);
-      mbar_init(b_s_empty + 8 * i, 128);
+    for (int i = 0; i < NK; ++i) {
+      mbar_init(b_k_full + 8 * i, 1);
+      mbar_init(b_k_empty + 8 * i, 1);
     }
-    mbar_init(b_p_full, 128);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(b_v_full + 8 * i, 1);
+      mbar_init(b_v_empty + 8 * i, 1);
+      mbar_init(b_s_full + 8 * i, 1);
+      mbar_init(b_s_empty + 8 * i, 8);
+    }
+    mbar_init(b_p_full, 8);
     mbar_init(b_o_full, 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -174,7 +216,7 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
-  const uint32_t t_s = tmem, t_o = tmem + 2 * BN;  // columns [0,128): S buffers, [128,256): O
+  const uint32_t t_s = tmem, t_o = tmem + 2 * BN;  // columns [0,128): S buffers (P_j aliases the first 32 of S_j), [128,256): O
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
@@ -183,15 +225,24 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       tma_load_2d(s_q, &map_q, h * DH, beg + qb * BM, b_q);
       tma_load_2d(s_q + kQBytes / 2, &map_q, h * DH + 64, beg + qb * BM, b_q);
       const int kcol = (hq + kvh) * DH, vcol = (hq + hkv + kvh) * DH;
-      for (int j = 0; j < n_blocks; ++j) {
-        const int st = j & 1, u = j >> 1;
-        if (!mbar_wait(b_kv_empty + 8 * st, (u & 1) ^ 1, err, abort_flag)) break;
-        const uint32_t sk = s_stage + st * kStageBytes, sv = sk + kKBytes;
-        mbar_expect_tx(b_kv_full + 8 * st, kStageBytes);
-        tma_load_2d(sk, &map_kv, kcol, beg + j * BN, b_kv_full + 8 * st);
-        tma_load_2d(sk + kKBytes / 2, &map_kv, kcol + 64, beg + j * BN, b_kv_full + 8 * st);
-        tma_load_2d(sv, &map_kv, vcol, beg + j * BN, b_kv_full + 8 * st);
-        tma_load_2d(sv + kVBytes / 2, &map_kv, vcol + 64, beg + j * BN, b_kv_full + 8 * st);
+      // K runs one block ahead of V: step t issues K_t, then V_{t-1}.
+      for (int t = 0; t <= n_blocks; ++t) {
+        if (t < n_blocks) {
+          const int st = t % NK, u = t / NK;
+          if (!mbar_wait(b_k_empty + 8 * st, (u & 1) ^ 1, err, abort_flag)) break;
+          const uint32_t sk = s_k + st * kKBytes;
+          mbar_expect_tx(b_k_full + 8 * st, kKBytes);
+          tma_load_2d(sk, &map_kv, kcol, beg + t * BN, b_k_full + 8 * st);
+          tma_load_2d(sk + kKBytes / 2, &map_kv, kcol + 64, beg + t * BN, b_k_full + 8 * st);
+        }
+        if (t >= 1) {
+          const int j = t - 1, st = j & 1, u = j >> 1;
+          if (!mbar_wait(b_v_empty + 8 * st, (u & 1) ^ 1, err, abort_flag)) break;
+          const uint32_t sv = s_v + st * kVBytes;
+          mbar_expect_tx(b_v_full + 8 * st, kVBytes);
+          tma_load_2d(sv, &map_kv, vcol, beg + j * BN, b_v_full + 8 * st);
+          tma_load_2d(sv + kVBytes / 2, &map_kv, vcol + 64, beg + j * BN, b_v_full + 8 * st);
+        }
       }
     }
   } else if (warp == 1) {
@@ -200,90 +251,99 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       constexpr uint32_t kIdescS = idesc(BN, 0), kIdescO = idesc(DH, 1);
       bool ok = mbar_wait(b_q, 0, err, abort_flag);
       auto issue_qk = [&](int j) {
-        const int st = j & 1;
-        const uint32_t sk = s_stage + st * kStageBytes;
+        const int st = j % NK;
+        const uint32_t sk = s_k + st * kKBytes;
         tc_fence_after();
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk) {  // 16 head-dim elements per step; sub-tile switches at kk = 4
           const uint64_t da = smem_desc(s_q + (kk >> 2) * (kQBytes / 2) + (kk & 3) * 32, 16, 1024);
           const uint64_t db = smem_desc(sk + (kk >> 2) * (kKBytes / 2) + (kk & 3) * 32, 16, 1024);
-          umma_bf16(t_s + st * BN, da, db, kIdescS, kk != 0);
+          umma_bf16(t_s + (j & 1) * BN, da, db, kIdescS, kk != 0);
         }
-        umma_commit(b_s_full + 8 * st);
+        umma_commit(b_s_full + 8 * (j & 1));
+        umma_commit(b_k_empty + 8 * st);  // the K tile is free as soon as these MMAs have read it
       };
-      if (ok) ok = mbar_wait(b_kv_full, 0, err, abort_flag);
+      if (ok) ok = mbar_wait(b_k_full, 0, err, abort_flag);
       if (ok) issue_qk(0);
       for (int j = 0; j < n_blocks && ok; ++j) {
         if (j + 1 < n_blocks) {
           const int b = (j + 1) & 1, u = (j + 1) >> 1;
-          if (!mbar_wait(b_kv_full + 8 * b, u & 1, err, abort_flag)) { ok = false; break; }
+          if (!mbar_wait(b_k_full + 8 * ((j + 1) % NK), ((j + 1) / NK) & 1, err, abort_flag)) { ok = false; break; }
           if (!mbar_wait(b_s_empty + 8 * b, (u & 1) ^ 1, err, abort_flag)) { ok = false; break; }
           issue_qk(j + 1);
         }
         if (!mbar_wait(b_p_full, j & 1, err, abort_flag)) { ok = false; break; }
+        if (!mbar_wait(b_v_full + 8 * (j & 1), (j >> 1) & 1, err, abort_flag)) { ok = false; break; }
         tc_fence_after();
-        const int st = j & 1;
-        const uint32_t sp = s_stage + st * kStageBytes, sv = sp + kKBytes;
+        const uint32_t sv = s_v + (j & 1) * kVBytes;
 #pragma unroll
-        for (int kk = 0; kk < 4; ++kk) {  // 16 keys per step
-          const uint64_t da = smem_desc(sp + kk * 32, 16, 1024);               // P: K-major, one 64-key atom
+        for (int kk = 0; kk < 4; ++kk) {  // 16 keys per step: 8 packed columns of P, 16 rows of V
           const uint64_t db = smem_desc(sv + kk * 2048, kVBytes / 2, 1024);    // V: MN-major, two 64-wide dh atoms
-          umma_bf16(t_o, da, db, kIdescO, (j | kk) != 0);
+          umma_bf16_ts(t_o, t_s + (j & 1) * BN + kk * 8, db, kIdescO, (j | kk) != 0);
         }
         umma_commit(b_o_full);
-        umma_commit(b_kv_empty + 8 * st);
+        umma_commit(b_v_empty + 8 * (j & 1));
       }
     }
   } else {
-    // ------------------------------------------------------------------ softmax + output (128 rows)
+    // ------------------------------------------------------------------ softmax + output (128 rows x 2 column halves)
     const int quarter = warp & 3;
+    const int colhalf = (warp - 2) >> 2;           // which 32 of a block's 64 keys / which 64 of the 128 output columns
     const int r = quarter * 32 + lane;             // row inside the tile = TMEM lane
     const int qrow = qb * BM + r;                  // row inside the sequence
     const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
-    float m_ref = 0.f, l = 0.f;                    // reference maximum (raw score units), running sum
+    const int pair_bar = 1 + quarter;              // named barrier of the two warps that share these rows
+    float m_ref = 0.f, l = 0.f;                    // reference maximum (raw score units), this thread's partial sum
     bool ok = true;
     for (int j = 0; j < n_blocks; ++j) {
       const int b = j & 1, u = j >> 1;
-      // Parity waits are only meaningful one phase at a time: observe every completion of O += P V in
-      // order (PV(j-2) finished long ago, so this costs nothing) before a later wait may target PV(j-1).
-      if (j >= 2 && !mbar_wait(b_o_full, (j - 2) & 1, err, abort_flag)) { ok = false; break; }
       if (!mbar_wait(b_s_full + 8 * b, u & 1, err, abort_flag)) { ok = false; break; }
       tc_fence_after();
-      uint32_t sr[64];
-      tmem_ld32(t_s + lane_base + b * BN, sr);
-      tmem_ld32(t_s + lane_base + b * BN + 32, sr + 32);
+      uint32_t sr[32];
+      tmem_ld32(t_s + lane_base + b * BN + colhalf * 32, sr);
       tmem_ld_wait();
       tc_fence_before();
-      mbar_arrive(b_s_empty + 8 * b);
-      const int key0 = j * BN;
-      if ((causal && key0 + BN - 1 > qb * BM) || key0 + BN > len) {
+      __syncwarp();
+      if (lane == 0) mbar_arrive(b_s_empty + 8 * b);  // one arrival per warp
+      const int key0 = j * BN + colhalf * 32;
+      if ((causal && j * BN + BN - 1 > qb * BM) || j * BN + BN > len) {
 #pragma unroll
-        for (int c = 0; c < 64; ++c) {
+        for (int c = 0; c < 32; ++c) {
           const int key = key0 + c;
           if (key >= len || (causal && key > qrow)) sr[c] = 0xff800000u;  // -inf
         }
       }
       float bm = -INFINITY;
 #pragma unroll
-      for (int c = 0; c < 64; ++c) bm = fmaxf(bm, __uint_as_float(sr[c]));
+      for (int c = 0; c < 32; ++c) bm = fmaxf(bm, __uint_as_float(sr[c]));
+      // Row maximum over both halves.  The value only serves as a reference for the exponentials, so it
+      // is exchanged rounded up to bf16; both threads of a row use the same two rounded numbers.
+      const __nv_bfloat16 bmr = __float2bfloat16_ru(bm);
+      xch[colhalf * 128 + r] = bmr;
+      asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
+      bm = fmaxf(__bfloat162float(bmr), __bfloat162float(xch[(colhalf ^ 1) * 128 + r]));
+      asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");  // both have read before the next block writes
+      bool saw_pv = false;  // has this thread already observed the completion of P_{j-1} V_{j-1}?
       if (j == 0) {
         m_ref = (bm == -INFINITY) ? 0.f : bm;
       } else {
-        // Rescale O only when this row's maximum outgrew the reference by more than 2^8 (rare).
+        // Rescale O only when this row's maximum outgrew the reference by more than 2^8 (rare).  Both
+        // threads of a row see the same bm and m_ref, so both warps of the pair take the same branch.
         const bool need = (bm - m_ref) * scale_log2 > 8.f;
         if (__any_sync(0xffffffffu, need)) {
           if (!mbar_wait(b_o_full, (j - 1) & 1, err, abort_flag)) { ok = false; break; }
+          saw_pv = true;
           tc_fence_after();
           const float m_new = need ? bm : m_ref;
           const float f = exp2f((m_ref - m_new) * scale_log2);
 #pragma unroll 1
-          for (int c = 0; c < 4; ++c) {
+          for (int c = 0; c < 2; ++c) {
             uint32_t o[32];
-            tmem_ld32(t_o + lane_base + c * 32, o);
+            tmem_ld32(t_o + lane_base + colhalf * 64 + c * 32, o);
             tmem_ld_wait();
 #pragma unroll
             for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * f);
-            tmem_st32(t_o + lane_base + c * 32, o);
+            tmem_st32(t_o + lane_base + colhalf * 64 + c * 32, o);
           }
           tmem_st_wait();
           l *= f;
@@ -291,36 +351,42 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         }
       }
       const float ms = m_ref * scale_log2;
-      const uint32_t sp = s_stage + b * kStageBytes;  // P_j overwrites K_j (its MMAs have completed)
       float rs = 0.f;
+      uint32_t pk[16];
 #pragma unroll
-      for (int c = 0; c < 8; ++c) {
-        float p[8];
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-          p[e] = exp2f(__uint_as_float(sr[c * 8 + e]) * scale_log2 - ms);
-          rs += p[e];
-        }
-        const uint32_t dst = sp + r * 128 + ((c ^ (r & 7)) << 4);
-        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(pack_bf16(p[0], p[1])),
-                     "r"(pack_bf16(p[2], p[3])), "r"(pack_bf16(p[4], p[5])), "r"(pack_bf16(p[6], p[7])) : "memory");
+      for (int c = 0; c < 16; ++c) {
+        const float p0 = ex2(fmaf(__uint_as_float(sr[2 * c]), scale_log2, -ms));
+        const float p1 = ex2(fmaf(__uint_as_float(sr[2 * c + 1]), scale_log2, -ms));
+        rs += p0 + p1;
+        pk[c] = pack_bf16(p0, p1);  // key 2c in the low half, key 2c+1 in the high half
       }
       l += rs;
-      fence_async_smem();
+      // P_j (packed bf16) goes over the first 32 columns of the S_j buffer: both threads of the row have
+      // loaded their S values (they met at the pair barrier above), and Q K_{j+2}^T is only issued after
+      // P_j V_j, so nothing else touches these columns meanwhile.
+      tmem_st16(t_s + lane_base + b * BN + colhalf * 16, pk);
+      tmem_st_wait();
       tc_fence_before();
-      // A warp that runs ahead must not let its arrival for block j be counted in block j-1's phase.
+      // mbarrier parity only tells the current phase from the previous one, so every thread observes
+      // every phase, in order, while the next one cannot complete yet: P_j V_j needs this thread's
+      // arrival below, hence the o_full barrier is at phase j-1 or j here and the wait is unambiguous
+      // (P_{j-1} V_{j-1} was issued a whole block ago, so it has normally finished).  Likewise p_full:
+      // a warp that runs ahead must not have its arrival for block j counted in block j-1's phase.
+      if (j > 0 && !saw_pv && !mbar_wait(b_o_full, (j - 1) & 1, err, abort_flag)) { ok = false; break; }
       if (j > 0 && !mbar_wait(b_p_full, (j - 1) & 1, err, abort_flag)) { ok = false; break; }
-      mbar_arrive(b_p_full);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(b_p_full);  // one arrival per warp
     }
-    if (ok && n_blocks >= 2) ok = mbar_wait(b_o_full, (n_blocks - 2) & 1, err, abort_flag);
     if (ok && mbar_wait(b_o_full, (n_blocks - 1) & 1, err, abort_flag)) {
       tc_fence_after();
-      const float inv = 1.f / l;
-      __nv_bfloat16* orow = out + (size_t)(beg + qrow) * ((size_t)hq * DH) + (size_t)h * DH;
+      xch_l[colhalf * 128 + r] = l;  // the row's sum is the sum of the two partial sums
+      asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
+      const float inv = 1.f / (l + xch_l[(colhalf ^ 1) * 128 + r]);
+      __nv_bfloat16* orow = out + (size_t)(beg + qrow) * ((size_t)hq * DH) + (size_t)h * DH + colhalf * 64;
 #pragma unroll 1
-      for (int c = 0; c < 4; ++c) {
+      for (int c = 0; c < 2; ++c) {
         uint32_t o[32];
-        tmem_ld32(t_o + lane_base + c * 32, o);
+        tmem_ld32(t_o + lane_base + colhalf * 64 + c * 32, o);
         tmem_ld_wait();
         if (qrow < len) {
 #pragma unroll

@@ -69,7 +69,8 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* er
   uint32_t it = 0;
   while (!mbar_try(bar, parity)) {
     if ((++it & 0x3ff) == 0) {
-      if (*abort_flag || clock64() - t0 > kWaitCycles) {
+      // a timeout anywhere on the device (recorded in the error word) ends every other wait quickly
+      if (*abort_flag || (*reinterpret_cast<volatile int*>(err) & kErrTimeout) || clock64() - t0 > kWaitCycles) {
         *abort_flag = 1;
         atomicOr(err, kErrTimeout);
         return false;

@@ -26,6 +26,8 @@ def main():
     ap.add_argument("request", type=int)
     ap.add_argument("--candidates", default=None, help="a:b slice of candidate indices")
     ap.add_argument("--out", default=None)
+    ap.add_argument("--act", default="exact", choices=["exact", "bf16"],
+                    help="bf16: round every stored activation to bfloat16 (the bf16 precision contract)")
     a = ap.parse_args()
     wl = synth.workload(a.workload)
     cfg = wl.model
@@ -39,12 +41,12 @@ def main():
     weights = dict(W.make_globals(cfg, wl.weight_seed))
     weights["layers"] = W.iter_layers(cfg, wl.weight_seed)        # lazily, one layer at a time
     t0 = time.time()
-    S = oracle.score_matrix(r["query"], r["cand_tokens"], r["cand_offsets"], weights, cfg, layers, candidates=ids)
+    S = oracle.score_matrix(r["query"], r["cand_tokens"], r["cand_offsets"], weights, cfg, layers, candidates=ids, act=a.act)
     dt = time.time() - t0
     out = a.out or os.path.join(os.path.dirname(os.path.abspath(__file__)),
                                 f"{wl.name}_scores_r{a.request}.txt")
     with open(out, "w") as f:
-        f.write(f"# oracle scores (fp64 forward, bf16-rounded weights where the workload is bf16)\n")
+        f.write(f"# oracle scores (fp64 forward, bf16-rounded weights where the workload is bf16), activations: {a.act}\n")
         f.write(f"# workload {wl.name} request {a.request} weight_seed {wl.weight_seed} candidates {ids[0]}..{ids[-1]}\n")
         f.write(f"# written by tests/golden/make_scores.py in {dt:.0f} s; one line per layer: layer then scores\n")
         for l in layers:

@@ -25,10 +25,8 @@ def traced_score_fn(trace):
     return lambda layer, ids: np.asarray([table[(layer, int(i))] for i in ids], np.float32)
 
 
-def check_scores(trace, S: Dict[int, np.ndarray], tol: float, ids_known: Sequence[int] | None = None,
-                 rel: float = 0.0) -> float:
-    """Every traced score against the oracle's.  The bound is `tol` absolute; `rel` > 0 widens it to
-    rel*|oracle score| for scores of large magnitude (used only where the test says why)."""
+def check_scores(trace, S: Dict[int, np.ndarray], tol: float, ids_known: Sequence[int] | None = None) -> float:
+    """Every traced score against the oracle's, within `tol` absolute."""
     worst = 0.0
     known = None if ids_known is None else {int(c): j for j, c in enumerate(ids_known)}
     for rec in trace.records:
@@ -41,8 +39,7 @@ def check_scores(trace, S: Dict[int, np.ndarray], tol: float, ids_known: Sequenc
                 ref = S[rec.layer][int(i)]
             err = abs(float(s) - float(ref))
             worst = max(worst, err)
-            bound = max(tol, rel * abs(float(ref)))
-            assert err <= bound, f"layer {rec.layer} candidate {i}: cuda {s} oracle {ref} |diff| {err} > {bound}"
+            assert err <= tol, f"layer {rec.layer} candidate {i}: cuda {s} oracle {ref} |diff| {err} > {tol}"
     return worst
 
 

@@ -243,3 +243,24 @@ def test_float32_forward_agrees_with_float64():
         got[li] = float(y @ torch.tensor(w["score_head"][0] - w["score_head"][1]))
     for l in (1, 2):
         assert abs(got[l] - ours[l]) < 1e-5
+
+
+def test_bf16_activation_mode_rounds_like_a_library_and_stays_close():
+    """The optional bf16-activation mode of the oracle: its rounding equals torch's float32 -> bfloat16
+    conversion bit for bit (ties to even included), rounding is idempotent, and on the tiny model the
+    mode moves the scores only by rounding noise."""
+    torch = pytest.importorskip("torch")
+    from oracle.reranker import to_bf16
+    rng = np.random.default_rng(0)
+    x = np.concatenate([rng.normal(size=5000) * 10.0 ** rng.integers(-6, 6, size=5000),
+                        np.array([1.0 + 2.0 ** -8, 1.0 + 3 * 2.0 ** -8, -(1.0 + 2.0 ** -8), 0.0, 65280.0])]).astype(np.float32)
+    ref = torch.from_numpy(x).to(torch.bfloat16).to(torch.float32).numpy().astype(np.float64)
+    got = to_bf16(x)
+    assert np.array_equal(got, ref)
+    assert np.array_equal(to_bf16(got), got)
+    wl, cfg, w = _tiny()
+    toks = np.random.default_rng(5).integers(0, cfg.vocab, size=40)
+    exact = oracle.candidate_scores(toks, w, cfg, [1, 2])
+    rounded = oracle.candidate_scores(toks, w, cfg, [1, 2], act="bf16")
+    for l in (1, 2):
+        assert 0 < abs(exact[l] - rounded[l]) < 5e-2
