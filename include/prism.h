@@ -193,6 +193,40 @@ PRISM_API int prism_select_host(prism_handle* h, const int32_t* query_tokens, in
                       const prism_prune_schedule* sched, int32_t* topk_idx, float* topk_scores,
                       int32_t* n_out, prism_trace* trace, void* cuda_stream);
 
+/* Automatic calibration of the dispersion threshold (Sec. 4.1, last paragraph): the user states a
+ * minimum precision; requests are sampled at a fixed frequency, the sampled ones are re-run without
+ * pruning to obtain the ground-truth top-K, and after every `window` samples the mean
+ * precision = |top-K with pruning  intersect  top-K without| / min(K, N) is compared with the target:
+ * below it the threshold is raised (more conservative), otherwise lowered (more pruning).
+ * The paper does not say by how much; here the threshold is multiplied by raise_factor (> 1) or
+ * lower_factor (< 1) and clamped to [min_threshold, max_threshold].  The re-run happens inside the
+ * call (the paper defers it to idle time); the caller owns the struct and may persist it. */
+typedef struct {
+  double threshold;         /* in/out: dispersion threshold used for the next request */
+  double target_precision;  /* in: e.g. 0.99 */
+  double raise_factor;      /* in: > 1 */
+  double lower_factor;      /* in: in (0, 1) */
+  double min_threshold;     /* in */
+  double max_threshold;     /* in */
+  int32_t sample_every;     /* in: every sample_every-th request is also run unpruned (>= 1) */
+  int32_t window;           /* in: samples per adjustment (>= 1) */
+  int32_t n_in_window;      /* state: samples collected since the last adjustment */
+  int32_t n_adjustments;    /* out: adjustments made so far */
+  int64_t n_requests;       /* out: requests served */
+  int64_t n_sampled;        /* out: requests re-run unpruned */
+  double precision_sum;     /* state: sum of the window's precisions */
+  double last_precision;    /* out: precision of the last sampled request */
+  double last_window_precision; /* out: mean precision of the last completed window */
+} prism_calibrator;
+
+/* prism_select with the threshold taken from (and maintained in) `cal`.  sched must be a
+ * PRISM_PRUNE_CLUSTER schedule; its cv_threshold field is ignored.  Outputs are those of the pruned
+ * run.  Errors: those of prism_select, plus INVALID_ARG for a malformed calibrator. */
+PRISM_API int prism_select_calibrated(prism_handle* h, const int32_t* query_tokens, int32_t query_len,
+                                      const int32_t* cand_tokens, const int32_t* cand_offsets, int32_t N, int32_t K,
+                                      const prism_prune_schedule* sched, prism_calibrator* cal, int32_t* topk_idx,
+                                      float* topk_scores, int32_t* n_out, prism_trace* trace, void* cuda_stream);
+
 /* Free the handle and its workspaces (NULL is allowed).  Caller memory is untouched. */
 PRISM_API void prism_destroy(prism_handle* h);
 

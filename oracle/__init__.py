@@ -11,3 +11,4 @@ from .reranker import (rmsnorm, rope_rotate, attention, layer_forward,  # noqa: 
 from .prune_rule import (coefficient_of_variation, rank_order, optimal_partition,  # noqa: F401
                          route_clusters, replay_select, MODE_NONE, MODE_FIXED_KEEP, MODE_CLUSTER)
 from .select import oracle_select  # noqa: F401
+from .calibrate import Calibrator, calibrated_step, precision_at_k  # noqa: F401

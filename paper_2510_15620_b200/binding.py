@@ -60,6 +60,15 @@ class _Trace(C.Structure):
                 ("workspace_bytes", C.c_int64)]
 
 
+class Calibrator(C.Structure):
+    """Mirror of prism_calibrator; create with the `in` fields set, pass to PrismModel.select_calibrated."""
+    _fields_ = [("threshold", C.c_double), ("target_precision", C.c_double), ("raise_factor", C.c_double),
+                ("lower_factor", C.c_double), ("min_threshold", C.c_double), ("max_threshold", C.c_double),
+                ("sample_every", C.c_int32), ("window", C.c_int32), ("n_in_window", C.c_int32),
+                ("n_adjustments", C.c_int32), ("n_requests", C.c_int64), ("n_sampled", C.c_int64),
+                ("precision_sum", C.c_double), ("last_precision", C.c_double), ("last_window_precision", C.c_double)]
+
+
 def lib() -> C.CDLL:
     """The loaded C-ABI library.  Raises if it has not been built (no fallback exists)."""
     global _lib
@@ -82,6 +91,8 @@ def lib() -> C.CDLL:
         for f in (L.prism_select, L.prism_select_host):
             f.restype = C.c_int
             f.argtypes = sel
+        L.prism_select_calibrated.restype = C.c_int
+        L.prism_select_calibrated.argtypes = sel[:8] + [C.POINTER(Calibrator)] + sel[8:]
         _lib = L
     return _lib
 
@@ -216,6 +227,21 @@ class PrismModel:
         n_out, trace = self._call(lib().prism_select, query.data_ptr(), query.numel(), cand_tokens.data_ptr(),
                                   cand_offsets.data_ptr(), n, k, sched, idx.data_ptr(), sc.data_ptr(), want_trace, stream)
         return idx[:n_out], sc[:n_out], trace
+
+    def select_calibrated(self, query: torch.Tensor, cand_tokens: torch.Tensor, cand_offsets: torch.Tensor, k: int, sched,
+                          cal: Calibrator):
+        """prism_select_calibrated: the threshold comes from `cal`, which is updated in place."""
+        n = cand_offsets.numel() - 1
+        idx = torch.empty(max(k, 1), dtype=torch.int32, device=query.device)
+        sc = torch.empty(max(k, 1), dtype=torch.float32, device=query.device)
+        s = self._schedule(sched)
+        n_out = C.c_int32(0)
+        rc = lib().prism_select_calibrated(self._h, query.data_ptr(), query.numel(), cand_tokens.data_ptr(),
+                                           cand_offsets.data_ptr(), n, k, C.byref(s), C.byref(cal), idx.data_ptr(),
+                                           sc.data_ptr(), C.byref(n_out), None, torch.cuda.current_stream().cuda_stream)
+        if rc != 0:
+            raise PrismError(rc, lib().prism_last_error(self._h).decode())
+        return idx[:n_out.value], sc[:n_out.value]
 
     def select_host(self, query: np.ndarray, cand_tokens: np.ndarray, cand_offsets: np.ndarray, k: int, sched=None,
                     want_trace: bool = False, idx_out: Optional[np.ndarray] = None, sc_out: Optional[np.ndarray] = None):

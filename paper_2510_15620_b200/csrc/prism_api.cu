@@ -4,6 +4,7 @@
 #include <algorithm>
 #include <cstdio>
 #include <cstring>
+#include <iterator>
 #include <new>
 #include <string>
 #include <vector>
@@ -734,6 +735,64 @@ int prism_select(prism_handle* h, const int32_t* query_tokens, int32_t query_len
     if (h->copy_stream) cudaStreamSynchronize(h->copy_stream);
   }
   return rc;
+}
+
+int prism_select_calibrated(prism_handle* h, const int32_t* query_tokens, int32_t query_len, const int32_t* cand_tokens,
+                            const int32_t* cand_offsets, int32_t N, int32_t K, const prism_prune_schedule* sched,
+                            prism_calibrator* cal, int32_t* topk_idx, float* topk_scores, int32_t* n_out, prism_trace* trace,
+                            void* cuda_stream) {
+  int rc = check_args(h, query_tokens, query_len, cand_tokens, cand_offsets, N, K, topk_idx, topk_scores, n_out);
+  if (rc != PRISM_OK) return rc;
+  *n_out = 0;
+  if (!cal || !sched || sched->mode != PRISM_PRUNE_CLUSTER) return fail(h, PRISM_ERR_INVALID_ARG, "calibration needs a CLUSTER schedule and a calibrator");
+  if (!(cal->raise_factor > 1.0) || !(cal->lower_factor > 0.0 && cal->lower_factor < 1.0) || cal->sample_every < 1 ||
+      cal->window < 1 || !(cal->min_threshold <= cal->max_threshold) || !(cal->threshold == cal->threshold) ||
+      !(cal->target_precision >= 0.0 && cal->target_precision <= 1.0))
+    return fail(h, PRISM_ERR_INVALID_ARG, "malformed calibrator");
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  prism_prune_schedule s = *sched;
+  s.cv_threshold = cal->threshold;
+  rc = select_impl(h, query_tokens, query_len, cand_tokens, cand_offsets, N, K, &s, topk_idx, topk_scores, n_out, trace, st);
+  if (rc != PRISM_OK) {
+    *n_out = 0;
+    cudaStreamSynchronize(st);
+    if (h->copy_stream) cudaStreamSynchronize(h->copy_stream);
+    return rc;
+  }
+  const bool sample = (cal->n_requests % cal->sample_every) == 0;
+  cal->n_requests++;
+  const int k_eff = *n_out;
+  if (!sample || k_eff == 0) return PRISM_OK;
+  // ground truth: the same request without pruning, into the handle's own output buffers
+  std::vector<int> pruned(k_eff), full(k_eff);
+  PRISM_CUDA(h, cudaMemcpyAsync(pruned.data(), topk_idx, (size_t)k_eff * sizeof(int), cudaMemcpyDeviceToHost, st));
+  PRISM_CUDA(h, cudaStreamSynchronize(st));
+  prism_prune_schedule none{};
+  none.mode = PRISM_PRUNE_NONE;
+  int n_full = 0;
+  rc = select_impl(h, query_tokens, query_len, cand_tokens, cand_offsets, N, K, &none, h->out_idx, h->out_score, &n_full, nullptr, st);
+  if (rc != PRISM_OK) return rc;
+  PRISM_CUDA(h, cudaMemcpyAsync(full.data(), h->out_idx, (size_t)k_eff * sizeof(int), cudaMemcpyDeviceToHost, st));
+  PRISM_CUDA(h, cudaStreamSynchronize(st));
+  std::sort(pruned.begin(), pruned.end());
+  std::sort(full.begin(), full.end());
+  std::vector<int> both;
+  std::set_intersection(pruned.begin(), pruned.end(), full.begin(), full.end(), std::back_inserter(both));
+  const double precision = (double)both.size() / (double)k_eff;
+  cal->last_precision = precision;
+  cal->precision_sum += precision;
+  cal->n_sampled++;
+  if (++cal->n_in_window >= cal->window) {
+    const double mean = cal->precision_sum / (double)cal->n_in_window;
+    cal->last_window_precision = mean;
+    double t = cal->threshold * (mean < cal->target_precision ? cal->raise_factor : cal->lower_factor);
+    t = std::min(cal->max_threshold, std::max(cal->min_threshold, t));
+    cal->threshold = t;
+    cal->n_in_window = 0;
+    cal->precision_sum = 0.0;
+    cal->n_adjustments++;
+  }
+  return PRISM_OK;
 }
 
 int prism_select_host(prism_handle* h, const int32_t* query_tokens, int32_t query_len, const int32_t* cand_tokens,

@@ -175,6 +175,43 @@ def test_runs_are_bitwise_repeatable(P, tiny):
     model.close()
 
 
+def test_threshold_calibration_follows_the_oracle_loop(P, tiny):
+    """Sec. 4.1 auto-calibration: the library's loop (pruned run, sampled unpruned re-run, precision,
+    multiplicative adjustment) must walk the same threshold trajectory as the oracle's loop fed with the
+    oracle's own scores, request after request."""
+    import ctypes
+    from oracle.calibrate import Calibrator as OCal, calibrated_step
+    wl, w, _, _ = tiny
+    cfg = wl.model
+    sched = Schedule(MODE_CLUSTER, (1,), cv_threshold=0.0, n_clusters=3)
+    reqs = [synth.make_request(wl, r) for r in range(10)]
+    lens = [np.diff(r["cand_offsets"]) + wl.query_len for r in reqs]
+    tw = P.upload_weights(w, cfg.dtype)
+    model = P.PrismModel(cfg, tw, int(max(l.max() for l in lens)), wl.n_candidates, int(max(l.sum() for l in lens)))
+    kw = dict(threshold=0.05, target_precision=0.99, raise_factor=2.0, lower_factor=0.75, min_threshold=0.01,
+              max_threshold=64.0, sample_every=1, window=2)
+    cal = P.Calibrator(**kw)
+    ocal = OCal(**kw)
+    k = 4
+    for r in reqs:
+        S = oracle.score_matrix(r["query"], r["cand_tokens"], r["cand_offsets"], w, cfg, [1, 2])
+
+        def orun(thr, S=S, r=r):
+            s = Schedule(MODE_NONE) if thr is None else Schedule(MODE_CLUSTER, (1,), cv_threshold=thr, n_clusters=3)
+            return oracle.oracle_select(r["query"], r["cand_tokens"], r["cand_offsets"], k, w, cfg, s, S=S).topk_idx
+        expect = calibrated_step(ocal, orun)
+        idx, _ = model.select_calibrated(dev_i32(r["query"]), dev_i32(r["cand_tokens"]), dev_i32(r["cand_offsets"]), k, sched, cal)
+        assert sorted(idx.cpu().numpy().tolist()) == sorted(expect)
+        assert cal.threshold == ocal.threshold and cal.last_precision == ocal.last_precision
+        assert (cal.n_requests, cal.n_sampled, cal.n_adjustments) == (ocal.n_requests, ocal.n_sampled, ocal.n_adjustments)
+    assert ocal.n_adjustments == 5 and len({ocal.threshold, 0.05}) == 2      # the threshold really moved
+    bad = P.Calibrator(**dict(kw, raise_factor=0.5))
+    with pytest.raises(P.PrismError) as e:
+        model.select_calibrated(dev_i32(reqs[0]["query"]), dev_i32(reqs[0]["cand_tokens"]), dev_i32(reqs[0]["cand_offsets"]), k, sched, bad)
+    assert e.value.status == -1
+    model.close()
+
+
 # ------------------------------------------------------------------------------------------ bf16, mid-size (tensor-core path)
 MID = ModelCfg(n_layers=6, hidden=1024, n_q_heads=16, n_kv_heads=8, head_dim=128, ffn=3072, vocab=4096,
                rope_theta=1e6, qk_norm=1, dtype=DTYPE_BF16, yes_id=3, no_id=4)

@@ -251,3 +251,28 @@ def test_fixed_keep():
     keep = sorted(sorted(range(n), key=lambda i: (-table[1][i], i))[:8])
     assert res.active_per_layer == [list(range(n)), keep]
     assert res.topk_idx == sorted(keep, key=lambda i: (-table[2][i], i))[:3]
+
+
+# ---------------------------------------------------------------- threshold auto-calibration (Sec. 4.1)
+def test_calibration_raises_below_target_and_lowers_otherwise():
+    from oracle.calibrate import Calibrator, calibrated_step, precision_at_k
+    assert precision_at_k([1, 2, 3, 4], [4, 3, 9, 8]) == 0.5 and precision_at_k([], []) == 1.0
+    full = list(range(10))
+    # scripted service: pruning at a threshold below 1.0 loses 3 of 10, at or above 1.0 loses none
+    run = lambda thr: full if thr is None or thr >= 1.0 else full[:7] + [97, 98, 99]
+    cal = Calibrator(threshold=0.25, target_precision=0.9, raise_factor=2.0, lower_factor=0.5, min_threshold=0.125,
+                     max_threshold=8.0, sample_every=2, window=2)
+    trail = []
+    for _ in range(16):
+        calibrated_step(cal, run)
+        trail.append(cal.threshold)
+    # every 2nd request is sampled, every 2 samples adjust: requests 1-4 at 0.25 (precision 0.7 -> x2), 5-8 at 0.5
+    # (0.7 -> x2), 9-12 at 1.0 (precision 1.0 -> x0.5), 13-16 at 0.5 (0.7 -> x2)
+    assert trail == [0.25, 0.25, 0.5, 0.5, 0.5, 0.5, 1.0, 1.0, 1.0, 1.0, 0.5, 0.5, 0.5, 0.5, 1.0, 1.0]
+    assert cal.n_requests == 16 and cal.n_sampled == 8 and cal.n_adjustments == 4
+    assert cal.last_window_precision == 0.7
+    # clamping
+    cal = Calibrator(threshold=0.2, target_precision=0.0, raise_factor=2.0, lower_factor=0.5, min_threshold=0.15,
+                     max_threshold=8.0)
+    calibrated_step(cal, run)
+    assert cal.threshold == 0.15
