@@ -13,7 +13,8 @@ PRISM_FP32, PRISM_BF16 = 0, 1
 PRISM_IMPL_AUTO, PRISM_IMPL_SIMT, PRISM_IMPL_MMA = 0, 1, 2
 PRISM_MAX_CLUSTERS = 8
 
-_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "lib", "libprism.so")
+# PRISM_LIBRARY overrides the in-tree library (e.g. an instrumented build of the same sources).
+_LIB_PATH = os.environ.get("PRISM_LIBRARY") or os.path.join(os.path.dirname(os.path.abspath(__file__)), "lib", "libprism.so")
 _lib = None
 
 

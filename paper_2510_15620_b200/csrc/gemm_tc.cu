@@ -257,9 +257,33 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
     const int colhalf = (warp - 2) >> 2;  // 0: first half of the tile's columns, 1: second half
     bool ok = true;
     int it = 0;
+    // QKV epilogue: the row's position and the first half of its rotary table rows do not depend on the
+    // accumulator, so they are requested before the wait for it (their L2 latency hides behind the MMAs).
+    [[maybe_unused]] int rope_pos = 0;
+    [[maybe_unused]] float4 tv[8];
+    [[maybe_unused]] auto rope_row_pos = [&](int t) {
+      const int rw = (t / n_tiles) * BM + quarter * 32 + lane;
+      return qa.pos[rw < m ? rw : 0];
+    };
+    [[maybe_unused]] auto rope_fetch = [&](int half) {
+#pragma unroll
+      for (int i8 = 0; i8 < 8; ++i8) {
+        const int rr = (colhalf * 8 + i8) * 2 + (lane >> 4);  // this warp fetches 16 of the quarter's 32 rows
+        const int p = __shfl_sync(0xffffffffu, rope_pos, rr);
+        tv[i8] = __ldg(reinterpret_cast<const float4*>(qa.tab + (size_t)p * 128 + half * 64) + (lane & 15));
+      }
+    };
+    if constexpr (kEpi == kEpiQkvRope) {
+      if ((int)blockIdx.x < num_tiles) rope_pos = rope_row_pos(blockIdx.x);
+    }
     for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++it) {
       const uint32_t acc = it & 1, acc_phase = (it >> 1) & 1;
       const int mt = tile / n_tiles, nt = tile % n_tiles;
+      [[maybe_unused]] int rope_pos_next = 0;
+      if constexpr (kEpi == kEpiQkvRope) {
+        if (nt * 2 < qa.hq + qa.hkv) rope_fetch(0);
+        if (tile + (int)gridDim.x < num_tiles) rope_pos_next = rope_row_pos(tile + gridDim.x);
+      }
       if (!mbar_wait(bar_acc_full + 8 * acc, acc_phase, err, abort_flag)) { ok = false; break; }
       tc_fence_after();
       const int row = mt * BM + quarter * 32 + lane;
@@ -322,8 +346,6 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
         // they are.  The rotary table rows of the quarter's 32 rows are fetched coalesced (256 bytes per
         // row and half) into a staging buffer shared by the two warps of the quarter, 16-byte chunks
         // XOR-swizzled by row so that every thread reads its own row without bank conflicts.
-        const int prow = row < m ? row : 0;
-        const int my_pos = qa.pos[prow];
         const uint32_t stage = epi_stage + (uint32_t)quarter * 2 * kEpiBufBytes;  // 8 KB = 32 rows x 256 B
         const int pair_bar = 1 + quarter;                                         // named barrier of the two warps
         const int head = nt * 2 + colhalf;
@@ -331,17 +353,6 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
         const bool rot = live && head < qa.hq + qa.hkv;
         const bool any_rot = nt * 2 < qa.hq + qa.hkv;  // same for both warps of the pair
         const uint32_t th = taddr + colhalf * 128;
-        // Table rows are requested one half ahead of their use, so that the L2 round trip overlaps the
-        // TMEM passes and the arithmetic.  This warp fetches 16 of the quarter's 32 rows.
-        float4 tv[8];
-        auto fetch_table = [&](int half) {
-#pragma unroll
-          for (int i8 = 0; i8 < 8; ++i8) {
-            const int rr = (colhalf * 8 + i8) * 2 + (lane >> 4);
-            const int p = __shfl_sync(0xffffffffu, my_pos, rr);
-            tv[i8] = __ldg(reinterpret_cast<const float4*>(qa.tab + (size_t)p * 128 + half * 64) + (lane & 15));
-          }
-        };
         auto stage_table = [&]() {
 #pragma unroll
           for (int i8 = 0; i8 < 8; ++i8) {
@@ -351,7 +362,6 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
                          "f"(tv[i8].w) : "memory");
           }
         };
-        if (any_rot) fetch_table(0);
         float rnh = 1.f;
         if (rot && qa.qk_norm) {
           float ss = 0.f;
@@ -374,7 +384,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
             asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
             stage_table();
             asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
-            if (half == 0) fetch_table(1);
+            if (half == 0) rope_fetch(1);
           }
           if (!live) continue;
           uint32_t a[32], b[32];
@@ -469,6 +479,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
           }
         }
       }
+      if constexpr (kEpi == kEpiQkvRope) rope_pos = rope_pos_next;
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_acc_empty + 8 * acc);

@@ -358,6 +358,25 @@ def test_route_matches_oracle_rule_bit_exact(P, n_clusters, winners):
         assert list(rsc[2:2 + left]) == [np.float32(x) for x in ref.topk_scores[:left]]
 
 
+def test_route_at_the_maximum_candidate_count(P):
+    """n = PRISM_MAX_CANDIDATES (4096), with ties, against the oracle's rule."""
+    rng = np.random.default_rng(77)
+    n, k = 4096, 50
+    sc = (rng.normal(size=n) * 2).astype(np.float32)
+    sc[rng.integers(0, n, size=500)] = sc[7]
+    ids = np.arange(n, dtype=np.int32)
+    lens = rng.integers(1, 20, size=n)
+    st, cu_new, s2o_new, oon, ridx, rsc, rec, cu = _run_route(P, sc, ids, lens, k, 0, dict(cv_threshold=0.1, n_clusters=4))
+    sched = Schedule(MODE_CLUSTER, (1,), cv_threshold=0.1, n_clusters=4)
+    ref = replay_select(lambda l, a: sc[np.asarray(a)], n, k, 2, sched)
+    t = ref.trace[0]
+    assert (rec.fired, rec.n_selected, rec.n_dropped, rec.n_deferred) == (t.fired, t.n_selected, t.n_dropped, t.n_deferred)
+    assert [rec.cuts[i] for i in range(rec.n_cuts)] == t.cuts and rec.cv == t.cv
+    survivors = ref.active_per_layer[1]
+    assert list(oon[: int(st[0])]) == survivors
+    assert list(cu_new[: len(survivors) + 1]) == list(np.concatenate([[0], np.cumsum(lens[survivors])]))
+
+
 def test_route_fixed_keep_and_final(P):
     rng = np.random.default_rng(9)
     n = 40

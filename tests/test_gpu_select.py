@@ -239,6 +239,24 @@ def test_bf16_paths_match_oracle(P, mid, gemm_impl, attn_impl):
     model.close()
 
 
+def test_bidirectional_attention_end_to_end(P, mid):
+    """causal = 0 (encoder-style attention) through every attention implementation against the oracle."""
+    w, req, _ = mid
+    cfg = replace(MID, causal=0, n_layers=3)
+    wb = dict(w, layers=w["layers"][:3])
+    S = oracle.score_matrix(req["query"], req["cand_tokens"], req["cand_offsets"], wb, cfg, [1, 2, 3])
+    S_causal = oracle.score_matrix(req["query"], req["cand_tokens"], req["cand_offsets"], wb, replace(cfg, causal=1), [3],
+                                   candidates=[0, 1])
+    assert abs(S_causal[3][0] - S[3][0]) > 1e-3                       # the flag matters
+    sched = Schedule(MODE_CLUSTER, (1, 2), cv_threshold=1e30)
+    for attn_impl in (0, 1, 2):
+        model = make_model(P, cfg, wb, req, attention_impl=attn_impl)
+        idx, sc, tr = run(P, model, req, MID_WL.top_k, sched)
+        check_scores(tr, S, TOL_BF16)
+        check_replay(tr, idx, sc, MID_WL.n_candidates, MID_WL.top_k, cfg.n_layers, sched)
+        model.close()
+
+
 def test_chunked_and_streamed_are_result_neutral(P, mid):
     """Chunked execution (Sec. 4.3) and overlapped layer streaming (Sec. 4.2) change where data lives
     and when it moves, never the values."""
