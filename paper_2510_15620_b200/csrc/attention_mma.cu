@@ -207,12 +207,8 @@ __global__ void __launch_bounds__(128) k_attention_mma(const __nv_bfloat16* __re
 cudaError_t launch_attention_mma(const void* qkv, void* out, const int* cu, int seq0, int nseq, int row0,
                                  int max_len, int n_q_heads, int n_kv_heads, int causal, cudaStream_t st) {
   if (nseq <= 0 || max_len <= 0) return cudaSuccess;
-  static bool attr = false;
-  if (!attr) {
-    cudaError_t e = cudaFuncSetAttribute(k_attention_mma, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmem);
-    if (e != cudaSuccess) return e;
-    attr = true;
-  }
+  static std::atomic<unsigned long long> smem_set{0};
+  if (cudaError_t e = ensure_dynamic_smem(k_attention_mma, kAttnSmem, smem_set)) return e;
   dim3 grid((max_len + kBM - 1) / kBM, n_q_heads, nseq);
   const float scale_log2 = 1.4426950408889634f / sqrtf((float)kDh);
   k_attention_mma<<<grid, 128, kAttnSmem, st>>>((const __nv_bfloat16*)qkv, (__nv_bfloat16*)out, cu, seq0, row0,

@@ -416,12 +416,8 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 cudaError_t launch_attention_tc(const void* qkv, void* out, const int* cu, int seq0, int nseq, int row0, int rows,
                                 int max_len, int n_q_heads, int n_kv_heads, int causal, int* err, cudaStream_t st) {
   if (nseq <= 0 || max_len <= 0 || rows <= 0) return cudaSuccess;
-  static bool attr = false;
-  if (!attr) {
-    cudaError_t e = cudaFuncSetAttribute(k_attention_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-    if (e != cudaSuccess) return e;
-    attr = true;
-  }
+  static std::atomic<unsigned long long> smem_set{0};
+  if (cudaError_t e = ensure_dynamic_smem(k_attention_tc, kSmemBytes, smem_set)) return e;
   // Exactly `rows` rows are described, so tiles that run past the batch read zeros, never stale memory.
   const uint64_t ld = (uint64_t)(n_q_heads + 2 * n_kv_heads) * DH;
   TmaDesc mq, mkv;

@@ -5,6 +5,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 namespace prism {
 
 constexpr int kMaxCandidates = 4096;
@@ -70,6 +72,21 @@ constexpr size_t route_scratch_bytes(int n) {
          + ((size_t)n + 1) * sizeof(int) * kMaxClusters  // argmin table
          + ((size_t)n + 1) * sizeof(int) * 2             // valid flags, sorted positions
          + 256;
+}
+
+// Raise a kernel's dynamic shared-memory limit once per device (the attribute is per device; `done` is a
+// bit mask over device ordinals, so concurrent callers at worst set it twice).
+template <typename Kernel>
+inline cudaError_t ensure_dynamic_smem(Kernel kernel, int bytes, std::atomic<unsigned long long>& done) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  const unsigned long long bit = 1ull << (dev & 63);
+  if (done.load(std::memory_order_acquire) & bit) return cudaSuccess;
+  e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e != cudaSuccess) return e;
+  done.fetch_or(bit, std::memory_order_release);
+  return cudaSuccess;
 }
 
 // Opaque 128-byte TMA tensor map (mirrors CUtensorMap so that headers need not include cuda.h).

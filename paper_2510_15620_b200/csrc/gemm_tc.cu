@@ -534,12 +534,14 @@ cudaError_t make_tma_2d_bf16(TmaDesc* out, const void* base, uint64_t rows, uint
 }
 
 int gemm_tc_sm_count() {
-  static int sms = 0;
+  static std::atomic<int> cached{0};  // every GPU of a node is the same part
+  int sms = cached.load(std::memory_order_relaxed);
   if (!sms) {
     int dev = 0;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     if (sms <= 0) sms = 148;
+    cached.store(sms, std::memory_order_relaxed);
   }
   return sms;
 }
@@ -562,15 +564,14 @@ cudaError_t launch_gemm_tc(const TmaDesc& a, const TmaDesc& b0, const TmaDesc& b
                            int n, int k, int epilogue, const QkvRopeArgs* qa, int* err, cudaStream_t st) {
   if (m <= 0 || n <= 0) return cudaSuccess;
   if (k <= 0 || (k % 8) || (n % 8)) return cudaErrorInvalidValue;
-  static bool attr = false;
-  if (!attr) {
-    cudaError_t e;
-    if ((e = cudaFuncSetAttribute(k_gemm_tc<kEpiStore>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes)) ||
-        (e = cudaFuncSetAttribute(k_gemm_tc<kEpiResidual>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes)) ||
-        (e = cudaFuncSetAttribute(k_gemm_tc<kEpiSwiGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes)) ||
-        (e = cudaFuncSetAttribute(k_gemm_tc<kEpiQkvRope>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes)))
-      return e;
-    attr = true;
+  static std::atomic<unsigned long long> smem_set[4];
+  {
+    cudaError_t e = cudaErrorInvalidValue;
+    if (epilogue == kEpiStore) e = ensure_dynamic_smem(k_gemm_tc<kEpiStore>, kSmemBytes, smem_set[0]);
+    else if (epilogue == kEpiResidual) e = ensure_dynamic_smem(k_gemm_tc<kEpiResidual>, kSmemBytes, smem_set[1]);
+    else if (epilogue == kEpiSwiGLU) e = ensure_dynamic_smem(k_gemm_tc<kEpiSwiGLU>, kSmemBytes, smem_set[2]);
+    else if (epilogue == kEpiQkvRope) e = ensure_dynamic_smem(k_gemm_tc<kEpiQkvRope>, kSmemBytes, smem_set[3]);
+    if (e != cudaSuccess) return e;
   }
   const int out_cols = epilogue == kEpiSwiGLU ? 128 : 256;
   const long long tiles = (long long)((m + BM - 1) / BM) * ((n + out_cols - 1) / out_cols);

@@ -320,12 +320,8 @@ cudaError_t launch_route(const float* scores, const int* cu_old, const int* seq2
                          const RouteParams& p, int* cu_new, int* seq2orig_new, int* old_of_new,
                          RouteState* state, int* res_idx, float* res_score, ProbeRecordDev* rec,
                          float* trace_scores, int* trace_ids, void* scratch, cudaStream_t st) {
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(k_route, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(Shared));
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static std::atomic<unsigned long long> smem_set{0};
+  if (cudaError_t e = ensure_dynamic_smem(k_route, (int)sizeof(Shared), smem_set)) return e;
   if (n < 0 || n > kMaxCandidates) return cudaErrorInvalidValue;
   k_route<<<1, kThreads, sizeof(Shared), st>>>(scores, cu_old, seq2orig_old, n, p, cu_new, seq2orig_new,
                                                old_of_new, state, res_idx, res_score, rec, trace_scores,
