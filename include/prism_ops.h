@@ -125,6 +125,12 @@ PRISM_API int prism_op_route_static(const float* scores, const int32_t* cu_old, 
 PRISM_API int prism_op_compact(const float* x_old, float* x_new, const int32_t* cu_old, const int32_t* cu_new,
                      const int32_t* old_of_new, int32_t n_new, int32_t total_new, int32_t d, void* stream);
 
+/* Self-test of the bounded device-side wait that every tensor-core kernel uses (PRISM_ERR_TIMEOUT path):
+ * one thread waits on a barrier that nothing arrives at, gives up after limit_cycles (1 .. 2e9 SM clock
+ * cycles), sets bit 4 of err_word (device int32, zeroed by the caller) and the kernel returns.  Nothing
+ * hangs or faults; the device stays usable. */
+PRISM_API int prism_op_wait_selftest(uint64_t limit_cycles, int32_t* err_word, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

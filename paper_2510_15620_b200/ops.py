@@ -28,6 +28,8 @@ def _L():
         L.prism_op_route.argtypes = [vp, vp, vp, i32, i32, i32, f64, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
         L.prism_op_route_static.argtypes = L.prism_op_route.argtypes
         L.prism_op_route_static.restype = C.c_int
+        L.prism_op_wait_selftest.argtypes = [C.c_uint64, vp, vp]
+        L.prism_op_wait_selftest.restype = C.c_int
         L.prism_op_compact.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, vp]
         for n in ("pack", "embed", "rmsnorm", "qknorm_rope", "gemm", "attention", "probe", "route", "compact"):
             getattr(L, "prism_op_" + n).restype = C.c_int
@@ -105,6 +107,10 @@ def prism_op_route_static(scores, cu_old, seq2orig_old, n, mode, keep_count, cv_
 def prism_op_compact(x_old, x_new, cu_old, cu_new, old_of_new, n_new, total_new):
     _check(_L().prism_op_compact(_p(x_old), _p(x_new), _p(cu_old), _p(cu_new), _p(old_of_new), n_new, total_new,
                                  x_old.shape[1], _stream()), "compact")
+
+
+def prism_op_wait_selftest(limit_cycles, err_word):
+    _check(_L().prism_op_wait_selftest(int(limit_cycles), _p(err_word), _stream()), "wait_selftest")
 
 
 RECORD_BYTES = C.sizeof(_ProbeRecord)

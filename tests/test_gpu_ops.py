@@ -294,6 +294,24 @@ def test_attention_tc_rescales_when_the_maximum_grows(P):
         assert np.max(np.abs(out.float().cpu().numpy() - ref)) < 2e-2 * max(1.0, np.max(np.abs(ref)))
 
 
+def test_bounded_wait_gives_up_and_reports(P):
+    """The wait every tensor-core kernel uses: on a barrier nothing arrives at it returns after its limit
+    and sets the time-out bit; nothing hangs, the device keeps working."""
+    err = torch.zeros(1, dtype=torch.int32, device="cuda")
+    t0 = torch.cuda.Event(enable_timing=True)
+    t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    P.ops.prism_op_wait_selftest(20_000_000, err)              # about 10 ms
+    t1.record()
+    torch.cuda.synchronize()
+    assert int(err.item()) == 4                                  # kErrTimeout and nothing else
+    assert 2.0 < t0.elapsed_time(t1) < 500.0
+    x = torch.arange(10, device="cuda").sum()                    # the context is intact
+    assert int(x.item()) == 45
+    with pytest.raises(P.PrismError):
+        P.ops.prism_op_wait_selftest(0, err)
+
+
 # ------------------------------------------------------------------------------------------ route / compact
 def _run_route(P, scores, ids, lens, k_rem, n_result, sched_kw, is_final=0, layer=3):
     n = len(scores)
