@@ -65,11 +65,12 @@ typedef struct prism_handle prism_handle;
  * architecture of the rerankers the paper evaluates (Sec. 6.1, Table 1). */
 typedef struct {
   int32_t n_layers;   /* 1..PRISM_MAX_LAYERS */
-  int32_t hidden;     /* D; multiple of 64 in bf16 mode, of 4 in fp32 mode */
+  int32_t hidden;     /* D <= 8192; multiple of 8 in bf16 mode, of 4 in fp32 mode */
   int32_t n_q_heads;  /* Hq, multiple of n_kv_heads */
   int32_t n_kv_heads; /* Hkv */
-  int32_t head_dim;   /* dh: 128 in bf16 mode; even, <= 256 in fp32 mode */
-  int32_t ffn;        /* F; multiple of 128 in bf16 mode */
+  int32_t head_dim;   /* dh: 128 for the tensor-core attention kernels (bf16, attention_impl AUTO or MMA);
+                         even and <= 256 for the CUDA-core path (fp32 mode, or attention_impl SIMT) */
+  int32_t ffn;        /* F; multiple of 128 for the tensor-core GEMM (bf16, gemm_impl AUTO), of 8 otherwise in bf16 */
   int32_t vocab;
   float rope_theta;
   float rms_eps;
