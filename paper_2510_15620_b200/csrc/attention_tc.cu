@@ -4,17 +4,19 @@
 // One CTA = 128 query rows of one (sequence, head); two CTAs fit on an SM.  Warp-specialised:
 //   warp 0      TMA producer: Q once, then K_j tiles (64 keys) into a 3-deep ring and V_j tiles into a
 //               2-deep ring; a K slot is released as soon as its Q K^T has run, a V slot after P V
-//   warp 1      MMA issuer:   S_j = Q K_j^T (tcgen05.mma M128 N64 K16 x 8) into one of two TMEM buffers,
-//                             O += P_j V_j  (M128 N128 K16 x 4; P read from TENSOR MEMORY, V as an
-//                             MN-major shared-memory operand) into TMEM
+//   warp 1      score issuer: S_j = Q K_j^T (tcgen05.mma M128 N64 K16 x 8) into one of two TMEM buffers
+//   warp 10     output issuer: O += P_j V_j (M128 N128 K16 x 4; P read from TENSOR MEMORY, V as an
+//               MN-major shared-memory operand) into TMEM.  Two issuing threads, so that the next
+//               scores never queue behind the wait for the current probabilities.
 //   warps 2..9  softmax: two threads per query row (warps w and w+4 share a 32-row TMEM lane quarter and
 //               take 32 of the 64 key columns each); read S_j from TMEM, exchange the row maximum,
 //               exponentiate against a running reference maximum and store P_j as packed bf16 back
 //               into the first 32 columns of the S_j buffer (tcgen05.st); O stays in TMEM and is
 //               rescaled (TMEM read-modify-write) only when a row's maximum outgrows the reference by
 //               more than 2^8.
-// S_{j+1} is issued before P_j is awaited, so the tensor core computes the next scores while the
-// softmax warps work.  Every mbarrier wait is bounded; on expiry the kernel records kErrTimeout, all
+// S_{j+1} and S_{j+2}... are issued as soon as their K tile has landed and their TMEM buffer is free (the
+// output issuer releases buffer j&1 with a commit after P_j V_j), so the tensor core computes the next
+// scores while the softmax warps work.  Every mbarrier wait is bounded; on expiry the kernel records kErrTimeout, all
 // roles drain to the common exit and the tensor memory is freed.  No cluster multicast.
 #include "tc_common.cuh"
 
@@ -35,7 +37,7 @@ constexpr int kTileBytes = kQBytes + NK * kKBytes + NV * kVBytes;  // 112 KB
 // shared window starts on a 1024-byte boundary (the swizzled tiles need it) and reports if not.
 constexpr int kSmemBytes = kTileBytes + 256 + kXchBytes;
 static_assert(2 * (kSmemBytes + 1024) <= 233472, "two CTAs per SM must fit in 228 KB of shared memory");
-constexpr int kThreads = 320;                 // TMA warp, MMA warp, 8 softmax warps
+constexpr int kThreads = 352;                 // TMA warp, score-MMA warp, 8 softmax warps, output-MMA warp
 constexpr int kTmemCols = 256;                // S: 2 x 64, O: 128
 
 __device__ __forceinline__ float ex2(float x) {  // 2^x on the special-function unit; -inf -> 0
@@ -86,7 +88,7 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       mbar_init(b_v_full + 8 * i, 1);
       mbar_init(b_v_empty + 8 * i, 1);
       mbar_init(b_s_full + 8 * i, 1);
-      mbar_init(b_s_empty + 8 * i, 8);
+      mbar_init(b_s_empty + 8 * i, 1);  // released by a commit of the output issuer
     }
     mbar_init(b_p_full, 8);
     mbar_init(b_o_full, 1);
@@ -131,34 +133,34 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       }
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer
+    // ------------------------------------------------------------------ score issuer: S_j = Q K_j^T
     if (lane == 0) {
-      constexpr uint32_t kIdescS = idesc_bf16(BM, BN, 0), kIdescO = idesc_bf16(BM, DH, 1);
+      constexpr uint32_t kIdescS = idesc_bf16(BM, BN, 0);
       bool ok = mbar_wait(b_q, 0, err, abort_flag);
-      auto issue_qk = [&](int j) {
-        const int st = j % NK;
+      for (int j = 0; j < n_blocks && ok; ++j) {
+        const int st = j % NK, b = j & 1, u = j >> 1;
+        if (!mbar_wait(b_k_full + 8 * st, (j / NK) & 1, err, abort_flag)) break;
+        // buffer b held S_{j-2} and then P_{j-2}; it is free once P_{j-2} V_{j-2} has completed
+        if (!mbar_wait(b_s_empty + 8 * b, (u & 1) ^ 1, err, abort_flag)) break;
         const uint32_t sk = s_k + st * kKBytes;
         tc_fence_after();
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk) {  // 16 head-dim elements per step; sub-tile switches at kk = 4
           const uint64_t da = smem_desc(s_q + (kk >> 2) * (kQBytes / 2) + (kk & 3) * 32, 16, 1024);
           const uint64_t db = smem_desc(sk + (kk >> 2) * (kKBytes / 2) + (kk & 3) * 32, 16, 1024);
-          umma_bf16(t_s + (j & 1) * BN, da, db, kIdescS, kk != 0);
+          umma_bf16(t_s + b * BN, da, db, kIdescS, kk != 0);
         }
-        umma_commit(b_s_full + 8 * (j & 1));
+        umma_commit(b_s_full + 8 * b);
         umma_commit(b_k_empty + 8 * st);  // the K tile is free as soon as these MMAs have read it
-      };
-      if (ok) ok = mbar_wait(b_k_full, 0, err, abort_flag);
-      if (ok) issue_qk(0);
-      for (int j = 0; j < n_blocks && ok; ++j) {
-        if (j + 1 < n_blocks) {
-          const int b = (j + 1) & 1, u = (j + 1) >> 1;
-          if (!mbar_wait(b_k_full + 8 * ((j + 1) % NK), ((j + 1) / NK) & 1, err, abort_flag)) { ok = false; break; }
-          if (!mbar_wait(b_s_empty + 8 * b, (u & 1) ^ 1, err, abort_flag)) { ok = false; break; }
-          issue_qk(j + 1);
-        }
-        if (!mbar_wait(b_p_full, j & 1, err, abort_flag)) { ok = false; break; }
-        if (!mbar_wait(b_v_full + 8 * (j & 1), (j >> 1) & 1, err, abort_flag)) { ok = false; break; }
+      }
+    }
+  } else if (warp == 10) {
+    // ------------------------------------------------------------------ output issuer: O += P_j V_j
+    if (lane == 0) {
+      constexpr uint32_t kIdescO = idesc_bf16(BM, DH, 1);
+      for (int j = 0; j < n_blocks; ++j) {
+        if (!mbar_wait(b_p_full, j & 1, err, abort_flag)) break;
+        if (!mbar_wait(b_v_full + 8 * (j & 1), (j >> 1) & 1, err, abort_flag)) break;
         tc_fence_after();
         const uint32_t sv = s_v + (j & 1) * kVBytes;
 #pragma unroll
@@ -168,6 +170,7 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         }
         umma_commit(b_o_full);
         umma_commit(b_v_empty + 8 * (j & 1));
+        umma_commit(b_s_empty + 8 * (j & 1));  // S/P buffer j&1 may be overwritten by Q K_{j+2}^T
       }
     }
   } else {
@@ -187,9 +190,6 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       uint32_t sr[32];
       tmem_ld32(t_s + lane_base + b * BN + colhalf * 32, sr);
       tmem_ld_wait();
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(b_s_empty + 8 * b);  // one arrival per warp
       const int key0 = j * BN + colhalf * 32;
       if ((causal && j * BN + BN - 1 > qb * BM) || j * BN + BN > len) {
 #pragma unroll
@@ -247,8 +247,8 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       }
       l += rs;
       // P_j (packed bf16) goes over the first 32 columns of the S_j buffer: both threads of the row have
-      // loaded their S values (they met at the pair barrier above), and Q K_{j+2}^T is only issued after
-      // P_j V_j, so nothing else touches these columns meanwhile.
+      // loaded their S values (they met at the pair barrier above), and Q K_{j+2}^T is only issued once
+      // P_j V_j has completed (s_empty), so nothing else touches these columns meanwhile.
       tmem_st16(t_s + lane_base + b * BN + colhalf * 16, pk);
       tmem_st_wait();
       tc_fence_before();
