@@ -236,15 +236,20 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         }
       }
       const float ms = m_ref * scale_log2;
-      float rs = 0.f;
       uint32_t pk[16];
+      const uint64_t sc2 = f2_pack(scale_log2, scale_log2), nm2 = f2_pack(-ms, -ms);
+      uint64_t rs2 = f2_pack(0.f, 0.f);
 #pragma unroll
       for (int c = 0; c < 16; ++c) {
-        const float p0 = ex2(fmaf(__uint_as_float(sr[2 * c]), scale_log2, -ms));
-        const float p1 = ex2(fmaf(__uint_as_float(sr[2 * c + 1]), scale_log2, -ms));
-        rs += p0 + p1;
+        float x0, x1;
+        f2_unpack(f2_fma(f2_pack(__uint_as_float(sr[2 * c]), __uint_as_float(sr[2 * c + 1])), sc2, nm2), x0, x1);
+        const float p0 = ex2(x0), p1 = ex2(x1);
+        rs2 = f2_add(rs2, f2_pack(p0, p1));
         pk[c] = pack_bf16(p0, p1);  // key 2c in the low half, key 2c+1 in the high half
       }
+      float rs, rs_hi;
+      f2_unpack(rs2, rs, rs_hi);
+      rs += rs_hi;
       l += rs;
       // P_j (packed bf16) goes over the first 32 columns of the S_j buffer: both threads of the row have
       // loaded their S values (they met at the pair barrier above), and Q K_{j+2}^T is only issued once
