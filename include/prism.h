@@ -54,9 +54,11 @@ typedef enum {
 enum { PRISM_FP32 = 0, PRISM_BF16 = 1 };
 enum { PRISM_WEIGHTS_DEVICE = 0, PRISM_WEIGHTS_HOST_STREAMED = 1 };
 enum { PRISM_PRUNE_NONE = 0, PRISM_PRUNE_FIXED_KEEP = 1, PRISM_PRUNE_CLUSTER = 2 };
-/* Implementation selectors (validation): AUTO picks the tcgen05 tensor-core kernels in bf16 mode,
- * SIMT the CUDA-core kernels, MMA (attention only) the warp-level mma.sync flash-attention kernel. */
-enum { PRISM_IMPL_AUTO = 0, PRISM_IMPL_SIMT = 1, PRISM_IMPL_MMA = 2 };
+/* Implementation selectors (validation): AUTO picks the tcgen05 tensor-core kernels in bf16 mode (the GEMM on
+ * CTA pairs: cta_group::2, one 256x256 tile per two-CTA cluster), SIMT the CUDA-core kernels, MMA (attention
+ * only) the warp-level mma.sync flash-attention kernel, SOLO (GEMM only) the single-CTA tcgen05 kernel with
+ * 128x256 tiles. */
+enum { PRISM_IMPL_AUTO = 0, PRISM_IMPL_SIMT = 1, PRISM_IMPL_MMA = 2, PRISM_IMPL_SOLO = 3 };
 
 typedef struct prism_handle prism_handle;
 

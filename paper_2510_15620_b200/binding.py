@@ -10,7 +10,7 @@ import numpy as np
 import torch
 
 PRISM_FP32, PRISM_BF16 = 0, 1
-PRISM_IMPL_AUTO, PRISM_IMPL_SIMT, PRISM_IMPL_MMA = 0, 1, 2
+PRISM_IMPL_AUTO, PRISM_IMPL_SIMT, PRISM_IMPL_MMA, PRISM_IMPL_SOLO = 0, 1, 2, 3
 PRISM_MAX_CLUSTERS = 8
 
 # PRISM_LIBRARY overrides the in-tree library (e.g. an instrumented build of the same sources).

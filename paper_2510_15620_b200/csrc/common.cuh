@@ -132,6 +132,9 @@ cudaError_t make_tma_2d_bf16(TmaDesc* out, const void* base, uint64_t rows, uint
 // projections, the gate and the up matrix for kEpiSwiGLU.
 cudaError_t launch_gemm_tc(const TmaDesc& a, const TmaDesc& b0, const TmaDesc& b1, void* out, float* resid, int m,
                            int n, int k, int epilogue, const QkvRopeArgs* qa, int* err, cudaStream_t st);
+// The same GEMM on CTA pairs (tcgen05 cta_group::2, 256x256 tiles per cluster of two CTAs).
+cudaError_t launch_gemm_tc2(const TmaDesc& a, const TmaDesc& b0, const TmaDesc& b1, void* out, float* resid, int m,
+                            int n, int k, int epilogue, const QkvRopeArgs* qa, int* err, cudaStream_t st);
 cudaError_t launch_attention_tc(const void* qkv, void* out, const int* cu, int seq0, int nseq, int row0, int rows,
                                 int max_len, int n_q_heads, int n_kv_heads, int causal, int* err, cudaStream_t st);
 cudaError_t launch_attention_mma(const void* qkv, void* out, const int* cu, int seq0, int nseq, int row0,

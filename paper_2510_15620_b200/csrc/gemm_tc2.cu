@@ -1,0 +1,500 @@
+// The projection GEMMs of gemm_tc.cu on CTA PAIRS (tcgen05 cta_group::2): a cluster of two CTAs computes a
+// 256x256 tile; each CTA loads its own 128 rows of A and ONE HALF (128 rows) of the B tile, the leader's
+// elected thread issues M256 N256 K16 MMAs that read both CTAs' shared memory, and each CTA's tensor
+// memory receives its own 128 accumulator rows.  Per SM this halves the B operand traffic through shared
+// memory, which is the co-limit of the single-CTA kernel.  Epilogues are the same code as in gemm_tc.cu.
+//
+// Protocol: full[s] lives in the leader and counts the bytes of BOTH CTAs' TMA loads; empty[s] and
+// acc_full[a] exist in both CTAs and are signalled by multicast commits; acc_empty[a] lives in the leader
+// and is arrived on by the epilogue warps of both CTAs.  No TMA multicast is used.  Every wait is bounded.
+#include "tc_common.cuh"
+
+namespace prism {
+
+namespace {
+
+using namespace tc;
+
+constexpr int BM = 128, BN = 256, BK = 64, UMMA_K = 16;
+constexpr int kStages = 6;
+constexpr int kABytes = BM * BK * 2;           // 16 KB
+constexpr int kBBytes = (BN / 2) * BK * 2;     // 16 KB: this CTA's half of the B tile
+constexpr int kStageBytes = kABytes + kBBytes; // 32 KB
+constexpr int kEpiBufBytes = 32 * 32 * 4;      // one 32x32 fp32 sub-tile staged for a TMA reduce-add
+constexpr int kEpiStageBytes = 4 * 2 * kEpiBufBytes;  // 4 epilogue warps x 2 buffers
+constexpr int kSmemBytes = kStages * kStageBytes + kEpiStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int kThreads = 320;  // TMA warp, MMA warp, 8 epilogue warps
+
+// x[tile] += smem tile (fp32), performed by the TMA unit / L2; rows and columns outside the tensor are clipped.
+__device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap* map, uint32_t src, int c0, int c1) {
+  asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3}], [%1];"
+               ::"l"(map), "r"(src), "r"(c0), "r"(c1)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait() { asm volatile("cp.async.bulk.wait_group %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// Address of the same shared-memory offset in CTA `rank` of the cluster.
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// TMA tile load of the pair form: data lands in this CTA, the byte count is reported to `bar`, which may
+// be a barrier of the other CTA of the pair (a shared::cluster address).
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void umma_bf16_pair(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc,
+                                               uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// Arrives on the barrier at this offset in BOTH CTAs once all MMAs issued so far have completed.
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"((uint16_t)3) : "memory");
+}
+
+// kind::f16 instruction descriptor: D fp32, A/B bf16, both K-major, M=128, N=256.
+constexpr uint32_t kIdesc = idesc_bf16(2 * BM, BN, 0);  // the pair's instruction: M = 256
+
+template <int kEpi>
+__global__ void __launch_bounds__(kThreads, 1)
+k_gemm_tc2(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b0,
+          const __grid_constant__ CUtensorMap map_b1, const __grid_constant__ CUtensorMap map_r,
+          __nv_bfloat16* __restrict__ out, int m, int n, int k, const QkvRopeArgs qa, int* __restrict__ err) {
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t tiles = (raw + 1023u) & ~1023u;  // swizzled tiles need 1024-byte alignment
+  unsigned char* gen_tiles = smem_raw + (tiles - raw);
+  const uint32_t epi_stage = tiles + kStages * kStageBytes;  // 1024-byte aligned
+  uint64_t* bars = reinterpret_cast<uint64_t*>(gen_tiles + kStages * kStageBytes + kEpiStageBytes);
+  // bars: full[kStages], empty[kStages], acc_full[2], acc_empty[2]; then tmem base and abort flag
+  const uint32_t bar_full = smem_u32(bars), bar_empty = smem_u32(bars + kStages);
+  const uint32_t bar_acc_full = smem_u32(bars + 2 * kStages), bar_acc_empty = smem_u32(bars + 2 * kStages + 2);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 4);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  // Output tile width: SwiGLU tiles hold 128 gate + 128 up columns and produce 128 outputs.
+  constexpr int kOutCols = (kEpi == kEpiSwiGLU) ? 128 : 256;
+  (void)epi_stage;
+  // A pair works on 256 rows: its tile index t names rows [256*(t / n_tiles), +256), of which this CTA owns
+  // the half selected by its rank in the cluster.
+  const uint32_t rank = cluster_ctarank();
+  const bool leader = rank == 0;
+  const int pair_id = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+  const int m_tiles2 = (m + 2 * BM - 1) / (2 * BM), n_tiles = (n + kOutCols - 1) / kOutCols;
+  const int num_tiles = m_tiles2 * n_tiles, num_kb = (k + BK - 1) / BK;
+  auto my_m_tile = [&](int t) { return (t / n_tiles) * 2 + (int)rank; };  // in units of 128 rows
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(bar_full + 8 * s, 1);
+      mbar_init(bar_empty + 8 * s, 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(bar_acc_full + 8 * a, 1);
+      mbar_init(bar_acc_empty + 8 * a, 16);  // 8 epilogue warps of each CTA of the pair (used in the leader)
+    }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  cluster_sync();  // both CTAs' barriers exist before anything can signal them
+  if (warp == 1) {  // both CTAs of the pair allocate all 512 tensor-memory columns (two 256-column accumulators)
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512));
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::);
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const uint32_t leader_full = map_to_cta(bar_full, 0);            // full[] of the leader, as seen from this CTA
+  const uint32_t leader_acc_empty = map_to_cta(bar_acc_empty, 0);  // acc_empty[] of the leader
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer (one per CTA)
+    if (lane == 0) {
+      uint32_t stage = 0, phase = 0;
+      bool ok = true;
+      for (int tile = pair_id; tile < num_tiles && ok; tile += n_pairs) {
+        const int mt = my_m_tile(tile), nt = tile % n_tiles;
+        const int row_a = mt * BM;
+        // this CTA's half of the B tile: rows [128*rank, +128) of the 256-row tile, or for SwiGLU the gate
+        // rows (rank 0) / the up rows (rank 1) of the tile's 128 outputs
+        const CUtensorMap* map_b = (kEpi == kEpiSwiGLU && rank == 1) ? &map_b1 : &map_b0;
+        const int row_b = (kEpi == kEpiSwiGLU) ? nt * 128 : nt * BN + (int)rank * 128;
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1, err, abort_flag)) { ok = false; break; }
+          const uint32_t sa = tiles + stage * kStageBytes, sb = sa + kABytes;
+          // the leader's barrier collects the bytes of both CTAs
+          if (leader) mbar_expect_tx(bar_full + 8 * stage, 2 * kStageBytes);
+          tma_load_2d_pair(sa, &map_a, kb * BK, row_a, leader_full + 8 * stage);
+          tma_load_2d_pair(sb, map_b, kb * BK, row_b, leader_full + 8 * stage);
+          if (++stage == kStages) { stage = 0; phase ^= 1; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer (leader CTA only)
+    if (lane == 0 && leader) {
+      uint32_t stage = 0, phase = 0;
+      bool ok = true;
+      int it = 0;
+      for (int tile = pair_id; tile < num_tiles && ok; tile += n_pairs, ++it) {
+        const uint32_t acc = it & 1, acc_phase = (it >> 1) & 1;
+        if (!mbar_wait(bar_acc_empty + 8 * acc, acc_phase ^ 1, err, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + acc * BN;
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!mbar_wait(bar_full + 8 * stage, phase, err, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = tiles + stage * kStageBytes, sb = sa + kABytes;
+          const uint64_t da = smem_desc(sa, 16, 1024), db = smem_desc(sb, 16, 1024);
+#pragma unroll
+          for (int kk = 0; kk < BK / UMMA_K; ++kk) {
+            umma_bf16_pair(d_tmem, da + 2 * kk, db + 2 * kk, kIdesc, (kb | kk) != 0);
+          }
+          umma_commit_pair(bar_empty + 8 * stage);  // the stage is free in both CTAs once these MMAs have read it
+          if (++stage == kStages) { stage = 0; phase ^= 1; }
+        }
+        if (ok) umma_commit_pair(bar_acc_full + 8 * acc);  // both CTAs' halves of the accumulator are complete
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue (8 warps, 128 rows x 2 column halves)
+    const int quarter = warp & 3;        // TMEM lane quarter this warp may read
+    const int colhalf = (warp - 2) >> 2;  // 0: first half of the tile's columns, 1: second half
+    bool ok = true;
+    int it = 0;
+    // QKV epilogue: the row's position and the first half of its rotary table rows do not depend on the
+    // accumulator, so they are requested before the wait for it (their L2 latency hides behind the MMAs).
+    [[maybe_unused]] int rope_pos = 0;
+    [[maybe_unused]] float4 tv[8];
+    [[maybe_unused]] auto rope_row_pos = [&](int t) {
+      const int rw = my_m_tile(t) * BM + quarter * 32 + lane;
+      return qa.pos[rw < m ? rw : 0];
+    };
+    [[maybe_unused]] auto rope_fetch = [&](int half) {
+#pragma unroll
+      for (int i8 = 0; i8 < 8; ++i8) {
+        const int rr = (colhalf * 8 + i8) * 2 + (lane >> 4);  // this warp fetches 16 of the quarter's 32 rows
+        const int p = __shfl_sync(0xffffffffu, rope_pos, rr);
+        tv[i8] = __ldg(reinterpret_cast<const float4*>(qa.tab + (size_t)p * 128 + half * 64) + (lane & 15));
+      }
+    };
+    if constexpr (kEpi == kEpiQkvRope) {
+      if (pair_id < num_tiles) rope_pos = rope_row_pos(pair_id);
+    }
+    for (int tile = pair_id; tile < num_tiles && ok; tile += n_pairs, ++it) {
+      const uint32_t acc = it & 1, acc_phase = (it >> 1) & 1;
+      const int mt = my_m_tile(tile), nt = tile % n_tiles;
+      [[maybe_unused]] int rope_pos_next = 0;
+      if constexpr (kEpi == kEpiQkvRope) {
+        if (nt * 2 < qa.hq + qa.hkv) rope_fetch(0);
+        if (tile + n_pairs < num_tiles) rope_pos_next = rope_row_pos(tile + n_pairs);
+      }
+      if (!mbar_wait(bar_acc_full + 8 * acc, acc_phase, err, abort_flag)) { ok = false; break; }
+      tc_fence_after();
+      const int row = mt * BM + quarter * 32 + lane;
+      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN;
+      const int col0 = nt * kOutCols;
+      if constexpr (kEpi == kEpiSwiGLU) {
+#pragma unroll 1
+        for (int cc = 0; cc < 2; ++cc) {
+          const int c = colhalf * 2 + cc;  // 32 of the tile's 128 outputs: gate columns c*32.., up columns 128 + c*32..
+          uint32_t g[32], u[32];
+          tmem_ld32(taddr + c * 32, g);
+          tmem_ld32(taddr + 128 + c * 32, u);
+          tmem_ld_wait();
+          if (row < m) {
+            __nv_bfloat16* o = out + (size_t)row * n + col0 + c * 32;
+#pragma unroll
+            for (int v = 0; v < 4; ++v) {
+              if (col0 + c * 32 + v * 8 < n) {
+                uint32_t pk[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                  const float g0 = __uint_as_float(g[v * 8 + 2 * e]), g1 = __uint_as_float(g[v * 8 + 2 * e + 1]);
+                  const float u0 = __uint_as_float(u[v * 8 + 2 * e]), u1 = __uint_as_float(u[v * 8 + 2 * e + 1]);
+                  pk[e] = pack_bf16(__fdividef(g0, 1.f + __expf(-g0)) * u0, __fdividef(g1, 1.f + __expf(-g1)) * u1);
+                }
+                *reinterpret_cast<uint4*>(o + v * 8) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+              }
+            }
+          }
+        }
+      } else if constexpr (kEpi == kEpiResidual) {
+        // 32x32 fp32 sub-tiles go through this warp's staging buffer (128-byte swizzle) into a TMA reduce-add.
+        const uint32_t buf = epi_stage + (uint32_t)(warp - 2) * kEpiBufBytes;
+#pragma unroll 1
+        for (int cc = 0; cc < 4; ++cc) {
+          const int c = colhalf * 4 + cc;
+          // sub-tiles outside the matrix are skipped (warp-uniform)
+          if (col0 + c * 32 >= n || mt * BM + quarter * 32 >= m) break;
+          uint32_t r[32];
+          tmem_ld32(taddr + c * 32, r);
+          if (lane == 0) bulk_wait_read<0>();  // the previous reduce has finished reading the buffer
+          __syncwarp();
+          tmem_ld_wait();
+#pragma unroll
+          for (int v = 0; v < 8; ++v) {
+            const uint32_t dst = buf + lane * 128 + ((v ^ (lane & 7)) << 4);
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(r[4 * v]), "r"(r[4 * v + 1]),
+                         "r"(r[4 * v + 2]), "r"(r[4 * v + 3]) : "memory");
+          }
+          fence_async_smem();
+          __syncwarp();
+          if (lane == 0) {
+            tma_reduce_add_2d(&map_r, buf, col0 + c * 32, mt * BM + quarter * 32);
+            bulk_commit();
+          }
+        }
+      } else if constexpr (kEpi == kEpiQkvRope) {
+        // A 256-column tile is two heads; this warp owns head `colhalf` of the tile.  q and k heads:
+        // optional RMSNorm over the head, then the rotation of pairs (i, i+64); v heads are stored as
+        // they are.  The rotary table rows of the quarter's 32 rows are fetched coalesced (256 bytes per
+        // row and half) into a staging buffer shared by the two warps of the quarter, 16-byte chunks
+        // XOR-swizzled by row so that every thread reads its own row without bank conflicts.
+        const uint32_t stage = epi_stage + (uint32_t)quarter * 2 * kEpiBufBytes;  // 8 KB = 32 rows x 256 B
+        const int pair_bar = 1 + quarter;                                         // named barrier of the two warps
+        const int head = nt * 2 + colhalf;
+        const bool live = head * 128 < n;
+        const bool rot = live && head < qa.hq + qa.hkv;
+        const bool any_rot = nt * 2 < qa.hq + qa.hkv;  // same for both warps of the pair
+        const uint32_t th = taddr + colhalf * 128;
+        auto stage_table = [&]() {
+#pragma unroll
+          for (int i8 = 0; i8 < 8; ++i8) {
+            const int rr = (colhalf * 8 + i8) * 2 + (lane >> 4), ch = lane & 15;
+            const uint32_t dst = stage + rr * 256 + ((ch ^ (rr & 7)) << 4);
+            asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "f"(tv[i8].x), "f"(tv[i8].y), "f"(tv[i8].z),
+                         "f"(tv[i8].w) : "memory");
+          }
+        };
+        float rnh = 1.f;
+        if (rot && qa.qk_norm) {
+          float ss = 0.f;
+#pragma unroll 1
+          for (int c = 0; c < 4; ++c) {
+            uint32_t r[32];
+            tmem_ld32(th + c * 32, r);
+            tmem_ld_wait();
+#pragma unroll
+            for (int e = 0; e < 32; ++e) ss = fmaf(__uint_as_float(r[e]), __uint_as_float(r[e]), ss);
+          }
+          rnh = 1.0f / sqrtf(ss * (1.f / 128.f) + qa.eps);
+        }
+        __nv_bfloat16* o = out + (size_t)row * n + (size_t)head * 128;
+        const __nv_bfloat16* gain = head < qa.hq ? qa.g_q : qa.g_k;
+#pragma unroll 1
+        for (int half = 0; half < 2; ++half) {
+          if (any_rot) {
+            // both warps are done reading the previous half before it is overwritten
+            asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
+            stage_table();
+            asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
+            if (half == 0) rope_fetch(1);
+          }
+          if (!live) continue;
+          uint32_t a[32], b[32];
+          tmem_ld32(th + half * 32, a);
+          tmem_ld32(th + 64 + half * 32, b);
+          tmem_ld_wait();
+          if (!rot) {  // v head: plain store of the two 32-column pieces
+            if (row < m) {
+#pragma unroll
+              for (int v = 0; v < 4; ++v) {
+                uint4 pa, pb;
+                pa.x = pack_bf16(__uint_as_float(a[v * 8 + 0]), __uint_as_float(a[v * 8 + 1]));
+                pa.y = pack_bf16(__uint_as_float(a[v * 8 + 2]), __uint_as_float(a[v * 8 + 3]));
+                pa.z = pack_bf16(__uint_as_float(a[v * 8 + 4]), __uint_as_float(a[v * 8 + 5]));
+                pa.w = pack_bf16(__uint_as_float(a[v * 8 + 6]), __uint_as_float(a[v * 8 + 7]));
+                pb.x = pack_bf16(__uint_as_float(b[v * 8 + 0]), __uint_as_float(b[v * 8 + 1]));
+                pb.y = pack_bf16(__uint_as_float(b[v * 8 + 2]), __uint_as_float(b[v * 8 + 3]));
+                pb.z = pack_bf16(__uint_as_float(b[v * 8 + 4]), __uint_as_float(b[v * 8 + 5]));
+                pb.w = pack_bf16(__uint_as_float(b[v * 8 + 6]), __uint_as_float(b[v * 8 + 7]));
+                *reinterpret_cast<uint4*>(o + half * 32 + v * 8) = pa;
+                *reinterpret_cast<uint4*>(o + 64 + half * 32 + v * 8) = pb;
+              }
+            }
+            continue;
+          }
+#pragma unroll
+          for (int v = 0; v < 4; ++v) {
+            float x0[8], x1[8], cs[8], sn[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+              x0[e] = __uint_as_float(a[v * 8 + e]);
+              x1[e] = __uint_as_float(b[v * 8 + e]);
+            }
+            if (qa.qk_norm) {
+              const uint4 g0 = __ldg(reinterpret_cast<const uint4*>(gain + half * 32 + v * 8));
+              const uint4 g1 = __ldg(reinterpret_cast<const uint4*>(gain + 64 + half * 32 + v * 8));
+              const __nv_bfloat16* p0 = reinterpret_cast<const __nv_bfloat16*>(&g0);
+              const __nv_bfloat16* p1 = reinterpret_cast<const __nv_bfloat16*>(&g1);
+#pragma unroll
+              for (int e = 0; e < 8; ++e) {
+                x0[e] = x0[e] * rnh * __bfloat162float(p0[e]);
+                x1[e] = x1[e] * rnh * __bfloat162float(p1[e]);
+              }
+            }
+            // staged row: chunks 0..7 = cos(32*half + 0..31), chunks 8..15 = sin
+#pragma unroll
+            for (int q4 = 0; q4 < 2; ++q4) {
+              const int cc = v * 2 + q4;
+              const uint32_t ca = stage + lane * 256 + ((cc ^ (lane & 7)) << 4);
+              const uint32_t sa = stage + lane * 256 + (((cc + 8) ^ (lane & 7)) << 4);
+              asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                           : "=f"(cs[q4 * 4]), "=f"(cs[q4 * 4 + 1]), "=f"(cs[q4 * 4 + 2]), "=f"(cs[q4 * 4 + 3]) : "r"(ca));
+              asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                           : "=f"(sn[q4 * 4]), "=f"(sn[q4 * 4 + 1]), "=f"(sn[q4 * 4 + 2]), "=f"(sn[q4 * 4 + 3]) : "r"(sa));
+            }
+            uint32_t lo[4], hi[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const float y0 = x0[2 * e] * cs[2 * e] - x1[2 * e] * sn[2 * e];
+              const float y1 = x0[2 * e + 1] * cs[2 * e + 1] - x1[2 * e + 1] * sn[2 * e + 1];
+              const float z0 = x1[2 * e] * cs[2 * e] + x0[2 * e] * sn[2 * e];
+              const float z1 = x1[2 * e + 1] * cs[2 * e + 1] + x0[2 * e + 1] * sn[2 * e + 1];
+              lo[e] = pack_bf16(y0, y1);
+              hi[e] = pack_bf16(z0, z1);
+            }
+            if (row < m) {
+              *reinterpret_cast<uint4*>(o + half * 32 + v * 8) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+              *reinterpret_cast<uint4*>(o + 64 + half * 32 + v * 8) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+            }
+          }
+        }
+      } else {
+#pragma unroll 1
+        for (int cc = 0; cc < 4; ++cc) {
+          const int c = colhalf * 4 + cc;
+          uint32_t r[32];
+          tmem_ld32(taddr + c * 32, r);
+          tmem_ld_wait();
+          if (row < m) {
+            __nv_bfloat16* o = out + (size_t)row * n + col0 + c * 32;
+#pragma unroll
+            for (int v = 0; v < 4; ++v) {
+              if (col0 + c * 32 + v * 8 < n) {
+                uint4 pk;
+                pk.x = pack_bf16(__uint_as_float(r[v * 8 + 0]), __uint_as_float(r[v * 8 + 1]));
+                pk.y = pack_bf16(__uint_as_float(r[v * 8 + 2]), __uint_as_float(r[v * 8 + 3]));
+                pk.z = pack_bf16(__uint_as_float(r[v * 8 + 4]), __uint_as_float(r[v * 8 + 5]));
+                pk.w = pack_bf16(__uint_as_float(r[v * 8 + 6]), __uint_as_float(r[v * 8 + 7]));
+                *reinterpret_cast<uint4*>(o + v * 8) = pk;
+              }
+            }
+          }
+        }
+      }
+      if constexpr (kEpi == kEpiQkvRope) rope_pos = rope_pos_next;
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(leader_acc_empty + 8 * acc);  // the leader's MMA thread waits for both CTAs
+    }
+    if constexpr (kEpi == kEpiResidual) {
+      if (lane == 0) bulk_wait<0>();  // all reduce-adds of this warp have completed
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync();  // neither CTA frees its shared or tensor memory while the other may still use or signal it
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512));
+  }
+}
+
+}  // namespace
+
+cudaError_t make_tma_2d_f32_box32(TmaDesc* out, const void* base, uint64_t rows, uint64_t cols);
+int gemm_tc_sm_count();
+
+cudaError_t launch_gemm_tc2(const TmaDesc& a, const TmaDesc& b0, const TmaDesc& b1, void* out, float* resid, int m,
+                           int n, int k, int epilogue, const QkvRopeArgs* qa, int* err, cudaStream_t st) {
+  if (m <= 0 || n <= 0) return cudaSuccess;
+  if (k <= 0 || (k % 8) || (n % 8)) return cudaErrorInvalidValue;
+  static std::atomic<unsigned long long> smem_set[4];
+  {
+    cudaError_t e = cudaErrorInvalidValue;
+    if (epilogue == kEpiStore) e = ensure_dynamic_smem(k_gemm_tc2<kEpiStore>, kSmemBytes, smem_set[0]);
+    else if (epilogue == kEpiResidual) e = ensure_dynamic_smem(k_gemm_tc2<kEpiResidual>, kSmemBytes, smem_set[1]);
+    else if (epilogue == kEpiSwiGLU) e = ensure_dynamic_smem(k_gemm_tc2<kEpiSwiGLU>, kSmemBytes, smem_set[2]);
+    else if (epilogue == kEpiQkvRope) e = ensure_dynamic_smem(k_gemm_tc2<kEpiQkvRope>, kSmemBytes, smem_set[3]);
+    if (e != cudaSuccess) return e;
+  }
+  const int out_cols = epilogue == kEpiSwiGLU ? 128 : 256;
+  const long long tiles = (long long)((m + 2 * BM - 1) / (2 * BM)) * ((n + out_cols - 1) / out_cols);
+  const int pairs = gemm_tc_sm_count() / 2;
+  const int grid = 2 * (int)(tiles < pairs ? tiles : pairs);
+  const CUtensorMap& ma = reinterpret_cast<const CUtensorMap&>(a);
+  const CUtensorMap& mb0 = reinterpret_cast<const CUtensorMap&>(b0);
+  const CUtensorMap& mb1 = reinterpret_cast<const CUtensorMap&>(b1);
+  TmaDesc rdesc = a;  // placeholder for the epilogues that do not use it
+  QkvRopeArgs q{};
+  if (epilogue == kEpiResidual) {
+    // the residual rows of this launch, exactly m of them, so that the TMA unit clips the ragged last tile
+    cudaError_t e = make_tma_2d_f32_box32(&rdesc, resid, (uint64_t)m, (uint64_t)n);
+    if (e != cudaSuccess) return e;
+  }
+  if (epilogue == kEpiQkvRope) {
+    if (!qa || n % 128) return cudaErrorInvalidValue;
+    q = *qa;
+  }
+  const CUtensorMap& mr = reinterpret_cast<const CUtensorMap&>(rdesc);
+  __nv_bfloat16* o = (__nv_bfloat16*)out;
+  // clusters of two CTAs along x
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = kSmemBytes;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaError_t le;
+  if (epilogue == kEpiStore)
+    le = cudaLaunchKernelEx(&cfg, k_gemm_tc2<kEpiStore>, ma, mb0, mb1, mr, o, m, n, k, q, err);
+  else if (epilogue == kEpiResidual)
+    le = cudaLaunchKernelEx(&cfg, k_gemm_tc2<kEpiResidual>, ma, mb0, mb1, mr, o, m, n, k, q, err);
+  else if (epilogue == kEpiSwiGLU)
+    le = cudaLaunchKernelEx(&cfg, k_gemm_tc2<kEpiSwiGLU>, ma, mb0, mb1, mr, o, m, n, k, q, err);
+  else if (epilogue == kEpiQkvRope)
+    le = cudaLaunchKernelEx(&cfg, k_gemm_tc2<kEpiQkvRope>, ma, mb0, mb1, mr, o, m, n, k, q, err);
+  else
+    return cudaErrorInvalidValue;
+  if (le != cudaSuccess) return le;
+  return cudaGetLastError();
+}
+
+}  // namespace prism

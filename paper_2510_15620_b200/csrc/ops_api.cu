@@ -60,13 +60,15 @@ int prism_op_gemm(const void* a, const void* b, const void* b2, void* out, float
   if (!a || !b || m < 0 || n < 1 || k < 1 || epilogue < 0 || epilogue > 2) return PRISM_ERR_INVALID_ARG;
   if (epilogue == kEpiSwiGLU && !b2) return PRISM_ERR_INVALID_ARG;
   if (epilogue == kEpiResidual ? !resid : !out) return PRISM_ERR_INVALID_ARG;
-  if (dtype == PRISM_BF16 && impl == PRISM_IMPL_AUTO) {
+  if (dtype == PRISM_BF16 && (impl == PRISM_IMPL_AUTO || impl == PRISM_IMPL_SOLO)) {
     if (!err_word || (k % 8) || (n % 8) || (epilogue == kEpiSwiGLU && n % 128)) return PRISM_ERR_UNSUPPORTED;
     TmaDesc ma, mb0, mb1;
     cudaError_t e = make_tma_2d_bf16(&ma, a, (uint64_t)m, (uint64_t)k, 128, 64);
     if (e == cudaSuccess) e = make_tma_2d_bf16(&mb0, b, (uint64_t)n, (uint64_t)k, 128, 64);
     if (e == cudaSuccess) e = make_tma_2d_bf16(&mb1, epilogue == kEpiSwiGLU ? b2 : b, (uint64_t)n, (uint64_t)k, 128, 64);
-    if (e == cudaSuccess) e = launch_gemm_tc(ma, mb0, mb1, out, resid, m, n, k, epilogue, nullptr, err_word, S(stream));
+    if (e == cudaSuccess)
+      e = impl == PRISM_IMPL_AUTO ? launch_gemm_tc2(ma, mb0, mb1, out, resid, m, n, k, epilogue, nullptr, err_word, S(stream))
+                                  : launch_gemm_tc(ma, mb0, mb1, out, resid, m, n, k, epilogue, nullptr, err_word, S(stream));
     return st_of(e);
   }
   return st_of(launch_gemm_simt(a, b, b2, out, resid, m, n, k, dtype, epilogue, S(stream)));
@@ -103,7 +105,7 @@ int prism_op_gemm_qkv_rope(const void* a, const void* w_qkv, void* out, int32_t 
   if (e == cudaSuccess) e = make_tma_2d_bf16(&ma, a, (uint64_t)m, (uint64_t)k, 128, 64);
   if (e == cudaSuccess) e = make_tma_2d_bf16(&mb, w_qkv, (uint64_t)n, (uint64_t)k, 128, 64);
   QkvRopeArgs qa{pos, tab, (const __nv_bfloat16*)g_q, (const __nv_bfloat16*)g_k, n_q_heads, n_kv_heads, qk_norm, eps};
-  if (e == cudaSuccess) e = launch_gemm_tc(ma, mb, mb, out, nullptr, m, n, k, kEpiQkvRope, &qa, err_word, S(stream));
+  if (e == cudaSuccess) e = launch_gemm_tc2(ma, mb, mb, out, nullptr, m, n, k, kEpiQkvRope, &qa, err_word, S(stream));
   return st_of(e);
 }
 

@@ -36,6 +36,7 @@ struct prism_handle {
   int esz = 4;
   int chunk_tokens = 0;
   bool tc = false;  // tensor-core GEMM path
+  bool pair = false;  // ... on CTA pairs (the default) rather than single CTAs
   int fa = 0;       // attention path: 0 SIMT, 1 tcgen05, 2 warp-level MMA
 
   std::vector<void*> dev_allocs;
@@ -257,7 +258,7 @@ int validate_cfg(const prism_model_cfg& c, std::string* why) {
   if (c.hidden % 4 || c.hidden > 8192) return unsup("hidden must be a multiple of 4 and <= 8192");
   if (c.dtype == PRISM_BF16) {
     if (c.hidden % 8 || c.ffn % 8 || c.head_dim % 8) return unsup("bf16 mode needs hidden, ffn, head_dim multiples of 8");
-    if (c.gemm_impl == PRISM_IMPL_AUTO && (c.ffn % 128)) return unsup("tensor-core SwiGLU needs ffn multiple of 128");
+    if (c.gemm_impl != PRISM_IMPL_SIMT && (c.ffn % 128)) return unsup("tensor-core SwiGLU needs ffn multiple of 128");
     if (c.attention_impl != PRISM_IMPL_SIMT && c.head_dim != 128) return unsup("tensor-core attention needs head_dim 128");
   }
   return PRISM_OK;
@@ -320,7 +321,8 @@ static int create_impl(prism_handle* h, const prism_model_cfg* cfg, const prism_
   const prism_model_cfg& c = *cfg;
   h->cfg = c;
   h->esz = c.dtype == PRISM_BF16 ? 2 : 4;
-  h->tc = c.dtype == PRISM_BF16 && c.gemm_impl == PRISM_IMPL_AUTO;
+  h->tc = c.dtype == PRISM_BF16 && (c.gemm_impl == PRISM_IMPL_AUTO || c.gemm_impl == PRISM_IMPL_SOLO);
+  h->pair = c.gemm_impl == PRISM_IMPL_AUTO;
   h->fa = c.dtype != PRISM_BF16 ? 0 : (c.attention_impl == PRISM_IMPL_AUTO ? 1 : (c.attention_impl == PRISM_IMPL_MMA ? 2 : 0));
   const bool streamed = c.weight_residency == PRISM_WEIGHTS_HOST_STREAMED;
   if (!w->embed || !w->g_final || !w->score_head || !w->layers) return fail(h, PRISM_ERR_INVALID_ARG, "null weight pointer");
@@ -478,6 +480,12 @@ int validate_schedule(const prism_handle* h, const prism_prune_schedule* s, int 
   return PRISM_OK;
 }
 
+cudaError_t gemm_tc_any(const prism_handle* h, const TmaDesc& a, const TmaDesc& b0, const TmaDesc& b1, void* out, float* resid,
+                        int m, int n, int k, int epi, const QkvRopeArgs* qa, cudaStream_t st) {
+  return h->pair ? launch_gemm_tc2(a, b0, b1, out, resid, m, n, k, epi, qa, h->errword, st)
+                 : launch_gemm_tc(a, b0, b1, out, resid, m, n, k, epi, qa, h->errword, st);
+}
+
 // One decoder block over rows [r0, r0+rows) (sequences [s0, s1)) of the live batch.
 int run_layer_chunk(prism_handle* h, const LayerDev& W, const LayerMaps* maps, float* x, const int* cu_dev, int s0, int s1,
                     int r0, int rows, int max_len, cudaStream_t st) {
@@ -498,10 +506,10 @@ int run_layer_chunk(prism_handle* h, const LayerDev& W, const LayerMaps* maps, f
     QkvRopeArgs qa{h->pos + r0, h->rope_fused, (const __nv_bfloat16*)W.g_q, (const __nv_bfloat16*)W.g_k,
                    c.n_q_heads, c.n_kv_heads, c.qk_norm, c.rms_eps};
     PRISM_LAUNCH_P(h, st, PRISM_K_GEMM_QKV, 2.0 * R * nqkv * D,
-                   launch_gemm_tc(h->map_a_norm, maps->qkv, maps->qkv, h->qkv, nullptr, rows, nqkv, D, kEpiQkvRope, &qa, h->errword, st));
+                   gemm_tc_any(h, h->map_a_norm, maps->qkv, maps->qkv, h->qkv, nullptr, rows, nqkv, D, kEpiQkvRope, &qa, st));
   } else if (h->tc)
     PRISM_LAUNCH_P(h, st, PRISM_K_GEMM_QKV, 2.0 * R * nqkv * D,
-                   launch_gemm_tc(h->map_a_norm, maps->qkv, maps->qkv, h->qkv, nullptr, rows, nqkv, D, kEpiStore, nullptr, h->errword, st));
+                   gemm_tc_any(h, h->map_a_norm, maps->qkv, maps->qkv, h->qkv, nullptr, rows, nqkv, D, kEpiStore, nullptr, st));
   else
     PRISM_LAUNCH_P(h, st, PRISM_K_GEMM_QKV, 2.0 * R * nqkv * D,
                    launch_gemm_simt(h->a_norm, W.w_qkv, nullptr, h->qkv, nullptr, rows, nqkv, D, c.dtype, kEpiStore, st));
@@ -522,20 +530,20 @@ int run_layer_chunk(prism_handle* h, const LayerDev& W, const LayerMaps* maps, f
                                          c.causal, c.dtype, st));
   if (h->tc)
     PRISM_LAUNCH_P(h, st, PRISM_K_GEMM_O, 2.0 * R * D * hd,
-                   launch_gemm_tc(h->map_attn, maps->o, maps->o, nullptr, xr, rows, D, hd, kEpiResidual, nullptr, h->errword, st));
+                   gemm_tc_any(h, h->map_attn, maps->o, maps->o, nullptr, xr, rows, D, hd, kEpiResidual, nullptr, st));
   else
     PRISM_LAUNCH_P(h, st, PRISM_K_GEMM_O, 2.0 * R * D * hd,
                    launch_gemm_simt(h->attn, W.w_o, nullptr, nullptr, xr, rows, D, hd, c.dtype, kEpiResidual, st));
   PRISM_LAUNCH_P(h, st, PRISM_K_RMSNORM, norm_bytes, launch_rmsnorm(xr, W.g_ffn, c.dtype, rows, D, c.rms_eps, h->a_norm, st));
   if (h->tc)
     PRISM_LAUNCH_P(h, st, PRISM_K_GEMM_GATEUP, 4.0 * R * c.ffn * D,
-                   launch_gemm_tc(h->map_a_norm, maps->gate, maps->up, h->hbuf, nullptr, rows, c.ffn, D, kEpiSwiGLU, nullptr, h->errword, st));
+                   gemm_tc_any(h, h->map_a_norm, maps->gate, maps->up, h->hbuf, nullptr, rows, c.ffn, D, kEpiSwiGLU, nullptr, st));
   else
     PRISM_LAUNCH_P(h, st, PRISM_K_GEMM_GATEUP, 4.0 * R * c.ffn * D,
                    launch_gemm_simt(h->a_norm, W.w_gate, W.w_up, h->hbuf, nullptr, rows, c.ffn, D, c.dtype, kEpiSwiGLU, st));
   if (h->tc)
     PRISM_LAUNCH_P(h, st, PRISM_K_GEMM_DOWN, 2.0 * R * D * c.ffn,
-                   launch_gemm_tc(h->map_hbuf, maps->down, maps->down, nullptr, xr, rows, D, c.ffn, kEpiResidual, nullptr, h->errword, st));
+                   gemm_tc_any(h, h->map_hbuf, maps->down, maps->down, nullptr, xr, rows, D, c.ffn, kEpiResidual, nullptr, st));
   else
     PRISM_LAUNCH_P(h, st, PRISM_K_GEMM_DOWN, 2.0 * R * D * c.ffn,
                    launch_gemm_simt(h->hbuf, W.w_down, nullptr, nullptr, xr, rows, D, c.ffn, c.dtype, kEpiResidual, st));

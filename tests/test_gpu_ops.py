@@ -11,7 +11,7 @@ torch = pytest.importorskip("torch")
 pytestmark = pytest.mark.gpu
 
 FP32, BF16 = 0, 1
-AUTO, SIMT = 0, 1
+AUTO, SIMT, SOLO = 0, 1, 3
 
 
 @pytest.fixture(scope="module")
@@ -161,12 +161,14 @@ def test_gemm_fp32_simt(P, m, n, k, epi):
     assert np.max(np.abs(got - ref)) < 1e-5 * max(1.0, np.max(np.abs(ref)))      # fp32 accumulation over k terms
 
 
-@pytest.mark.parametrize("impl", [AUTO, SIMT])
+@pytest.mark.parametrize("impl", [AUTO, SOLO, SIMT])
 @pytest.mark.parametrize("epi", [0, 1, 2])
-@pytest.mark.parametrize("m,n,k", [(1, 256, 64), (300, 512, 320), (1000, 1024, 1024), (777, 384, 200), (4100, 2560, 512)])
+@pytest.mark.parametrize("m,n,k", [(1, 256, 64), (129, 256, 72), (300, 512, 320), (1000, 1024, 1024), (777, 384, 200),
+                                   (4100, 2560, 512)])
 def test_gemm_bf16(P, m, n, k, epi, impl):
-    """tcgen05 kernel (AUTO) and the CUDA-core kernel on the same bf16 inputs vs an fp64 matmul.
-    Shapes span several 128x256 tiles, ragged M/N/K tails and more tiles than SMs."""
+    """tcgen05 kernels (AUTO: CTA pairs, 256x256 tiles; SOLO: single CTAs, 128x256) and the CUDA-core kernel on the
+    same bf16 inputs vs an fp64 matmul.  Shapes span several tiles, ragged M/N/K tails (one where only the pair's
+    first CTA has rows, one where the second has a single row) and more tiles than SMs."""
     rng = np.random.default_rng(m * 7 + n + k + epi)
     a = round_to_bf16(rng.normal(size=(m, k)).astype(np.float32))
     b = round_to_bf16((rng.normal(size=(n, k)) * 0.05).astype(np.float32))

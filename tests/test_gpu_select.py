@@ -227,7 +227,7 @@ def mid(P):
     return w, req, S
 
 
-@pytest.mark.parametrize("gemm_impl,attn_impl", [(1, 1), (0, 1), (1, 0), (0, 0)])
+@pytest.mark.parametrize("gemm_impl,attn_impl", [(1, 1), (0, 1), (1, 0), (0, 0), (3, 0)])
 def test_bf16_paths_match_oracle(P, mid, gemm_impl, attn_impl):
     w, req, S = mid
     model = make_model(P, MID, w, req, gemm_impl=gemm_impl, attention_impl=attn_impl)
