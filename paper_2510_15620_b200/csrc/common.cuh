@@ -128,6 +128,11 @@ cudaError_t launch_attention_simt(const void* qkv, void* out, const int* cu, int
 // fetched in boxes of box_rows x 64 columns with the 128-byte swizzle the MMA descriptors expect.
 cudaError_t make_tma_2d_bf16(TmaDesc* out, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows,
                              uint32_t box_cols);
+// Store-side maps of the GEMM epilogues: fp32 [rows, cols] in 32x32 boxes (128-byte swizzle) and bf16
+// [rows, cols] in 32x32 boxes (64-byte swizzle).
+cudaError_t make_tma_2d_f32_box32(TmaDesc* out, const void* base, uint64_t rows, uint64_t cols);
+cudaError_t make_tma_2d_bf16_box32_sw64(TmaDesc* out, const void* base, uint64_t rows, uint64_t cols);
+int gemm_tc_sm_count();
 // b0/b1 describe the first and second 128 weight rows of a tile: the same matrix for plain
 // projections, the gate and the up matrix for kEpiSwiGLU.
 cudaError_t launch_gemm_tc(const TmaDesc& a, const TmaDesc& b0, const TmaDesc& b1, void* out, float* resid, int m,

@@ -16,18 +16,27 @@ namespace {
 using namespace tc;
 
 constexpr int BM = 128, BN = 256, BK = 64, UMMA_K = 16;
-constexpr int kStages = 6;
 constexpr int kABytes = BM * BK * 2;           // 16 KB
 constexpr int kBBytes = (BN / 2) * BK * 2;     // 16 KB: this CTA's half of the B tile
 constexpr int kStageBytes = kABytes + kBBytes; // 32 KB
-constexpr int kEpiBufBytes = 32 * 32 * 4;      // one 32x32 fp32 sub-tile staged for a TMA reduce-add
-constexpr int kEpiStageBytes = 4 * 2 * kEpiBufBytes;  // 4 epilogue warps x 2 buffers
-constexpr int kSmemBytes = kStages * kStageBytes + kEpiStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int kEpiBufBytes = 32 * 32 * 4;      // one 32-row, 128-byte-wide sub-tile staged for a TMA store or reduce-add
+// Operand ring and epilogue staging share 224 KB: the residual and SwiGLU epilogues stage one 4 KB sub-tile per
+// warp and keep six operand stages; the plain store stages 8 KB per warp (two buffers), the QKV epilogue 32 KB
+// of rotary-table rows and 4 KB of output per warp, and these keep five.
+__host__ __device__ constexpr int stages_of(int epi) { return (epi == kEpiResidual || epi == kEpiSwiGLU) ? 6 : 5; }
+__host__ __device__ constexpr int epi_stage_bytes_of(int epi) { return (7 - stages_of(epi)) * kStageBytes; }
+constexpr int kSmemBytes = 7 * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
 constexpr int kThreads = 320;  // TMA warp, MMA warp, 8 epilogue warps
 
 // x[tile] += smem tile (fp32), performed by the TMA unit / L2; rows and columns outside the tensor are clipped.
 __device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap* map, uint32_t src, int c0, int c1) {
   asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3}], [%1];"
+               ::"l"(map), "r"(src), "r"(c0), "r"(c1)
+               : "memory");
+}
+// smem tile -> global tile (bf16), rows and columns outside the tensor are clipped.
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int c0, int c1) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%2, %3}], [%1];"
                ::"l"(map), "r"(src), "r"(c0), "r"(c1)
                : "memory");
 }
@@ -86,6 +95,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 k_gemm_tc2(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b0,
           const __grid_constant__ CUtensorMap map_b1, const __grid_constant__ CUtensorMap map_r,
           __nv_bfloat16* __restrict__ out, int m, int n, int k, const QkvRopeArgs qa, int* __restrict__ err) {
+  constexpr int kStages = stages_of(kEpi), kEpiStageBytes = epi_stage_bytes_of(kEpi);
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t tiles = (raw + 1023u) & ~1023u;  // swizzled tiles need 1024-byte alignment
@@ -190,6 +200,7 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
     const int colhalf = (warp - 2) >> 2;  // 0: first half of the tile's columns, 1: second half
     bool ok = true;
     int it = 0;
+    [[maybe_unused]] uint32_t n_stores = 0;  // TMA stores issued by this warp (selects its staging buffer)
     // QKV epilogue: the row's position and the first half of its rotary table rows do not depend on the
     // accumulator, so they are requested before the wait for it (their L2 latency hides behind the MMAs).
     [[maybe_unused]] int rope_pos = 0;
@@ -219,32 +230,42 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
       }
       if (!mbar_wait(bar_acc_full + 8 * acc, acc_phase, err, abort_flag)) { ok = false; break; }
       tc_fence_after();
-      const int row = mt * BM + quarter * 32 + lane;
+      [[maybe_unused]] const int row = mt * BM + quarter * 32 + lane;
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN;
       const int col0 = nt * kOutCols;
       if constexpr (kEpi == kEpiSwiGLU) {
+        // This warp's 32 rows x 64 outputs (columns colhalf*64.. of the tile's 128) are staged as bf16 in its
+        // buffer (128-byte rows, 128-byte swizzle) and leave as one TMA store per tile.
+        if (col0 + colhalf * 64 < n && mt * BM + quarter * 32 < m) {
+          const uint32_t buf = epi_stage + (uint32_t)(warp - 2) * kEpiBufBytes;
+          if (lane == 0) bulk_wait_read<0>();  // the previous tile's store has read the buffer
+          __syncwarp();
 #pragma unroll 1
-        for (int cc = 0; cc < 2; ++cc) {
-          const int c = colhalf * 2 + cc;  // 32 of the tile's 128 outputs: gate columns c*32.., up columns 128 + c*32..
-          uint32_t g[32], u[32];
-          tmem_ld32(taddr + c * 32, g);
-          tmem_ld32(taddr + 128 + c * 32, u);
-          tmem_ld_wait();
-          if (row < m) {
-            __nv_bfloat16* o = out + (size_t)row * n + col0 + c * 32;
+          for (int cc = 0; cc < 2; ++cc) {
+            const int c = colhalf * 2 + cc;  // 32 of the tile's 128 outputs: gate columns c*32.., up columns 128 + c*32..
+            uint32_t g[32], u[32];
+            tmem_ld32(taddr + c * 32, g);
+            tmem_ld32(taddr + 128 + c * 32, u);
+            tmem_ld_wait();
 #pragma unroll
             for (int v = 0; v < 4; ++v) {
-              if (col0 + c * 32 + v * 8 < n) {
-                uint32_t pk[4];
+              uint32_t pk[4];
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                  const float g0 = __uint_as_float(g[v * 8 + 2 * e]), g1 = __uint_as_float(g[v * 8 + 2 * e + 1]);
-                  const float u0 = __uint_as_float(u[v * 8 + 2 * e]), u1 = __uint_as_float(u[v * 8 + 2 * e + 1]);
-                  pk[e] = pack_bf16(__fdividef(g0, 1.f + __expf(-g0)) * u0, __fdividef(g1, 1.f + __expf(-g1)) * u1);
-                }
-                *reinterpret_cast<uint4*>(o + v * 8) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+              for (int e = 0; e < 4; ++e) {
+                const float g0 = __uint_as_float(g[v * 8 + 2 * e]), g1 = __uint_as_float(g[v * 8 + 2 * e + 1]);
+                const float u0 = __uint_as_float(u[v * 8 + 2 * e]), u1 = __uint_as_float(u[v * 8 + 2 * e + 1]);
+                pk[e] = pack_bf16(__fdividef(g0, 1.f + __expf(-g0)) * u0, __fdividef(g1, 1.f + __expf(-g1)) * u1);
               }
+              const uint32_t dst = buf + lane * 128 + (((cc * 4 + v) ^ (lane & 7)) << 4);
+              asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(pk[0]), "r"(pk[1]), "r"(pk[2]), "r"(pk[3])
+                           : "memory");
             }
+          }
+          fence_async_smem();
+          __syncwarp();
+          if (lane == 0) {
+            tma_store_2d(&map_r, buf, col0 + colhalf * 64, mt * BM + quarter * 32);
+            bulk_commit();
           }
         }
       } else if constexpr (kEpi == kEpiResidual) {
@@ -308,7 +329,7 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
           }
           rnh = 1.0f / sqrtf(ss * (1.f / 128.f) + qa.eps);
         }
-        __nv_bfloat16* o = out + (size_t)row * n + (size_t)head * 128;
+        const uint32_t out_stage = epi_stage + 8 * kEpiBufBytes + (uint32_t)(warp - 2) * kEpiBufBytes;  // 2 boxes of 2 KB
         const __nv_bfloat16* gain = head < qa.hq ? qa.g_q : qa.g_k;
 #pragma unroll 1
         for (int half = 0; half < 2; ++half) {
@@ -319,30 +340,34 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
             asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
             if (half == 0) rope_fetch(1);
           }
-          if (!live) continue;
+          if (!live || mt * BM + quarter * 32 >= m) continue;  // warp-uniform
           uint32_t a[32], b[32];
           tmem_ld32(th + half * 32, a);
           tmem_ld32(th + 64 + half * 32, b);
+          if (lane == 0) bulk_wait_read<0>();  // the previous half's stores have read the two output boxes
+          __syncwarp();
           tmem_ld_wait();
-          if (!rot) {  // v head: plain store of the two 32-column pieces
-            if (row < m) {
+          // output columns [32*half, +32) and [64 + 32*half, +32) of the head: two 32-row x 64-byte boxes
+          // (64-byte swizzle), each leaving as one TMA store
+          const uint32_t box_lo = out_stage + lane * 64, box_hi = box_lo + 2048;
+          const uint32_t sw = (uint32_t)(lane >> 1) & 3u;
+          if (!rot) {  // v head: stored as it is
 #pragma unroll
-              for (int v = 0; v < 4; ++v) {
-                uint4 pa, pb;
-                pa.x = pack_bf16(__uint_as_float(a[v * 8 + 0]), __uint_as_float(a[v * 8 + 1]));
-                pa.y = pack_bf16(__uint_as_float(a[v * 8 + 2]), __uint_as_float(a[v * 8 + 3]));
-                pa.z = pack_bf16(__uint_as_float(a[v * 8 + 4]), __uint_as_float(a[v * 8 + 5]));
-                pa.w = pack_bf16(__uint_as_float(a[v * 8 + 6]), __uint_as_float(a[v * 8 + 7]));
-                pb.x = pack_bf16(__uint_as_float(b[v * 8 + 0]), __uint_as_float(b[v * 8 + 1]));
-                pb.y = pack_bf16(__uint_as_float(b[v * 8 + 2]), __uint_as_float(b[v * 8 + 3]));
-                pb.z = pack_bf16(__uint_as_float(b[v * 8 + 4]), __uint_as_float(b[v * 8 + 5]));
-                pb.w = pack_bf16(__uint_as_float(b[v * 8 + 6]), __uint_as_float(b[v * 8 + 7]));
-                *reinterpret_cast<uint4*>(o + half * 32 + v * 8) = pa;
-                *reinterpret_cast<uint4*>(o + 64 + half * 32 + v * 8) = pb;
-              }
+            for (int v = 0; v < 4; ++v) {
+              asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(box_lo + ((v ^ sw) << 4)),
+                           "r"(pack_bf16(__uint_as_float(a[v * 8 + 0]), __uint_as_float(a[v * 8 + 1]))),
+                           "r"(pack_bf16(__uint_as_float(a[v * 8 + 2]), __uint_as_float(a[v * 8 + 3]))),
+                           "r"(pack_bf16(__uint_as_float(a[v * 8 + 4]), __uint_as_float(a[v * 8 + 5]))),
+                           "r"(pack_bf16(__uint_as_float(a[v * 8 + 6]), __uint_as_float(a[v * 8 + 7])))
+                           : "memory");
+              asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(box_hi + ((v ^ sw) << 4)),
+                           "r"(pack_bf16(__uint_as_float(b[v * 8 + 0]), __uint_as_float(b[v * 8 + 1]))),
+                           "r"(pack_bf16(__uint_as_float(b[v * 8 + 2]), __uint_as_float(b[v * 8 + 3]))),
+                           "r"(pack_bf16(__uint_as_float(b[v * 8 + 4]), __uint_as_float(b[v * 8 + 5]))),
+                           "r"(pack_bf16(__uint_as_float(b[v * 8 + 6]), __uint_as_float(b[v * 8 + 7])))
+                           : "memory");
             }
-            continue;
-          }
+          } else {
 #pragma unroll
           for (int v = 0; v < 4; ++v) {
             float x0[8], x1[8], cs[8], sn[8];
@@ -383,33 +408,51 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
               lo[e] = pack_bf16(y0, y1);
               hi[e] = pack_bf16(z0, z1);
             }
-            if (row < m) {
-              *reinterpret_cast<uint4*>(o + half * 32 + v * 8) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
-              *reinterpret_cast<uint4*>(o + 64 + half * 32 + v * 8) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-            }
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(box_lo + ((v ^ sw) << 4)), "r"(lo[0]), "r"(lo[1]),
+                         "r"(lo[2]), "r"(lo[3]) : "memory");
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(box_hi + ((v ^ sw) << 4)), "r"(hi[0]), "r"(hi[1]),
+                         "r"(hi[2]), "r"(hi[3]) : "memory");
+          }
+          }
+          fence_async_smem();
+          __syncwarp();
+          if (lane == 0) {
+            tma_store_2d(&map_r, out_stage, head * 128 + half * 32, mt * BM + quarter * 32);
+            tma_store_2d(&map_r, out_stage + 2048, head * 128 + 64 + half * 32, mt * BM + quarter * 32);
+            bulk_commit();
           }
         }
       } else {
+        // 32 rows x 64 columns at a time: bf16 into one of the warp's two staging buffers (128-byte rows,
+        // 128-byte swizzle), then one TMA store, which clips the ragged edges of the matrix.
 #pragma unroll 1
-        for (int cc = 0; cc < 4; ++cc) {
-          const int c = colhalf * 4 + cc;
-          uint32_t r[32];
-          tmem_ld32(taddr + c * 32, r);
+        for (int cc = 0; cc < 2; ++cc) {
+          const int c = colhalf * 2 + cc;  // 64-column piece of the tile
+          if (col0 + c * 64 >= n || mt * BM + quarter * 32 >= m) break;  // warp-uniform; later pieces are outside too
+          uint32_t r[64];
+          tmem_ld32(taddr + c * 64, r);
+          tmem_ld32(taddr + c * 64 + 32, r + 32);
+          const uint32_t buf = epi_stage + (uint32_t)(warp - 2) * 2 * kEpiBufBytes + (n_stores & 1) * kEpiBufBytes;
+          if (lane == 0) bulk_wait_read<1>();  // the store that last used this buffer has read it
+          __syncwarp();
           tmem_ld_wait();
-          if (row < m) {
-            __nv_bfloat16* o = out + (size_t)row * n + col0 + c * 32;
 #pragma unroll
-            for (int v = 0; v < 4; ++v) {
-              if (col0 + c * 32 + v * 8 < n) {
-                uint4 pk;
-                pk.x = pack_bf16(__uint_as_float(r[v * 8 + 0]), __uint_as_float(r[v * 8 + 1]));
-                pk.y = pack_bf16(__uint_as_float(r[v * 8 + 2]), __uint_as_float(r[v * 8 + 3]));
-                pk.z = pack_bf16(__uint_as_float(r[v * 8 + 4]), __uint_as_float(r[v * 8 + 5]));
-                pk.w = pack_bf16(__uint_as_float(r[v * 8 + 6]), __uint_as_float(r[v * 8 + 7]));
-                *reinterpret_cast<uint4*>(o + v * 8) = pk;
-              }
-            }
+          for (int v = 0; v < 8; ++v) {
+            const uint32_t dst = buf + lane * 128 + ((v ^ (lane & 7)) << 4);
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst),
+                         "r"(pack_bf16(__uint_as_float(r[v * 8 + 0]), __uint_as_float(r[v * 8 + 1]))),
+                         "r"(pack_bf16(__uint_as_float(r[v * 8 + 2]), __uint_as_float(r[v * 8 + 3]))),
+                         "r"(pack_bf16(__uint_as_float(r[v * 8 + 4]), __uint_as_float(r[v * 8 + 5]))),
+                         "r"(pack_bf16(__uint_as_float(r[v * 8 + 6]), __uint_as_float(r[v * 8 + 7])))
+                         : "memory");
           }
+          fence_async_smem();
+          __syncwarp();
+          if (lane == 0) {
+            tma_store_2d(&map_r, buf, col0 + c * 64, mt * BM + quarter * 32);
+            bulk_commit();
+          }
+          ++n_stores;
         }
       }
       if constexpr (kEpi == kEpiQkvRope) rope_pos = rope_pos_next;
@@ -417,9 +460,7 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(leader_acc_empty + 8 * acc);  // the leader's MMA thread waits for both CTAs
     }
-    if constexpr (kEpi == kEpiResidual) {
-      if (lane == 0) bulk_wait<0>();  // all reduce-adds of this warp have completed
-    }
+    if (lane == 0) bulk_wait<0>();  // all TMA stores / reduce-adds of this warp have completed
   }
 
   tc_fence_before();
@@ -432,9 +473,6 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
 }
 
 }  // namespace
-
-cudaError_t make_tma_2d_f32_box32(TmaDesc* out, const void* base, uint64_t rows, uint64_t cols);
-int gemm_tc_sm_count();
 
 cudaError_t launch_gemm_tc2(const TmaDesc& a, const TmaDesc& b0, const TmaDesc& b1, void* out, float* resid, int m,
                            int n, int k, int epilogue, const QkvRopeArgs* qa, int* err, cudaStream_t st) {
@@ -456,7 +494,7 @@ cudaError_t launch_gemm_tc2(const TmaDesc& a, const TmaDesc& b0, const TmaDesc& 
   const CUtensorMap& ma = reinterpret_cast<const CUtensorMap&>(a);
   const CUtensorMap& mb0 = reinterpret_cast<const CUtensorMap&>(b0);
   const CUtensorMap& mb1 = reinterpret_cast<const CUtensorMap&>(b1);
-  TmaDesc rdesc = a;  // placeholder for the epilogues that do not use it
+  TmaDesc rdesc = a;  // the output (or residual) rows of this launch, exactly m of them: the TMA unit clips the ragged last tile
   QkvRopeArgs q{};
   if (epilogue == kEpiResidual) {
     // the residual rows of this launch, exactly m of them, so that the TMA unit clips the ragged last tile
@@ -466,6 +504,12 @@ cudaError_t launch_gemm_tc2(const TmaDesc& a, const TmaDesc& b0, const TmaDesc& 
   if (epilogue == kEpiQkvRope) {
     if (!qa || n % 128) return cudaErrorInvalidValue;
     q = *qa;
+    cudaError_t e = make_tma_2d_bf16_box32_sw64(&rdesc, out, (uint64_t)m, (uint64_t)n);
+    if (e != cudaSuccess) return e;
+  }
+  if (epilogue == kEpiStore || epilogue == kEpiSwiGLU) {
+    cudaError_t e = make_tma_2d_bf16(&rdesc, out, (uint64_t)m, (uint64_t)n, 32, 64);
+    if (e != cudaSuccess) return e;
   }
   const CUtensorMap& mr = reinterpret_cast<const CUtensorMap&>(rdesc);
   __nv_bfloat16* o = (__nv_bfloat16*)out;
