@@ -31,10 +31,10 @@ UNIT = "candidate-tokens/s"
 KERNEL_CLASSES = ["pack", "embed", "rmsnorm", "gemm_qkv", "rope", "attention", "gemm_o", "gemm_gateup", "gemm_down",
                   "probe", "route", "compact"]
 GEMM_CLASSES = ("gemm_qkv", "gemm_o", "gemm_gateup", "gemm_down")
-# dram__bytes_read.sum + dram__bytes_write.sum of one k_gemm_tc launch at M = 8192 with the cfg1 weight
-# shapes, from the ncu captures summarised under profiles/ (down-proj: A + W + residual, not captured).
+# dram__bytes_read.sum + dram__bytes_write.sum of one k_gemm_tc2 launch at M = 8192 with the cfg1 weight
+# shapes, from the ncu captures summarised under profiles/gemm_tc2_*.md.
 # Reads grow in proportion to M; writes are mostly absorbed by the 126 MB L2 inside the kernel's window.
-NCU_TRAFFIC_M8192 = {"gemm_qkv": 41.7e6, "gemm_o": 71.6e6, "gemm_gateup": 31.7e6, "gemm_down": 90.2e6}
+NCU_TRAFFIC_M8192 = {"gemm_qkv": 42.6e6, "gemm_o": 72.5e6, "gemm_gateup": 36.8e6, "gemm_down": 94.5e6}
 CFG1_NK = {"gemm_qkv": (4096, 1024), "gemm_o": (1024, 2048), "gemm_gateup": (6144, 1024), "gemm_down": (1024, 3072)}
 
 
@@ -319,7 +319,7 @@ def run_prism(args):
                             "flops_per_launch": g_fl / g_n if g_n else 0, "avg_launch_ms": g_ms / g_n if g_n else 0,
                             "traffic": traffic,
                             "traffic_note": "bytes per launch: ncu dram read+write of each GEMM shape at M = 8192 "
-                                            "(profiles/gemm_tc_*.md) scaled by the rows each launch processed",
+                                            "(profiles/gemm_tc2_*.md) scaled by the rows each launch processed",
                             "share_of_kernel_time": g_ms / tot_ms if tot_ms else None}
         line["kernels"] = {n: {"ms_per_step": round(v["ms_per_step"], 4), "share": round(v["ms_per_step"] / tot_ms, 4),
                                "launches_per_step": v["launches_per_step"],
