@@ -142,6 +142,9 @@ cudaError_t launch_gemm_tc2(const TmaDesc& a, const TmaDesc& b0, const TmaDesc& 
                             int n, int k, int epilogue, const QkvRopeArgs* qa, int* err, cudaStream_t st);
 cudaError_t launch_attention_tc(const void* qkv, void* out, const int* cu, int seq0, int nseq, int row0, int rows,
                                 int max_len, int n_q_heads, int n_kv_heads, int causal, int* err, cudaStream_t st);
+// Two query heads of a key/value group per CTA, persistent (needs an even group size n_q_heads / n_kv_heads).
+cudaError_t launch_attention_tc2(const void* qkv, void* out, const int* cu, int seq0, int nseq, int row0, int rows,
+                                int max_len, int n_q_heads, int n_kv_heads, int causal, int* err, cudaStream_t st);
 cudaError_t launch_attention_mma(const void* qkv, void* out, const int* cu, int seq0, int nseq, int row0,
                                  int max_len, int n_q_heads, int n_kv_heads, int causal, cudaStream_t st);
 

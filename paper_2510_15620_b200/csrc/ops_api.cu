@@ -115,8 +115,11 @@ int prism_op_attention(const void* qkv, void* out, const int32_t* cu, int32_t n_
   if (!qkv || !out || !cu || n_seq < 0 || total < 0 || n_kv_heads < 1 || n_q_heads % n_kv_heads) return PRISM_ERR_INVALID_ARG;
   if (dtype == PRISM_BF16 && impl != PRISM_IMPL_SIMT) {
     if (head_dim != 128) return PRISM_ERR_UNSUPPORTED;
-    if (impl == PRISM_IMPL_AUTO) {
+    if (impl == PRISM_IMPL_AUTO || impl == PRISM_IMPL_SOLO) {
       if (!err_word) return PRISM_ERR_INVALID_ARG;
+      if (impl == PRISM_IMPL_AUTO && ((n_q_heads / n_kv_heads) & 1) == 0)
+        return st_of(launch_attention_tc2(qkv, out, cu, 0, n_seq, 0, total, max_len, n_q_heads, n_kv_heads, causal,
+                                          err_word, S(stream)));
       return st_of(launch_attention_tc(qkv, out, cu, 0, n_seq, 0, total, max_len, n_q_heads, n_kv_heads, causal, err_word,
                                        S(stream)));
     }

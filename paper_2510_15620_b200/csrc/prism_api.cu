@@ -323,7 +323,11 @@ static int create_impl(prism_handle* h, const prism_model_cfg* cfg, const prism_
   h->esz = c.dtype == PRISM_BF16 ? 2 : 4;
   h->tc = c.dtype == PRISM_BF16 && (c.gemm_impl == PRISM_IMPL_AUTO || c.gemm_impl == PRISM_IMPL_SOLO);
   h->pair = c.gemm_impl == PRISM_IMPL_AUTO;
-  h->fa = c.dtype != PRISM_BF16 ? 0 : (c.attention_impl == PRISM_IMPL_AUTO ? 1 : (c.attention_impl == PRISM_IMPL_MMA ? 2 : 0));
+  // 0: CUDA cores, 1: tcgen05 one query head per CTA, 2: mma.sync, 3: tcgen05 two query heads per CTA (even groups)
+  h->fa = c.dtype != PRISM_BF16 ? 0
+          : c.attention_impl == PRISM_IMPL_AUTO ? ((((c.n_q_heads / c.n_kv_heads) & 1) == 0) ? 3 : 1)
+          : c.attention_impl == PRISM_IMPL_SOLO ? 1
+          : c.attention_impl == PRISM_IMPL_MMA  ? 2 : 0;
   const bool streamed = c.weight_residency == PRISM_WEIGHTS_HOST_STREAMED;
   if (!w->embed || !w->g_final || !w->score_head || !w->layers) return fail(h, PRISM_ERR_INVALID_ARG, "null weight pointer");
   h->embed = w->embed;
@@ -517,7 +521,11 @@ int run_layer_chunk(prism_handle* h, const LayerDev& W, const LayerMaps* maps, f
   PRISM_LAUNCH_P(h, st, PRISM_K_ROPE, 2.0 * R * (c.n_q_heads + c.n_kv_heads) * dh * esz,
                  launch_qknorm_rope(h->qkv, c.dtype, h->pos + r0, rows, c.n_q_heads, c.n_kv_heads, dh, c.qk_norm, W.g_q, W.g_k,
                                     c.rms_eps, h->rope_cos, h->rope_sin, st));
-  if (h->fa == 1)
+  if (h->fa == 3)
+    PRISM_LAUNCH_P(h, st, PRISM_K_ATTENTION, attn_flops,
+                   launch_attention_tc2(h->qkv, h->attn, cu_dev, s0, s1 - s0, r0, rows, max_len, c.n_q_heads, c.n_kv_heads, c.causal,
+                                        h->errword, st));
+  else if (h->fa == 1)
     PRISM_LAUNCH_P(h, st, PRISM_K_ATTENTION, attn_flops,
                    launch_attention_tc(h->qkv, h->attn, cu_dev, s0, s1 - s0, r0, rows, max_len, c.n_q_heads, c.n_kv_heads, c.causal,
                                        h->errword, st));

@@ -250,10 +250,13 @@ def _attn_ref(qkv, cu, hq, hkv, dh, causal):
 
 
 @pytest.mark.parametrize("causal", [1, 0])
-@pytest.mark.parametrize("dtype,impl,dh", [(FP32, SIMT, 64), (BF16, SIMT, 128), (BF16, AUTO, 128), (BF16, 2, 128)])
-def test_attention(P, dtype, impl, dh, causal):
+@pytest.mark.parametrize("dtype,impl,dh,hq,hkv", [(FP32, SIMT, 64, 4, 2), (BF16, SIMT, 128, 4, 2), (BF16, AUTO, 128, 4, 2),
+                                                  (BF16, AUTO, 128, 8, 2), (BF16, AUTO, 128, 3, 1), (BF16, 2, 128, 4, 2),
+                                                  (BF16, SOLO, 128, 4, 2)])
+def test_attention(P, dtype, impl, dh, hq, hkv, causal):
+    """AUTO runs the two-heads-per-CTA tcgen05 kernel for even group sizes (2 and 4 here) and the one-head kernel
+    otherwise (group 3); SOLO forces the one-head kernel; 2 is the mma.sync kernel."""
     rng = np.random.default_rng(dh + causal)
-    hq, hkv = 4, 2
     lens = np.array([1, 7, 64, 65, 130, 200, 63, 128, 129, 300, 513])      # below, at and across the 64/128-row tiles
     cu = np.zeros(len(lens) + 1, np.int32)
     cu[1:] = np.cumsum(lens)
@@ -294,6 +297,39 @@ def test_attention_tc_rescales_when_the_maximum_grows(P):
         assert int(err.item()) == 0
         ref = _attn_ref(qkv, cu, hq, hkv, dh, bool(causal))
         assert np.max(np.abs(out.float().cpu().numpy() - ref)) < 2e-2 * max(1.0, np.max(np.abs(ref)))
+
+
+@pytest.mark.parametrize("impl", [AUTO, SOLO])
+def test_attention_tc_scores_far_above_the_first_key(P, impl):
+    """The two-head kernel exponentiates against the row's score on key 0 and moves that reference only when a
+    row sum leaves fp32's comfortable range.  Here later keys score hundreds of powers of two above key 0
+    (and, in other rows, far below it), inside one 32-key chunk, across chunks and across key blocks, so the
+    reference must move (repeatedly) and O, l and the probabilities already written must follow exactly."""
+    rng = np.random.default_rng(11)
+    hq, hkv, dh = 4, 2, 128
+    lens = np.array([300, 40, 129])
+    cu = np.zeros(len(lens) + 1, np.int32)
+    cu[1:] = np.cumsum(lens)
+    tot = int(cu[-1])
+    qkv = rng.normal(size=(tot, (hq + 2 * hkv) * dh)).astype(np.float32)
+    pos = np.concatenate([np.arange(l) for l in lens])
+    # key norm: a staircase over positions (x1 ... x40) with jumps inside chunks, between chunks and between blocks;
+    # q . k / sqrt(dh) then spans roughly +-(4 * 40 * sqrt(128) / sqrt(128)) ~ +-500 in natural-log units
+    stair = 1.0 + 39.0 * (((pos * 7) % 97) / 96.0) * (pos > 0) + 20.0 * (pos % 50 == 17)
+    qkv[:, hq * dh:(hq + hkv) * dh] *= stair[:, None]
+    qkv[:, : hq * dh] *= 2.0
+    qkv = round_to_bf16(qkv)
+    out = torch.zeros(tot, hq * dh, dtype=torch.bfloat16, device="cuda")
+    err = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for causal in (1, 0):
+        P.ops.prism_op_attention(dev(qkv, torch.bfloat16), out, dev(cu), len(lens), int(lens.max()), hq, hkv, dh, causal,
+                                 BF16, impl, err)
+        torch.cuda.synchronize()
+        assert int(err.item()) == 0
+        ref = _attn_ref(qkv, cu, hq, hkv, dh, bool(causal))
+        got = out.float().cpu().numpy()
+        assert np.isfinite(got).all()
+        assert np.max(np.abs(got - ref)) < 2e-2 * max(1.0, np.max(np.abs(ref))), np.max(np.abs(got - ref))
 
 
 def test_bounded_wait_gives_up_and_reports(P):
