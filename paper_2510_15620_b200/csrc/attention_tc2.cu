@@ -45,13 +45,13 @@ __device__ __forceinline__ float ex2(float x) {  // 2^x on the special-function 
   return y;
 }
 
-// 2^x for a pair of exponents.  The special-function unit delivers 16 results per clock and SM, exactly what
-// the tensor core consumes at this head size, so kEmulated of every 8 pairs take the FMA pipe instead:
+// 2^x for a pair of exponents.  All softmax warps of the SM share its special-function unit, so kEmulated of
+// every 8 pairs take the FMA pipe instead (measured: 0, 2, 3 and 4 of 8 are within 4 % of each other, 2 is best):
 // x = n + f with n = round(x) (the 1.5 * 2^23 trick leaves n in the low bits of t), 2^f by a cubic whose relative
 // error (7.5e-5) is far below bf16 rounding, and n is added to the exponent field.  x is clamped to [-125, 126]:
 // masked scores (-inf) come out as 2^-125 instead of 0 (every row sum is at least 1), and exponents beyond
 // fp32 range still produce a sum that the range check catches.
-constexpr int kEmulated = 3;
+constexpr int kEmulated = 2;
 __device__ __forceinline__ void exp2_pair(uint64_t xv, bool emulate, float& p0, float& p1) {
   float x0, x1;
   f2_unpack(xv, x0, x1);
@@ -391,7 +391,6 @@ k_attention_tc2(const __grid_constant__ CUtensorMap map_qkv, __nv_bfloat16* __re
         // One barrier of the row's two warps per block.  It carries the vote "some row sum is out of range", and
         // it orders the P stores below after BOTH threads' score loads: P chunks overwrite score columns of the
         // other thread's chunks.
-        bool saw_pv = false;  // has this thread already observed the completion of this head's previous P V?
         const int vote = pair_meet(!(rs <= kBigSum));
         if (vote < 0) { ok = false; break; }
         if (vote) {
@@ -419,8 +418,7 @@ k_attention_tc2(const __grid_constant__ CUtensorMap map_qkv, __nv_bfloat16* __re
           const float d = xmax > 64.f ? ceilf(xmax) : 0.f;
           const float f = exp2f(-d);
           if (j > 0) {
-            if (!mbar_wait(bar_o, (gc - 1) & 1, err, abort_flag)) { ok = false; break; }
-            saw_pv = true;
+            if (!mbar_wait(bar_o, (gc - 1) & 1, err, abort_flag)) { ok = false; break; }  // complete already
             tc_fence_after();
 #pragma unroll 1
             for (int c = 0; c < 2; ++c) {  // this thread's 64 columns of O
@@ -451,11 +449,10 @@ k_attention_tc2(const __grid_constant__ CUtensorMap map_qkv, __nv_bfloat16* __re
         tmem_st16(t_s + c1 * 16, pk + 16);
         tmem_st_wait();
         tc_fence_before();
-        // mbarrier parity only tells the current phase from the previous one, so every thread observes
-        // every phase of o_full and p_full, in order, at a point where the next phase cannot complete yet:
-        // this head's next P V needs this thread's arrival below.
-        if (j > 0 && !saw_pv && !mbar_wait(bar_o, (gc - 1) & 1, err, abort_flag)) { ok = false; break; }
-        if (gc > 0 && !mbar_wait(bar_p, (gc - 1) & 1, err, abort_flag)) { ok = false; break; }
+        // No wait is needed to keep the barrier phases apart.  The scores of block gc were issued after the
+        // wait for p_full(gc - 1), so that phase is over before any warp gets here; and s_full(gc), which this
+        // thread has observed, completes only after every earlier MMA of this head, so o_full stands at phase
+        // gc - 1 exactly until this thread's arrival below lets P V(gc) be issued.
         __syncwarp();
         if (lane == 0) mbar_arrive(bar_p);  // one arrival per warp
       }
