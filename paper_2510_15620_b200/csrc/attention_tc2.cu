@@ -78,12 +78,14 @@ __device__ __forceinline__ void exp2_pair(uint64_t xv, bool emulate, float& p0, 
 __device__ __forceinline__ void tmem_ld1(uint32_t taddr, uint32_t& v) {
   asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];" : "=r"(v) : "r"(taddr));
 }
-// Work distribution.  Candidate index i names (query block, sequence, head pair) with the query block
-// descending, so that the heaviest items are handed out first; candidates whose block lies beyond the
-// sequence's end are skipped.  CTAs draw candidates from a device-wide counter (the items differ in cost by the
-// number of key blocks, and a fixed assignment leaves a quarter of the SMs idle at the end).  The producer
-// thread draws, and publishes each item through a small ring in shared memory to the other roles, which
-// read the ring in order.
+// Work distribution.  Sequences are taken in groups of `gsz` (as many as keep their q/k/v rows well inside L2);
+// candidate index i names (group, query block, sequence of the group, head pair) with the query block
+// descending inside a group: a sequence's K and V rows are fetched from DRAM once and found in L2 by its
+// other query blocks and head pairs, and the last items of the launch are the light ones.
+// Candidates whose block lies beyond the sequence's end are skipped.  CTAs draw candidates from a device-wide
+// counter (the items differ in cost by the number of key blocks, and a fixed assignment leaves a quarter of
+// the SMs idle at the end).  The producer thread draws, and publishes each item through a small ring in
+// shared memory to the other roles, which read the ring in order.
 struct ItemRec {
   int qb, pair, beg, len, n_blocks;  // n_blocks == 0: no more items
 };
@@ -112,8 +114,8 @@ struct ItemReader {
 
 __global__ void __launch_bounds__(kThreads, 1)
 k_attention_tc2(const __grid_constant__ CUtensorMap map_qkv, __nv_bfloat16* __restrict__ out,
-                const int* __restrict__ cu, int seq0, int nseq, int row0, int nqb, int hq, int hkv, int causal,
-                float scale_log2, int* __restrict__ sched, int* __restrict__ err) {
+                const int* __restrict__ cu, int seq0, int nseq, int row0, int nqb, int gsz, int hq, int hkv,
+                int causal, float scale_log2, int* __restrict__ sched, int* __restrict__ err) {
   extern __shared__ unsigned char smem_raw[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t raw = smem_u32(smem_raw);
@@ -166,15 +168,18 @@ k_attention_tc2(const __grid_constant__ CUtensorMap map_qkv, __nv_bfloat16* __re
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
       ItemRec it;
-      const int per_qb = nseq * npairs, total = nqb * per_qb;
+      const int per_qb = gsz * npairs, per_group = nqb * per_qb;
+      const int total = ((nseq + gsz - 1) / gsz) * per_group;
       uint32_t kc = 0, vc = 0, ic = 0;  // K tiles, V tiles, items issued so far
       bool ok = true;
       while (ok) {
         // draw candidates until one is a real item
         it.n_blocks = 0;
         for (int i = atomicAdd(sched, 1); i < total; i = atomicAdd(sched, 1)) {
-          it.qb = nqb - 1 - i / per_qb;
-          const int rem = i % per_qb, s = seq0 + rem / npairs;
+          const int in_group = i % per_group, rem = in_group % per_qb, sl = (i / per_group) * gsz + rem / npairs;
+          if (sl >= nseq) continue;
+          const int s = seq0 + sl;
+          it.qb = nqb - 1 - in_group / per_qb;
           it.pair = rem % npairs;
           const int b = __ldg(cu + s);
           it.len = __ldg(cu + s + 1) - b;
@@ -537,7 +542,11 @@ cudaError_t launch_attention_tc2(const void* qkv, void* out, const int* cu, int 
   cudaError_t e = make_tma_2d_bf16(&mq, qkv, (uint64_t)rows, ld, 128, 64);
   if (e != cudaSuccess) return e;
   const int nqb = (max_len + BM - 1) / BM;
-  const long long total = (long long)nqb * nseq * (n_q_heads / 2);
+  // sequences per scheduling group: their q/k/v rows (at most max_len each) stay within 48 MB
+  const long long seq_bytes = (long long)nqb * BM * (long long)ld * 2;
+  int gsz = (int)((48ll << 20) / seq_bytes);
+  gsz = gsz < 1 ? 1 : (gsz > nseq ? nseq : gsz);
+  const long long total = (long long)((nseq + gsz - 1) / gsz) * gsz * nqb * (n_q_heads / 2);
   if (total > 0x7fffffffLL) return cudaErrorInvalidValue;
   const int sms = gemm_tc_sm_count();
   const int grid = (int)(total < sms ? total : sms);
@@ -556,7 +565,7 @@ cudaError_t launch_attention_tc2(const void* qkv, void* out, const int* cu, int 
   int* sched = sb + 2 * (ticket.fetch_add(1, std::memory_order_relaxed) % kTickets);
   const float scale_log2 = 1.4426950408889634f / sqrtf((float)DH);
   k_attention_tc2<<<grid, kThreads, kSmemBytes, st>>>(reinterpret_cast<const CUtensorMap&>(mq), (__nv_bfloat16*)out, cu,
-                                                      seq0, nseq, row0, nqb, n_q_heads, n_kv_heads, causal, scale_log2,
+                                                      seq0, nseq, row0, nqb, gsz, n_q_heads, n_kv_heads, causal, scale_log2,
                                                       sched, err);
   return cudaGetLastError();
 }
