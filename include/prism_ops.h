@@ -46,9 +46,10 @@ PRISM_API int prism_op_qknorm_rope(void* qkv, int32_t dtype, const int32_t* pos,
  *   epilogue 0: out[m,n] = C                      (dtype elements)
  *   epilogue 1: resid[m,n] += C                   (float residual stream; out unused)
  *   epilogue 2: out[m,n] = silu(A*B^T) * (A*B2^T) (SwiGLU; B = gate rows, B2 = up rows)
- * impl PRISM_IMPL_AUTO uses the tcgen05 tensor-core kernel in bf16 mode (k, n multiples of 8; n a
- * multiple of 128 for epilogue 2), PRISM_IMPL_SIMT the CUDA-core kernel.  The tensor-core kernel
- * reports an expired bounded wait in err_word bit 4 (nullable for SIMT). */
+ * impl PRISM_IMPL_AUTO uses the tcgen05 tensor-core kernel on CTA pairs in bf16 mode (k, n multiples of 8;
+ * n a multiple of 128 for epilogue 2; out and resid 16-byte aligned: they are written through TMA),
+ * PRISM_IMPL_SOLO the single-CTA tcgen05 kernel, PRISM_IMPL_SIMT the CUDA-core kernel.  The tensor-core
+ * kernels report an expired bounded wait in err_word bit 4 (nullable for SIMT). */
 PRISM_API int prism_op_gemm(const void* a, const void* b, const void* b2, void* out, float* resid, int32_t m, int32_t n,
                   int32_t k, int32_t dtype, int32_t epilogue, int32_t impl, int32_t* err_word, void* stream);
 
@@ -66,8 +67,9 @@ PRISM_API int prism_op_gemm_qkv_rope(const void* a, const void* w_qkv, void* out
 /* Attention over packed sequences: for sequence s (rows cu[s]..cu[s+1]) and query head h (kv head
  * h / (Hq/Hkv)): out = softmax(q k^T / sqrt(head_dim) [+ causal mask]) v.  qkv [total, (Hq+2Hkv)*dh],
  * out [total, Hq*dh].  total = cu[n_seq] rows; max_len >= the longest sequence.  impl: PRISM_IMPL_AUTO =
- * tcgen05 kernel (bf16, head_dim 128; reports an expired bounded wait in err_word bit 4),
- * PRISM_IMPL_MMA = warp-level MMA kernel (bf16, head_dim 128), PRISM_IMPL_SIMT = CUDA cores. */
+ * tcgen05 kernel (bf16, head_dim 128; two query heads of a KV group per CTA when Hq/Hkv is even, else one
+ * head per CTA; reports an expired bounded wait in err_word bit 4), PRISM_IMPL_SOLO = the one-head tcgen05
+ * kernel, PRISM_IMPL_MMA = warp-level MMA kernel (bf16, head_dim 128), PRISM_IMPL_SIMT = CUDA cores. */
 PRISM_API int prism_op_attention(const void* qkv, void* out, const int32_t* cu, int32_t n_seq, int32_t total,
                                  int32_t max_len, int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim,
                                  int32_t causal, int32_t dtype, int32_t impl, int32_t* err_word, void* stream);

@@ -17,7 +17,7 @@
 // S_{j+1} and S_{j+2}... are issued as soon as their K tile has landed and their TMEM buffer is free (the
 // output issuer releases buffer j&1 with a commit after P_j V_j), so the tensor core computes the next
 // scores while the softmax warps work.  Every mbarrier wait is bounded; on expiry the kernel records kErrTimeout, all
-// roles drain to the common exit and the tensor memory is freed.  No cluster multicast.
+// roles drain to the common exit and the tensor memory is freed.  Every TMA load is a plain per-CTA load.
 #include "tc_common.cuh"
 
 namespace prism {

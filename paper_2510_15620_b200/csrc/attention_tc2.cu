@@ -20,7 +20,7 @@
 // Tensor memory: S_A, S_B, O_A, O_B, 128 columns each.  S_x(g+1) overwrites the columns P_x(g) occupies;
 // it is issued after PV_x(g) by the same thread with the same instruction shape, and such MMAs execute
 // in issue order.  Every mbarrier wait is bounded; on expiry the kernel records kErrTimeout, all roles
-// drain to the common exit and the tensor memory is freed.  No cluster multicast.
+// drain to the common exit and the tensor memory is freed.  Every TMA load is a plain per-CTA load.
 #include "tc_common.cuh"
 
 namespace prism {

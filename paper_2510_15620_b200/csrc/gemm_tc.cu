@@ -18,7 +18,7 @@
 // depend on where it sits in the batch (duplicated candidates give bit-identical scores).
 //
 // Every mbarrier wait is bounded: on expiry the kernel records kErrTimeout and all roles drain to
-// the common exit, which frees the tensor memory.  No cluster multicast is used anywhere.
+// the common exit, which frees the tensor memory.  Every TMA load is a plain per-CTA load.
 #include "tc_common.cuh"
 
 namespace prism {

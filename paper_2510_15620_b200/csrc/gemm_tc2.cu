@@ -5,8 +5,8 @@
 // memory, which is the co-limit of the single-CTA kernel.  Epilogues are the same code as in gemm_tc.cu.
 //
 // Protocol: full[s] lives in the leader and counts the bytes of BOTH CTAs' TMA loads; empty[s] and
-// acc_full[a] exist in both CTAs and are signalled by multicast commits; acc_empty[a] lives in the leader
-// and is arrived on by the epilogue warps of both CTAs.  No TMA multicast is used.  Every wait is bounded.
+// acc_full[a] exist in both CTAs and are signalled by commits that arrive in both CTAs; acc_empty[a] lives in the leader
+// and is arrived on by the epilogue warps of both CTAs.  Every TMA load is a plain per-CTA load.  Every wait is bounded.
 #include "tc_common.cuh"
 
 namespace prism {

@@ -299,6 +299,59 @@ def test_attention_tc_rescales_when_the_maximum_grows(P):
         assert np.max(np.abs(out.float().cpu().numpy() - ref)) < 2e-2 * max(1.0, np.max(np.abs(ref)))
 
 
+def test_attention_tc_many_items_per_cta(P):
+    """More work items than SMs x ring depth, mixed lengths from 1 to 6 key blocks, group size 4: the item ring of
+    the two-head kernel wraps many times, items of different cost interleave, and the counters of one launch are
+    rearmed for a later one.  Run twice on the same buffers: both runs must match the oracle and each other bit
+    for bit (the dynamic hand-out changes which SM computes what, never the arithmetic of a row)."""
+    rng = np.random.default_rng(21)
+    hq, hkv, dh = 8, 2, 128
+    lens = rng.integers(1, 700, size=96)
+    lens[:4] = [1, 128, 129, 699]
+    cu = np.zeros(len(lens) + 1, np.int32)
+    cu[1:] = np.cumsum(lens)
+    tot = int(cu[-1])
+    qkv = round_to_bf16(rng.normal(size=(tot, (hq + 2 * hkv) * dh)).astype(np.float32))
+    err = torch.zeros(1, dtype=torch.int32, device="cuda")
+    dq, dcu = dev(qkv, torch.bfloat16), dev(cu)
+    outs = []
+    for _ in range(2):
+        out = torch.zeros(tot, hq * dh, dtype=torch.bfloat16, device="cuda")
+        P.ops.prism_op_attention(dq, out, dcu, len(lens), int(lens.max()), hq, hkv, dh, 1, BF16, AUTO, err)
+        torch.cuda.synchronize()
+        assert int(err.item()) == 0
+        outs.append(out)
+    assert torch.equal(outs[0], outs[1])
+    ref = _attn_ref(qkv, cu, hq, hkv, dh, True)
+    assert np.max(np.abs(outs[0].float().cpu().numpy() - ref)) < 2e-2
+
+
+def test_attention_tc_work_counters_are_rearmed(P):
+    """Each launch of the two-head kernel takes the next pair of device work counters from a table of 1024 and
+    must leave it zeroed.  1100 small launches wrap the table; a counter left non-zero would make a later launch
+    skip its work, so the last outputs are checked against the first."""
+    rng = np.random.default_rng(5)
+    hq, hkv, dh = 4, 2, 128
+    lens = np.array([70, 130, 5])
+    cu = np.zeros(len(lens) + 1, np.int32)
+    cu[1:] = np.cumsum(lens)
+    tot = int(cu[-1])
+    qkv = dev(round_to_bf16(rng.normal(size=(tot, (hq + 2 * hkv) * dh)).astype(np.float32)), torch.bfloat16)
+    dcu = dev(cu)
+    err = torch.zeros(1, dtype=torch.int32, device="cuda")
+    first = torch.zeros(tot, hq * dh, dtype=torch.bfloat16, device="cuda")
+    P.ops.prism_op_attention(qkv, first, dcu, len(lens), 130, hq, hkv, dh, 1, BF16, AUTO, err)
+    out = torch.zeros_like(first)
+    for i in range(1100):
+        if i >= 1096:
+            out.zero_()
+        P.ops.prism_op_attention(qkv, out, dcu, len(lens), 130, hq, hkv, dh, 1, BF16, AUTO, err)
+        if i >= 1096:
+            torch.cuda.synchronize()
+            assert int(err.item()) == 0
+            assert torch.equal(out, first), i
+
+
 @pytest.mark.parametrize("impl", [AUTO, SOLO])
 def test_attention_tc_scores_far_above_the_first_key(P, impl):
     """The two-head kernel exponentiates against the row's score on key 0 and moves that reference only when a
