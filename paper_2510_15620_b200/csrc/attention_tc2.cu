@@ -115,7 +115,7 @@ struct ItemReader {
 __global__ void __launch_bounds__(kThreads, 1)
 k_attention_tc2(const __grid_constant__ CUtensorMap map_qkv, __nv_bfloat16* __restrict__ out,
                 const int* __restrict__ cu, int seq0, int nseq, int row0, int nqb, int gsz, int hq, int hkv,
-                int causal, float scale_log2, int* __restrict__ sched, int* __restrict__ err) {
+                int causal, int reverse, float scale_log2, int* __restrict__ sched, int* __restrict__ err) {
   extern __shared__ unsigned char smem_raw[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t raw = smem_u32(smem_raw);
@@ -176,7 +176,8 @@ k_attention_tc2(const __grid_constant__ CUtensorMap map_qkv, __nv_bfloat16* __re
         // draw candidates until one is a real item
         it.n_blocks = 0;
         for (int i = atomicAdd(sched, 1); i < total; i = atomicAdd(sched, 1)) {
-          const int in_group = i % per_group, rem = in_group % per_qb, sl = (i / per_group) * gsz + rem / npairs;
+          const int n_groups = (nseq + gsz - 1) / gsz, grp = reverse ? n_groups - 1 - i / per_group : i / per_group;
+          const int in_group = i % per_group, rem = in_group % per_qb, sl = grp * gsz + rem / npairs;
           if (sl >= nseq) continue;
           const int s = seq0 + sl;
           it.qb = nqb - 1 - in_group / per_qb;
@@ -531,7 +532,8 @@ __device__ int g_sched[kTickets][2];
 }  // namespace
 
 cudaError_t launch_attention_tc2(const void* qkv, void* out, const int* cu, int seq0, int nseq, int row0, int rows,
-                                 int max_len, int n_q_heads, int n_kv_heads, int causal, int* err, cudaStream_t st) {
+                                 int max_len, int n_q_heads, int n_kv_heads, int causal, int* err, cudaStream_t st,
+                                 bool reverse) {
   if (nseq <= 0 || max_len <= 0 || rows <= 0) return cudaSuccess;
   if (n_kv_heads < 1 || n_q_heads % n_kv_heads || ((n_q_heads / n_kv_heads) & 1)) return cudaErrorInvalidValue;
   static std::atomic<unsigned long long> smem_set{0};
@@ -565,7 +567,8 @@ cudaError_t launch_attention_tc2(const void* qkv, void* out, const int* cu, int 
   int* sched = sb + 2 * (ticket.fetch_add(1, std::memory_order_relaxed) % kTickets);
   const float scale_log2 = 1.4426950408889634f / sqrtf((float)DH);
   k_attention_tc2<<<grid, kThreads, kSmemBytes, st>>>(reinterpret_cast<const CUtensorMap&>(mq), (__nv_bfloat16*)out, cu,
-                                                      seq0, nseq, row0, nqb, gsz, n_q_heads, n_kv_heads, causal, scale_log2,
+                                                      seq0, nseq, row0, nqb, gsz, n_q_heads, n_kv_heads, causal, reverse ? 1 : 0,
+                                                      scale_log2,
                                                       sched, err);
   return cudaGetLastError();
 }

@@ -104,7 +104,7 @@ cudaError_t launch_positions(const int* cu, int n, int total, int* pos, cudaStre
 cudaError_t launch_embed(const void* table, int dtype, const int* tokens, int total, int d, float* x,
                          cudaStream_t st);
 cudaError_t launch_rmsnorm(const float* x, const void* gain, int dtype, int rows, int d, float eps,
-                           void* out, cudaStream_t st);
+                           void* out, cudaStream_t st, bool reverse = false);
 cudaError_t launch_rope_table(float* cos_t, float* sin_t, int max_pos, int head_dim, float theta,
                               cudaStream_t st);
 cudaError_t launch_rope_table_fused(float* tab, int max_pos, float theta, cudaStream_t st);
@@ -139,12 +139,12 @@ cudaError_t launch_gemm_tc(const TmaDesc& a, const TmaDesc& b0, const TmaDesc& b
                            int n, int k, int epilogue, const QkvRopeArgs* qa, int* err, cudaStream_t st);
 // The same GEMM on CTA pairs (tcgen05 cta_group::2, 256x256 tiles per cluster of two CTAs).
 cudaError_t launch_gemm_tc2(const TmaDesc& a, const TmaDesc& b0, const TmaDesc& b1, void* out, float* resid, int m,
-                            int n, int k, int epilogue, const QkvRopeArgs* qa, int* err, cudaStream_t st);
+                            int n, int k, int epilogue, const QkvRopeArgs* qa, int* err, cudaStream_t st, bool reverse = false);
 cudaError_t launch_attention_tc(const void* qkv, void* out, const int* cu, int seq0, int nseq, int row0, int rows,
                                 int max_len, int n_q_heads, int n_kv_heads, int causal, int* err, cudaStream_t st);
 // Two query heads of a key/value group per CTA, persistent (needs an even group size n_q_heads / n_kv_heads).
 cudaError_t launch_attention_tc2(const void* qkv, void* out, const int* cu, int seq0, int nseq, int row0, int rows,
-                                int max_len, int n_q_heads, int n_kv_heads, int causal, int* err, cudaStream_t st);
+                                int max_len, int n_q_heads, int n_kv_heads, int causal, int* err, cudaStream_t st, bool reverse = false);
 cudaError_t launch_attention_mma(const void* qkv, void* out, const int* cu, int seq0, int nseq, int row0,
                                  int max_len, int n_q_heads, int n_kv_heads, int causal, cudaStream_t st);
 

@@ -138,9 +138,9 @@ __global__ void __launch_bounds__(128) k_embed(const WT* __restrict__ table, con
 // S2/S7 RMSNorm: y = x * rsqrt(mean(x^2) + eps) * g.  One block per row; the row stays in registers.
 template <typename OT, int kVec>
 __global__ void __launch_bounds__(256) k_rmsnorm(const float* __restrict__ x, const OT* __restrict__ gain, int d,
-                                                 float eps, OT* __restrict__ out) {
+                                                 float eps, OT* __restrict__ out, int reverse) {
   __shared__ float red[32];
-  const size_t row = blockIdx.x;
+  const size_t row = reverse ? gridDim.x - 1 - blockIdx.x : blockIdx.x;  // last rows first: see launch_rmsnorm
   const float4* xr = reinterpret_cast<const float4*>(x + row * d);
   const int nv = d >> 2;
   float4 v[kVec];
@@ -178,9 +178,10 @@ __global__ void __launch_bounds__(256) k_rmsnorm(const float* __restrict__ x, co
 // flight, which hides HBM latency better than one block per row when the row is only a few KB.
 template <typename OT, int kPer>
 __global__ void __launch_bounds__(256) k_rmsnorm_warp(const float* __restrict__ x, const OT* __restrict__ gain,
-                                                      int rows, int d, float eps, OT* __restrict__ out) {
+                                                      int rows, int d, float eps, OT* __restrict__ out, int reverse) {
   const int lane = threadIdx.x & 31;
-  const long long row = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
+  const long long blk = reverse ? (long long)gridDim.x - 1 - blockIdx.x : blockIdx.x;
+  const long long row = blk * 8 + (threadIdx.x >> 5);
   if (row >= rows) return;
   const float4* xr = reinterpret_cast<const float4*>(x + (size_t)row * d);
   const int nv = d >> 2;
@@ -380,14 +381,17 @@ cudaError_t launch_embed(const void* table, int dtype, const int* tokens, int to
   return cudaGetLastError();
 }
 
+// reverse: blocks take the rows from the end of the matrix backwards.  The driver alternates the direction
+// from one kernel of a layer to the next, so that a kernel starts on the rows its predecessor wrote last,
+// which are the ones still in L2 when the tensors are larger than L2.
 cudaError_t launch_rmsnorm(const float* x, const void* gain, int dtype, int rows, int d, float eps,
-                           void* out, cudaStream_t st) {
+                           void* out, cudaStream_t st, bool reverse) {
   if (rows <= 0) return cudaSuccess;
   const int nv = d >> 2;
   if (nv > 8 * 256) return cudaErrorInvalidValue;
   if (nv <= 16 * 32) {  // rows of up to 8 KB: one warp per row
     const unsigned grid = (unsigned)((rows + 7) / 8);
-#define PRISM_NORMW(OT, V) k_rmsnorm_warp<OT, V><<<grid, 256, 0, st>>>(x, (const OT*)gain, rows, d, eps, (OT*)out)
+#define PRISM_NORMW(OT, V) k_rmsnorm_warp<OT, V><<<grid, 256, 0, st>>>(x, (const OT*)gain, rows, d, eps, (OT*)out, reverse ? 1 : 0)
     if (dtype == 1) {
       if (nv <= 128) PRISM_NORMW(__nv_bfloat16, 4);
       else if (nv <= 256) PRISM_NORMW(__nv_bfloat16, 8);
@@ -401,7 +405,7 @@ cudaError_t launch_rmsnorm(const float* x, const void* gain, int dtype, int rows
     return cudaGetLastError();
   }
 #define PRISM_NORM(OT, V) \
-  k_rmsnorm<OT, V><<<rows, 256, 0, st>>>(x, (const OT*)gain, d, eps, (OT*)out)
+  k_rmsnorm<OT, V><<<rows, 256, 0, st>>>(x, (const OT*)gain, d, eps, (OT*)out, reverse ? 1 : 0)
   if (dtype == 1) {
     if (nv <= 256) PRISM_NORM(__nv_bfloat16, 1);
     else if (nv <= 512) PRISM_NORM(__nv_bfloat16, 2);

@@ -94,7 +94,8 @@ template <int kEpi>
 __global__ void __launch_bounds__(kThreads, 1)
 k_gemm_tc2(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b0,
           const __grid_constant__ CUtensorMap map_b1, const __grid_constant__ CUtensorMap map_r,
-          __nv_bfloat16* __restrict__ out, int m, int n, int k, const QkvRopeArgs qa, int* __restrict__ err) {
+          __nv_bfloat16* __restrict__ out, int m, int n, int k, const QkvRopeArgs qa, int reverse,
+          int* __restrict__ err) {
   constexpr int kStages = stages_of(kEpi), kEpiStageBytes = epi_stage_bytes_of(kEpi);
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
@@ -119,7 +120,11 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
   const int pair_id = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
   const int m_tiles2 = (m + 2 * BM - 1) / (2 * BM), n_tiles = (n + kOutCols - 1) / kOutCols;
   const int num_tiles = m_tiles2 * n_tiles, num_kb = (k + BK - 1) / BK;
-  auto my_m_tile = [&](int t) { return (t / n_tiles) * 2 + (int)rank; };  // in units of 128 rows
+  // reverse: the row tiles are taken from the end of the matrix backwards (launch_gemm_tc2 says why)
+  auto my_m_tile = [&](int t) {  // in units of 128 rows
+    const int mrow2 = t / n_tiles;
+    return (reverse ? m_tiles2 - 1 - mrow2 : mrow2) * 2 + (int)rank;
+  };
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
@@ -474,8 +479,10 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
 
 }  // namespace
 
+// reverse: see launch_rmsnorm; the result is the same bit for bit in either direction (every tile has the same
+// shape and K order, and each output element is written or reduced into exactly once).
 cudaError_t launch_gemm_tc2(const TmaDesc& a, const TmaDesc& b0, const TmaDesc& b1, void* out, float* resid, int m,
-                           int n, int k, int epilogue, const QkvRopeArgs* qa, int* err, cudaStream_t st) {
+                           int n, int k, int epilogue, const QkvRopeArgs* qa, int* err, cudaStream_t st, bool reverse) {
   if (m <= 0 || n <= 0) return cudaSuccess;
   if (k <= 0 || (k % 8) || (n % 8)) return cudaErrorInvalidValue;
   static std::atomic<unsigned long long> smem_set[4];
@@ -528,13 +535,13 @@ cudaError_t launch_gemm_tc2(const TmaDesc& a, const TmaDesc& b0, const TmaDesc& 
   cfg.numAttrs = 1;
   cudaError_t le;
   if (epilogue == kEpiStore)
-    le = cudaLaunchKernelEx(&cfg, k_gemm_tc2<kEpiStore>, ma, mb0, mb1, mr, o, m, n, k, q, err);
+    le = cudaLaunchKernelEx(&cfg, k_gemm_tc2<kEpiStore>, ma, mb0, mb1, mr, o, m, n, k, q, reverse ? 1 : 0, err);
   else if (epilogue == kEpiResidual)
-    le = cudaLaunchKernelEx(&cfg, k_gemm_tc2<kEpiResidual>, ma, mb0, mb1, mr, o, m, n, k, q, err);
+    le = cudaLaunchKernelEx(&cfg, k_gemm_tc2<kEpiResidual>, ma, mb0, mb1, mr, o, m, n, k, q, reverse ? 1 : 0, err);
   else if (epilogue == kEpiSwiGLU)
-    le = cudaLaunchKernelEx(&cfg, k_gemm_tc2<kEpiSwiGLU>, ma, mb0, mb1, mr, o, m, n, k, q, err);
+    le = cudaLaunchKernelEx(&cfg, k_gemm_tc2<kEpiSwiGLU>, ma, mb0, mb1, mr, o, m, n, k, q, reverse ? 1 : 0, err);
   else if (epilogue == kEpiQkvRope)
-    le = cudaLaunchKernelEx(&cfg, k_gemm_tc2<kEpiQkvRope>, ma, mb0, mb1, mr, o, m, n, k, q, err);
+    le = cudaLaunchKernelEx(&cfg, k_gemm_tc2<kEpiQkvRope>, ma, mb0, mb1, mr, o, m, n, k, q, reverse ? 1 : 0, err);
   else
     return cudaErrorInvalidValue;
   if (le != cudaSuccess) return le;

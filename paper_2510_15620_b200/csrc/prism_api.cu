@@ -37,6 +37,8 @@ struct prism_handle {
   int chunk_tokens = 0;
   bool tc = false;  // tensor-core GEMM path
   bool pair = false;  // ... on CTA pairs (the default) rather than single CTAs
+  bool flip = true;   // consecutive kernels of a layer walk the rows in opposite directions (L2 reuse)
+  bool last_rev = false;  // direction of the kernel launched last
   int fa = 0;       // attention path: 0 SIMT, 1 tcgen05, 2 warp-level MMA
 
   std::vector<void*> dev_allocs;
@@ -484,9 +486,19 @@ int validate_schedule(const prism_handle* h, const prism_prune_schedule* s, int 
   return PRISM_OK;
 }
 
-cudaError_t gemm_tc_any(const prism_handle* h, const TmaDesc& a, const TmaDesc& b0, const TmaDesc& b1, void* out, float* resid,
+// The direction the next kernel takes the rows in: opposite to its predecessor's, so that it starts on what
+// was written last and is still in L2 (the layer's tensors are larger than L2 at full batch).  Kernels
+// without a direction argument count as forward.
+bool next_dir(prism_handle* h, bool supported) {
+  const bool rev = supported && h->flip && !h->last_rev;
+  h->last_rev = rev;
+  return rev;
+}
+
+cudaError_t gemm_tc_any(prism_handle* h, const TmaDesc& a, const TmaDesc& b0, const TmaDesc& b1, void* out, float* resid,
                         int m, int n, int k, int epi, const QkvRopeArgs* qa, cudaStream_t st) {
-  return h->pair ? launch_gemm_tc2(a, b0, b1, out, resid, m, n, k, epi, qa, h->errword, st)
+  const bool rev = next_dir(h, h->pair);
+  return h->pair ? launch_gemm_tc2(a, b0, b1, out, resid, m, n, k, epi, qa, h->errword, st, rev)
                  : launch_gemm_tc(a, b0, b1, out, resid, m, n, k, epi, qa, h->errword, st);
 }
 
@@ -504,7 +516,7 @@ int run_layer_chunk(prism_handle* h, const LayerDev& W, const LayerMaps* maps, f
     const double L = h->h_cu[s + 1] - h->h_cu[s];
     attn_flops += (c.causal ? 2.0 : 4.0) * L * L * c.n_q_heads * dh;
   }
-  PRISM_LAUNCH_P(h, st, PRISM_K_RMSNORM, norm_bytes, launch_rmsnorm(xr, W.g_attn, c.dtype, rows, D, c.rms_eps, h->a_norm, st));
+  PRISM_LAUNCH_P(h, st, PRISM_K_RMSNORM, norm_bytes, launch_rmsnorm(xr, W.g_attn, c.dtype, rows, D, c.rms_eps, h->a_norm, st, next_dir(h, true)));
   const bool fused_rope = h->tc && dh == 128;  // QK-norm + RoPE inside the QKV GEMM's epilogue
   if (fused_rope) {
     QkvRopeArgs qa{h->pos + r0, h->rope_fused, (const __nv_bfloat16*)W.g_q, (const __nv_bfloat16*)W.g_k,
@@ -524,8 +536,11 @@ int run_layer_chunk(prism_handle* h, const LayerDev& W, const LayerMaps* maps, f
   if (h->fa == 3)
     PRISM_LAUNCH_P(h, st, PRISM_K_ATTENTION, attn_flops,
                    launch_attention_tc2(h->qkv, h->attn, cu_dev, s0, s1 - s0, r0, rows, max_len, c.n_q_heads, c.n_kv_heads, c.causal,
-                                        h->errword, st));
-  else if (h->fa == 1)
+                                        h->errword, st, next_dir(h, true)));
+  else
+    next_dir(h, false);
+  if (h->fa == 3) {
+  } else if (h->fa == 1)
     PRISM_LAUNCH_P(h, st, PRISM_K_ATTENTION, attn_flops,
                    launch_attention_tc(h->qkv, h->attn, cu_dev, s0, s1 - s0, r0, rows, max_len, c.n_q_heads, c.n_kv_heads, c.causal,
                                        h->errword, st));
@@ -542,7 +557,7 @@ int run_layer_chunk(prism_handle* h, const LayerDev& W, const LayerMaps* maps, f
   else
     PRISM_LAUNCH_P(h, st, PRISM_K_GEMM_O, 2.0 * R * D * hd,
                    launch_gemm_simt(h->attn, W.w_o, nullptr, nullptr, xr, rows, D, hd, c.dtype, kEpiResidual, st));
-  PRISM_LAUNCH_P(h, st, PRISM_K_RMSNORM, norm_bytes, launch_rmsnorm(xr, W.g_ffn, c.dtype, rows, D, c.rms_eps, h->a_norm, st));
+  PRISM_LAUNCH_P(h, st, PRISM_K_RMSNORM, norm_bytes, launch_rmsnorm(xr, W.g_ffn, c.dtype, rows, D, c.rms_eps, h->a_norm, st, next_dir(h, true)));
   if (h->tc)
     PRISM_LAUNCH_P(h, st, PRISM_K_GEMM_GATEUP, 4.0 * R * c.ffn * D,
                    gemm_tc_any(h, h->map_a_norm, maps->gate, maps->up, h->hbuf, nullptr, rows, c.ffn, D, kEpiSwiGLU, nullptr, st));
