@@ -533,14 +533,12 @@ int run_layer_chunk(prism_handle* h, const LayerDev& W, const LayerMaps* maps, f
   PRISM_LAUNCH_P(h, st, PRISM_K_ROPE, 2.0 * R * (c.n_q_heads + c.n_kv_heads) * dh * esz,
                  launch_qknorm_rope(h->qkv, c.dtype, h->pos + r0, rows, c.n_q_heads, c.n_kv_heads, dh, c.qk_norm, W.g_q, W.g_k,
                                     c.rms_eps, h->rope_cos, h->rope_sin, st));
+  if (h->fa != 3) next_dir(h, false);  // the other attention kernels walk forward
   if (h->fa == 3)
     PRISM_LAUNCH_P(h, st, PRISM_K_ATTENTION, attn_flops,
                    launch_attention_tc2(h->qkv, h->attn, cu_dev, s0, s1 - s0, r0, rows, max_len, c.n_q_heads, c.n_kv_heads, c.causal,
                                         h->errword, st, next_dir(h, true)));
-  else
-    next_dir(h, false);
-  if (h->fa == 3) {
-  } else if (h->fa == 1)
+  else if (h->fa == 1)
     PRISM_LAUNCH_P(h, st, PRISM_K_ATTENTION, attn_flops,
                    launch_attention_tc(h->qkv, h->attn, cu_dev, s0, s1 - s0, r0, rows, max_len, c.n_q_heads, c.n_kv_heads, c.causal,
                                        h->errword, st));
