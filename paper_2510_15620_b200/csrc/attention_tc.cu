@@ -1,5 +1,6 @@
 // S5 on the 5th-generation tensor cores: varlen flash attention over packed sequences, bf16,
-// head_dim 128, GQA, causal or bidirectional.
+// head_dim 128, GQA, causal or bidirectional.  One query head per CTA: this kernel serves odd group sizes
+// Hq/Hkv and PRISM_IMPL_SOLO; even group sizes take the two-heads-per-CTA kernel of attention_tc2.cu.
 //
 // One CTA = 128 query rows of one (sequence, head); two CTAs fit on an SM.  Warp-specialised:
 //   warp 0      TMA producer: Q once, then K_j tiles (64 keys) into a 3-deep ring and V_j tiles into a

@@ -1,3 +1,5 @@
+// The single-CTA version of the projection GEMMs (PRISM_IMPL_SOLO; the default is the CTA-pair kernel of
+// gemm_tc2.cu, which this file also serves with the tensor-map builders).
 // Projection GEMMs of the decoder block on the 5th-generation tensor cores (sm_100a):
 //   C[M,N] = A[M,K] * B[N,K]^T, bf16 operands (both K-major), fp32 accumulation in tensor memory.
 //

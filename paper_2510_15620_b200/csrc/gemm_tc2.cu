@@ -2,7 +2,19 @@
 // 256x256 tile; each CTA loads its own 128 rows of A and ONE HALF (128 rows) of the B tile, the leader's
 // elected thread issues M256 N256 K16 MMAs that read both CTAs' shared memory, and each CTA's tensor
 // memory receives its own 128 accumulator rows.  Per SM this halves the B operand traffic through shared
-// memory, which is the co-limit of the single-CTA kernel.  Epilogues are the same code as in gemm_tc.cu.
+// memory, which is the co-limit of the single-CTA kernel.
+//
+// Epilogues (8 warps per CTA, one accumulator row per thread) compute what gemm_tc.cu's do, but every result
+// leaves through a swizzled shared-memory staging buffer and a TMA operation whose tensor map has exactly M
+// rows (the ragged last tile is clipped by the TMA unit):
+//   store     bf16, 32-row x 128-byte boxes, two buffers per warp
+//   residual  x += acc as a TMA reduce-add (no read of x by the SM, one add per element: deterministic)
+//   SwiGLU    rank 0 of the pair loads the tile's gate rows, rank 1 the up rows, so each CTA's accumulator
+//             holds gate and up of its rows side by side; silu(gate) * up, one 64-column box per warp and tile
+//   QKV       per-head RMSNorm (QK-norm) and rotary embedding on the q and k heads (a 256-column tile is two
+//             heads of 128); rotary-table rows staged per 32-row quarter; 32x32 boxes with the 64-byte swizzle
+// Every tile has the same shape and K order whatever M is, and the row tiles can be walked in either
+// direction, so a row's result does not depend on where it sits in the batch or on the direction.
 //
 // Protocol: full[s] lives in the leader and counts the bytes of BOTH CTAs' TMA loads; empty[s] and
 // acc_full[a] exist in both CTAs and are signalled by commits that arrive in both CTAs; acc_empty[a] lives in the leader
