@@ -208,12 +208,18 @@ def run_prism(args):
     wl = synth.workload(args.workload)
     cfg = wl.model
     n_req = max(args.requests, 1)
-    seeds = shard_requests(rank, world, n_req)
+    by_cand = args.shard == "candidates"
+    seeds = list(range(n_req)) if by_cand else shard_requests(rank, world, n_req)
     reqs = [synth.make_request(wl, s) for s in seeds]
     lq = wl.query_len
     lens_all = [np.diff(r["cand_offsets"]) + lq for r in reqs]
     max_seq = int(max(l.max() for l in lens_all))
     max_tot = int(max(l.sum() for l in lens_all))
+    # candidate sharding: every rank computes the same partition; this rank runs the candidates it owns
+    owned = [(P.shard_candidates(l, world) == rank).astype(np.uint8) for l in lens_all] if by_cand else None
+    if by_cand:
+        max_tot = int(max(l[o != 0].sum() for l, o in zip(lens_all, owned))) or 1
+    reduce = (lambda t: P.all_reduce_scores(t)) if (by_cand and world > 1) else (lambda t: None)
     w_np = synth.make_weights(cfg, wl.weight_seed)
     tw = P.upload_weights(w_np, cfg.dtype, device=str(dev), layers_pinned_host=bool(wl.stream_weights))
     model = P.PrismModel(cfg, tw, max_seq, wl.n_candidates, max_tot, activation_budget_bytes=wl.activation_budget_bytes,
@@ -255,11 +261,20 @@ def run_prism(args):
 
     def dev_step(i, s=sched):
         q, c, o = dreqs[i % n_req]
-        model.select(q, c, o, wl.top_k, s, want_trace=False)
+        if by_cand:
+            model.select_sharded(q, c, o, wl.top_k, s, owned[i % n_req], reduce, want_trace=False)
+        else:
+            model.select(q, c, o, wl.top_k, s, want_trace=False)
 
     def host_step(i):
         q, c, o = hreqs[i % n_req]
-        model.select_host(q, c, o, wl.top_k, sched, idx_out=hidx, sc_out=hsc)
+        if by_cand:  # the sharded entry point takes device buffers: the copies are made here, inside the timed region
+            tq, tc, to = (torch.from_numpy(a).to(dev, non_blocking=True) for a in (q, c, o))
+            idx, sc, _ = model.select_sharded(tq, tc, to, wl.top_k, sched, owned[i % n_req], reduce, want_trace=False)
+            hidx[: idx.numel()] = idx.cpu().numpy()
+            hsc[: sc.numel()] = sc.cpu().numpy()
+        else:
+            model.select_host(q, c, o, wl.top_k, sched, idx_out=hidx, sc_out=hsc)
 
     tokens_of = lambda i: int(lens_all[i % n_req].sum())
     K, W = args.steps, args.warmup
@@ -270,7 +285,7 @@ def run_prism(args):
     clocks = sampler.stop()
     total_ms = max_over_ranks(total_ms, world, dev)
     toks = sum(tokens_of(W + i) for i in range(K))
-    toks_all = sum_over_ranks(float(toks), world, dev)
+    toks_all = float(toks) if by_cand else sum_over_ranks(float(toks), world, dev)  # shared requests count once
     value = toks_all / (total_ms * 1e-3)
 
     e2e_ms, e2e_lat, _ = timed(host_step, K, W)
@@ -283,20 +298,26 @@ def run_prism(args):
     off_ms = max_over_ranks(off_ms / max(3, K // 4), world, dev)
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
-            "ms_per_step": total_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "ms_per_step": total_ms / K, "higher_is_better": True, "scaling": "strong" if by_cand else "weak", "vs_baseline": None,
             "dtype": "bf16" if cfg.dtype == 1 else "f32", "data": "synthetic",
             "config": {"workload": wl.name, "requests_cycled": n_req, "candidates": wl.n_candidates, "top_k": wl.top_k,
                        "tokens_per_request": int(np.mean([l.sum() for l in lens_all])),
                        "schedule": {"mode": sched.mode, "probe_layers": list(sched.probe_layers),
                                     "cv_threshold": sched.cv_threshold, "n_clusters": sched.n_clusters},
                        "l2": "no flush: each step streams 0.9 GB of weights and >1 GB of activations, far beyond the 126 MB L2",
-                       "parallelism": f"dp{world} over requests"},
+                       "parallelism": (f"{world} ranks share each request's candidates, one score all-reduce per probe"
+                                       if by_cand else f"dp{world} over requests")},
             "latency_ms": {"p50": float(np.percentile(lat, 50)), "p99": float(np.percentile(lat, 99))},
             "pruning_off_ms_per_step": off_ms, "pruning_speedup": off_ms / (total_ms / K),
             "e2e": {"value": toks_all / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "p50_ms": float(np.percentile(e2e_lat, 50))},
             "gpu_launches": int(launches), "clocks": clocks}
 
+    psteps = max(3, min(K, 10))
+    if by_cand and world > 1 and rank != 0:
+        for i in range(psteps):      # rank 0's profiled steps below contain all-reduces: take part in them
+            dev_step(W + i)
+        torch.cuda.synchronize()
     if rank == 0:
         # per-kernel device time, measured live with CUDA events around every launch of profiled steps
         lib = P.lib()
@@ -308,7 +329,6 @@ def run_prism(args):
         lib.prism_profile_read.argtypes = [C.c_void_p, C.POINTER(Stat), C.c_int]
         stats = (Stat * len(KERNEL_CLASSES))()
         lib.prism_profile(model._h, 1)
-        psteps = max(3, min(K, 10))
         for i in range(psteps):
             dev_step(W + i)
         torch.cuda.synchronize()
@@ -371,6 +391,9 @@ def main():
     ap.add_argument("--workload", type=int, default=1)
     ap.add_argument("--requests", type=int, default=10, help="distinct request seeds cycled through")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--shard", default="requests", choices=["requests", "candidates"],
+                    help="requests: every rank serves its own requests (weak scaling, the default); candidates: all "
+                         "ranks share each request, one score all-reduce per probe (strong scaling)")
     args = ap.parse_args()
     if args.impl == "reference":
         args.steps = 5 if args.steps is None else args.steps

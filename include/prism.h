@@ -188,6 +188,30 @@ PRISM_API int prism_select(prism_handle* h, const int32_t* query_tokens, int32_t
                  const prism_prune_schedule* sched, int32_t* topk_idx, float* topk_scores,
                  int32_t* n_out, prism_trace* trace, void* cuda_stream);
 
+/* One request over several GPUs, one process (rank) per GPU: the candidates are partitioned over the ranks (the
+ * sequences never attend to each other, so a candidate's hidden states and scores do not depend on which rank
+ * runs it), every rank runs the layers on its own candidates only, and the one global step of the method, the
+ * prune decision after a probe (Sec. 4.1), is taken by every rank on the same complete score vector.
+ *   owned      host uint8[N]: 1 for the candidates this rank runs.  Every candidate must be owned by exactly
+ *              one rank; the library cannot check that.
+ *   exchange   device float[N], caller-owned.  Before every prune decision the library writes the scores of
+ *              the n still-active candidates to exchange[0..n) on cuda_stream (0 for candidates of other
+ *              ranks) and calls reduce.
+ *   reduce     must replace exchange[0..n) by its element-wise sum over all ranks, ordered after the work
+ *              already enqueued on cuda_stream and before work enqueued there later (an all-reduce on that
+ *              stream, or a stream synchronisation around a host-side reduction); returns 0 on success.  n is
+ *              the same on every rank.  The sum is exact (one non-zero term per element), so all ranks
+ *              decide on bit-identical numbers and stay in step without any other communication.
+ * All other arguments, the outputs (identical on every rank) and the errors are those of prism_select; every
+ * rank passes the complete cand_tokens / cand_offsets.  max_total_tokens bounds the rank's own tokens.
+ * The paper runs on one device and has no counterpart of this entry point. */
+typedef int (*prism_exchange_fn)(void* ctx, int32_t n, void* cuda_stream);
+PRISM_API int prism_select_sharded(prism_handle* h, const int32_t* query_tokens, int32_t query_len,
+                 const int32_t* cand_tokens, const int32_t* cand_offsets, int32_t N, int32_t K,
+                 const prism_prune_schedule* sched, const uint8_t* owned, float* exchange,
+                 prism_exchange_fn reduce, void* ctx, int32_t* topk_idx, float* topk_scores,
+                 int32_t* n_out, prism_trace* trace, void* cuda_stream);
+
 /* Same request with HOST buffers: copies the three inputs to the device, runs prism_select's path
  * and copies topk_idx / topk_scores back (all on cuda_stream, inside the call).  Pinned buffers
  * make the copies asynchronous; pageable ones work too. */

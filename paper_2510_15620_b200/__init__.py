@@ -3,5 +3,6 @@
 Every step of the path runs in the CUDA kernels of lib/libprism.so; this package only marshals
 arguments.  Importing it without a built library raises: there is no CPU fallback."""
 from .binding import (PrismModel, PrismError, Calibrator, Trace, ProbeRecord, lib, upload_weights,  # noqa: F401
-                      status_str, PRISM_FP32, PRISM_BF16, PRISM_IMPL_AUTO, PRISM_IMPL_SIMT, PRISM_IMPL_MMA, PRISM_IMPL_SOLO)
+                      status_str, PRISM_FP32, PRISM_BF16, PRISM_IMPL_AUTO, PRISM_IMPL_SIMT, PRISM_IMPL_MMA, PRISM_IMPL_SOLO,
+                      shard_candidates, all_reduce_scores)
 from . import ops  # noqa: F401

@@ -4,7 +4,7 @@ from __future__ import annotations
 import ctypes as C
 import os
 from dataclasses import dataclass, field
-from typing import Dict, List, Optional, Sequence
+from typing import Callable, Dict, List, Optional, Sequence
 
 import numpy as np
 import torch
@@ -16,6 +16,30 @@ PRISM_MAX_CLUSTERS = 8
 # PRISM_LIBRARY overrides the in-tree library (e.g. an instrumented build of the same sources).
 _LIB_PATH = os.environ.get("PRISM_LIBRARY") or os.path.join(os.path.dirname(os.path.abspath(__file__)), "lib", "libprism.so")
 _lib = None
+
+
+
+EXCHANGE_FN = C.CFUNCTYPE(C.c_int, C.c_void_p, C.c_int32, C.c_void_p)
+
+
+def shard_candidates(lengths: Sequence[int], world_size: int) -> np.ndarray:
+    """Owner rank of every candidate: longest first, each to the rank with the fewest tokens so far (ties: lowest
+    rank).  Deterministic, so every rank computes the same partition from the same lengths."""
+    lengths = np.asarray(lengths, dtype=np.int64)
+    owner = np.zeros(len(lengths), dtype=np.int32)
+    load = np.zeros(max(world_size, 1), dtype=np.int64)
+    for i in np.argsort(-lengths, kind="stable"):
+        r = int(np.argmin(load))
+        owner[i] = r
+        load[r] += lengths[i]
+    return owner
+
+
+def all_reduce_scores(t: torch.Tensor, group=None) -> None:
+    """The `reduce` argument of select_sharded for torch.distributed: a SUM all-reduce (NCCL on GPUs), enqueued
+    on the current stream."""
+    import torch.distributed as dist
+    dist.all_reduce(t, op=dist.ReduceOp.SUM, group=group)
 
 
 class PrismError(RuntimeError):
@@ -94,6 +118,8 @@ def lib() -> C.CDLL:
             f.argtypes = sel
         L.prism_select_calibrated.restype = C.c_int
         L.prism_select_calibrated.argtypes = sel[:8] + [C.POINTER(Calibrator)] + sel[8:]
+        L.prism_select_sharded.restype = C.c_int
+        L.prism_select_sharded.argtypes = sel[:8] + [C.c_void_p, C.c_void_p, EXCHANGE_FN, C.c_void_p] + sel[8:]
         _lib = L
     return _lib
 
@@ -227,6 +253,44 @@ class PrismModel:
         stream = torch.cuda.current_stream().cuda_stream
         n_out, trace = self._call(lib().prism_select, query.data_ptr(), query.numel(), cand_tokens.data_ptr(),
                                   cand_offsets.data_ptr(), n, k, sched, idx.data_ptr(), sc.data_ptr(), want_trace, stream)
+        return idx[:n_out], sc[:n_out], trace
+
+    def select_sharded(self, query: torch.Tensor, cand_tokens: torch.Tensor, cand_offsets: torch.Tensor, k: int, sched,
+                       owned: np.ndarray, reduce: Callable[[torch.Tensor], None], want_trace: bool = True):
+        """prism_select_sharded: this rank runs the candidates with owned[i] != 0; `reduce(t)` must sum the float32
+        device tensor t over all ranks in place, ordered on the current stream (see all_reduce_scores).  The
+        outputs are the same on every rank."""
+        n = cand_offsets.numel() - 1
+        owned = np.ascontiguousarray(owned, dtype=np.uint8)
+        if owned.shape != (n,):
+            raise ValueError("owned must have one entry per candidate")
+        idx = torch.empty(max(k, 1), dtype=torch.int32, device=query.device)
+        sc = torch.empty(max(k, 1), dtype=torch.float32, device=query.device)
+        exchange = torch.zeros(max(n, 1), dtype=torch.float32, device=query.device)
+        failure = []
+
+        def on_exchange(_ctx, n_active, _stream):
+            try:
+                reduce(exchange[:n_active])
+                return 0
+            except BaseException as e:  # must not propagate into the C caller
+                failure.append(e)
+                return 1
+
+        cb = EXCHANGE_FN(on_exchange)
+        stream = torch.cuda.current_stream().cuda_stream
+
+        def fn(h, q, lq, c, o, n_, k_, s_, idx_, sc_, n_out_, tr_, st_):
+            return lib().prism_select_sharded(h, q, lq, c, o, n_, k_, s_, owned.ctypes.data, exchange.data_ptr(), cb, None,
+                                              idx_, sc_, n_out_, tr_, st_)
+
+        try:
+            n_out, trace = self._call(fn, query.data_ptr(), query.numel(), cand_tokens.data_ptr(), cand_offsets.data_ptr(),
+                                      n, k, sched, idx.data_ptr(), sc.data_ptr(), want_trace, stream)
+        except PrismError:
+            if failure:
+                raise failure[0]
+            raise
         return idx[:n_out], sc[:n_out], trace
 
     def select_calibrated(self, query: torch.Tensor, cand_tokens: torch.Tensor, cand_offsets: torch.Tensor, k: int, sched,

@@ -95,8 +95,9 @@ struct alignas(64) TmaDesc {
 };
 
 // ---- launchers (each returns the CUDA error of the launch; none synchronises) -----------------
+// owned (nullable, device, n bytes): candidates with owned[i] == 0 get length zero (candidate-sharded runs).
 cudaError_t launch_pack_offsets(const int* cand_offsets, int n, int query_len, int* cu, int* seq2orig,
-                                int* err, cudaStream_t st);
+                                int* err, cudaStream_t st, const unsigned char* owned = nullptr);
 cudaError_t launch_pack_tokens(const int* query, int query_len, const int* cand_tokens,
                                const int* cand_offsets, const int* cu, int n, int total, int vocab,
                                int* tokens, int* pos, int* err, cudaStream_t st);

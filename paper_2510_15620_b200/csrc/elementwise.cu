@@ -41,10 +41,12 @@ __device__ __forceinline__ int seq_of_row(const int* __restrict__ cu, int n, int
 }
 
 // ------------------------------------------------------------------------------------------------
-// S0 pack: cu = exclusive scan of (query_len + doc_len_i), seq2orig = identity.  One block.
+// S0 pack: cu = exclusive scan of (query_len + doc_len_i), seq2orig = identity.  One block.  With an ownership
+// mask (candidate-sharded runs) the candidates of other ranks become sequences of length zero: they keep their
+// place in every per-sequence array and take no rows.
 __global__ void __launch_bounds__(1024) k_pack_offsets(const int* __restrict__ off, int n, int lq,
-                                                       int* __restrict__ cu, int* __restrict__ seq2orig,
-                                                       int* __restrict__ err) {
+                                                       const unsigned char* __restrict__ owned, int* __restrict__ cu,
+                                                       int* __restrict__ seq2orig, int* __restrict__ err) {
   __shared__ int warp_tot[32];
   __shared__ int carry;
   if (threadIdx.x == 0) {
@@ -58,7 +60,7 @@ __global__ void __launch_bounds__(1024) k_pack_offsets(const int* __restrict__ o
     if (i < n) {
       int dl = off[i + 1] - off[i];
       if (dl < 0) { atomicOr(err, kErrBadOffsets); dl = 0; }
-      len = lq + dl;
+      len = (owned && !owned[i]) ? 0 : lq + dl;
       seq2orig[i] = i;
     }
     int v = len;
@@ -294,6 +296,10 @@ __global__ void __launch_bounds__(256) k_probe(const float* __restrict__ x, cons
                                                float eps, float* __restrict__ scores) {
   __shared__ float red[32];
   const int i = blockIdx.x;
+  if (cu[i + 1] == cu[i]) {  // a sequence without rows (another rank's candidate): its score comes from there
+    if (threadIdx.x == 0) scores[i] = 0.f;
+    return;
+  }
   const float* row = x + (size_t)(cu[i + 1] - 1) * d;
   float ss = 0.f, dot = 0.f;
   for (int c = threadIdx.x * 4; c < d; c += blockDim.x * 4) {
@@ -351,8 +357,8 @@ inline int grid_for(long long work, int block, int cap = 148 * 16) {
 }  // namespace
 
 cudaError_t launch_pack_offsets(const int* cand_offsets, int n, int query_len, int* cu, int* seq2orig,
-                                int* err, cudaStream_t st) {
-  k_pack_offsets<<<1, 1024, 0, st>>>(cand_offsets, n, query_len, cu, seq2orig, err);
+                                int* err, cudaStream_t st, const unsigned char* owned) {
+  k_pack_offsets<<<1, 1024, 0, st>>>(cand_offsets, n, query_len, owned, cu, seq2orig, err);
   return cudaGetLastError();
 }
 

@@ -57,6 +57,7 @@ struct prism_handle {
   ProbeRecordDev* recs = nullptr;
   float* trace_scores = nullptr;
   int* trace_ids = nullptr;
+  unsigned char* owned_dev = nullptr;  // candidate-sharded runs: which candidates this rank runs
   void* route_scratch = nullptr;
   int *in_query = nullptr, *in_cand = nullptr, *in_off = nullptr, *out_idx = nullptr;
   float* out_score = nullptr;
@@ -384,6 +385,7 @@ static int create_impl(prism_handle* h, const prism_model_cfg* cfg, const prism_
   PRISM_CUDA(h, dev_alloc(h, &h->recs, (size_t)c.n_layers));
   PRISM_CUDA(h, dev_alloc(h, &h->trace_scores, (size_t)c.n_layers * N));
   PRISM_CUDA(h, dev_alloc(h, &h->trace_ids, (size_t)c.n_layers * N));
+  PRISM_CUDA(h, dev_alloc(h, &h->owned_dev, N));
   PRISM_CUDA(h, dev_alloc(h, (unsigned char**)&h->route_scratch, route_scratch_bytes((int)N)));
   PRISM_CUDA(h, dev_alloc(h, &h->in_query, (size_t)c.max_seq_len));
   PRISM_CUDA(h, dev_alloc(h, &h->in_cand, T));
@@ -571,9 +573,19 @@ int run_layer_chunk(prism_handle* h, const LayerDev& W, const LayerMaps* maps, f
   return PRISM_OK;
 }
 
+// Candidate-sharded runs (Shard non-null): this rank packs only the candidates it owns (the others are sequences
+// of length zero), probes write 0 for them, and before every prune decision `reduce` sums the score vector over
+// the ranks, after which every rank evaluates the same rule on the same numbers.
+struct Shard {
+  const uint8_t* owned;  // host, N bytes
+  float* exchange;       // device, N floats
+  prism_exchange_fn reduce;
+  void* ctx;
+};
+
 int select_impl(prism_handle* h, const int32_t* query, int32_t lq, const int32_t* cand, const int32_t* off, int32_t N,
                 int32_t K, const prism_prune_schedule* sched, int32_t* topk_idx, float* topk_scores, int32_t* n_out,
-                prism_trace* trace, cudaStream_t st) {
+                prism_trace* trace, cudaStream_t st, const Shard* shard = nullptr) {
   const prism_model_cfg& c = h->cfg;
   h->err.clear();
   if (trace) {
@@ -604,6 +616,10 @@ int select_impl(prism_handle* h, const int32_t* query, int32_t lq, const int32_t
   for (int i = 0; i < N; ++i)
     if (h->h_off[i + 1] < h->h_off[i]) return fail(h, PRISM_ERR_BAD_INPUT, "cand_offsets not monotone");
   for (int i = 0; i < N; ++i) {
+    if (shard && !shard->owned[i]) {  // another rank's candidate: no rows here
+      h->h_cu[i + 1] = (int)total;
+      continue;
+    }
     const long long dl = (long long)h->h_off[i + 1] - h->h_off[i];
     if (dl + lq > c.max_seq_len) return fail(h, PRISM_ERR_SHAPE_LIMIT, "a sequence exceeds max_seq_len");
     if (dl + lq > h->chunk_tokens) return fail(h, PRISM_ERR_BUDGET, "a sequence exceeds the chunk the activation budget allows");
@@ -622,7 +638,13 @@ int select_impl(prism_handle* h, const int32_t* query, int32_t lq, const int32_t
   PRISM_CUDA(h, cudaMemsetAsync(h->errword, 0, sizeof(int), st));
 
   int cur = 0;  // ping-pong index of x / cu / seq2orig
-  PRISM_LAUNCH_P(h, st, PRISM_K_PACK, 8.0 * N, launch_pack_offsets(off, N, lq, h->cu[cur], h->seq2orig[cur], h->errword, st));
+  const unsigned char* owned_dev = nullptr;
+  if (shard) {
+    PRISM_CUDA(h, cudaMemcpyAsync(h->owned_dev, shard->owned, (size_t)N, cudaMemcpyHostToDevice, st));
+    owned_dev = h->owned_dev;
+  }
+  PRISM_LAUNCH_P(h, st, PRISM_K_PACK, 8.0 * N,
+                 launch_pack_offsets(off, N, lq, h->cu[cur], h->seq2orig[cur], h->errword, st, owned_dev));
   PRISM_LAUNCH_P(h, st, PRISM_K_PACK, 12.0 * total,
                  launch_pack_tokens(query, lq, cand, off, h->cu[cur], N, (int)total, c.vocab, h->tokens, h->pos, h->errword, st));
   PRISM_LAUNCH_P(h, st, PRISM_K_EMBED, (double)total * c.hidden * (4.0 + h->esz),
@@ -674,9 +696,11 @@ int select_impl(prism_handle* h, const int32_t* query, int32_t lq, const int32_t
       p.is_final = is_final ? 1 : 0;
       p.layer = layers_run;
       const int nxt = cur ^ 1;
+      float* score_buf = shard ? shard->exchange : h->scores;
       PRISM_LAUNCH_P(h, st, PRISM_K_PROBE, 4.0 * n * c.hidden,
-                     launch_probe(h->x[cur], h->cu[cur], n, c.hidden, h->g_final, c.dtype, h->w_diff, c.rms_eps, h->scores, st));
-      PRISM_LAUNCH_P(h, st, PRISM_K_ROUTE, 8.0 * n, launch_route(h->scores, h->cu[cur], h->seq2orig[cur], n, p, h->cu[nxt], h->seq2orig[nxt], h->old_of_new,
+                     launch_probe(h->x[cur], h->cu[cur], n, c.hidden, h->g_final, c.dtype, h->w_diff, c.rms_eps, score_buf, st));
+      if (shard && shard->reduce(shard->ctx, n, st) != 0) return fail(h, PRISM_ERR_CUDA, "the score exchange callback failed");
+      PRISM_LAUNCH_P(h, st, PRISM_K_ROUTE, 8.0 * n, launch_route(score_buf, h->cu[cur], h->seq2orig[cur], n, p, h->cu[nxt], h->seq2orig[nxt], h->old_of_new,
                                    h->state, h->res_idx, h->res_score, h->recs + n_rec,
                                    h->trace_scores + (size_t)n_rec * c.max_candidates,
                                    h->trace_ids + (size_t)n_rec * c.max_candidates, h->route_scratch, st));
@@ -822,6 +846,27 @@ int prism_select_calibrated(prism_handle* h, const int32_t* query_tokens, int32_
     cal->n_adjustments++;
   }
   return PRISM_OK;
+}
+
+int prism_select_sharded(prism_handle* h, const int32_t* query_tokens, int32_t query_len, const int32_t* cand_tokens,
+                         const int32_t* cand_offsets, int32_t N, int32_t K, const prism_prune_schedule* sched,
+                         const uint8_t* owned, float* exchange, prism_exchange_fn reduce, void* ctx, int32_t* topk_idx,
+                         float* topk_scores, int32_t* n_out, prism_trace* trace, void* cuda_stream) {
+  int rc = check_args(h, query_tokens, query_len, cand_tokens, cand_offsets, N, K, topk_idx, topk_scores, n_out);
+  if (rc != PRISM_OK) return rc;
+  *n_out = 0;
+  if (!owned || !exchange || !reduce) return fail(h, PRISM_ERR_INVALID_ARG, "owned, exchange or reduce is null");
+  if (N > h->cfg.max_candidates) return fail(h, PRISM_ERR_SHAPE_LIMIT, "N exceeds max_candidates");
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  const Shard shard{owned, exchange, reduce, ctx};
+  rc = select_impl(h, query_tokens, query_len, cand_tokens, cand_offsets, N, K, sched, topk_idx, topk_scores, n_out, trace, st,
+                   &shard);
+  if (rc != PRISM_OK) {
+    *n_out = 0;
+    cudaStreamSynchronize(st);
+    if (h->copy_stream) cudaStreamSynchronize(h->copy_stream);
+  }
+  return rc;
 }
 
 int prism_select_host(prism_handle* h, const int32_t* query_tokens, int32_t query_len, const int32_t* cand_tokens,
