@@ -48,7 +48,7 @@ class HostSum:
         return reduce
 
 
-def run_sharded(P, cfg, w, req, k, sched, owner, world):
+def run_sharded(P, cfg, w, req, k, sched, owner, world, **model_kw):
     out, errs = [None] * world, []
     hs = HostSum(world)
 
@@ -56,7 +56,7 @@ def run_sharded(P, cfg, w, req, k, sched, owner, world):
         try:
             torch.cuda.set_device(0)
             with torch.cuda.stream(torch.cuda.Stream()):
-                model = make_model(P, cfg, w, req)
+                model = make_model(P, cfg, w, req, **model_kw)
                 idx, sc, tr = model.select_sharded(dev_i32(req["query"]), dev_i32(req["cand_tokens"]),
                                                    dev_i32(req["cand_offsets"]), k, sched,
                                                    (owner == rank).astype(np.uint8), hs.reducer(rank))
@@ -126,6 +126,37 @@ def test_sharded_with_an_idle_rank_and_a_single_owner(P, mid_case):
         for idx, sc, _tr in out:
             assert np.array_equal(idx, ref_idx)
             assert np.array_equal(sc.view(np.uint32), ref_sc.view(np.uint32))
+    base.close()
+
+
+def test_sharded_fp32_path_and_chunked_streamed_models(P, mid_case):
+    """The CUDA-core fp32 path (cfg 0) and a bf16 model that runs chunked under an activation budget with its
+    layer weights streamed from pinned host memory: sharded over two ranks, both must return what the plain
+    handle returns.  In the chunked case some chunks of a rank consist of other ranks' rowless sequences only."""
+    wl = synth.workload(0)
+    w0 = synth.make_weights(wl.model)
+    r0 = synth.make_request(wl, 0)
+    base = make_model(P, wl.model, w0, r0)
+    ref = run(P, base, r0, wl.top_k, wl.schedule)
+    owner = P.shard_candidates(np.diff(r0["cand_offsets"]) + len(r0["query"]), 2)
+    for o in (owner, np.zeros_like(owner)):
+        out, _ = run_sharded(P, wl.model, w0, r0, wl.top_k, wl.schedule, o, 2)
+        for idx, sc, _tr in out:
+            assert np.array_equal(idx, ref[0]) and np.array_equal(sc.view(np.uint32), ref[1].view(np.uint32))
+    base.close()
+
+    w, req = mid_case
+    lens = np.diff(req["cand_offsets"]) + len(req["query"])
+    per_tok = (1024 + 4096 + 2048 + 3072) * 2
+    budget = 2 * int(lens.sum()) * 1024 * 4 + per_tok * (int(lens.max()) + 50)     # about one long sequence per chunk
+    base = make_model(P, MID, w, req)
+    ref = run(P, base, req, MID_WL.top_k, MID_WL.schedule)
+    owner = (np.arange(MID_WL.n_candidates) >= MID_WL.n_candidates // 2).astype(np.int32)   # contiguous halves
+    out, _ = run_sharded(P, MID, w, req, MID_WL.top_k, MID_WL.schedule, owner, 2,
+                         activation_budget_bytes=budget, stream_weights=True)
+    for idx, sc, tr in out:
+        assert np.array_equal(idx, ref[0]) and np.array_equal(sc.view(np.uint32), ref[1].view(np.uint32))
+        assert tr.n_chunks_max > 3
     base.close()
 
 
