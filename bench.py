@@ -355,6 +355,7 @@ def run_prism(args):
                             "achieved": ach, "peak": peak, "unit": "TFLOP/s", "frac": ach / peak if peak else None,
                             "peak_source": f"bf16_tflops_sustained of {peaks['source']} (kernel timed inside a long step)",
                             "frac_of_burst_peak": ach / peaks["bf16_tflops"],
+                            "frac_of_nominal_2250": ach / 2250.0,
                             "flops_per_launch": g_fl / g_n if g_n else 0, "avg_launch_ms": g_ms / g_n if g_n else 0,
                             "traffic": traffic,
                             "traffic_note": "bytes per launch: ncu dram read+write of each GEMM shape at M = 8192 "
