@@ -91,6 +91,12 @@ typedef struct {
                       stream while layer l computes (overlapped layer streaming, Sec. 4.2) */
   int32_t gemm_impl;      /* PRISM_IMPL_* */
   int32_t attention_impl; /* PRISM_IMPL_* */
+  int32_t embed_cache_rows; /* 0: `embed` is a device table.  > 0: embedding table caching (Sec. 4.4): `embed` is
+                      the complete table in PINNED HOST memory and the device holds this many of its rows,
+                      replaced least-recently-used first.  Every request first collects its distinct tokens
+                      (one device-to-host copy of the token ids) and brings the missing rows into the cache
+                      before the layers start.  A request with more distinct tokens than rows fails with
+                      PRISM_ERR_SHAPE_LIMIT.  The paper sizes the cache at 10 % of the vocabulary. */
 } prism_model_cfg;
 
 typedef struct {
@@ -211,6 +217,10 @@ PRISM_API int prism_select_sharded(prism_handle* h, const int32_t* query_tokens,
                  const prism_prune_schedule* sched, const uint8_t* owned, float* exchange,
                  prism_exchange_fn reduce, void* ctx, int32_t* topk_idx, float* topk_scores,
                  int32_t* n_out, prism_trace* trace, void* cuda_stream);
+
+/* Counters of the embedding-row cache since prism_create: rows found in the cache, rows fetched from the host
+ * table, and fetched rows that replaced another token's row.  All zero when embed_cache_rows == 0. */
+PRISM_API int prism_embed_cache_stats(const prism_handle* h, int64_t* hits, int64_t* misses, int64_t* evictions);
 
 /* Same request with HOST buffers: copies the three inputs to the device, runs prism_select's path
  * and copies topk_idx / topk_scores back (all on cuda_stream, inside the call).  Pinned buffers

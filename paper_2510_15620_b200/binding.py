@@ -54,7 +54,7 @@ class _ModelCfg(C.Structure):
                 ("rms_eps", C.c_float), ("causal", C.c_int32), ("qk_norm", C.c_int32), ("dtype", C.c_int32),
                 ("max_seq_len", C.c_int32), ("max_candidates", C.c_int32), ("max_total_tokens", C.c_int32),
                 ("activation_budget_bytes", C.c_int64), ("weight_residency", C.c_int32), ("gemm_impl", C.c_int32),
-                ("attention_impl", C.c_int32)]
+                ("attention_impl", C.c_int32), ("embed_cache_rows", C.c_int32)]
 
 
 class _LayerWeights(C.Structure):
@@ -109,6 +109,8 @@ def lib() -> C.CDLL:
         L.prism_launch_count.argtypes = [C.c_void_p]
         L.prism_create.restype = C.c_int
         L.prism_create.argtypes = [C.POINTER(_ModelCfg), C.POINTER(_Weights), C.POINTER(C.c_void_p)]
+        L.prism_embed_cache_stats.restype = C.c_int
+        L.prism_embed_cache_stats.argtypes = [C.c_void_p, C.POINTER(C.c_int64), C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
         L.prism_destroy.restype = None
         L.prism_destroy.argtypes = [C.c_void_p]
         sel = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.POINTER(_Schedule),
@@ -153,10 +155,11 @@ class Trace:
     workspace_bytes: int
 
 
-def upload_weights(w: Dict[str, object], dtype: int, device: str = "cuda", layers_pinned_host: bool = False):
+def upload_weights(w: Dict[str, object], dtype: int, device: str = "cuda", layers_pinned_host: bool = False,
+                   embed_pinned_host: bool = False):
     """numpy weights (as produced by the synthetic generator: float32 values, already bf16-rounded in
     bf16 mode) -> torch tensors of the library's element type.  Layer tensors go to pinned host memory
-    when they are to be streamed."""
+    when they are to be streamed, the embedding table when it is to be cached row by row."""
     def conv(a: np.ndarray, pinned: bool) -> torch.Tensor:
         t = torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32))
         if dtype == PRISM_BF16:
@@ -164,7 +167,7 @@ def upload_weights(w: Dict[str, object], dtype: int, device: str = "cuda", layer
         if pinned:
             return t.pin_memory()
         return t.to(device)
-    out: Dict[str, object] = {k: conv(w[k], False) for k in ("embed", "g_final", "score_head")}
+    out: Dict[str, object] = {k: conv(w[k], embed_pinned_host and k == "embed") for k in ("embed", "g_final", "score_head")}
     out["layers"] = [{k: conv(v, layers_pinned_host) for k, v in lw.items()} for lw in w["layers"]]
     return out
 
@@ -174,13 +177,14 @@ class PrismModel:
 
     def __init__(self, cfg, weights: Dict[str, object], max_seq_len: int, max_candidates: int, max_total_tokens: int,
                  activation_budget_bytes: int = 0, stream_weights: bool = False, gemm_impl: int = PRISM_IMPL_AUTO,
-                 attention_impl: int = PRISM_IMPL_AUTO):
+                 attention_impl: int = PRISM_IMPL_AUTO, embed_cache_rows: int = 0):
         self._h = C.c_void_p()
         self.cfg = cfg
         self._weights = weights            # keep the tensors alive for the life of the handle
         c = _ModelCfg(cfg.n_layers, cfg.hidden, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.ffn, cfg.vocab,
                       cfg.rope_theta, cfg.rms_eps, cfg.causal, cfg.qk_norm, cfg.dtype, max_seq_len, max_candidates,
-                      max_total_tokens, activation_budget_bytes, 1 if stream_weights else 0, gemm_impl, attention_impl)
+                      max_total_tokens, activation_budget_bytes, 1 if stream_weights else 0, gemm_impl, attention_impl,
+                      embed_cache_rows)
         layers = (_LayerWeights * cfg.n_layers)()
         for i, lw in enumerate(weights["layers"]):
             for k, _ in _LayerWeights._fields_:
@@ -201,6 +205,12 @@ class PrismModel:
             self.close()
         except Exception:
             pass
+
+    def embed_cache_stats(self):
+        """(hits, misses, evictions) of the embedding-row cache since the handle was created."""
+        h, m, e = C.c_int64(0), C.c_int64(0), C.c_int64(0)
+        lib().prism_embed_cache_stats(self._h, C.byref(h), C.byref(m), C.byref(e))
+        return int(h.value), int(m.value), int(e.value)
 
     @property
     def launch_count(self) -> int:

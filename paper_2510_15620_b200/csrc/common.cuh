@@ -103,7 +103,10 @@ cudaError_t launch_pack_tokens(const int* query, int query_len, const int* cand_
                                int* tokens, int* pos, int* err, cudaStream_t st);
 cudaError_t launch_positions(const int* cu, int n, int total, int* pos, cudaStream_t st);
 cudaError_t launch_embed(const void* table, int dtype, const int* tokens, int total, int d, float* x,
-                         cudaStream_t st);
+                         cudaStream_t st, const int* tok2slot = nullptr);
+// Sec. 4.4 embedding table caching: rows of the pinned host table into rows of the device cache.
+cudaError_t launch_cache_fill(const void* host_table, void* cache, const int* pairs, int n_rows, int row_bytes,
+                              int* tok2slot, cudaStream_t st);
 cudaError_t launch_rmsnorm(const float* x, const void* gain, int dtype, int rows, int d, float eps,
                            void* out, cudaStream_t st, bool reverse = false);
 cudaError_t launch_rope_table(float* cos_t, float* sin_t, int max_pos, int head_dim, float theta,

@@ -115,11 +115,13 @@ __global__ void k_positions(const int* __restrict__ cu, int n, int total, int* _
 
 // ------------------------------------------------------------------------------------------------
 // S1 embedding gather into the fp32 residual stream.  One block per token row.
+// With a row cache (Sec. 4.4) `table` is the cache and tok2slot maps a token id to its row there.
 template <typename WT>
 __global__ void __launch_bounds__(128) k_embed(const WT* __restrict__ table, const int* __restrict__ tokens,
-                                               int d, float* __restrict__ x) {
+                                               const int* __restrict__ tok2slot, int d, float* __restrict__ x) {
   const int t = blockIdx.x;
-  const WT* src = table + (size_t)tokens[t] * d;
+  const int tok = tokens[t];
+  const WT* src = table + (size_t)(tok2slot ? tok2slot[tok] : tok) * d;
   float* dst = x + (size_t)t * d;
   if constexpr (sizeof(WT) == 2) {
     for (int c = threadIdx.x * 8; c < d; c += blockDim.x * 8) {
@@ -378,12 +380,32 @@ cudaError_t launch_positions(const int* cu, int n, int total, int* pos, cudaStre
 }
 
 cudaError_t launch_embed(const void* table, int dtype, const int* tokens, int total, int d, float* x,
-                         cudaStream_t st) {
+                         cudaStream_t st, const int* tok2slot) {
   if (total <= 0) return cudaSuccess;
   if (dtype == 1)
-    k_embed<__nv_bfloat16><<<total, 128, 0, st>>>((const __nv_bfloat16*)table, tokens, d, x);
+    k_embed<__nv_bfloat16><<<total, 128, 0, st>>>((const __nv_bfloat16*)table, tokens, tok2slot, d, x);
   else
-    k_embed<float><<<total, 128, 0, st>>>((const float*)table, tokens, d, x);
+    k_embed<float><<<total, 128, 0, st>>>((const float*)table, tokens, tok2slot, d, x);
+  return cudaGetLastError();
+}
+
+// Embedding-row cache fill: row pairs[2i] of the host table (pinned, read over the host link) goes to cache row
+// pairs[2i+1], and the token's entry in tok2slot follows.  One block per row, 16-byte pieces.
+__global__ void __launch_bounds__(128) k_cache_fill(const unsigned char* __restrict__ host_table,
+                                                    unsigned char* __restrict__ cache, const int* __restrict__ pairs,
+                                                    int row_bytes, int* __restrict__ tok2slot) {
+  const int tok = pairs[2 * blockIdx.x], slot = pairs[2 * blockIdx.x + 1];
+  const uint4* src = reinterpret_cast<const uint4*>(host_table + (size_t)tok * row_bytes);
+  uint4* dst = reinterpret_cast<uint4*>(cache + (size_t)slot * row_bytes);
+  for (int c = threadIdx.x; c < row_bytes / 16; c += blockDim.x) dst[c] = src[c];
+  if (threadIdx.x == 0) tok2slot[tok] = slot;
+}
+
+cudaError_t launch_cache_fill(const void* host_table, void* cache, const int* pairs, int n_rows, int row_bytes,
+                              int* tok2slot, cudaStream_t st) {
+  if (n_rows <= 0) return cudaSuccess;
+  if (row_bytes % 16) return cudaErrorInvalidValue;
+  k_cache_fill<<<n_rows, 128, 0, st>>>((const unsigned char*)host_table, (unsigned char*)cache, pairs, row_bytes, tok2slot);
   return cudaGetLastError();
 }
 

@@ -58,6 +58,19 @@ struct prism_handle {
   float* trace_scores = nullptr;
   int* trace_ids = nullptr;
   unsigned char* owned_dev = nullptr;  // candidate-sharded runs: which candidates this rank runs
+
+  // Embedding table caching (Sec. 4.4): `embed` is the pinned host table, the device holds cache_rows rows.
+  int cache_rows = 0;
+  unsigned char* cache_dev = nullptr;  // [cache_rows, D] in the table's element type
+  int* tok2slot_dev = nullptr;         // [vocab]: row of a token in the cache (valid for the tokens of the request)
+  int* pairs_dev = nullptr;            // (token, slot) of the rows to fetch
+  int* h_tokens = nullptr;             // pinned: the request's token ids
+  int* h_pairs = nullptr;              // pinned
+  std::vector<int> slot_of_tok, tok_of_slot;
+  std::vector<uint64_t> slot_stamp;    // request number of the slot's last use (0 = never)
+  std::vector<uint64_t> tok_seen;      // request number in which the token was last looked up
+  uint64_t request_no = 0;
+  int64_t cache_hits = 0, cache_misses = 0, cache_evictions = 0;
   void* route_scratch = nullptr;
   int *in_query = nullptr, *in_cand = nullptr, *in_off = nullptr, *out_idx = nullptr;
   float* out_score = nullptr;
@@ -256,6 +269,7 @@ int validate_cfg(const prism_model_cfg& c, std::string* why) {
   if (c.weight_residency != PRISM_WEIGHTS_DEVICE && c.weight_residency != PRISM_WEIGHTS_HOST_STREAMED)
     return bad("unknown weight_residency");
   if (!(c.rope_theta > 0.f) || !(c.rms_eps >= 0.f)) return bad("rope_theta must be > 0 and rms_eps >= 0");
+  if (c.embed_cache_rows < 0) return bad("negative embed_cache_rows");
   auto unsup = [&](const char* m) { *why = m; return PRISM_ERR_UNSUPPORTED; };
   if (c.head_dim % 2 || c.head_dim > 256) return unsup("head_dim must be even and <= 256");
   if (c.hidden % 4 || c.hidden > 8192) return unsup("hidden must be a multiple of 4 and <= 8192");
@@ -289,6 +303,14 @@ const char* prism_status_str(int s) {
 const char* prism_last_error(const prism_handle* h) { return h ? h->err.c_str() : ""; }
 
 int64_t prism_launch_count(const prism_handle* h) { return h ? h->launches : 0; }
+
+int prism_embed_cache_stats(const prism_handle* h, int64_t* hits, int64_t* misses, int64_t* evictions) {
+  if (!h) return PRISM_ERR_INVALID_ARG;
+  if (hits) *hits = h->cache_hits;
+  if (misses) *misses = h->cache_misses;
+  if (evictions) *evictions = h->cache_evictions;
+  return PRISM_OK;
+}
 
 int prism_profile(prism_handle* h, int enable) {
   if (!h) return PRISM_ERR_INVALID_ARG;
@@ -386,6 +408,27 @@ static int create_impl(prism_handle* h, const prism_model_cfg* cfg, const prism_
   PRISM_CUDA(h, dev_alloc(h, &h->trace_scores, (size_t)c.n_layers * N));
   PRISM_CUDA(h, dev_alloc(h, &h->trace_ids, (size_t)c.n_layers * N));
   PRISM_CUDA(h, dev_alloc(h, &h->owned_dev, N));
+  if (c.embed_cache_rows > 0) {
+    if ((reinterpret_cast<uintptr_t>(w->embed) & 15) || (D * h->esz) % 16)
+      return fail(h, PRISM_ERR_INVALID_ARG, "the host embedding table must be 16-byte aligned with rows of a multiple of 16 bytes");
+    cudaPointerAttributes pa{};
+    if (cudaPointerGetAttributes(&pa, w->embed) != cudaSuccess || pa.type != cudaMemoryTypeHost) {
+      cudaGetLastError();
+      return fail(h, PRISM_ERR_INVALID_ARG, "embed_cache_rows > 0 needs the embedding table in pinned host memory");
+    }
+    h->cache_rows = std::min(c.embed_cache_rows, c.vocab);
+    const size_t C = (size_t)h->cache_rows, ntok = T + (size_t)c.max_seq_len;
+    PRISM_CUDA(h, dev_alloc(h, &h->cache_dev, C * D * h->esz));
+    PRISM_CUDA(h, dev_alloc(h, &h->tok2slot_dev, (size_t)c.vocab));
+    PRISM_CUDA(h, dev_alloc(h, &h->pairs_dev, 2 * C));
+    PRISM_CUDA(h, host_alloc(h, &h->h_tokens, ntok));
+    PRISM_CUDA(h, host_alloc(h, &h->h_pairs, 2 * C));
+    PRISM_CUDA(h, cudaMemset(h->tok2slot_dev, 0, (size_t)c.vocab * sizeof(int)));
+    h->slot_of_tok.assign((size_t)c.vocab, -1);
+    h->tok_of_slot.assign(C, -1);
+    h->slot_stamp.assign(C, 0);
+    h->tok_seen.assign((size_t)c.vocab, 0);
+  }
   PRISM_CUDA(h, dev_alloc(h, (unsigned char**)&h->route_scratch, route_scratch_bytes((int)N)));
   PRISM_CUDA(h, dev_alloc(h, &h->in_query, (size_t)c.max_seq_len));
   PRISM_CUDA(h, dev_alloc(h, &h->in_cand, T));
@@ -573,6 +616,69 @@ int run_layer_chunk(prism_handle* h, const LayerDev& W, const LayerMaps* maps, f
   return PRISM_OK;
 }
 
+// Embedding table caching (Sec. 4.4).  The request's token ids come to the host; every distinct token either has a
+// row in the device cache (hit) or gets one: a free row first, else the row whose last use lies furthest back
+// among those this request does not use.  The missing rows are then read from the pinned host table by one kernel.
+// Token ids outside the vocabulary are skipped here; the pack kernel reports them.
+int cache_prepare(prism_handle* h, const int* query, int lq, const int* cand, int n_cand, cudaStream_t st) {
+  const prism_model_cfg& c = h->cfg;
+  if (n_cand < 0 || (long long)n_cand + lq > (long long)c.max_total_tokens + c.max_seq_len)
+    return fail(h, PRISM_ERR_SHAPE_LIMIT, "token total exceeds max_total_tokens");
+  if (lq > 0) PRISM_CUDA(h, cudaMemcpyAsync(h->h_tokens, query, (size_t)lq * sizeof(int), cudaMemcpyDeviceToHost, st));
+  if (n_cand > 0)
+    PRISM_CUDA(h, cudaMemcpyAsync(h->h_tokens + lq, cand, (size_t)n_cand * sizeof(int), cudaMemcpyDeviceToHost, st));
+  PRISM_CUDA(h, cudaStreamSynchronize(st));
+  const uint64_t now = ++h->request_no;
+  std::vector<int> missing;
+  int64_t distinct = 0;
+  for (int i = 0; i < lq + n_cand; ++i) {
+    const int t = h->h_tokens[i];
+    if (t < 0 || t >= c.vocab || h->tok_seen[t] == now) continue;
+    h->tok_seen[t] = now;
+    ++distinct;
+    const int s = h->slot_of_tok[t];
+    if (s >= 0) h->slot_stamp[s] = now;
+    else missing.push_back(t);
+  }
+  if (distinct > h->cache_rows) {
+    // undo the stamps of this request so that the cache state is as before
+    for (int i = 0; i < lq + n_cand; ++i) {
+      const int t = h->h_tokens[i];
+      if (t >= 0 && t < c.vocab) h->tok_seen[t] = 0;
+    }
+    return fail(h, PRISM_ERR_SHAPE_LIMIT, "the request has more distinct tokens than the embedding cache has rows");
+  }
+  h->cache_hits += distinct - (int64_t)missing.size();
+  h->cache_misses += (int64_t)missing.size();
+  if (missing.empty()) return PRISM_OK;
+  // rows this request does not use, least recently used first (never-used rows have stamp 0)
+  std::vector<int> victims;
+  victims.reserve((size_t)h->cache_rows);
+  for (int s = 0; s < h->cache_rows; ++s)
+    if (h->slot_stamp[s] != now) victims.push_back(s);
+  const size_t need = missing.size();
+  std::partial_sort(victims.begin(), victims.begin() + (std::ptrdiff_t)need, victims.end(), [&](int a, int b) {
+    return h->slot_stamp[a] != h->slot_stamp[b] ? h->slot_stamp[a] < h->slot_stamp[b] : a < b;
+  });
+  for (size_t i = 0; i < need; ++i) {
+    const int t = missing[i], s = victims[i];
+    if (h->tok_of_slot[s] >= 0) {
+      h->slot_of_tok[h->tok_of_slot[s]] = -1;
+      ++h->cache_evictions;
+    }
+    h->tok_of_slot[s] = t;
+    h->slot_of_tok[t] = s;
+    h->slot_stamp[s] = now;
+    h->h_pairs[2 * i] = t;
+    h->h_pairs[2 * i + 1] = s;
+  }
+  PRISM_CUDA(h, cudaMemcpyAsync(h->pairs_dev, h->h_pairs, 2 * need * sizeof(int), cudaMemcpyHostToDevice, st));
+  PRISM_LAUNCH(h, launch_cache_fill(h->embed, h->cache_dev, h->pairs_dev, (int)need, c.hidden * (int)h->esz, h->tok2slot_dev, st));
+  // the pinned pair list is reused by the next request: this one's copy must have left it
+  PRISM_CUDA(h, cudaStreamSynchronize(st));
+  return PRISM_OK;
+}
+
 // Candidate-sharded runs (Shard non-null): this rank packs only the candidates it owns (the others are sequences
 // of length zero), probes write 0 for them, and before every prune decision `reduce` sums the score vector over
 // the ranks, after which every rank evaluates the same rule on the same numbers.
@@ -637,6 +743,8 @@ int select_impl(prism_handle* h, const int32_t* query, int32_t lq, const int32_t
   PRISM_CUDA(h, cudaMemcpyAsync(h->state, h->h_state, sizeof(RouteState), cudaMemcpyHostToDevice, st));
   PRISM_CUDA(h, cudaMemsetAsync(h->errword, 0, sizeof(int), st));
 
+  if (h->cache_rows > 0 && (rc = cache_prepare(h, query, lq, cand, h->h_off[N], st)) != PRISM_OK) return rc;
+
   int cur = 0;  // ping-pong index of x / cu / seq2orig
   const unsigned char* owned_dev = nullptr;
   if (shard) {
@@ -648,7 +756,8 @@ int select_impl(prism_handle* h, const int32_t* query, int32_t lq, const int32_t
   PRISM_LAUNCH_P(h, st, PRISM_K_PACK, 12.0 * total,
                  launch_pack_tokens(query, lq, cand, off, h->cu[cur], N, (int)total, c.vocab, h->tokens, h->pos, h->errword, st));
   PRISM_LAUNCH_P(h, st, PRISM_K_EMBED, (double)total * c.hidden * (4.0 + h->esz),
-                 launch_embed(h->embed, c.dtype, h->tokens, (int)total, c.hidden, h->x[cur], st));
+                 launch_embed(h->cache_rows > 0 ? h->cache_dev : h->embed, c.dtype, h->tokens, (int)total, c.hidden, h->x[cur], st,
+                              h->cache_rows > 0 ? h->tok2slot_dev : nullptr));
 
   if (streamed) {
     // The previous request drained both streams before returning, so both slots are free.
