@@ -97,6 +97,12 @@ typedef struct {
                       (one device-to-host copy of the token ids) and brings the missing rows into the cache
                       before the layers start.  A request with more distinct tokens than rows fails with
                       PRISM_ERR_SHAPE_LIMIT.  The paper sizes the cache at 10 % of the vocabulary. */
+  int32_t hidden_offload;   /* 1: dynamic offloading of the hidden states (Sec. 4.3): the hidden states of all
+                      sequences live in pinned host memory (allocated by the library) and at most three chunks
+                      are on the device at a time: the one being computed, the one being written back and the
+                      one being fetched.  Needs activation_budget_bytes > 0, which then has to hold three
+                      chunks of hidden states plus one chunk's intermediates.  Embedding, probe and compaction
+                      work on the host copy directly.  0: hidden states stay on the device. */
 } prism_model_cfg;
 
 typedef struct {

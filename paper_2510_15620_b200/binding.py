@@ -54,7 +54,7 @@ class _ModelCfg(C.Structure):
                 ("rms_eps", C.c_float), ("causal", C.c_int32), ("qk_norm", C.c_int32), ("dtype", C.c_int32),
                 ("max_seq_len", C.c_int32), ("max_candidates", C.c_int32), ("max_total_tokens", C.c_int32),
                 ("activation_budget_bytes", C.c_int64), ("weight_residency", C.c_int32), ("gemm_impl", C.c_int32),
-                ("attention_impl", C.c_int32), ("embed_cache_rows", C.c_int32)]
+                ("attention_impl", C.c_int32), ("embed_cache_rows", C.c_int32), ("hidden_offload", C.c_int32)]
 
 
 class _LayerWeights(C.Structure):
@@ -177,14 +177,14 @@ class PrismModel:
 
     def __init__(self, cfg, weights: Dict[str, object], max_seq_len: int, max_candidates: int, max_total_tokens: int,
                  activation_budget_bytes: int = 0, stream_weights: bool = False, gemm_impl: int = PRISM_IMPL_AUTO,
-                 attention_impl: int = PRISM_IMPL_AUTO, embed_cache_rows: int = 0):
+                 attention_impl: int = PRISM_IMPL_AUTO, embed_cache_rows: int = 0, hidden_offload: bool = False):
         self._h = C.c_void_p()
         self.cfg = cfg
         self._weights = weights            # keep the tensors alive for the life of the handle
         c = _ModelCfg(cfg.n_layers, cfg.hidden, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.ffn, cfg.vocab,
                       cfg.rope_theta, cfg.rms_eps, cfg.causal, cfg.qk_norm, cfg.dtype, max_seq_len, max_candidates,
                       max_total_tokens, activation_budget_bytes, 1 if stream_weights else 0, gemm_impl, attention_impl,
-                      embed_cache_rows)
+                      embed_cache_rows, 1 if hidden_offload else 0)
         layers = (_LayerWeights * cfg.n_layers)()
         for i, lw in enumerate(weights["layers"]):
             for k, _ in _LayerWeights._fields_:

@@ -59,6 +59,16 @@ struct prism_handle {
   int* trace_ids = nullptr;
   unsigned char* owned_dev = nullptr;  // candidate-sharded runs: which candidates this rank runs
 
+  // Dynamic offloading of the hidden states (Sec. 4.3): x[0], x[1] are pinned host memory, the layers run on one
+  // of three device chunk buffers; chunk c is fetched on in_stream, computed on the request's stream and written
+  // back on out_stream.
+  bool offload = false;
+  float* xc[3] = {nullptr, nullptr, nullptr};
+  cudaStream_t in_stream = nullptr, out_stream = nullptr;
+  cudaEvent_t ev_in[3] = {nullptr, nullptr, nullptr}, ev_done[3] = {nullptr, nullptr, nullptr},
+              ev_slot_out[3] = {nullptr, nullptr, nullptr}, ev_main = nullptr;
+  std::vector<cudaEvent_t> ev_chunk_out;  // per chunk index: its last write-back
+
   // Embedding table caching (Sec. 4.4): `embed` is the pinned host table, the device holds cache_rows rows.
   int cache_rows = 0;
   unsigned char* cache_dev = nullptr;  // [cache_rows, D] in the table's element type
@@ -270,6 +280,8 @@ int validate_cfg(const prism_model_cfg& c, std::string* why) {
     return bad("unknown weight_residency");
   if (!(c.rope_theta > 0.f) || !(c.rms_eps >= 0.f)) return bad("rope_theta must be > 0 and rms_eps >= 0");
   if (c.embed_cache_rows < 0) return bad("negative embed_cache_rows");
+  if (c.hidden_offload != 0 && c.hidden_offload != 1) return bad("hidden_offload must be 0 or 1");
+  if (c.hidden_offload && c.activation_budget_bytes <= 0) return bad("hidden_offload needs an activation budget");
   auto unsup = [&](const char* m) { *why = m; return PRISM_ERR_UNSUPPORTED; };
   if (c.head_dim % 2 || c.head_dim > 256) return unsup("head_dim must be even and <= 256");
   if (c.hidden % 4 || c.hidden > 8192) return unsup("hidden must be a multiple of 4 and <= 8192");
@@ -337,6 +349,15 @@ void prism_destroy(prism_handle* h) {
     if (h->ev_freed[s]) cudaEventDestroy(h->ev_freed[s]);
   }
   if (h->copy_stream) cudaStreamDestroy(h->copy_stream);
+  if (h->in_stream) cudaStreamDestroy(h->in_stream);
+  if (h->out_stream) cudaStreamDestroy(h->out_stream);
+  for (int i = 0; i < 3; ++i) {
+    if (h->ev_in[i]) cudaEventDestroy(h->ev_in[i]);
+    if (h->ev_done[i]) cudaEventDestroy(h->ev_done[i]);
+    if (h->ev_slot_out[i]) cudaEventDestroy(h->ev_slot_out[i]);
+  }
+  if (h->ev_main) cudaEventDestroy(h->ev_main);
+  for (cudaEvent_t e : h->ev_chunk_out) cudaEventDestroy(e);
   for (auto& p : h->prof_pending) { cudaEventDestroy(p.a); cudaEventDestroy(p.b); }
   for (cudaEvent_t e : h->prof_pool) cudaEventDestroy(e);
   delete h;
@@ -374,7 +395,14 @@ static int create_impl(prism_handle* h, const prism_model_cfg* cfg, const prism_
   const size_t hidden_bytes = 2 * T * D * sizeof(float);
   const size_t ptb = per_token_bytes(c, h->esz);
   size_t chunk = T;
-  if (c.activation_budget_bytes > 0) {
+  h->offload = c.hidden_offload != 0;
+  if (h->offload) {
+    // three chunks of hidden states and one chunk of intermediates on the device
+    const size_t per_row = 3 * D * sizeof(float) + ptb;
+    chunk = std::min(T, (size_t)c.activation_budget_bytes / per_row);
+    if (chunk < (size_t)c.max_seq_len)
+      return fail(h, PRISM_ERR_BUDGET, "activation budget cannot hold three chunks of one max_seq_len sequence");
+  } else if (c.activation_budget_bytes > 0) {
     const size_t budget = (size_t)c.activation_budget_bytes;
     if (budget <= hidden_bytes || (budget - hidden_bytes) / ptb < (size_t)c.max_seq_len)
       return fail(h, PRISM_ERR_BUDGET, "activation budget cannot hold the hidden states plus one max_seq_len sequence");
@@ -382,8 +410,22 @@ static int create_impl(prism_handle* h, const prism_model_cfg* cfg, const prism_
   }
   h->chunk_tokens = (int)chunk;
 
-  PRISM_CUDA(h, dev_alloc(h, &h->x[0], T * D));
-  PRISM_CUDA(h, dev_alloc(h, &h->x[1], T * D));
+  if (h->offload) {
+    PRISM_CUDA(h, host_alloc(h, &h->x[0], T * D));
+    PRISM_CUDA(h, host_alloc(h, &h->x[1], T * D));
+    for (int i = 0; i < 3; ++i) {
+      PRISM_CUDA(h, dev_alloc(h, &h->xc[i], chunk * D));
+      PRISM_CUDA(h, cudaEventCreateWithFlags(&h->ev_in[i], cudaEventDisableTiming));
+      PRISM_CUDA(h, cudaEventCreateWithFlags(&h->ev_done[i], cudaEventDisableTiming));
+      PRISM_CUDA(h, cudaEventCreateWithFlags(&h->ev_slot_out[i], cudaEventDisableTiming));
+    }
+    PRISM_CUDA(h, cudaEventCreateWithFlags(&h->ev_main, cudaEventDisableTiming));
+    PRISM_CUDA(h, cudaStreamCreateWithFlags(&h->in_stream, cudaStreamNonBlocking));
+    PRISM_CUDA(h, cudaStreamCreateWithFlags(&h->out_stream, cudaStreamNonBlocking));
+  } else {
+    PRISM_CUDA(h, dev_alloc(h, &h->x[0], T * D));
+    PRISM_CUDA(h, dev_alloc(h, &h->x[1], T * D));
+  }
   PRISM_CUDA(h, dev_alloc(h, &h->tokens, T));
   PRISM_CUDA(h, dev_alloc(h, &h->pos, T));
   for (int i = 0; i < 2; ++i) {
@@ -548,12 +590,13 @@ cudaError_t gemm_tc_any(prism_handle* h, const TmaDesc& a, const TmaDesc& b0, co
 }
 
 // One decoder block over rows [r0, r0+rows) (sequences [s0, s1)) of the live batch.
+// x is the whole batch's hidden-state matrix, or (x_is_chunk) the buffer holding just this chunk's rows.
 int run_layer_chunk(prism_handle* h, const LayerDev& W, const LayerMaps* maps, float* x, const int* cu_dev, int s0, int s1,
-                    int r0, int rows, int max_len, cudaStream_t st) {
+                    int r0, int rows, int max_len, cudaStream_t st, bool x_is_chunk = false) {
   const prism_model_cfg& c = h->cfg;
   const int D = c.hidden, dh = c.head_dim;
   const int nqkv = (c.n_q_heads + 2 * c.n_kv_heads) * dh, hd = c.n_q_heads * dh;
-  float* xr = x + (size_t)r0 * D;
+  float* xr = x_is_chunk ? x : x + (size_t)r0 * D;
   const double esz = h->esz, R = rows;
   const double norm_bytes = R * D * (4.0 + esz);
   double attn_flops = 0.0;
@@ -767,6 +810,15 @@ int select_impl(prism_handle* h, const int32_t* query, int32_t lq, const int32_t
 
   int n = N, T = (int)total, n_rec = 0, probe_j = 0, layers_run = 0, chunks_max = 0;
   bool done = false;
+  // hidden-state offload bookkeeping
+  bool main_dirty = true, slot_used[3] = {false, false, false};
+  int chunk_out_valid = 0;  // chunk indices below this have a write-back event from the previous layer
+  int last_out = -1;        // chunk index of the latest write-back enqueued on out_stream
+  if (h->offload) {
+    // a failed request may have left copies in flight
+    PRISM_CUDA(h, cudaStreamSynchronize(h->in_stream));
+    PRISM_CUDA(h, cudaStreamSynchronize(h->out_stream));
+  }
   for (int l = 0; l < c.n_layers && !done; ++l) {
     const int s = l & 1;
     LayerDev W = streamed ? layer_in_slot(h, s) : layer_resident(h, l);
@@ -781,10 +833,46 @@ int select_impl(prism_handle* h, const int32_t* query, int32_t lq, const int32_t
         ++s1;
       }
       const int r0 = h->h_cu[s0], rows = h->h_cu[s1] - r0;
-      if ((rc = run_layer_chunk(h, W, maps, h->x[cur], h->cu[cur], s0, s1, r0, rows, max_len, st)) != PRISM_OK) return rc;
+      if (!h->offload) {
+        if ((rc = run_layer_chunk(h, W, maps, h->x[cur], h->cu[cur], s0, s1, r0, rows, max_len, st)) != PRISM_OK) return rc;
+      } else if (rows > 0) {
+        // Chunk `chunks` goes through device buffer chunks % 3: fetched on in_stream once the buffer's previous
+        // occupant has been written back and this chunk's rows on the host are final (its own write-back of the
+        // previous layer, or the request stream's embedding / compaction), computed here, written back on
+        // out_stream.  The host enqueues chunk after chunk, so the fetch of chunk c + 1 and the write-back of
+        // chunk c - 1 run under the computation of chunk c: at most three chunks are on the device.
+        const int slot = chunks % 3;
+        const size_t bytes = (size_t)rows * c.hidden * sizeof(float);
+        float* hx = h->x[cur] + (size_t)r0 * c.hidden;
+        while ((size_t)chunks >= h->ev_chunk_out.size()) {
+          cudaEvent_t e = nullptr;
+          PRISM_CUDA(h, cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+          h->ev_chunk_out.push_back(e);
+        }
+        if (main_dirty) {  // the request stream wrote the host copy (embedding, compaction) since the last fetch
+          PRISM_CUDA(h, cudaEventRecord(h->ev_main, st));
+          main_dirty = false;
+          chunk_out_valid = 0;
+        }
+        PRISM_CUDA(h, cudaStreamWaitEvent(h->in_stream, h->ev_main, 0));
+        if (slot_used[slot]) PRISM_CUDA(h, cudaStreamWaitEvent(h->in_stream, h->ev_slot_out[slot], 0));
+        if (chunks < chunk_out_valid) PRISM_CUDA(h, cudaStreamWaitEvent(h->in_stream, h->ev_chunk_out[chunks], 0));
+        PRISM_CUDA(h, cudaMemcpyAsync(h->xc[slot], hx, bytes, cudaMemcpyHostToDevice, h->in_stream));
+        PRISM_CUDA(h, cudaEventRecord(h->ev_in[slot], h->in_stream));
+        PRISM_CUDA(h, cudaStreamWaitEvent(st, h->ev_in[slot], 0));
+        if ((rc = run_layer_chunk(h, W, maps, h->xc[slot], h->cu[cur], s0, s1, r0, rows, max_len, st, true)) != PRISM_OK) return rc;
+        PRISM_CUDA(h, cudaEventRecord(h->ev_done[slot], st));
+        PRISM_CUDA(h, cudaStreamWaitEvent(h->out_stream, h->ev_done[slot], 0));
+        PRISM_CUDA(h, cudaMemcpyAsync(hx, h->xc[slot], bytes, cudaMemcpyDeviceToHost, h->out_stream));
+        PRISM_CUDA(h, cudaEventRecord(h->ev_slot_out[slot], h->out_stream));
+        PRISM_CUDA(h, cudaEventRecord(h->ev_chunk_out[chunks], h->out_stream));
+        slot_used[slot] = true;
+        last_out = chunks;
+      }
       s0 = s1;
       ++chunks;
     }
+    if (h->offload) chunk_out_valid = chunks;  // the next layer's chunk c waits for this layer's write-back of chunk c
     chunks_max = std::max(chunks_max, chunks);
     if (trace && trace->tokens_per_layer) trace->tokens_per_layer[l] = T;
     layers_run = l + 1;
@@ -794,6 +882,12 @@ int select_impl(prism_handle* h, const int32_t* query, int32_t lq, const int32_t
 
     const bool is_final = (layers_run == c.n_layers);
     const bool is_probe = probe_j < n_probes && sched->probe_layers[probe_j] == layers_run;
+    if (h->offload && (is_final || is_probe) && last_out >= 0) {
+      // probe and compaction read the host copy on the request's stream: every write-back must have landed
+      // (out_stream is in order, so its latest event covers them all)
+      PRISM_CUDA(h, cudaStreamWaitEvent(st, h->ev_chunk_out[last_out], 0));
+      main_dirty = true;  // whatever the request stream does to the host copy now must precede later fetches
+    }
     if (is_final || is_probe) {
       RouteParams p{};
       p.mode = mode;
