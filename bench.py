@@ -223,7 +223,7 @@ def run_prism(args):
     w_np = synth.make_weights(cfg, wl.weight_seed)
     tw = P.upload_weights(w_np, cfg.dtype, device=str(dev), layers_pinned_host=bool(wl.stream_weights))
     model = P.PrismModel(cfg, tw, max_seq, wl.n_candidates, max_tot, activation_budget_bytes=wl.activation_budget_bytes,
-                         stream_weights=bool(wl.stream_weights))
+                         stream_weights=bool(wl.stream_weights), shared_prefix=args.shared_prefix == "on")
     d = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(dev)
     dreqs = [(d(r["query"]), d(r["cand_tokens"]), d(r["cand_offsets"])) for r in reqs]
     pin = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).pin_memory().numpy()
@@ -266,6 +266,10 @@ def run_prism(args):
         else:
             model.select(q, c, o, wl.top_k, s, want_trace=False)
 
+    prefix_rows = 0  # what the library reports for this workload (one untimed traced request)
+    if not by_cand:
+        prefix_rows = model.select(*dreqs[0], wl.top_k, sched, want_trace=True)[2].shared_prefix_rows
+
     def host_step(i):
         q, c, o = hreqs[i % n_req]
         if by_cand:  # the sharded entry point takes device buffers: the copies are made here, inside the timed region
@@ -302,6 +306,10 @@ def run_prism(args):
             "dtype": "bf16" if cfg.dtype == 1 else "f32", "data": "synthetic",
             "config": {"workload": wl.name, "requests_cycled": n_req, "candidates": wl.n_candidates, "top_k": wl.top_k,
                        "tokens_per_request": int(np.mean([l.sum() for l in lens_all])),
+                       # causal attention: the query's rows are computed once per request instead of once per
+                       # candidate (same scores bit for bit); the metric keeps counting query + document per candidate
+                       "shared_query_prefix_rows": prefix_rows,
+                       "rows_computed_first_layer": int(np.mean([l.sum() - (len(l) - 1) * prefix_rows for l in lens_all])),
                        "schedule": {"mode": sched.mode, "probe_layers": list(sched.probe_layers),
                                     "cv_threshold": sched.cv_threshold, "n_clusters": sched.n_clusters},
                        "l2": "no flush: each step streams 0.9 GB of weights and >1 GB of activations, far beyond the 126 MB L2",
@@ -392,6 +400,9 @@ def main():
     ap.add_argument("--workload", type=int, default=1)
     ap.add_argument("--requests", type=int, default=10, help="distinct request seeds cycled through")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--shared-prefix", default="on", choices=["on", "off"],
+                    help="on: the query's rows are stored and computed once per request where the path supports it "
+                         "(causal attention; results are bit-identical); off: one query copy per candidate")
     ap.add_argument("--shard", default="requests", choices=["requests", "candidates"],
                     help="requests: every rank serves its own requests (weak scaling, the default); candidates: all "
                          "ranks share each request, one score all-reduce per probe (strong scaling)")

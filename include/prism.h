@@ -60,6 +60,9 @@ enum { PRISM_PRUNE_NONE = 0, PRISM_PRUNE_FIXED_KEEP = 1, PRISM_PRUNE_CLUSTER = 2
  * 128x256 tiles. */
 enum { PRISM_IMPL_AUTO = 0, PRISM_IMPL_SIMT = 1, PRISM_IMPL_MMA = 2, PRISM_IMPL_SOLO = 3 };
 
+/* shared_prefix of prism_model_cfg */
+enum { PRISM_PREFIX_AUTO = 0, PRISM_PREFIX_OFF = 1 };
+
 typedef struct prism_handle prism_handle;
 
 /* Model description: a pre-norm decoder block stack (RMSNorm -> GQA attention with optional
@@ -103,6 +106,15 @@ typedef struct {
                       one being fetched.  Needs activation_budget_bytes > 0, which then has to hold three
                       chunks of hidden states plus one chunk's intermediates.  Embedding, probe and compaction
                       work on the host copy directly.  0: hidden states stay on the device. */
+  int32_t shared_prefix;    /* PRISM_PREFIX_AUTO (0): under causal attention the query's rows do not depend on the
+                      document behind them, so the batch stores and computes them ONCE, in front of all documents,
+                      and every sequence attends to those rows followed by its own (Sec. 3.1's batch, minus the
+                      N - 1 repeated copies of the query).  Scores, selections and traces are bit-identical to the
+                      batch with one query copy per sequence; tokens_per_layer and tokens_before keep counting
+                      query_len + document length per sequence.  Taken when: causal, bf16 tensor-core path with an
+                      even Hq / Hkv, 8 <= query_len <= 120 and query_len a multiple of 8, N >= 2, the request
+                      fits one chunk, no hidden_offload, not prism_select_sharded.  Otherwise, or with
+                      PRISM_PREFIX_OFF (1), every sequence carries its own copy of the query. */
 } prism_model_cfg;
 
 typedef struct {
@@ -173,6 +185,8 @@ typedef struct {
   int32_t* tokens_per_layer;   /* out, nullable: [n_layers] live tokens forwarded through each layer */
   int32_t n_chunks_max;        /* out: largest number of chunks used for one layer */
   int64_t workspace_bytes;     /* out: device bytes held by the handle */
+  int32_t shared_prefix_rows;  /* out: query rows stored once for all sequences (0: one copy per sequence) */
+  int32_t reserved;
 } prism_trace;
 
 /* Validate cfg, take the weight pointers, allocate every workspace the handle will ever need

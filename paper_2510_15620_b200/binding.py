@@ -54,7 +54,8 @@ class _ModelCfg(C.Structure):
                 ("rms_eps", C.c_float), ("causal", C.c_int32), ("qk_norm", C.c_int32), ("dtype", C.c_int32),
                 ("max_seq_len", C.c_int32), ("max_candidates", C.c_int32), ("max_total_tokens", C.c_int32),
                 ("activation_budget_bytes", C.c_int64), ("weight_residency", C.c_int32), ("gemm_impl", C.c_int32),
-                ("attention_impl", C.c_int32), ("embed_cache_rows", C.c_int32), ("hidden_offload", C.c_int32)]
+                ("attention_impl", C.c_int32), ("embed_cache_rows", C.c_int32), ("hidden_offload", C.c_int32),
+                ("shared_prefix", C.c_int32)]
 
 
 class _LayerWeights(C.Structure):
@@ -82,7 +83,7 @@ class _Trace(C.Structure):
     _fields_ = [("capacity", C.c_int32), ("n_records", C.c_int32), ("records", C.POINTER(_ProbeRecord)),
                 ("scores", C.POINTER(C.c_float)), ("ids", C.POINTER(C.c_int32)), ("layers_run", C.c_int32),
                 ("tokens_per_layer", C.POINTER(C.c_int32)), ("n_chunks_max", C.c_int32),
-                ("workspace_bytes", C.c_int64)]
+                ("workspace_bytes", C.c_int64), ("shared_prefix_rows", C.c_int32), ("reserved", C.c_int32)]
 
 
 class Calibrator(C.Structure):
@@ -153,6 +154,7 @@ class Trace:
     tokens_per_layer: List[int]
     n_chunks_max: int
     workspace_bytes: int
+    shared_prefix_rows: int = 0
 
 
 def upload_weights(w: Dict[str, object], dtype: int, device: str = "cuda", layers_pinned_host: bool = False,
@@ -177,14 +179,15 @@ class PrismModel:
 
     def __init__(self, cfg, weights: Dict[str, object], max_seq_len: int, max_candidates: int, max_total_tokens: int,
                  activation_budget_bytes: int = 0, stream_weights: bool = False, gemm_impl: int = PRISM_IMPL_AUTO,
-                 attention_impl: int = PRISM_IMPL_AUTO, embed_cache_rows: int = 0, hidden_offload: bool = False):
+                 attention_impl: int = PRISM_IMPL_AUTO, embed_cache_rows: int = 0, hidden_offload: bool = False,
+                 shared_prefix: bool = True):
         self._h = C.c_void_p()
         self.cfg = cfg
         self._weights = weights            # keep the tensors alive for the life of the handle
         c = _ModelCfg(cfg.n_layers, cfg.hidden, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.ffn, cfg.vocab,
                       cfg.rope_theta, cfg.rms_eps, cfg.causal, cfg.qk_norm, cfg.dtype, max_seq_len, max_candidates,
                       max_total_tokens, activation_budget_bytes, 1 if stream_weights else 0, gemm_impl, attention_impl,
-                      embed_cache_rows, 1 if hidden_offload else 0)
+                      embed_cache_rows, 1 if hidden_offload else 0, 0 if shared_prefix else 1)
         layers = (_LayerWeights * cfg.n_layers)()
         for i, lw in enumerate(weights["layers"]):
             for k, _ in _LayerWeights._fields_:
@@ -237,7 +240,7 @@ class PrismModel:
             ids = np.zeros((cap, max(n, 1)), np.int32)
             tpl = (C.c_int32 * self.cfg.n_layers)()
             tr = _Trace(cap, 0, recs, sc.ctypes.data_as(C.POINTER(C.c_float)), ids.ctypes.data_as(C.POINTER(C.c_int32)),
-                        0, tpl, 0, 0)
+                        0, tpl, 0, 0, 0, 0)
         rc = fn(self._h, q_ptr, lq, c_ptr, o_ptr, n, k, C.byref(s) if s is not None else None, idx_ptr, sc_ptr,
                 C.byref(n_out), C.byref(tr) if tr is not None else None, stream)
         if rc != 0:
@@ -251,7 +254,8 @@ class PrismModel:
                 out.append(ProbeRecord(x.layer, na, x.fired, x.n_selected, x.n_dropped, x.n_deferred, x.k_rem_after,
                                        [x.cuts[i] for i in range(x.n_cuts)], x.tokens_before, x.cv,
                                        [int(v) for v in ids[r, :na]], sc[r, :na].copy()))
-            trace = Trace(out, tr.layers_run, [tpl[i] for i in range(tr.layers_run)], tr.n_chunks_max, tr.workspace_bytes)
+            trace = Trace(out, tr.layers_run, [tpl[i] for i in range(tr.layers_run)], tr.n_chunks_max, tr.workspace_bytes,
+                          tr.shared_prefix_rows)
         return int(n_out.value), trace
 
     def select(self, query: torch.Tensor, cand_tokens: torch.Tensor, cand_offsets: torch.Tensor, k: int, sched=None,

@@ -88,13 +88,14 @@ __device__ __forceinline__ void tmem_ld1(uint32_t taddr, uint32_t& v) {
 // shared memory to the other roles, which read the ring in order.
 struct ItemRec {
   int qb, pair, beg, len, n_blocks;  // n_blocks == 0: no more items
+  int first;                         // the launch's first sequence (it stores the rows of a shared prefix)
 };
 constexpr int NI = 4;  // ring depth
 
 struct ItemReader {
   volatile ItemRec* ring;
   uint32_t b_full, b_empty, n;
-  int qb, pair, beg, len, n_blocks;  // the current item
+  int qb, pair, beg, len, n_blocks, first;  // the current item
   __device__ __forceinline__ void init(ItemRec* ring_, uint32_t b_full_, uint32_t b_empty_) {
     ring = ring_, b_full = b_full_, b_empty = b_empty_, n = 0;
     n_blocks = 0;
@@ -105,6 +106,7 @@ struct ItemReader {
     if (!mbar_wait(b_full + 8 * slot, (n / NI) & 1, err, abort_flag)) return false;
     qb = ring[slot].qb, pair = ring[slot].pair, beg = ring[slot].beg, len = ring[slot].len;
     n_blocks = ring[slot].n_blocks;
+    first = ring[slot].first;
     return n_blocks > 0;
   }
   // The caller (one thread per arriving party) is done with the current item's record.
@@ -113,9 +115,11 @@ struct ItemReader {
 };
 
 __global__ void __launch_bounds__(kThreads, 1)
-k_attention_tc2(const __grid_constant__ CUtensorMap map_qkv, __nv_bfloat16* __restrict__ out,
+k_attention_tc2(const __grid_constant__ CUtensorMap map_qkv, const __grid_constant__ CUtensorMap map_pre,
+                const __grid_constant__ CUtensorMap map_rest, __nv_bfloat16* __restrict__ out,
                 const int* __restrict__ cu, int seq0, int nseq, int row0, int nqb, int gsz, int hq, int hkv,
-                int causal, int reverse, float scale_log2, int* __restrict__ sched, int* __restrict__ err) {
+                int causal, int reverse, int prefix, float scale_log2, int* __restrict__ sched,
+                int* __restrict__ err) {
   extern __shared__ unsigned char smem_raw[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t raw = smem_u32(smem_raw);
@@ -182,10 +186,13 @@ k_attention_tc2(const __grid_constant__ CUtensorMap map_qkv, __nv_bfloat16* __re
           const int s = seq0 + sl;
           it.qb = nqb - 1 - in_group / per_qb;
           it.pair = rem % npairs;
+          // Shared query prefix: rows 0 .. prefix-1 of the batch belong to every sequence, cu[s] is the first row
+          // of the sequence's own part.  Row v of the sequence is batch row v (v < prefix) or beg + v - prefix.
           const int b = __ldg(cu + s);
-          it.len = __ldg(cu + s + 1) - b;
+          it.len = prefix + __ldg(cu + s + 1) - b;
           if (it.qb * BM >= it.len) continue;
           it.beg = b - row0;
+          it.first = sl == 0;
           const int kv_end = causal ? min(it.len, (it.qb + 1) * BM) : it.len;
           it.n_blocks = (kv_end + BN - 1) / BN;
           break;
@@ -198,22 +205,32 @@ k_attention_tc2(const __grid_constant__ CUtensorMap map_qkv, __nv_bfloat16* __re
         if (it.n_blocks == 0) break;
         const int h0 = it.pair * 2, kvh = h0 / group;
         const int kcol = (hq + kvh) * DH, vcol = (hq + hkv + kvh) * DH;
-        const int qrow0 = it.beg + it.qb * BM;
+        // 128 rows of the sequence starting at row 128 * blk, columns col .. col + 127, as two 64-column
+        // sub-tiles.  The block that holds a shared prefix is put together from two row ranges (prefix rows, then
+        // the sequence's own first 128 - prefix rows; prefix is a multiple of 8, so the second part starts on a
+        // swizzle-atom boundary); the boxes add up to a full tile, so the byte count is the same.
+        auto load_tile = [&](uint32_t dst, int col, int blk, uint32_t bar) {
+          mbar_expect_tx(bar, kTile);
+          if (prefix > 0 && blk == 0) {
+            tma_load_2d(dst, &map_pre, col, 0, bar);
+            tma_load_2d(dst + kTile / 2, &map_pre, col + 64, 0, bar);
+            tma_load_2d(dst + prefix * 128, &map_rest, col, it.beg, bar);
+            tma_load_2d(dst + kTile / 2 + prefix * 128, &map_rest, col + 64, it.beg, bar);
+          } else {
+            const int row = it.beg + blk * 128 - prefix;
+            tma_load_2d(dst, &map_qkv, col, row, bar);
+            tma_load_2d(dst + kTile / 2, &map_qkv, col + 64, row, bar);
+          }
+        };
         auto load_q = [&](int x) {
           if (!mbar_wait(b_q_empty + 8 * x, (ic & 1) ^ 1, err, abort_flag)) return false;
-          const uint32_t dst = s_q + x * kTile;
-          mbar_expect_tx(b_q_full + 8 * x, kTile);
-          tma_load_2d(dst, &map_qkv, (h0 + x) * DH, qrow0, b_q_full + 8 * x);
-          tma_load_2d(dst + kTile / 2, &map_qkv, (h0 + x) * DH + 64, qrow0, b_q_full + 8 * x);
+          load_tile(s_q + x * kTile, (h0 + x) * DH, it.qb, b_q_full + 8 * x);
           return true;
         };
         auto load_kv = [&](int col, int t, uint32_t ring, uint32_t b_full, uint32_t b_empty, uint32_t& cnt, int depth) {
           const uint32_t st = cnt % depth, u = cnt / depth;
           if (!mbar_wait(b_empty + 8 * st, (u & 1) ^ 1, err, abort_flag)) return false;
-          const uint32_t dst = ring + st * kTile;
-          mbar_expect_tx(b_full + 8 * st, kTile);
-          tma_load_2d(dst, &map_qkv, col, it.beg + t * BN, b_full + 8 * st);
-          tma_load_2d(dst + kTile / 2, &map_qkv, col + 64, it.beg + t * BN, b_full + 8 * st);
+          load_tile(ring + st * kTile, col, t, b_full + 8 * st);
           ++cnt;
           return true;
         };
@@ -475,8 +492,7 @@ k_attention_tc2(const __grid_constant__ CUtensorMap map_qkv, __nv_bfloat16* __re
       // This thread's 64 columns of O_x / l as bf16, 32 columns at a time through the warp's staging rows
       // (64 bytes each, 16-byte chunks XOR-swizzled), so that global stores are 64 contiguous bytes per row.
       const int row_w = it.qb * BM + quarter * 32;  // first row of this warp inside the sequence
-      __nv_bfloat16* obase =
-          out + (size_t)(it.beg + row_w) * ((size_t)hq * DH) + (size_t)(it.pair * 2 + x) * DH + hf * 64;
+      __nv_bfloat16* ocol = out + (size_t)(it.pair * 2 + x) * DH + hf * 64;
 #pragma unroll 1
       for (int part = 0; part < 2; ++part) {
         uint32_t o[32];
@@ -500,8 +516,13 @@ k_attention_tc2(const __grid_constant__ CUtensorMap map_qkv, __nv_bfloat16* __re
           asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
                        : "=r"(val.x), "=r"(val.y), "=r"(val.z), "=r"(val.w)
                        : "r"(stg + rr * 64 + ((chn ^ ((rr >> 1) & 3)) << 4)));
-          if (row_w + rr < it.len)
-            *reinterpret_cast<uint4*>(obase + (size_t)rr * ((size_t)hq * DH) + part * 32 + chn * 8) = val;
+          // row v of the sequence: its own row beg + v - prefix, or row v of the shared prefix, which only the
+          // launch's first sequence writes (every sequence computes the same values for it)
+          const int v = row_w + rr;
+          if (v < it.len && (v >= prefix || it.first)) {
+            const size_t prow = v < prefix ? (size_t)v : (size_t)(it.beg + v - prefix);
+            *reinterpret_cast<uint4*>(ocol + prow * ((size_t)hq * DH) + part * 32 + chn * 8) = val;
+          }
         }
         __syncwarp();
       }
@@ -533,16 +554,25 @@ __device__ int g_sched[kTickets][2];
 
 cudaError_t launch_attention_tc2(const void* qkv, void* out, const int* cu, int seq0, int nseq, int row0, int rows,
                                  int max_len, int n_q_heads, int n_kv_heads, int causal, int* err, cudaStream_t st,
-                                 bool reverse) {
+                                 bool reverse, int prefix) {
   if (nseq <= 0 || max_len <= 0 || rows <= 0) return cudaSuccess;
   if (n_kv_heads < 1 || n_q_heads % n_kv_heads || ((n_q_heads / n_kv_heads) & 1)) return cudaErrorInvalidValue;
   static std::atomic<unsigned long long> smem_set{0};
   if (cudaError_t e = ensure_dynamic_smem(k_attention_tc2, kSmemBytes, smem_set)) return e;
   // Exactly `rows` rows are described, so tiles that run past the batch read zeros, never stale memory.
   const uint64_t ld = (uint64_t)(n_q_heads + 2 * n_kv_heads) * DH;
-  TmaDesc mq;
+  TmaDesc mq, mpre, mrest;
   cudaError_t e = make_tma_2d_bf16(&mq, qkv, (uint64_t)rows, ld, 128, 64);
   if (e != cudaSuccess) return e;
+  mpre = mq;
+  mrest = mq;
+  if (prefix) {
+    // shared query prefix: max_len counts prefix + own rows; the first block of every tile is two boxes
+    if (prefix < 8 || prefix > 120 || (prefix & 7) || row0 != 0 || seq0 != 0 || !causal) return cudaErrorInvalidValue;
+    e = make_tma_2d_bf16(&mpre, qkv, (uint64_t)rows, ld, (uint32_t)prefix, 64);
+    if (e == cudaSuccess) e = make_tma_2d_bf16(&mrest, qkv, (uint64_t)rows, ld, (uint32_t)(128 - prefix), 64);
+    if (e != cudaSuccess) return e;
+  }
   const int nqb = (max_len + BM - 1) / BM;
   // sequences per scheduling group: their q/k/v rows (at most max_len each) stay within 48 MB
   const long long seq_bytes = (long long)nqb * BM * (long long)ld * 2;
@@ -566,9 +596,11 @@ cudaError_t launch_attention_tc2(const void* qkv, void* out, const int* cu, int 
   }
   int* sched = sb + 2 * (ticket.fetch_add(1, std::memory_order_relaxed) % kTickets);
   const float scale_log2 = 1.4426950408889634f / sqrtf((float)DH);
-  k_attention_tc2<<<grid, kThreads, kSmemBytes, st>>>(reinterpret_cast<const CUtensorMap&>(mq), (__nv_bfloat16*)out, cu,
+  k_attention_tc2<<<grid, kThreads, kSmemBytes, st>>>(reinterpret_cast<const CUtensorMap&>(mq),
+                                                      reinterpret_cast<const CUtensorMap&>(mpre),
+                                                      reinterpret_cast<const CUtensorMap&>(mrest), (__nv_bfloat16*)out, cu,
                                                       seq0, nseq, row0, nqb, gsz, n_q_heads, n_kv_heads, causal, reverse ? 1 : 0,
-                                                      scale_log2,
+                                                      prefix, scale_log2,
                                                       sched, err);
   return cudaGetLastError();
 }

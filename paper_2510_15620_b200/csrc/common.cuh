@@ -45,6 +45,7 @@ struct RouteParams {
   int select_winners;
   int is_final;  // 1: last layer, append the best k_rem and stop
   int layer;
+  int prefix;    // shared query prefix: rows in front of the batch that belong to every sequence (0 = none)
 };
 
 // Request state that lives on the device and is mirrored to the host after every scored layer.
@@ -97,11 +98,13 @@ struct alignas(64) TmaDesc {
 // ---- launchers (each returns the CUDA error of the launch; none synchronises) -----------------
 // owned (nullable, device, n bytes): candidates with owned[i] == 0 get length zero (candidate-sharded runs).
 cudaError_t launch_pack_offsets(const int* cand_offsets, int n, int query_len, int* cu, int* seq2orig,
-                                int* err, cudaStream_t st, const unsigned char* owned = nullptr);
+                                int* err, cudaStream_t st, const unsigned char* owned = nullptr, bool shared_prefix = false);
 cudaError_t launch_pack_tokens(const int* query, int query_len, const int* cand_tokens,
                                const int* cand_offsets, const int* cu, int n, int total, int vocab,
-                               int* tokens, int* pos, int* err, cudaStream_t st);
-cudaError_t launch_positions(const int* cu, int n, int total, int* pos, cudaStream_t st);
+                               int* tokens, int* pos, int* err, cudaStream_t st, bool shared_prefix = false);
+// Shared query prefix (prefix = query_len > 0 below): the query's rows are stored once in front of the batch,
+// cu[i] is the first DOCUMENT row of sequence i, and a sequence is the prefix rows followed by its own rows.
+cudaError_t launch_positions(const int* cu, int n, int total, int* pos, cudaStream_t st, int prefix = 0);
 cudaError_t launch_embed(const void* table, int dtype, const int* tokens, int total, int d, float* x,
                          cudaStream_t st, const int* tok2slot = nullptr);
 // Sec. 4.4 embedding table caching: rows of the pinned host table into rows of the device cache.
@@ -117,10 +120,10 @@ cudaError_t launch_qknorm_rope(void* qkv, int dtype, const int* pos, int rows, i
                                const void* g_k, float eps, const float* cos_t, const float* sin_t,
                                cudaStream_t st);
 cudaError_t launch_probe(const float* x, const int* cu, int n, int d, const void* g_final, int dtype,
-                         const float* w_diff, float eps, float* scores, cudaStream_t st);
+                         const float* w_diff, float eps, float* scores, cudaStream_t st, int prefix = 0);
 cudaError_t launch_score_diff(const void* score_head, int dtype, int d, float* w_diff, cudaStream_t st);
 cudaError_t launch_compact_rows(const float* x_old, float* x_new, const int* cu_old, const int* cu_new,
-                                const int* old_of_new, int n_new, int total_new, int d, cudaStream_t st);
+                                const int* old_of_new, int n_new, int total_new, int d, cudaStream_t st, int prefix = 0);
 
 cudaError_t launch_gemm_simt(const void* a, const void* b, const void* b2, void* out, float* resid, int m,
                              int n, int k, int dtype, int epilogue, cudaStream_t st);
@@ -148,7 +151,7 @@ cudaError_t launch_attention_tc(const void* qkv, void* out, const int* cu, int s
                                 int max_len, int n_q_heads, int n_kv_heads, int causal, int* err, cudaStream_t st);
 // Two query heads of a key/value group per CTA, persistent (needs an even group size n_q_heads / n_kv_heads).
 cudaError_t launch_attention_tc2(const void* qkv, void* out, const int* cu, int seq0, int nseq, int row0, int rows,
-                                int max_len, int n_q_heads, int n_kv_heads, int causal, int* err, cudaStream_t st, bool reverse = false);
+                                int max_len, int n_q_heads, int n_kv_heads, int causal, int* err, cudaStream_t st, bool reverse = false, int prefix = 0);
 cudaError_t launch_attention_mma(const void* qkv, void* out, const int* cu, int seq0, int nseq, int row0,
                                  int max_len, int n_q_heads, int n_kv_heads, int causal, cudaStream_t st);
 

@@ -44,9 +44,12 @@ __device__ __forceinline__ int seq_of_row(const int* __restrict__ cu, int n, int
 // S0 pack: cu = exclusive scan of (query_len + doc_len_i), seq2orig = identity.  One block.  With an ownership
 // mask (candidate-sharded runs) the candidates of other ranks become sequences of length zero: they keep their
 // place in every per-sequence array and take no rows.
+// With a shared query prefix (shared = 1) the query's lq rows are stored once, in front of the batch, and
+// sequence i keeps only its document rows: cu[i] = lq + sum of the document lengths before i.
 __global__ void __launch_bounds__(1024) k_pack_offsets(const int* __restrict__ off, int n, int lq,
-                                                       const unsigned char* __restrict__ owned, int* __restrict__ cu,
-                                                       int* __restrict__ seq2orig, int* __restrict__ err) {
+                                                       const unsigned char* __restrict__ owned, int shared,
+                                                       int* __restrict__ cu, int* __restrict__ seq2orig,
+                                                       int* __restrict__ err) {
   __shared__ int warp_tot[32];
   __shared__ int carry;
   if (threadIdx.x == 0) {
@@ -60,7 +63,7 @@ __global__ void __launch_bounds__(1024) k_pack_offsets(const int* __restrict__ o
     if (i < n) {
       int dl = off[i + 1] - off[i];
       if (dl < 0) { atomicOr(err, kErrBadOffsets); dl = 0; }
-      len = (owned && !owned[i]) ? 0 : lq + dl;
+      len = (owned && !owned[i]) ? 0 : (shared ? dl : lq + dl);
       seq2orig[i] = i;
     }
     int v = len;
@@ -82,34 +85,44 @@ __global__ void __launch_bounds__(1024) k_pack_offsets(const int* __restrict__ o
       warp_tot[lane] = t;
     }
     __syncthreads();
-    int excl = carry + (w ? warp_tot[w - 1] : 0) + v - len;
+    int excl = carry + (w ? warp_tot[w - 1] : 0) + v - len + (shared ? lq : 0);
     if (i < n) cu[i] = excl;
     __syncthreads();
     if (threadIdx.x == blockDim.x - 1) carry += warp_tot[31];
     __syncthreads();
   }
-  if (threadIdx.x == 0) cu[n] = carry;
+  if (threadIdx.x == 0) cu[n] = carry + (shared ? lq : 0);
 }
 
 // Packed token ids (query in front of every document) and per-token positions.
 __global__ void k_pack_tokens(const int* __restrict__ query, int lq, const int* __restrict__ cand,
                               const int* __restrict__ off, const int* __restrict__ cu, int n, int total,
-                              int vocab, int* __restrict__ tokens, int* __restrict__ pos,
+                              int vocab, int shared, int* __restrict__ tokens, int* __restrict__ pos,
                               int* __restrict__ err) {
   for (int t = blockIdx.x * blockDim.x + threadIdx.x; t < total; t += gridDim.x * blockDim.x) {
-    int s = seq_of_row(cu, n, t);
-    int p = t - cu[s];
-    int tok = (p < lq) ? query[p] : cand[off[s] + (p - lq)];
+    int tok, p;
+    if (shared && t < lq) {  // the shared query prefix
+      p = t;
+      tok = query[t];
+    } else {
+      int s = seq_of_row(cu, n, t);
+      p = t - cu[s] + (shared ? lq : 0);  // position inside the sequence query || document
+      tok = (p < lq) ? query[p] : cand[off[s] + (p - lq)];
+    }
     if (tok < 0 || tok >= vocab) { atomicOr(err, kErrBadToken); tok = 0; }
     tokens[t] = tok;
     pos[t] = p;
   }
 }
 
-__global__ void k_positions(const int* __restrict__ cu, int n, int total, int* __restrict__ pos) {
+__global__ void k_positions(const int* __restrict__ cu, int n, int total, int prefix, int* __restrict__ pos) {
   for (int t = blockIdx.x * blockDim.x + threadIdx.x; t < total; t += gridDim.x * blockDim.x) {
-    int s = seq_of_row(cu, n, t);
-    pos[t] = t - cu[s];
+    if (t < prefix) {
+      pos[t] = t;
+    } else {
+      int s = seq_of_row(cu, n, t);
+      pos[t] = t - cu[s] + prefix;
+    }
   }
 }
 
@@ -295,14 +308,18 @@ __global__ void __launch_bounds__(256) k_qknorm_rope(T* __restrict__ qkv, const 
 template <typename WT>
 __global__ void __launch_bounds__(256) k_probe(const float* __restrict__ x, const int* __restrict__ cu, int d,
                                                const WT* __restrict__ g_final, const float* __restrict__ w_diff,
-                                               float eps, float* __restrict__ scores) {
+                                               float eps, int prefix, float* __restrict__ scores) {
   __shared__ float red[32];
   const int i = blockIdx.x;
-  if (cu[i + 1] == cu[i]) {  // a sequence without rows (another rank's candidate): its score comes from there
-    if (threadIdx.x == 0) scores[i] = 0.f;
-    return;
+  int last = cu[i + 1] - 1;
+  if (cu[i + 1] == cu[i]) {
+    if (prefix == 0) {  // a sequence without rows (another rank's candidate): its score comes from there
+      if (threadIdx.x == 0) scores[i] = 0.f;
+      return;
+    }
+    last = prefix - 1;  // shared query prefix and an empty document: the sequence ends with the query
   }
-  const float* row = x + (size_t)(cu[i + 1] - 1) * d;
+  const float* row = x + (size_t)last * d;
   float ss = 0.f, dot = 0.f;
   for (int c = threadIdx.x * 4; c < d; c += blockDim.x * 4) {
     float4 v = *reinterpret_cast<const float4*>(row + c);
@@ -328,11 +345,14 @@ __global__ void __launch_bounds__(256) k_compact_rows(const float* __restrict__ 
                                                       const int* __restrict__ cu_old,
                                                       const int* __restrict__ cu_new,
                                                       const int* __restrict__ old_of_new, int n_new,
-                                                      int total_new, int d) {
+                                                      int total_new, int d, int prefix) {
   const int nv = d >> 2;
   for (int t = blockIdx.x; t < total_new; t += gridDim.x) {
-    const int s = seq_of_row(cu_new, n_new, t);
-    const int src = cu_old[old_of_new[s]] + (t - cu_new[s]);
+    int src = t;  // rows of a shared query prefix stay where they are
+    if (t >= prefix) {
+      const int s = seq_of_row(cu_new, n_new, t);
+      src = cu_old[old_of_new[s]] + (t - cu_new[s]);
+    }
     const float4* a = reinterpret_cast<const float4*>(x_old + (size_t)src * d);
     float4* b = reinterpret_cast<float4*>(x_new + (size_t)t * d);
     for (int c = threadIdx.x; c < nv; c += 4 * 256) {
@@ -359,23 +379,23 @@ inline int grid_for(long long work, int block, int cap = 148 * 16) {
 }  // namespace
 
 cudaError_t launch_pack_offsets(const int* cand_offsets, int n, int query_len, int* cu, int* seq2orig,
-                                int* err, cudaStream_t st, const unsigned char* owned) {
-  k_pack_offsets<<<1, 1024, 0, st>>>(cand_offsets, n, query_len, owned, cu, seq2orig, err);
+                                int* err, cudaStream_t st, const unsigned char* owned, bool shared_prefix) {
+  k_pack_offsets<<<1, 1024, 0, st>>>(cand_offsets, n, query_len, owned, shared_prefix ? 1 : 0, cu, seq2orig, err);
   return cudaGetLastError();
 }
 
 cudaError_t launch_pack_tokens(const int* query, int query_len, const int* cand_tokens,
                                const int* cand_offsets, const int* cu, int n, int total, int vocab,
-                               int* tokens, int* pos, int* err, cudaStream_t st) {
+                               int* tokens, int* pos, int* err, cudaStream_t st, bool shared_prefix) {
   if (total <= 0) return cudaSuccess;
   k_pack_tokens<<<grid_for(total, 256), 256, 0, st>>>(query, query_len, cand_tokens, cand_offsets, cu, n,
-                                                      total, vocab, tokens, pos, err);
+                                                      total, vocab, shared_prefix ? 1 : 0, tokens, pos, err);
   return cudaGetLastError();
 }
 
-cudaError_t launch_positions(const int* cu, int n, int total, int* pos, cudaStream_t st) {
+cudaError_t launch_positions(const int* cu, int n, int total, int* pos, cudaStream_t st, int prefix) {
   if (total <= 0) return cudaSuccess;
-  k_positions<<<grid_for(total, 256), 256, 0, st>>>(cu, n, total, pos);
+  k_positions<<<grid_for(total, 256), 256, 0, st>>>(cu, n, total, prefix, pos);
   return cudaGetLastError();
 }
 
@@ -484,12 +504,12 @@ cudaError_t launch_qknorm_rope(void* qkv, int dtype, const int* pos, int rows, i
 }
 
 cudaError_t launch_probe(const float* x, const int* cu, int n, int d, const void* g_final, int dtype,
-                         const float* w_diff, float eps, float* scores, cudaStream_t st) {
+                         const float* w_diff, float eps, float* scores, cudaStream_t st, int prefix) {
   if (n <= 0) return cudaSuccess;
   if (dtype == 1)
-    k_probe<__nv_bfloat16><<<n, 256, 0, st>>>(x, cu, d, (const __nv_bfloat16*)g_final, w_diff, eps, scores);
+    k_probe<__nv_bfloat16><<<n, 256, 0, st>>>(x, cu, d, (const __nv_bfloat16*)g_final, w_diff, eps, prefix, scores);
   else
-    k_probe<float><<<n, 256, 0, st>>>(x, cu, d, (const float*)g_final, w_diff, eps, scores);
+    k_probe<float><<<n, 256, 0, st>>>(x, cu, d, (const float*)g_final, w_diff, eps, prefix, scores);
   return cudaGetLastError();
 }
 
@@ -502,10 +522,10 @@ cudaError_t launch_score_diff(const void* score_head, int dtype, int d, float* w
 }
 
 cudaError_t launch_compact_rows(const float* x_old, float* x_new, const int* cu_old, const int* cu_new,
-                                const int* old_of_new, int n_new, int total_new, int d, cudaStream_t st) {
+                                const int* old_of_new, int n_new, int total_new, int d, cudaStream_t st, int prefix) {
   if (total_new <= 0) return cudaSuccess;
   int grid = total_new < 148 * 8 ? total_new : 148 * 8;
-  k_compact_rows<<<grid, 256, 0, st>>>(x_old, x_new, cu_old, cu_new, old_of_new, n_new, total_new, d);
+  k_compact_rows<<<grid, 256, 0, st>>>(x_old, x_new, cu_old, cu_new, old_of_new, n_new, total_new, d, prefix);
   return cudaGetLastError();
 }
 

@@ -282,6 +282,7 @@ int validate_cfg(const prism_model_cfg& c, std::string* why) {
   if (c.embed_cache_rows < 0) return bad("negative embed_cache_rows");
   if (c.hidden_offload != 0 && c.hidden_offload != 1) return bad("hidden_offload must be 0 or 1");
   if (c.hidden_offload && c.activation_budget_bytes <= 0) return bad("hidden_offload needs an activation budget");
+  if (c.shared_prefix != PRISM_PREFIX_AUTO && c.shared_prefix != PRISM_PREFIX_OFF) return bad("shared_prefix must be 0 or 1");
   auto unsup = [&](const char* m) { *why = m; return PRISM_ERR_UNSUPPORTED; };
   if (c.head_dim % 2 || c.head_dim > 256) return unsup("head_dim must be even and <= 256");
   if (c.hidden % 4 || c.hidden > 8192) return unsup("hidden must be a multiple of 4 and <= 8192");
@@ -591,8 +592,10 @@ cudaError_t gemm_tc_any(prism_handle* h, const TmaDesc& a, const TmaDesc& b0, co
 
 // One decoder block over rows [r0, r0+rows) (sequences [s0, s1)) of the live batch.
 // x is the whole batch's hidden-state matrix, or (x_is_chunk) the buffer holding just this chunk's rows.
+// prefix > 0: rows [0, prefix) are the query shared by all sequences, cu holds the sequences' own rows, max_len
+// counts prefix + own rows (whole batch in one chunk, r0 = 0).
 int run_layer_chunk(prism_handle* h, const LayerDev& W, const LayerMaps* maps, float* x, const int* cu_dev, int s0, int s1,
-                    int r0, int rows, int max_len, cudaStream_t st, bool x_is_chunk = false) {
+                    int r0, int rows, int max_len, cudaStream_t st, bool x_is_chunk = false, int prefix = 0) {
   const prism_model_cfg& c = h->cfg;
   const int D = c.hidden, dh = c.head_dim;
   const int nqkv = (c.n_q_heads + 2 * c.n_kv_heads) * dh, hd = c.n_q_heads * dh;
@@ -601,7 +604,7 @@ int run_layer_chunk(prism_handle* h, const LayerDev& W, const LayerMaps* maps, f
   const double norm_bytes = R * D * (4.0 + esz);
   double attn_flops = 0.0;
   for (int s = s0; s < s1; ++s) {
-    const double L = h->h_cu[s + 1] - h->h_cu[s];
+    const double L = h->h_cu[s + 1] - h->h_cu[s] + prefix;
     attn_flops += (c.causal ? 2.0 : 4.0) * L * L * c.n_q_heads * dh;
   }
   PRISM_LAUNCH_P(h, st, PRISM_K_RMSNORM, norm_bytes, launch_rmsnorm(xr, W.g_attn, c.dtype, rows, D, c.rms_eps, h->a_norm, st, next_dir(h, true)));
@@ -625,7 +628,7 @@ int run_layer_chunk(prism_handle* h, const LayerDev& W, const LayerMaps* maps, f
   if (h->fa == 3)
     PRISM_LAUNCH_P(h, st, PRISM_K_ATTENTION, attn_flops,
                    launch_attention_tc2(h->qkv, h->attn, cu_dev, s0, s1 - s0, r0, rows, max_len, c.n_q_heads, c.n_kv_heads, c.causal,
-                                        h->errword, st, next_dir(h, true)));
+                                        h->errword, st, next_dir(h, true), prefix));
   else if (h->fa == 1)
     PRISM_LAUNCH_P(h, st, PRISM_K_ATTENTION, attn_flops,
                    launch_attention_tc(h->qkv, h->attn, cu_dev, s0, s1 - s0, r0, rows, max_len, c.n_q_heads, c.n_kv_heads, c.causal,
@@ -742,6 +745,7 @@ int select_impl(prism_handle* h, const int32_t* query, int32_t lq, const int32_t
     trace->layers_run = 0;
     trace->n_chunks_max = 0;
     trace->workspace_bytes = h->workspace_bytes;
+    trace->shared_prefix_rows = 0;
   }
   const int k_eff = std::min(K, N);
   std::string why;
@@ -764,6 +768,17 @@ int select_impl(prism_handle* h, const int32_t* query, int32_t lq, const int32_t
   h->h_cu[0] = 0;
   for (int i = 0; i < N; ++i)
     if (h->h_off[i + 1] < h->h_off[i]) return fail(h, PRISM_ERR_BAD_INPUT, "cand_offsets not monotone");
+  // Shared query prefix: under causal attention the query's rows are the same in every sequence, so they are
+  // stored and computed once in front of the documents (rows [0, lq)); cu then holds document rows only.
+  const int prefix = (c.shared_prefix == PRISM_PREFIX_AUTO && h->fa == 3 && c.causal && !h->offload && !shard && N >= 2 &&
+                      lq >= 8 && lq <= 120 && (lq & 7) == 0 && (long long)lq + h->h_off[N] <= h->chunk_tokens)
+                         ? lq
+                         : 0;
+  if (prefix) {
+    total = lq;
+    h->h_cu[0] = lq;
+    if (trace) trace->shared_prefix_rows = prefix;
+  }
   for (int i = 0; i < N; ++i) {
     if (shard && !shard->owned[i]) {  // another rank's candidate: no rows here
       h->h_cu[i + 1] = (int)total;
@@ -773,7 +788,7 @@ int select_impl(prism_handle* h, const int32_t* query, int32_t lq, const int32_t
     if (dl + lq > c.max_seq_len) return fail(h, PRISM_ERR_SHAPE_LIMIT, "a sequence exceeds max_seq_len");
     if (dl + lq > h->chunk_tokens) return fail(h, PRISM_ERR_BUDGET, "a sequence exceeds the chunk the activation budget allows");
     if (dl + lq < 1) return fail(h, PRISM_ERR_INVALID_ARG, "empty sequence (query_len = 0 and an empty document)");
-    total += dl + lq;
+    total += prefix ? dl : dl + lq;
     if (total > c.max_total_tokens) return fail(h, PRISM_ERR_SHAPE_LIMIT, "token total exceeds max_total_tokens");
     h->h_cu[i + 1] = (int)total;
   }
@@ -795,9 +810,10 @@ int select_impl(prism_handle* h, const int32_t* query, int32_t lq, const int32_t
     owned_dev = h->owned_dev;
   }
   PRISM_LAUNCH_P(h, st, PRISM_K_PACK, 8.0 * N,
-                 launch_pack_offsets(off, N, lq, h->cu[cur], h->seq2orig[cur], h->errword, st, owned_dev));
+                 launch_pack_offsets(off, N, lq, h->cu[cur], h->seq2orig[cur], h->errword, st, owned_dev, prefix > 0));
   PRISM_LAUNCH_P(h, st, PRISM_K_PACK, 12.0 * total,
-                 launch_pack_tokens(query, lq, cand, off, h->cu[cur], N, (int)total, c.vocab, h->tokens, h->pos, h->errword, st));
+                 launch_pack_tokens(query, lq, cand, off, h->cu[cur], N, (int)total, c.vocab, h->tokens, h->pos, h->errword, st,
+                                    prefix > 0));
   PRISM_LAUNCH_P(h, st, PRISM_K_EMBED, (double)total * c.hidden * (4.0 + h->esz),
                  launch_embed(h->cache_rows > 0 ? h->cache_dev : h->embed, c.dtype, h->tokens, (int)total, c.hidden, h->x[cur], st,
                               h->cache_rows > 0 ? h->tok2slot_dev : nullptr));
@@ -826,6 +842,14 @@ int select_impl(prism_handle* h, const int32_t* query, int32_t lq, const int32_t
     if (streamed) PRISM_CUDA(h, cudaStreamWaitEvent(st, h->ev_copied[s], 0));
     // chunks on sequence boundaries: the longest prefix of the remaining sequences that fits
     int s0 = 0, chunks = 0;
+    if (prefix) {  // one chunk: the prefix rows and every sequence's own rows
+      int max_len = 0;
+      for (int i = 0; i < n; ++i) max_len = std::max(max_len, h->h_cu[i + 1] - h->h_cu[i]);
+      if ((rc = run_layer_chunk(h, W, maps, h->x[cur], h->cu[cur], 0, n, 0, h->h_cu[n], prefix + max_len, st, false, prefix)) != PRISM_OK)
+        return rc;
+      s0 = n;
+      chunks = 1;
+    }
     while (s0 < n) {
       int s1 = s0 + 1, max_len = h->h_cu[s1] - h->h_cu[s0];
       while (s1 < n && h->h_cu[s1 + 1] - h->h_cu[s0] <= h->chunk_tokens) {
@@ -874,7 +898,7 @@ int select_impl(prism_handle* h, const int32_t* query, int32_t lq, const int32_t
     }
     if (h->offload) chunk_out_valid = chunks;  // the next layer's chunk c waits for this layer's write-back of chunk c
     chunks_max = std::max(chunks_max, chunks);
-    if (trace && trace->tokens_per_layer) trace->tokens_per_layer[l] = T;
+    if (trace && trace->tokens_per_layer) trace->tokens_per_layer[l] = prefix ? T - prefix + n * prefix : T;
     layers_run = l + 1;
     if (streamed) {
       PRISM_CUDA(h, cudaEventRecord(h->ev_freed[s], st));
@@ -898,10 +922,11 @@ int select_impl(prism_handle* h, const int32_t* query, int32_t lq, const int32_t
       p.select_winners = sched ? sched->select_winners : 1;
       p.is_final = is_final ? 1 : 0;
       p.layer = layers_run;
+      p.prefix = prefix;
       const int nxt = cur ^ 1;
       float* score_buf = shard ? shard->exchange : h->scores;
       PRISM_LAUNCH_P(h, st, PRISM_K_PROBE, 4.0 * n * c.hidden,
-                     launch_probe(h->x[cur], h->cu[cur], n, c.hidden, h->g_final, c.dtype, h->w_diff, c.rms_eps, score_buf, st));
+                     launch_probe(h->x[cur], h->cu[cur], n, c.hidden, h->g_final, c.dtype, h->w_diff, c.rms_eps, score_buf, st, prefix));
       if (shard && shard->reduce(shard->ctx, n, st) != 0) return fail(h, PRISM_ERR_CUDA, "the score exchange callback failed");
       PRISM_LAUNCH_P(h, st, PRISM_K_ROUTE, 8.0 * n, launch_route(score_buf, h->cu[cur], h->seq2orig[cur], n, p, h->cu[nxt], h->seq2orig[nxt], h->old_of_new,
                                    h->state, h->res_idx, h->res_score, h->recs + n_rec,
@@ -923,8 +948,8 @@ int select_impl(prism_handle* h, const int32_t* query, int32_t lq, const int32_t
         std::swap(h->h_cu, h->h_cu_next);
         PRISM_LAUNCH_P(h, st, PRISM_K_COMPACT, 8.0 * stt.n_tokens * c.hidden,
                        launch_compact_rows(h->x[cur], h->x[nxt], h->cu[cur], h->cu[nxt], h->old_of_new, stt.n_active,
-                                           stt.n_tokens, c.hidden, st));
-        PRISM_LAUNCH_P(h, st, PRISM_K_PACK, 4.0 * stt.n_tokens, launch_positions(h->cu[nxt], stt.n_active, stt.n_tokens, h->pos, st));
+                                           stt.n_tokens, c.hidden, st, prefix));
+        PRISM_LAUNCH_P(h, st, PRISM_K_PACK, 4.0 * stt.n_tokens, launch_positions(h->cu[nxt], stt.n_active, stt.n_tokens, h->pos, st, prefix));
         cur = nxt;
         n = stt.n_active;
         T = stt.n_tokens;

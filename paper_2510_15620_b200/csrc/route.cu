@@ -69,7 +69,8 @@ __global__ void __launch_bounds__(kThreads) k_route(const float* __restrict__ sc
 
   const int k_rem = state->k_rem;
   const int n_result = state->n_result;
-  const int tokens_before = cu_old[n];
+  // with a shared query prefix the batch holds the prefix rows once: report the sequences' own token count
+  const int tokens_before = p.prefix ? (cu_old[n] - p.prefix) + n * p.prefix : cu_old[n];
 
   for (int i = tid; i < n; i += kThreads) {
     const float raw = scores[i];
@@ -255,7 +256,7 @@ __global__ void __launch_bounds__(kThreads) k_route(const float* __restrict__ sc
   // ---- survivor offsets: stable compaction in batch order ---------------------------------
   int total_new = 0;
   if (!done) {
-    if (tid == 0) { sh.carry_a = 0; sh.carry_b = 0; }
+    if (tid == 0) { sh.carry_a = 0; sh.carry_b = p.prefix; }  // the prefix rows stay in front
     __syncthreads();
     for (int base = 0; base < n; base += kThreads) {
       const int i = base + tid;
