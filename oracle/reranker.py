@@ -146,6 +146,11 @@ def score_matrix(query: np.ndarray, cand_tokens: np.ndarray, cand_offsets: np.nd
     Layer-major over the weights (each layer's weights are materialised once, then applied to
     every requested candidate separately) so that 4B/8B-shaped weights need not be resident
     all at once; the values are those of the candidate-major loop."""
+    if getattr(cfg, "arch", 0) == 1:   # encoder-only stack: same contract, other model definition
+        from .encoder import encoder_score_matrix
+        if act != "exact":
+            raise ValueError("the encoder oracle has no rounded-activation mode")
+        return encoder_score_matrix(query, cand_tokens, cand_offsets, weights, cfg, score_layers, candidates)
     n = len(cand_offsets) - 1
     ids = list(range(n)) if candidates is None else [int(c) for c in candidates]
     want = sorted(set(int(l) for l in score_layers))

@@ -17,6 +17,9 @@ MODE_CLUSTER = 2     # progressive cluster pruning (Sec. 4.1)
 DTYPE_FP32 = 0
 DTYPE_BF16 = 1
 
+ARCH_DECODER = 0     # pre-norm decoder blocks (RMSNorm, rotary embedding, SwiGLU): the Qwen3 rerankers
+ARCH_ENCODER = 1     # post-norm encoder blocks (LayerNorm, learned positions, GELU, biases): the BGE-M3 reranker
+
 
 @dataclass(frozen=True)
 class ModelCfg:
@@ -34,6 +37,11 @@ class ModelCfg:
     dtype: int = DTYPE_BF16
     yes_id: int = 0   # vocab rows the two-row score head is taken from
     no_id: int = 1
+    # ARCH_ENCODER: rms_eps is the LayerNorm epsilon, n_kv_heads = n_q_heads, rope_theta and qk_norm are unused,
+    # positions are learned: token p of a sequence reads row p + pos_offset of a [max_positions, hidden] table
+    arch: int = ARCH_DECODER
+    max_positions: int = 0
+    pos_offset: int = 0
 
     @property
     def qkv_rows(self) -> int:
@@ -42,7 +50,8 @@ class ModelCfg:
     @property
     def params_per_layer(self) -> int:
         d = self.hidden
-        return d * self.qkv_rows + self.n_q_heads * self.head_dim * d + 3 * d * self.ffn
+        ffn_mats = 2 if self.arch == ARCH_ENCODER else 3
+        return d * self.qkv_rows + self.n_q_heads * self.head_dim * d + ffn_mats * d * self.ffn
 
 
 @dataclass(frozen=True)
@@ -79,6 +88,11 @@ _QWEN3_06B = ModelCfg(n_layers=28, hidden=1024, n_q_heads=16, n_kv_heads=8, head
                       ffn=3072, vocab=151669, rope_theta=1e6, yes_id=9693, no_id=2152)
 _QWEN3_4B = replace(_QWEN3_06B, n_layers=36, hidden=2560, n_q_heads=32, ffn=9728)
 _QWEN3_8B = replace(_QWEN3_06B, n_layers=36, hidden=4096, n_q_heads=32, ffn=12288)
+# The encoder-only reranker the paper evaluates next to the Qwen3 family (Table 1): BGE-M3's reranker is an
+# XLM-RoBERTa-large stack (24 post-norm blocks, 16 heads of 64, GELU FFN of 4096, learned positions offset by 2).
+_BGE_M3 = ModelCfg(n_layers=24, hidden=1024, n_q_heads=16, n_kv_heads=16, head_dim=64, ffn=4096, vocab=250002,
+                   rope_theta=1.0, rms_eps=1e-5, causal=0, qk_norm=0, arch=ARCH_ENCODER, max_positions=8194,
+                   pos_offset=2)
 _TINY = ModelCfg(n_layers=2, hidden=256, n_q_heads=4, n_kv_heads=2, head_dim=64, ffn=768,
                  vocab=4096, rope_theta=1e4, qk_norm=0, dtype=DTYPE_FP32, yes_id=7, no_id=11)
 
@@ -98,6 +112,9 @@ WORKLOADS: List[Workload] = [
     Workload("cfg4_stress_0p6b", _QWEN3_06B, 1000, 20, 32, ("lognormal", 256, 0.6, 32, 1024),
              Schedule(MODE_CLUSTER, tuple(range(4, 28, 2)), cv_threshold=0.5),
              dup_fraction=0.3, cfg_index=4),
+    # beyond the five benchmark configurations: the encoder stack on cfg 1's request recipe
+    Workload("cfg5_bge_m3_shaped", _BGE_M3, 100, 10, 32, ("uniform", 128, 512, 128, 512),
+             Schedule(MODE_CLUSTER, (6, 9, 12, 15, 18, 21), cv_threshold=0.5), cfg_index=5),
 ]
 
 

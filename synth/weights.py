@@ -14,7 +14,7 @@ from typing import Dict, Iterator, Tuple
 
 import numpy as np
 
-from .configs import DTYPE_BF16, ModelCfg
+from .configs import ARCH_ENCODER, DTYPE_BF16, ModelCfg
 
 W_STD = 0.02
 GAIN_JITTER = 0.1
@@ -63,6 +63,16 @@ def tensor(seed: int, name: str, shape: Tuple[int, ...], cfg: ModelCfg, gain: bo
 
 def layer_tensor_shapes(cfg: ModelCfg) -> Dict[str, Tuple[Tuple[int, ...], bool]]:
     d, dh = cfg.hidden, cfg.head_dim
+    if cfg.arch == ARCH_ENCODER:
+        # biases and LayerNorm shifts are drawn like matrix entries (non-zero, so that a dropped bias fails parity)
+        return {
+            "w_qkv": ((cfg.qkv_rows, d), False), "b_qkv": ((cfg.qkv_rows,), False),
+            "w_o": ((d, cfg.n_q_heads * dh), False), "b_o": ((d,), False),
+            "ln1_g": ((d,), True), "ln1_b": ((d,), False),
+            "w_ffn1": ((cfg.ffn, d), False), "b_ffn1": ((cfg.ffn,), False),
+            "w_ffn2": ((d, cfg.ffn), False), "b_ffn2": ((d,), False),
+            "ln2_g": ((d,), True), "ln2_b": ((d,), False),
+        }
     out = {
         "g_attn": ((d,), True),
         "w_qkv": ((cfg.qkv_rows, d), False),   # rows: all q heads, then k heads, then v heads
@@ -86,7 +96,16 @@ def make_layer(cfg: ModelCfg, layer: int, seed: int = 0) -> Dict[str, np.ndarray
 def make_globals(cfg: ModelCfg, seed: int = 0, embed_rows: np.ndarray | None = None) -> Dict[str, np.ndarray]:
     """embed [V, D], g_final [D], score_head [2, D] (row 0 = "yes", row 1 = "no").
 
-    The score head is a separate two-row matrix, not tied to the embedding table."""
+    The score head is a separate two-row matrix, not tied to the embedding table.
+    ARCH_ENCODER: embed, pos_embed [max_positions, D], type_embed [D], the embedding LayerNorm, and the
+    classification head: dense [D, D] + bias, tanh, out_proj [D] + bias [1]."""
+    if cfg.arch == ARCH_ENCODER:
+        d = cfg.hidden
+        shapes = {"embed": ((cfg.vocab, d), False), "pos_embed": ((cfg.max_positions, d), False),
+                  "type_embed": ((d,), False), "emb_ln_g": ((d,), True), "emb_ln_b": ((d,), False),
+                  "head_dense_w": ((d, d), False), "head_dense_b": ((d,), False),
+                  "head_out_w": ((d,), False), "head_out_b": ((1,), False)}
+        return {k: tensor(seed, k, shp, cfg, gain) for k, (shp, gain) in shapes.items()}
     out = {
         "embed": tensor(seed, "embed", (cfg.vocab, cfg.hidden), cfg),
         "g_final": tensor(seed, "g_final", (cfg.hidden,), cfg, gain=True),
