@@ -60,6 +60,13 @@ enum { PRISM_PRUNE_NONE = 0, PRISM_PRUNE_FIXED_KEEP = 1, PRISM_PRUNE_CLUSTER = 2
  * 128x256 tiles. */
 enum { PRISM_IMPL_AUTO = 0, PRISM_IMPL_SIMT = 1, PRISM_IMPL_MMA = 2, PRISM_IMPL_SOLO = 3 };
 
+/* arch of prism_model_cfg.  DECODER: the pre-norm blocks described at prism_model_cfg, created by prism_create.
+ * ENCODER: the encoder-only reranker the paper evaluates next to them (BGE-M3's, an XLM-RoBERTa stack; Sec. 6.1,
+ * Table 1), created by prism_create_encoder: token + learned position + token-type embedding, LayerNorm, then
+ * post-norm blocks x = LN1(x + O(attention(QKV x))), x = LN2(x + W2 gelu(W1 x + b1) + b2) with a bias on every
+ * linear map and the exact GELU x Phi(x); the classifier reads the FIRST token. */
+enum { PRISM_ARCH_DECODER = 0, PRISM_ARCH_ENCODER = 1 };
+
 /* shared_prefix of prism_model_cfg */
 enum { PRISM_PREFIX_AUTO = 0, PRISM_PREFIX_OFF = 1 };
 
@@ -115,6 +122,13 @@ typedef struct {
                       even Hq / Hkv, 8 <= query_len <= 120 and query_len a multiple of 8, N >= 2, the request
                       fits one chunk, no hidden_offload, not prism_select_sharded.  Otherwise, or with
                       PRISM_PREFIX_OFF (1), every sequence carries its own copy of the query. */
+  int32_t arch;             /* PRISM_ARCH_*.  For PRISM_ARCH_ENCODER: rms_eps is the LayerNorm epsilon; rope_theta and
+                      qk_norm are ignored (qk_norm must be 0); causal is normally 0; head_dim is 64 or 128 on the
+                      tensor-core path; ffn a multiple of 8; weight_residency must be PRISM_WEIGHTS_DEVICE,
+                      embed_cache_rows 0 and hidden_offload 0 (PRISM_ERR_UNSUPPORTED otherwise); gemm_impl AUTO or
+                      SIMT, attention_impl AUTO, SOLO or SIMT. */
+  int32_t max_positions;    /* encoder: rows of the learned position table; max_seq_len + pos_offset <= max_positions */
+  int32_t pos_offset;       /* encoder: token p of a sequence reads position row p + pos_offset (2 for XLM-RoBERTa) */
 } prism_model_cfg;
 
 typedef struct {
@@ -140,6 +154,37 @@ typedef struct {
   const void* score_head; /* [2, D]: row 0 = "yes" logit row, row 1 = "no"; score = yes - no */
   const prism_layer_weights* layers;
 } prism_weights;
+
+/* Weights of one encoder block.  Matrices have the element type of cfg.dtype and are device pointers, 16-byte
+ * aligned; the vectors (biases, LayerNorm gain and shift) have the same element type and are widened to fp32
+ * copies inside prism_create_encoder. */
+typedef struct {
+  const void* w_qkv;  /* [(Hq+2Hkv)*dh, D]: all q heads, then k heads, then v heads */
+  const void* b_qkv;  /* [(Hq+2Hkv)*dh] */
+  const void* w_o;    /* [D, Hq*dh] */
+  const void* b_o;    /* [D] */
+  const void* ln1_g;  /* [D] LayerNorm after the attention residual */
+  const void* ln1_b;  /* [D] */
+  const void* w_ffn1; /* [F, D] */
+  const void* b_ffn1; /* [F] */
+  const void* w_ffn2; /* [D, F] */
+  const void* b_ffn2; /* [D] */
+  const void* ln2_g;  /* [D] LayerNorm after the FFN residual */
+  const void* ln2_b;  /* [D] */
+} prism_encoder_layer_weights;
+
+typedef struct {
+  const void* embed;        /* [vocab, D] */
+  const void* pos_embed;    /* [max_positions, D] */
+  const void* type_embed;   /* [D]: the token-type-0 row */
+  const void* emb_ln_g;     /* [D] LayerNorm of the embedding sum */
+  const void* emb_ln_b;     /* [D] */
+  const void* head_dense_w; /* [D, D] classifier: dense + tanh ... */
+  const void* head_dense_b; /* [D] */
+  const void* head_out_w;   /* [D] ... then one logit, which is the score */
+  const void* head_out_b;   /* [1] */
+  const prism_encoder_layer_weights* layers; /* host array of n_layers structs, read during creation only */
+} prism_encoder_weights;
 
 /* When and how to prune (Sec. 4.1).  probe_layers[j] counts completed layers (1-based),
  * strictly increasing, each < n_layers; the last layer is always scored and never prunes.
@@ -194,6 +239,12 @@ typedef struct {
  * Errors: INVALID_ARG, UNSUPPORTED, BUDGET (budget below hidden states + one max_seq_len sequence),
  * NOMEM, CUDA.  On error *out = NULL. */
 PRISM_API int prism_create(const prism_model_cfg* cfg, const prism_weights* w, prism_handle** out);
+
+/* The same for the encoder stack (cfg->arch must be PRISM_ARCH_ENCODER).  The handle serves prism_select,
+ * prism_select_host, prism_select_calibrated and prism_select_sharded exactly like a decoder handle: packing,
+ * chunked execution, probe schedule, routing, compaction and the final top-K are shared; the probe after block l
+ * applies the classifier to the first token of block l's output.  Errors as prism_create. */
+PRISM_API int prism_create_encoder(const prism_model_cfg* cfg, const prism_encoder_weights* w, prism_handle** out);
 
 /* Top-K selection for one request (problem statement Sec. 2.1; method Sec. 3.3-4.3).
  *   query_tokens  device int32[query_len]

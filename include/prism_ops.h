@@ -67,12 +67,39 @@ PRISM_API int prism_op_gemm_qkv_rope(const void* a, const void* w_qkv, void* out
 /* Attention over packed sequences: for sequence s (rows cu[s]..cu[s+1]) and query head h (kv head
  * h / (Hq/Hkv)): out = softmax(q k^T / sqrt(head_dim) [+ causal mask]) v.  qkv [total, (Hq+2Hkv)*dh],
  * out [total, Hq*dh].  total = cu[n_seq] rows; max_len >= the longest sequence.  impl: PRISM_IMPL_AUTO =
- * tcgen05 kernel (bf16, head_dim 128; two query heads of a KV group per CTA when Hq/Hkv is even, else one
- * head per CTA; reports an expired bounded wait in err_word bit 4), PRISM_IMPL_SOLO = the one-head tcgen05
+ * tcgen05 kernel (bf16; head_dim 128: two query heads of a KV group per CTA when Hq/Hkv is even, else one
+ * head per CTA; head_dim 64: one head per CTA; reports an expired bounded wait in err_word bit 4), PRISM_IMPL_SOLO = the one-head tcgen05
  * kernel, PRISM_IMPL_MMA = warp-level MMA kernel (bf16, head_dim 128), PRISM_IMPL_SIMT = CUDA cores. */
 PRISM_API int prism_op_attention(const void* qkv, void* out, const int32_t* cu, int32_t n_seq, int32_t total,
                                  int32_t max_len, int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim,
                                  int32_t causal, int32_t dtype, int32_t impl, int32_t* err_word, void* stream);
+
+/* ---- encoder stack (the encoder-only reranker of Sec. 6.1, Table 1; see PRISM_ARCH_ENCODER in prism.h) ---- */
+
+/* Linear map with a bias: C = A[m,k] B[n,k]^T + bias[n] (bias fp32, device, 16-byte aligned).
+ * epilogue 0: out[m,n] = C in element type `dtype`; 1: resid[m,n] += C (fp32); 2: out = gelu(C), gelu(x) = x Phi(x).
+ * impl: PRISM_IMPL_AUTO = the tcgen05 kernel on CTA pairs (bf16; n and k multiples of 8; err_word as for
+ * prism_op_gemm), PRISM_IMPL_SIMT = CUDA cores (fp32 or bf16). */
+PRISM_API int prism_op_gemm_bias(const void* a, const void* b, const float* bias, void* out, float* resid, int32_t m, int32_t n,
+                       int32_t k, int32_t dtype, int32_t epilogue, int32_t impl, int32_t* err_word, void* stream);
+
+/* LayerNorm over rows of d (multiple of 4, <= 8192) fp32 values, IN PLACE: x = (x - mean) / sqrt(var + eps) * gain +
+ * shift (biased variance; gain and shift fp32), and the same values in element type `dtype` to out[rows, d]. */
+PRISM_API int prism_op_layernorm(float* x, const float* gain, const float* shift, int32_t dtype, int32_t rows, int32_t d, float eps,
+                       void* out, void* stream);
+
+/* Encoder input embedding: x[t,:] = table[tokens[t],:] + pos_table[pos[t] + pos_offset,:] + type_row (fp32 sum;
+ * tables of element type `dtype`, type_row fp32).  The embedding LayerNorm is a separate prism_op_layernorm. */
+PRISM_API int prism_op_embed_encoder(const void* table, const void* pos_table, const float* type_row, int32_t dtype,
+                           const int32_t* tokens, const int32_t* pos, int32_t pos_offset, int32_t total, int32_t d, float* x,
+                           void* stream);
+
+/* Encoder score probe: for each sequence, LayerNorm (gain, shift, eps) of its FIRST row, then
+ * out_w . tanh(dense_w y + dense_b) + out_b[0].  dense_w [d, d] in element type `dtype`, all vectors fp32.
+ * A sequence without rows scores 0. */
+PRISM_API int prism_op_probe_encoder(const float* x, const int32_t* cu, int32_t n, int32_t d, const float* gain, const float* shift,
+                           float eps, const void* dense_w, int32_t dtype, const float* dense_b, const float* out_w,
+                           const float* out_b, float* scores, void* stream);
 
 /* Score probe (Sec. 4.1: the model's classifier on an intermediate hidden state): for each sequence,
  * final RMSNorm of its last row, then logit(score_head row 0) - logit(score_head row 1).

@@ -11,6 +11,7 @@ import torch
 
 PRISM_FP32, PRISM_BF16 = 0, 1
 PRISM_IMPL_AUTO, PRISM_IMPL_SIMT, PRISM_IMPL_MMA, PRISM_IMPL_SOLO = 0, 1, 2, 3
+PRISM_ARCH_DECODER, PRISM_ARCH_ENCODER = 0, 1
 PRISM_MAX_CLUSTERS = 8
 
 # PRISM_LIBRARY overrides the in-tree library (e.g. an instrumented build of the same sources).
@@ -55,7 +56,8 @@ class _ModelCfg(C.Structure):
                 ("max_seq_len", C.c_int32), ("max_candidates", C.c_int32), ("max_total_tokens", C.c_int32),
                 ("activation_budget_bytes", C.c_int64), ("weight_residency", C.c_int32), ("gemm_impl", C.c_int32),
                 ("attention_impl", C.c_int32), ("embed_cache_rows", C.c_int32), ("hidden_offload", C.c_int32),
-                ("shared_prefix", C.c_int32)]
+                ("shared_prefix", C.c_int32), ("arch", C.c_int32), ("max_positions", C.c_int32),
+                ("pos_offset", C.c_int32)]
 
 
 class _LayerWeights(C.Structure):
@@ -65,6 +67,19 @@ class _LayerWeights(C.Structure):
 class _Weights(C.Structure):
     _fields_ = [("embed", C.c_void_p), ("g_final", C.c_void_p), ("score_head", C.c_void_p),
                 ("layers", C.POINTER(_LayerWeights))]
+
+
+_ENC_LAYER_KEYS = ("w_qkv", "b_qkv", "w_o", "b_o", "ln1_g", "ln1_b", "w_ffn1", "b_ffn1", "w_ffn2", "b_ffn2", "ln2_g", "ln2_b")
+_ENC_GLOBAL_KEYS = ("embed", "pos_embed", "type_embed", "emb_ln_g", "emb_ln_b", "head_dense_w", "head_dense_b",
+                    "head_out_w", "head_out_b")
+
+
+class _EncLayerWeights(C.Structure):
+    _fields_ = [(k, C.c_void_p) for k in _ENC_LAYER_KEYS]
+
+
+class _EncWeights(C.Structure):
+    _fields_ = [(k, C.c_void_p) for k in _ENC_GLOBAL_KEYS] + [("layers", C.POINTER(_EncLayerWeights))]
 
 
 class _Schedule(C.Structure):
@@ -110,6 +125,8 @@ def lib() -> C.CDLL:
         L.prism_launch_count.argtypes = [C.c_void_p]
         L.prism_create.restype = C.c_int
         L.prism_create.argtypes = [C.POINTER(_ModelCfg), C.POINTER(_Weights), C.POINTER(C.c_void_p)]
+        L.prism_create_encoder.restype = C.c_int
+        L.prism_create_encoder.argtypes = [C.POINTER(_ModelCfg), C.POINTER(_EncWeights), C.POINTER(C.c_void_p)]
         L.prism_embed_cache_stats.restype = C.c_int
         L.prism_embed_cache_stats.argtypes = [C.c_void_p, C.POINTER(C.c_int64), C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
         L.prism_destroy.restype = None
@@ -169,7 +186,7 @@ def upload_weights(w: Dict[str, object], dtype: int, device: str = "cuda", layer
         if pinned:
             return t.pin_memory()
         return t.to(device)
-    out: Dict[str, object] = {k: conv(w[k], embed_pinned_host and k == "embed") for k in ("embed", "g_final", "score_head")}
+    out: Dict[str, object] = {k: conv(v, embed_pinned_host and k == "embed") for k, v in w.items() if k != "layers"}
     out["layers"] = [{k: conv(v, layers_pinned_host) for k, v in lw.items()} for lw in w["layers"]]
     return out
 
@@ -187,7 +204,19 @@ class PrismModel:
         c = _ModelCfg(cfg.n_layers, cfg.hidden, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.ffn, cfg.vocab,
                       cfg.rope_theta, cfg.rms_eps, cfg.causal, cfg.qk_norm, cfg.dtype, max_seq_len, max_candidates,
                       max_total_tokens, activation_budget_bytes, 1 if stream_weights else 0, gemm_impl, attention_impl,
-                      embed_cache_rows, 1 if hidden_offload else 0, 0 if shared_prefix else 1)
+                      embed_cache_rows, 1 if hidden_offload else 0, 0 if shared_prefix else 1,
+                      getattr(cfg, "arch", 0), getattr(cfg, "max_positions", 0), getattr(cfg, "pos_offset", 0))
+        if getattr(cfg, "arch", 0) == PRISM_ARCH_ENCODER:
+            elayers = (_EncLayerWeights * cfg.n_layers)()
+            for i, lw in enumerate(weights["layers"]):
+                for k in _ENC_LAYER_KEYS:
+                    setattr(elayers[i], k, lw[k].data_ptr())
+            ew = _EncWeights(*[weights[k].data_ptr() for k in _ENC_GLOBAL_KEYS], elayers)
+            rc = lib().prism_create_encoder(C.byref(c), C.byref(ew), C.byref(self._h))
+            if rc != 0:
+                raise PrismError(rc, "prism_create_encoder")
+            self.max_candidates = max_candidates
+            return
         layers = (_LayerWeights * cfg.n_layers)()
         for i, lw in enumerate(weights["layers"]):
             for k, _ in _LayerWeights._fields_:

@@ -1,5 +1,5 @@
 // S5 on the 5th-generation tensor cores: varlen flash attention over packed sequences, bf16,
-// head_dim 128, GQA, causal or bidirectional.  One query head per CTA: this kernel serves odd group sizes
+// head_dim 128 (the decoder rerankers) or 64 (the encoder stack), GQA, causal or bidirectional.  One query head per CTA: this kernel serves odd group sizes
 // Hq/Hkv and PRISM_IMPL_SOLO; even group sizes take the two-heads-per-CTA kernel of attention_tc2.cu.
 //
 // One CTA = 128 query rows of one (sequence, head); two CTAs fit on an SM.  Warp-specialised:
@@ -27,29 +27,32 @@ namespace {
 
 using namespace tc;
 
-constexpr int BM = 128, BN = 64, DH = 128;
-constexpr int kQBytes = BM * DH * 2;          // 32 KB: two [128 x 64] swizzled sub-tiles
-constexpr int kKBytes = BN * DH * 2;          // 16 KB: two [64 x 64] sub-tiles
-constexpr int kVBytes = BN * DH * 2;          // 16 KB: two [64 keys x 64 dh] sub-tiles
+constexpr int BM = 128, BN = 64;
 constexpr int NK = 3, NV = 2;                 // ring depths
 constexpr int kXchBytes = 2 * 128 * 2;        // per-row exchange of the block maximum (bf16) between the two threads of a row
-constexpr int kTileBytes = kQBytes + NK * kKBytes + NV * kVBytes;  // 112 KB
+// Tiles for head_dim DH (sizes for DH = 128; half of it for 64): Q 32 KB as DH/64 [128 x 64] swizzled sub-tiles,
+// K and V 16 KB each as DH/64 [64 x 64] sub-tiles; 112 KB in all.
 // No alignment slack: two CTAs per SM only fit if nothing is wasted.  The kernel checks that its
 // shared window starts on a 1024-byte boundary (the swizzled tiles need it) and reports if not.
-constexpr int kSmemBytes = kTileBytes + 256 + kXchBytes;
-static_assert(2 * (kSmemBytes + 1024) <= 233472, "two CTAs per SM must fit in 228 KB of shared memory");
+__host__ __device__ constexpr int tile_bytes_of(int dh) { return BM * dh * 2 + NK * BN * dh * 2 + NV * BN * dh * 2; }
+__host__ __device__ constexpr int smem_bytes_of(int dh) { return tile_bytes_of(dh) + 256 + kXchBytes; }
+static_assert(2 * (smem_bytes_of(128) + 1024) <= 233472, "two CTAs per SM must fit in 228 KB of shared memory");
 constexpr int kThreads = 352;                 // TMA warp, score-MMA warp, 8 softmax warps, output-MMA warp
-constexpr int kTmemCols = 256;                // S: 2 x 64, O: 128
+constexpr int kTmemCols = 256;                // S: 2 x 64, O: up to 128
 
 __device__ __forceinline__ float ex2(float x) {  // 2^x on the special-function unit; -inf -> 0
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+template <int DH>
 __global__ void __launch_bounds__(kThreads, 2)
 k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_kv,
                __nv_bfloat16* __restrict__ out, const int* __restrict__ cu, int seq0, int row0, int hq, int hkv,
                int causal, float scale_log2, int* __restrict__ err) {
+  constexpr int NS = DH / 64;  // 64-column sub-tiles per head
+  constexpr int kQBytes = BM * DH * 2, kKBytes = BN * DH * 2, kVBytes = BN * DH * 2;
+  constexpr int kTileBytes = tile_bytes_of(DH);
   extern __shared__ unsigned char smem_raw[];
   const int s = seq0 + blockIdx.z;
   const int beg = cu[s] - row0, len = cu[s + 1] - cu[s];
@@ -110,8 +113,8 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
       mbar_expect_tx(b_q, kQBytes);
-      tma_load_2d(s_q, &map_q, h * DH, beg + qb * BM, b_q);
-      tma_load_2d(s_q + kQBytes / 2, &map_q, h * DH + 64, beg + qb * BM, b_q);
+#pragma unroll
+      for (int x = 0; x < NS; ++x) tma_load_2d(s_q + x * (kQBytes / NS), &map_q, h * DH + 64 * x, beg + qb * BM, b_q);
       const int kcol = (hq + kvh) * DH, vcol = (hq + hkv + kvh) * DH;
       // K runs one block ahead of V: step t issues K_t, then V_{t-1}.
       for (int t = 0; t <= n_blocks; ++t) {
@@ -120,16 +123,18 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           if (!mbar_wait(b_k_empty + 8 * st, (u & 1) ^ 1, err, abort_flag)) break;
           const uint32_t sk = s_k + st * kKBytes;
           mbar_expect_tx(b_k_full + 8 * st, kKBytes);
-          tma_load_2d(sk, &map_kv, kcol, beg + t * BN, b_k_full + 8 * st);
-          tma_load_2d(sk + kKBytes / 2, &map_kv, kcol + 64, beg + t * BN, b_k_full + 8 * st);
+#pragma unroll
+          for (int x = 0; x < NS; ++x)
+            tma_load_2d(sk + x * (kKBytes / NS), &map_kv, kcol + 64 * x, beg + t * BN, b_k_full + 8 * st);
         }
         if (t >= 1) {
           const int j = t - 1, st = j & 1, u = j >> 1;
           if (!mbar_wait(b_v_empty + 8 * st, (u & 1) ^ 1, err, abort_flag)) break;
           const uint32_t sv = s_v + st * kVBytes;
           mbar_expect_tx(b_v_full + 8 * st, kVBytes);
-          tma_load_2d(sv, &map_kv, vcol, beg + j * BN, b_v_full + 8 * st);
-          tma_load_2d(sv + kVBytes / 2, &map_kv, vcol + 64, beg + j * BN, b_v_full + 8 * st);
+#pragma unroll
+          for (int x = 0; x < NS; ++x)
+            tma_load_2d(sv + x * (kVBytes / NS), &map_kv, vcol + 64 * x, beg + j * BN, b_v_full + 8 * st);
         }
       }
     }
@@ -146,9 +151,9 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         const uint32_t sk = s_k + st * kKBytes;
         tc_fence_after();
 #pragma unroll
-        for (int kk = 0; kk < 8; ++kk) {  // 16 head-dim elements per step; sub-tile switches at kk = 4
-          const uint64_t da = smem_desc(s_q + (kk >> 2) * (kQBytes / 2) + (kk & 3) * 32, 16, 1024);
-          const uint64_t db = smem_desc(sk + (kk >> 2) * (kKBytes / 2) + (kk & 3) * 32, 16, 1024);
+        for (int kk = 0; kk < DH / 16; ++kk) {  // 16 head-dim elements per step; sub-tile switches at kk = 4
+          const uint64_t da = smem_desc(s_q + (kk >> 2) * (kQBytes / NS) + (kk & 3) * 32, 16, 1024);
+          const uint64_t db = smem_desc(sk + (kk >> 2) * (kKBytes / NS) + (kk & 3) * 32, 16, 1024);
           umma_bf16(t_s + b * BN, da, db, kIdescS, kk != 0);
         }
         umma_commit(b_s_full + 8 * b);
@@ -166,7 +171,7 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         const uint32_t sv = s_v + (j & 1) * kVBytes;
 #pragma unroll
         for (int kk = 0; kk < 4; ++kk) {  // 16 keys per step: 8 packed columns of P, 16 rows of V
-          const uint64_t db = smem_desc(sv + kk * 2048, kVBytes / 2, 1024);    // V: MN-major, two 64-wide dh atoms
+          const uint64_t db = smem_desc(sv + kk * 2048, kVBytes / NS, 1024);   // V: MN-major, DH/64 atoms of 64 dh
           umma_bf16_ts(t_o, t_s + (j & 1) * BN + kk * 8, db, kIdescO, (j | kk) != 0);
         }
         umma_commit(b_o_full);
@@ -177,7 +182,7 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   } else {
     // ------------------------------------------------------------------ softmax + output (128 rows x 2 column halves)
     const int quarter = warp & 3;
-    const int colhalf = (warp - 2) >> 2;           // which 32 of a block's 64 keys / which 64 of the 128 output columns
+    const int colhalf = (warp - 2) >> 2;           // which 32 of a block's 64 keys / which half of the DH output columns
     const int r = quarter * 32 + lane;             // row inside the tile = TMEM lane
     const int qrow = qb * BM + r;                  // row inside the sequence
     const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
@@ -223,13 +228,13 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           const float m_new = need ? bm : m_ref;
           const float f = exp2f((m_ref - m_new) * scale_log2);
 #pragma unroll 1
-          for (int c = 0; c < 2; ++c) {
+          for (int c = 0; c < NS; ++c) {
             uint32_t o[32];
-            tmem_ld32(t_o + lane_base + colhalf * 64 + c * 32, o);
+            tmem_ld32(t_o + lane_base + colhalf * (DH / 2) + c * 32, o);
             tmem_ld_wait();
 #pragma unroll
             for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * f);
-            tmem_st32(t_o + lane_base + colhalf * 64 + c * 32, o);
+            tmem_st32(t_o + lane_base + colhalf * (DH / 2) + c * 32, o);
           }
           tmem_st_wait();
           l *= f;
@@ -273,11 +278,11 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       xch_l[colhalf * 128 + r] = l;  // the row's sum is the sum of the two partial sums
       asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
       const float inv = 1.f / (l + xch_l[(colhalf ^ 1) * 128 + r]);
-      __nv_bfloat16* orow = out + (size_t)(beg + qrow) * ((size_t)hq * DH) + (size_t)h * DH + colhalf * 64;
+      __nv_bfloat16* orow = out + (size_t)(beg + qrow) * ((size_t)hq * DH) + (size_t)h * DH + colhalf * (DH / 2);
 #pragma unroll 1
-      for (int c = 0; c < 2; ++c) {
+      for (int c = 0; c < NS; ++c) {
         uint32_t o[32];
-        tmem_ld32(t_o + lane_base + colhalf * 64 + c * 32, o);
+        tmem_ld32(t_o + lane_base + colhalf * (DH / 2) + c * 32, o);
         tmem_ld_wait();
         if (qrow < len) {
 #pragma unroll
@@ -305,10 +310,15 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 }  // namespace
 
 cudaError_t launch_attention_tc(const void* qkv, void* out, const int* cu, int seq0, int nseq, int row0, int rows,
-                                int max_len, int n_q_heads, int n_kv_heads, int causal, int* err, cudaStream_t st) {
+                                int max_len, int n_q_heads, int n_kv_heads, int causal, int* err, cudaStream_t st,
+                                int head_dim) {
   if (nseq <= 0 || max_len <= 0 || rows <= 0) return cudaSuccess;
-  static std::atomic<unsigned long long> smem_set{0};
-  if (cudaError_t e = ensure_dynamic_smem(k_attention_tc, kSmemBytes, smem_set)) return e;
+  if (head_dim != 128 && head_dim != 64) return cudaErrorInvalidValue;
+  const int DH = head_dim;
+  static std::atomic<unsigned long long> smem_set[2];
+  if (cudaError_t e = DH == 128 ? ensure_dynamic_smem(k_attention_tc<128>, smem_bytes_of(128), smem_set[0])
+                                : ensure_dynamic_smem(k_attention_tc<64>, smem_bytes_of(64), smem_set[1]))
+    return e;
   // Exactly `rows` rows are described, so tiles that run past the batch read zeros, never stale memory.
   const uint64_t ld = (uint64_t)(n_q_heads + 2 * n_kv_heads) * DH;
   TmaDesc mq, mkv;
@@ -317,9 +327,14 @@ cudaError_t launch_attention_tc(const void* qkv, void* out, const int* cu, int s
   if (e != cudaSuccess) return e;
   dim3 grid((max_len + BM - 1) / BM, n_q_heads, nseq);
   const float scale_log2 = 1.4426950408889634f / sqrtf((float)DH);
-  k_attention_tc<<<grid, kThreads, kSmemBytes, st>>>(reinterpret_cast<const CUtensorMap&>(mq),
-                                                     reinterpret_cast<const CUtensorMap&>(mkv), (__nv_bfloat16*)out, cu,
-                                                     seq0, row0, n_q_heads, n_kv_heads, causal, scale_log2, err);
+  if (DH == 128)
+    k_attention_tc<128><<<grid, kThreads, smem_bytes_of(128), st>>>(
+        reinterpret_cast<const CUtensorMap&>(mq), reinterpret_cast<const CUtensorMap&>(mkv), (__nv_bfloat16*)out, cu, seq0,
+        row0, n_q_heads, n_kv_heads, causal, scale_log2, err);
+  else
+    k_attention_tc<64><<<grid, kThreads, smem_bytes_of(64), st>>>(
+        reinterpret_cast<const CUtensorMap&>(mq), reinterpret_cast<const CUtensorMap&>(mkv), (__nv_bfloat16*)out, cu, seq0,
+        row0, n_q_heads, n_kv_heads, causal, scale_log2, err);
   return cudaGetLastError();
 }
 

@@ -24,6 +24,10 @@ enum Epilogue : int {
   kEpiResidual = 1,  // x[M,N] += acc, x fp32 residual stream        (O-proj, down-proj)
   kEpiSwiGLU = 2,    // out[M,N] = silu(acc_gate) * acc_up           (gate/up projection)
   kEpiQkvRope = 3,   // QKV projection with QK-norm + rotary embedding applied to the q and k heads
+  // encoder stack: every linear map has a bias (fp32 vector of n entries)
+  kEpiStoreBias = 4,     // out[M,N] = acc + bias                        (QKV projection)
+  kEpiGeluBias = 5,      // out[M,N] = gelu(acc + bias), gelu(x) = x Phi(x)   (first FFN map)
+  kEpiResidualBias = 6,  // x[M,N] += acc + bias                         (O-proj, second FFN map)
 };
 
 // Inputs of the fused QK-norm + RoPE epilogue (head_dim 128; rotary table rows of 64 floats).
@@ -121,12 +125,29 @@ cudaError_t launch_qknorm_rope(void* qkv, int dtype, const int* pos, int rows, i
                                cudaStream_t st);
 cudaError_t launch_probe(const float* x, const int* cu, int n, int d, const void* g_final, int dtype,
                          const float* w_diff, float eps, float* scores, cudaStream_t st, int prefix = 0);
+// ---- encoder stack (post-norm blocks with LayerNorm, learned positions, first-token classification head) ----
+// x[t,:] = table[tokens[t],:] + pos_table[pos[t] + pos_offset,:] + type_row (fp32 sum; the embedding LayerNorm is
+// the first norm of the first block)
+cudaError_t launch_embed_encoder(const void* table, const void* pos_table, const float* type_row, int dtype,
+                                 const int* tokens, const int* pos, int pos_offset, int total, int d, float* x,
+                                 cudaStream_t st);
+// In place: x[r,:] = (x[r,:] - mean) / sqrt(var + eps) * gain + shift (fp32), and the same values in element type
+// `dtype` to out (the next GEMM's input).
+cudaError_t launch_layernorm(float* x, const float* gain, const float* shift, int dtype, int rows, int d, float eps,
+                             void* out, cudaStream_t st, bool reverse = false);
+// Score of sequence i from its FIRST row: LayerNorm (gain, shift) of the row, then
+// out_w . tanh(dense_w y + dense_b) + out_b.  dense_w [d, d] has element type `dtype`, the vectors are fp32.
+cudaError_t launch_probe_encoder(const float* x, const int* cu, int n, int d, const float* gain, const float* shift,
+                                 float eps, const void* dense_w, int dtype, const float* dense_b, const float* out_w,
+                                 const float* out_b, float* scores, cudaStream_t st);
+// n values of element type `dtype` widened to fp32
+cudaError_t launch_to_f32(const void* src, int dtype, int n, float* dst, cudaStream_t st);
 cudaError_t launch_score_diff(const void* score_head, int dtype, int d, float* w_diff, cudaStream_t st);
 cudaError_t launch_compact_rows(const float* x_old, float* x_new, const int* cu_old, const int* cu_new,
                                 const int* old_of_new, int n_new, int total_new, int d, cudaStream_t st, int prefix = 0);
 
 cudaError_t launch_gemm_simt(const void* a, const void* b, const void* b2, void* out, float* resid, int m,
-                             int n, int k, int dtype, int epilogue, cudaStream_t st);
+                             int n, int k, int dtype, int epilogue, cudaStream_t st, const float* bias = nullptr);
 cudaError_t launch_attention_simt(const void* qkv, void* out, const int* cu, int seq0, int nseq, int row0,
                                   int max_len, int n_q_heads, int n_kv_heads, int head_dim, int causal,
                                   int dtype, cudaStream_t st);
@@ -146,9 +167,12 @@ cudaError_t launch_gemm_tc(const TmaDesc& a, const TmaDesc& b0, const TmaDesc& b
                            int n, int k, int epilogue, const QkvRopeArgs* qa, int* err, cudaStream_t st);
 // The same GEMM on CTA pairs (tcgen05 cta_group::2, 256x256 tiles per cluster of two CTAs).
 cudaError_t launch_gemm_tc2(const TmaDesc& a, const TmaDesc& b0, const TmaDesc& b1, void* out, float* resid, int m,
-                            int n, int k, int epilogue, const QkvRopeArgs* qa, int* err, cudaStream_t st, bool reverse = false);
+                            int n, int k, int epilogue, const QkvRopeArgs* qa, int* err, cudaStream_t st, bool reverse = false,
+                            const float* bias = nullptr);
+// head_dim 128 or 64
 cudaError_t launch_attention_tc(const void* qkv, void* out, const int* cu, int seq0, int nseq, int row0, int rows,
-                                int max_len, int n_q_heads, int n_kv_heads, int causal, int* err, cudaStream_t st);
+                                int max_len, int n_q_heads, int n_kv_heads, int causal, int* err, cudaStream_t st,
+                                int head_dim = 128);
 // Two query heads of a key/value group per CTA, persistent (needs an even group size n_q_heads / n_kv_heads).
 cudaError_t launch_attention_tc2(const void* qkv, void* out, const int* cu, int seq0, int nseq, int row0, int rows,
                                 int max_len, int n_q_heads, int n_kv_heads, int causal, int* err, cudaStream_t st, bool reverse = false, int prefix = 0);

@@ -235,6 +235,143 @@ __global__ void __launch_bounds__(256) k_rmsnorm_warp(const float* __restrict__ 
   }
 }
 
+
+// ------------------------------------------------------------------------------------------------
+// Encoder stack (post-norm blocks; Sec. 6.1 evaluates an encoder-only reranker next to the decoders).
+// Input embedding: token row + learned position row (position p reads row p + pos_offset) + the token-type row,
+// summed in fp32.  The LayerNorm that follows is the first norm of the first block.  One block per token row.
+template <typename WT>
+__global__ void __launch_bounds__(128) k_embed_encoder(const WT* __restrict__ table, const WT* __restrict__ pos_table,
+                                                       const float* __restrict__ type_row, const int* __restrict__ tokens,
+                                                       const int* __restrict__ pos, int pos_offset, int d,
+                                                       float* __restrict__ x) {
+  const int t = blockIdx.x;
+  const WT* a = table + (size_t)tokens[t] * d;
+  const WT* b = pos_table + (size_t)(pos[t] + pos_offset) * d;
+  float* dst = x + (size_t)t * d;
+  for (int c = threadIdx.x * 4; c < d; c += blockDim.x * 4) {
+    const float4 ty = *reinterpret_cast<const float4*>(type_row + c);
+    float4 o;
+    if constexpr (sizeof(WT) == 2) {
+      const uint2 ra = *reinterpret_cast<const uint2*>(a + c), rb = *reinterpret_cast<const uint2*>(b + c);
+      const __nv_bfloat16* pa = reinterpret_cast<const __nv_bfloat16*>(&ra);
+      const __nv_bfloat16* pb = reinterpret_cast<const __nv_bfloat16*>(&rb);
+      o = make_float4(to_f(pa[0]) + to_f(pb[0]) + ty.x, to_f(pa[1]) + to_f(pb[1]) + ty.y,
+                      to_f(pa[2]) + to_f(pb[2]) + ty.z, to_f(pa[3]) + to_f(pb[3]) + ty.w);
+    } else {
+      const float4 fa = *reinterpret_cast<const float4*>(a + c), fb = *reinterpret_cast<const float4*>(b + c);
+      o = make_float4(fa.x + fb.x + ty.x, fa.y + fb.y + ty.y, fa.z + fb.z + ty.z, fa.w + fb.w + ty.w);
+    }
+    *reinterpret_cast<float4*>(dst + c) = o;
+  }
+}
+
+// LayerNorm in place on the fp32 residual stream, plus a copy in the GEMM input type:
+// y = (x - mean) / sqrt(var + eps) * g + b, biased variance, two passes over the row held in registers.
+// kWarp: one warp per row (8 rows per block, lanes keep kPer float4), else one block of 256 threads per row.
+template <typename OT, int kPer, bool kWarp>
+__global__ void __launch_bounds__(256) k_layernorm(float* __restrict__ x, const float* __restrict__ gain,
+                                                   const float* __restrict__ shift, int rows, int d, float eps,
+                                                   OT* __restrict__ out, int reverse) {
+  __shared__ float red[32];
+  const int lane = kWarp ? (threadIdx.x & 31) : threadIdx.x;
+  constexpr int kStride = kWarp ? 32 : 256;
+  const long long blk = reverse ? (long long)gridDim.x - 1 - blockIdx.x : blockIdx.x;
+  const long long row = kWarp ? blk * 8 + (threadIdx.x >> 5) : blk;
+  if (kWarp && row >= rows) return;
+  float4* xr = reinterpret_cast<float4*>(x + (size_t)row * d);
+  const int nv = d >> 2;
+  float4 v[kPer];
+  float sum = 0.f;
+#pragma unroll
+  for (int i = 0; i < kPer; ++i) {
+    const int c = lane + i * kStride;
+    if (c < nv) v[i] = xr[c];
+  }
+#pragma unroll
+  for (int i = 0; i < kPer; ++i) {
+    const int c = lane + i * kStride;
+    if (c < nv) sum += (v[i].x + v[i].y) + (v[i].z + v[i].w);
+  }
+  sum = kWarp ? warp_sum(sum) : block_sum(sum, red);
+  const float mean = sum / (float)d;
+  float sq = 0.f;
+#pragma unroll
+  for (int i = 0; i < kPer; ++i) {
+    const int c = lane + i * kStride;
+    if (c < nv) {
+      v[i].x -= mean; v[i].y -= mean; v[i].z -= mean; v[i].w -= mean;
+      sq += v[i].x * v[i].x + v[i].y * v[i].y + v[i].z * v[i].z + v[i].w * v[i].w;
+    }
+  }
+  sq = kWarp ? warp_sum(sq) : block_sum(sq, red);
+  const float r = 1.0f / sqrtf(sq / (float)d + eps);
+  OT* orow = out + (size_t)row * d;
+#pragma unroll
+  for (int i = 0; i < kPer; ++i) {
+    const int c = lane + i * kStride;
+    if (c < nv) {
+      const float4 g = *reinterpret_cast<const float4*>(gain + 4 * c), b = *reinterpret_cast<const float4*>(shift + 4 * c);
+      const float4 o = make_float4(v[i].x * r * g.x + b.x, v[i].y * r * g.y + b.y, v[i].z * r * g.z + b.z,
+                                   v[i].w * r * g.w + b.w);
+      xr[c] = o;
+      if constexpr (sizeof(OT) == 2) {
+        __nv_bfloat162 lo = __floats2bfloat162_rn(o.x, o.y), hi = __floats2bfloat162_rn(o.z, o.w);
+        *reinterpret_cast<uint2*>(orow + 4 * c) = make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
+      } else {
+        *reinterpret_cast<float4*>(orow + 4 * c) = o;
+      }
+    }
+  }
+}
+
+// Score probe of the encoder stack (Sec. 4.1: the model's own classifier on an intermediate hidden state): the
+// FIRST row of sequence i goes through the pending LayerNorm of the block it leaves, then
+// score = out_w . tanh(dense_w y + dense_b) + out_b.  One block per sequence; the normed row sits in shared
+// memory, every warp takes output units w, w + 8, ... with the lanes striding the row (coalesced weight reads).
+template <typename WT>
+__global__ void __launch_bounds__(256) k_probe_encoder(const float* __restrict__ x, const int* __restrict__ cu, int d,
+                                                       const float* __restrict__ gain, const float* __restrict__ shift,
+                                                       float eps, const WT* __restrict__ dense_w,
+                                                       const float* __restrict__ dense_b, const float* __restrict__ out_w,
+                                                       const float* __restrict__ out_b, float* __restrict__ scores) {
+  extern __shared__ float y[];  // [d]
+  __shared__ float red[32];
+  const int i = blockIdx.x;
+  if (cu[i + 1] == cu[i]) {  // a sequence without rows (another rank's candidate)
+    if (threadIdx.x == 0) scores[i] = 0.f;
+    return;
+  }
+  const float* row = x + (size_t)cu[i] * d;
+  float sum = 0.f;
+  for (int c = threadIdx.x; c < d; c += 256) sum += row[c];
+  const float mean = block_sum(sum, red) / (float)d;
+  float sq = 0.f;
+  for (int c = threadIdx.x; c < d; c += 256) {
+    const float t = row[c] - mean;
+    sq += t * t;
+  }
+  const float r = 1.0f / sqrtf(block_sum(sq, red) / (float)d + eps);
+  for (int c = threadIdx.x; c < d; c += 256) y[c] = (row[c] - mean) * r * gain[c] + shift[c];
+  __syncthreads();
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  float acc = 0.f;  // lane 0 of each warp: sum over its units of out_w[j] * tanh(...)
+  for (int j = w; j < d; j += 8) {
+    const WT* wr = dense_w + (size_t)j * d;
+    float dot = 0.f;
+    for (int c = lane; c < d; c += 32) dot = fmaf(to_f(wr[c]), y[c], dot);
+    dot = warp_sum(dot);
+    if (lane == 0) acc += out_w[j] * tanhf(dot + dense_b[j]);
+  }
+  const float total = block_sum(lane == 0 ? acc : 0.f, red);
+  if (threadIdx.x == 0) scores[i] = total + out_b[0];
+}
+
+template <typename WT>
+__global__ void k_to_f32(const WT* __restrict__ src, int n, float* __restrict__ dst) {
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) dst[i] = to_f(src[i]);
+}
+
 // ------------------------------------------------------------------------------------------------
 // Rotary table in fp64, stored fp32: cos/sin(pos * theta^(-2j/dh)), j < dh/2.
 __global__ void k_rope_table(float* __restrict__ cos_t, float* __restrict__ sin_t, int max_pos, int half,
@@ -466,6 +603,74 @@ cudaError_t launch_rmsnorm(const float* x, const void* gain, int dtype, int rows
     else PRISM_NORM(float, 8);
   }
 #undef PRISM_NORM
+  return cudaGetLastError();
+}
+
+
+cudaError_t launch_embed_encoder(const void* table, const void* pos_table, const float* type_row, int dtype,
+                                 const int* tokens, const int* pos, int pos_offset, int total, int d, float* x,
+                                 cudaStream_t st) {
+  if (total <= 0) return cudaSuccess;
+  if (d % 4) return cudaErrorInvalidValue;
+  if (dtype == 1)
+    k_embed_encoder<__nv_bfloat16><<<total, 128, 0, st>>>((const __nv_bfloat16*)table, (const __nv_bfloat16*)pos_table,
+                                                          type_row, tokens, pos, pos_offset, d, x);
+  else
+    k_embed_encoder<float><<<total, 128, 0, st>>>((const float*)table, (const float*)pos_table, type_row, tokens, pos,
+                                                  pos_offset, d, x);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_layernorm(float* x, const float* gain, const float* shift, int dtype, int rows, int d, float eps,
+                             void* out, cudaStream_t st, bool reverse) {
+  if (rows <= 0) return cudaSuccess;
+  const int nv = d >> 2;
+  if ((d & 3) || nv > 8 * 256) return cudaErrorInvalidValue;
+  const int rev = reverse ? 1 : 0;
+#define PRISM_LN(OT, P, W, G) k_layernorm<OT, P, W><<<(G), 256, 0, st>>>(x, gain, shift, rows, d, eps, (OT*)out, rev)
+  if (nv <= 16 * 32) {  // rows of up to 8 KB: one warp per row
+    const unsigned grid = (unsigned)((rows + 7) / 8);
+    if (dtype == 1) {
+      if (nv <= 128) PRISM_LN(__nv_bfloat16, 4, true, grid);
+      else if (nv <= 256) PRISM_LN(__nv_bfloat16, 8, true, grid);
+      else PRISM_LN(__nv_bfloat16, 16, true, grid);
+    } else {
+      if (nv <= 128) PRISM_LN(float, 4, true, grid);
+      else if (nv <= 256) PRISM_LN(float, 8, true, grid);
+      else PRISM_LN(float, 16, true, grid);
+    }
+  } else {
+    if (dtype == 1) {
+      if (nv <= 1024) PRISM_LN(__nv_bfloat16, 4, false, rows);
+      else PRISM_LN(__nv_bfloat16, 8, false, rows);
+    } else {
+      if (nv <= 1024) PRISM_LN(float, 4, false, rows);
+      else PRISM_LN(float, 8, false, rows);
+    }
+  }
+#undef PRISM_LN
+  return cudaGetLastError();
+}
+
+cudaError_t launch_probe_encoder(const float* x, const int* cu, int n, int d, const float* gain, const float* shift,
+                                 float eps, const void* dense_w, int dtype, const float* dense_b, const float* out_w,
+                                 const float* out_b, float* scores, cudaStream_t st) {
+  if (n <= 0) return cudaSuccess;
+  const size_t smem = (size_t)d * sizeof(float);
+  if (dtype == 1)
+    k_probe_encoder<__nv_bfloat16><<<n, 256, smem, st>>>(x, cu, d, gain, shift, eps, (const __nv_bfloat16*)dense_w, dense_b,
+                                                         out_w, out_b, scores);
+  else
+    k_probe_encoder<float><<<n, 256, smem, st>>>(x, cu, d, gain, shift, eps, (const float*)dense_w, dense_b, out_w, out_b,
+                                                 scores);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_to_f32(const void* src, int dtype, int n, float* dst, cudaStream_t st) {
+  if (n <= 0) return cudaSuccess;
+  const int grid = grid_for(n, 256);
+  if (dtype == 1) k_to_f32<__nv_bfloat16><<<grid, 256, 0, st>>>((const __nv_bfloat16*)src, n, dst);
+  else k_to_f32<float><<<grid, 256, 0, st>>>((const float*)src, n, dst);
   return cudaGetLastError();
 }
 

@@ -35,7 +35,9 @@ constexpr int kEpiBufBytes = 32 * 32 * 4;      // one 32-row, 128-byte-wide sub-
 // Operand ring and epilogue staging share 224 KB: the residual and SwiGLU epilogues stage one 4 KB sub-tile per
 // warp and keep six operand stages; the plain store stages 8 KB per warp (two buffers), the QKV epilogue 32 KB
 // of rotary-table rows and 4 KB of output per warp, and these keep five.
-__host__ __device__ constexpr int stages_of(int epi) { return (epi == kEpiResidual || epi == kEpiSwiGLU) ? 6 : 5; }
+__host__ __device__ constexpr int stages_of(int epi) {
+  return (epi == kEpiResidual || epi == kEpiResidualBias || epi == kEpiSwiGLU) ? 6 : 5;
+}
 __host__ __device__ constexpr int epi_stage_bytes_of(int epi) { return (7 - stages_of(epi)) * kStageBytes; }
 constexpr int kSmemBytes = 7 * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
 constexpr int kThreads = 320;  // TMA warp, MMA warp, 8 epilogue warps
@@ -89,7 +91,10 @@ __global__ void __launch_bounds__(kThreads, 1)
 k_gemm_tc2(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b0,
           const __grid_constant__ CUtensorMap map_b1, const __grid_constant__ CUtensorMap map_r,
           __nv_bfloat16* __restrict__ out, int m, int n, int k, const QkvRopeArgs qa, int reverse,
-          int* __restrict__ err) {
+          int* __restrict__ err, const float* __restrict__ bias) {
+  // the bias variants share the staging and the TMA path of the plain store and of the residual reduce-add
+  constexpr bool kHasBias = kEpi == kEpiStoreBias || kEpi == kEpiGeluBias || kEpi == kEpiResidualBias;
+  constexpr bool kIsResidual = kEpi == kEpiResidual || kEpi == kEpiResidualBias;
   constexpr int kStages = stages_of(kEpi), kEpiStageBytes = epi_stage_bytes_of(kEpi);
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
@@ -267,7 +272,7 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
             bulk_commit();
           }
         }
-      } else if constexpr (kEpi == kEpiResidual) {
+      } else if constexpr (kIsResidual) {
         // 32x32 fp32 sub-tiles go through this warp's staging buffer (128-byte swizzle) into a TMA reduce-add.
         const uint32_t buf = epi_stage + (uint32_t)(warp - 2) * kEpiBufBytes;
 #pragma unroll 1
@@ -280,6 +285,19 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
           if (lane == 0) bulk_wait_read<0>();  // the previous reduce has finished reading the buffer
           __syncwarp();
           tmem_ld_wait();
+          if constexpr (kHasBias) {  // the same 32 bias values for every row: warp-uniform loads
+#pragma unroll
+            for (int v = 0; v < 8; ++v) {
+              const int cb = col0 + c * 32 + v * 4;
+              if (cb < n) {
+                const float4 bv = __ldg(reinterpret_cast<const float4*>(bias + cb));
+                r[4 * v] = __float_as_uint(__uint_as_float(r[4 * v]) + bv.x);
+                r[4 * v + 1] = __float_as_uint(__uint_as_float(r[4 * v + 1]) + bv.y);
+                r[4 * v + 2] = __float_as_uint(__uint_as_float(r[4 * v + 2]) + bv.z);
+                r[4 * v + 3] = __float_as_uint(__uint_as_float(r[4 * v + 3]) + bv.w);
+              }
+            }
+          }
 #pragma unroll
           for (int v = 0; v < 8; ++v) {
             const uint32_t dst = buf + lane * 128 + ((v ^ (lane & 7)) << 4);
@@ -435,6 +453,22 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
           if (lane == 0) bulk_wait_read<1>();  // the store that last used this buffer has read it
           __syncwarp();
           tmem_ld_wait();
+          if constexpr (kHasBias) {
+#pragma unroll
+            for (int v = 0; v < 16; ++v) {
+              const int cb = col0 + c * 64 + v * 4;
+              float4 bv = make_float4(0.f, 0.f, 0.f, 0.f);
+              if (cb < n) bv = __ldg(reinterpret_cast<const float4*>(bias + cb));  // warp-uniform address
+              float y[4] = {__uint_as_float(r[4 * v]) + bv.x, __uint_as_float(r[4 * v + 1]) + bv.y,
+                            __uint_as_float(r[4 * v + 2]) + bv.z, __uint_as_float(r[4 * v + 3]) + bv.w};
+              if constexpr (kEpi == kEpiGeluBias) {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) y[e] = 0.5f * y[e] * (1.f + erff(y[e] * 0.70710678118654752f));
+              }
+#pragma unroll
+              for (int e = 0; e < 4; ++e) r[4 * v + e] = __float_as_uint(y[e]);
+            }
+          }
 #pragma unroll
           for (int v = 0; v < 8; ++v) {
             const uint32_t dst = buf + lane * 128 + ((v ^ (lane & 7)) << 4);
@@ -476,16 +510,22 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
 // reverse: see launch_rmsnorm; the result is the same bit for bit in either direction (every tile has the same
 // shape and K order, and each output element is written or reduced into exactly once).
 cudaError_t launch_gemm_tc2(const TmaDesc& a, const TmaDesc& b0, const TmaDesc& b1, void* out, float* resid, int m,
-                           int n, int k, int epilogue, const QkvRopeArgs* qa, int* err, cudaStream_t st, bool reverse) {
+                           int n, int k, int epilogue, const QkvRopeArgs* qa, int* err, cudaStream_t st, bool reverse,
+                           const float* bias) {
   if (m <= 0 || n <= 0) return cudaSuccess;
   if (k <= 0 || (k % 8) || (n % 8)) return cudaErrorInvalidValue;
-  static std::atomic<unsigned long long> smem_set[4];
+  static std::atomic<unsigned long long> smem_set[7];
+  const bool has_bias = epilogue == kEpiStoreBias || epilogue == kEpiGeluBias || epilogue == kEpiResidualBias;
+  if (has_bias && (!bias || (reinterpret_cast<uintptr_t>(bias) & 15))) return cudaErrorInvalidValue;
   {
     cudaError_t e = cudaErrorInvalidValue;
     if (epilogue == kEpiStore) e = ensure_dynamic_smem(k_gemm_tc2<kEpiStore>, kSmemBytes, smem_set[0]);
     else if (epilogue == kEpiResidual) e = ensure_dynamic_smem(k_gemm_tc2<kEpiResidual>, kSmemBytes, smem_set[1]);
     else if (epilogue == kEpiSwiGLU) e = ensure_dynamic_smem(k_gemm_tc2<kEpiSwiGLU>, kSmemBytes, smem_set[2]);
     else if (epilogue == kEpiQkvRope) e = ensure_dynamic_smem(k_gemm_tc2<kEpiQkvRope>, kSmemBytes, smem_set[3]);
+    else if (epilogue == kEpiStoreBias) e = ensure_dynamic_smem(k_gemm_tc2<kEpiStoreBias>, kSmemBytes, smem_set[4]);
+    else if (epilogue == kEpiGeluBias) e = ensure_dynamic_smem(k_gemm_tc2<kEpiGeluBias>, kSmemBytes, smem_set[5]);
+    else if (epilogue == kEpiResidualBias) e = ensure_dynamic_smem(k_gemm_tc2<kEpiResidualBias>, kSmemBytes, smem_set[6]);
     if (e != cudaSuccess) return e;
   }
   const int out_cols = epilogue == kEpiSwiGLU ? 128 : 256;
@@ -497,7 +537,7 @@ cudaError_t launch_gemm_tc2(const TmaDesc& a, const TmaDesc& b0, const TmaDesc& 
   const CUtensorMap& mb1 = reinterpret_cast<const CUtensorMap&>(b1);
   TmaDesc rdesc = a;  // the output (or residual) rows of this launch, exactly m of them: the TMA unit clips the ragged last tile
   QkvRopeArgs q{};
-  if (epilogue == kEpiResidual) {
+  if (epilogue == kEpiResidual || epilogue == kEpiResidualBias) {
     // the residual rows of this launch, exactly m of them, so that the TMA unit clips the ragged last tile
     cudaError_t e = make_tma_2d_f32_box32(&rdesc, resid, (uint64_t)m, (uint64_t)n);
     if (e != cudaSuccess) return e;
@@ -508,7 +548,7 @@ cudaError_t launch_gemm_tc2(const TmaDesc& a, const TmaDesc& b0, const TmaDesc& 
     cudaError_t e = make_tma_2d_bf16_box32_sw64(&rdesc, out, (uint64_t)m, (uint64_t)n);
     if (e != cudaSuccess) return e;
   }
-  if (epilogue == kEpiStore || epilogue == kEpiSwiGLU) {
+  if (epilogue == kEpiStore || epilogue == kEpiSwiGLU || epilogue == kEpiStoreBias || epilogue == kEpiGeluBias) {
     cudaError_t e = make_tma_2d_bf16(&rdesc, out, (uint64_t)m, (uint64_t)n, 32, 64);
     if (e != cudaSuccess) return e;
   }
@@ -529,13 +569,19 @@ cudaError_t launch_gemm_tc2(const TmaDesc& a, const TmaDesc& b0, const TmaDesc& 
   cfg.numAttrs = 1;
   cudaError_t le;
   if (epilogue == kEpiStore)
-    le = cudaLaunchKernelEx(&cfg, k_gemm_tc2<kEpiStore>, ma, mb0, mb1, mr, o, m, n, k, q, reverse ? 1 : 0, err);
+    le = cudaLaunchKernelEx(&cfg, k_gemm_tc2<kEpiStore>, ma, mb0, mb1, mr, o, m, n, k, q, reverse ? 1 : 0, err, bias);
   else if (epilogue == kEpiResidual)
-    le = cudaLaunchKernelEx(&cfg, k_gemm_tc2<kEpiResidual>, ma, mb0, mb1, mr, o, m, n, k, q, reverse ? 1 : 0, err);
+    le = cudaLaunchKernelEx(&cfg, k_gemm_tc2<kEpiResidual>, ma, mb0, mb1, mr, o, m, n, k, q, reverse ? 1 : 0, err, bias);
   else if (epilogue == kEpiSwiGLU)
-    le = cudaLaunchKernelEx(&cfg, k_gemm_tc2<kEpiSwiGLU>, ma, mb0, mb1, mr, o, m, n, k, q, reverse ? 1 : 0, err);
+    le = cudaLaunchKernelEx(&cfg, k_gemm_tc2<kEpiSwiGLU>, ma, mb0, mb1, mr, o, m, n, k, q, reverse ? 1 : 0, err, bias);
   else if (epilogue == kEpiQkvRope)
-    le = cudaLaunchKernelEx(&cfg, k_gemm_tc2<kEpiQkvRope>, ma, mb0, mb1, mr, o, m, n, k, q, reverse ? 1 : 0, err);
+    le = cudaLaunchKernelEx(&cfg, k_gemm_tc2<kEpiQkvRope>, ma, mb0, mb1, mr, o, m, n, k, q, reverse ? 1 : 0, err, bias);
+  else if (epilogue == kEpiStoreBias)
+    le = cudaLaunchKernelEx(&cfg, k_gemm_tc2<kEpiStoreBias>, ma, mb0, mb1, mr, o, m, n, k, q, reverse ? 1 : 0, err, bias);
+  else if (epilogue == kEpiGeluBias)
+    le = cudaLaunchKernelEx(&cfg, k_gemm_tc2<kEpiGeluBias>, ma, mb0, mb1, mr, o, m, n, k, q, reverse ? 1 : 0, err, bias);
+  else if (epilogue == kEpiResidualBias)
+    le = cudaLaunchKernelEx(&cfg, k_gemm_tc2<kEpiResidualBias>, ma, mb0, mb1, mr, o, m, n, k, q, reverse ? 1 : 0, err, bias);
   else
     return cudaErrorInvalidValue;
   if (le != cudaSuccess) return le;

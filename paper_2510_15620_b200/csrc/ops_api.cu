@@ -74,6 +74,46 @@ int prism_op_gemm(const void* a, const void* b, const void* b2, void* out, float
   return st_of(launch_gemm_simt(a, b, b2, out, resid, m, n, k, dtype, epilogue, S(stream)));
 }
 
+int prism_op_gemm_bias(const void* a, const void* b, const float* bias, void* out, float* resid, int32_t m, int32_t n,
+                       int32_t k, int32_t dtype, int32_t epilogue, int32_t impl, int32_t* err_word, void* stream) {
+  if (!a || !b || !bias || m < 0 || n < 1 || k < 1 || epilogue < 0 || epilogue > 2) return PRISM_ERR_INVALID_ARG;
+  if (epilogue == 1 ? !resid : !out) return PRISM_ERR_INVALID_ARG;
+  const int epi = epilogue == 0 ? kEpiStoreBias : epilogue == 1 ? kEpiResidualBias : kEpiGeluBias;
+  if (dtype == PRISM_BF16 && impl == PRISM_IMPL_AUTO) {
+    if (!err_word || (k % 8) || (n % 8)) return PRISM_ERR_UNSUPPORTED;
+    TmaDesc ma, mb;
+    cudaError_t e = make_tma_2d_bf16(&ma, a, (uint64_t)m, (uint64_t)k, 128, 64);
+    if (e == cudaSuccess) e = make_tma_2d_bf16(&mb, b, (uint64_t)n, (uint64_t)k, 128, 64);
+    if (e == cudaSuccess) e = launch_gemm_tc2(ma, mb, mb, out, resid, m, n, k, epi, nullptr, err_word, S(stream), false, bias);
+    return st_of(e);
+  }
+  if (impl != PRISM_IMPL_SIMT && dtype == PRISM_BF16) return PRISM_ERR_UNSUPPORTED;
+  return st_of(launch_gemm_simt(a, b, nullptr, out, resid, m, n, k, dtype, epi, S(stream), bias));
+}
+
+int prism_op_layernorm(float* x, const float* gain, const float* shift, int32_t dtype, int32_t rows, int32_t d, float eps,
+                       void* out, void* stream) {
+  if (!x || !gain || !shift || !out || rows < 0 || d < 4 || (d % 4) || d > 8192) return PRISM_ERR_INVALID_ARG;
+  return st_of(launch_layernorm(x, gain, shift, dtype, rows, d, eps, out, S(stream)));
+}
+
+int prism_op_embed_encoder(const void* table, const void* pos_table, const float* type_row, int32_t dtype,
+                           const int32_t* tokens, const int32_t* pos, int32_t pos_offset, int32_t total, int32_t d, float* x,
+                           void* stream) {
+  if (!table || !pos_table || !type_row || !tokens || !pos || !x || total < 0 || (d % 4) || pos_offset < 0)
+    return PRISM_ERR_INVALID_ARG;
+  if (dtype == PRISM_BF16 && (d % 8)) return PRISM_ERR_INVALID_ARG;
+  return st_of(launch_embed_encoder(table, pos_table, type_row, dtype, tokens, pos, pos_offset, total, d, x, S(stream)));
+}
+
+int prism_op_probe_encoder(const float* x, const int32_t* cu, int32_t n, int32_t d, const float* gain, const float* shift,
+                           float eps, const void* dense_w, int32_t dtype, const float* dense_b, const float* out_w,
+                           const float* out_b, float* scores, void* stream) {
+  if (!x || !cu || !gain || !shift || !dense_w || !dense_b || !out_w || !out_b || !scores || n < 0 || d < 1 || d > 8192)
+    return PRISM_ERR_INVALID_ARG;
+  return st_of(launch_probe_encoder(x, cu, n, d, gain, shift, eps, dense_w, dtype, dense_b, out_w, out_b, scores, S(stream)));
+}
+
 int prism_op_gemm_qkv_rope(const void* a, const void* w_qkv, void* out, int32_t m, int32_t k, int32_t n_q_heads,
                            int32_t n_kv_heads, int32_t qk_norm, const void* g_q, const void* g_k, float eps,
                            const int32_t* pos, float theta, int32_t max_pos, int32_t* err_word, void* stream) {
@@ -114,14 +154,14 @@ int prism_op_attention(const void* qkv, void* out, const int32_t* cu, int32_t n_
                        int32_t impl, int32_t* err_word, void* stream) {
   if (!qkv || !out || !cu || n_seq < 0 || total < 0 || n_kv_heads < 1 || n_q_heads % n_kv_heads) return PRISM_ERR_INVALID_ARG;
   if (dtype == PRISM_BF16 && impl != PRISM_IMPL_SIMT) {
-    if (head_dim != 128) return PRISM_ERR_UNSUPPORTED;
+    if (head_dim != 128 && !(head_dim == 64 && impl != PRISM_IMPL_MMA)) return PRISM_ERR_UNSUPPORTED;
     if (impl == PRISM_IMPL_AUTO || impl == PRISM_IMPL_SOLO) {
       if (!err_word) return PRISM_ERR_INVALID_ARG;
-      if (impl == PRISM_IMPL_AUTO && ((n_q_heads / n_kv_heads) & 1) == 0)
+      if (impl == PRISM_IMPL_AUTO && head_dim == 128 && ((n_q_heads / n_kv_heads) & 1) == 0)
         return st_of(launch_attention_tc2(qkv, out, cu, 0, n_seq, 0, total, max_len, n_q_heads, n_kv_heads, causal,
                                           err_word, S(stream)));
       return st_of(launch_attention_tc(qkv, out, cu, 0, n_seq, 0, total, max_len, n_q_heads, n_kv_heads, causal, err_word,
-                                       S(stream)));
+                                       S(stream), head_dim));
     }
     return st_of(launch_attention_mma(qkv, out, cu, 0, n_seq, 0, max_len, n_q_heads, n_kv_heads, causal, S(stream)));
   }

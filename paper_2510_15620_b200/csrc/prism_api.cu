@@ -27,12 +27,22 @@ struct LayerMaps {  // TMA descriptors of the B operands
   TmaDesc qkv, o, gate, up, down;
 };
 
+struct EncVec {  // fp32 copies of one encoder block's vectors
+  const float *b_qkv, *b_o, *ln1_g, *ln1_b, *b_ffn1, *b_ffn2, *ln2_g, *ln2_b;
+};
+
 }  // namespace
 
 struct prism_handle {
   prism_model_cfg cfg{};
   std::vector<prism_layer_weights> layers;  // caller's pointers (device, or pinned host when streamed)
   const void *embed = nullptr, *g_final = nullptr, *score_head = nullptr;
+  // encoder stack (cfg.arch == PRISM_ARCH_ENCODER)
+  bool enc = false;
+  std::vector<prism_encoder_layer_weights> enc_layers;
+  std::vector<EncVec> enc_vec;
+  const void *pos_embed = nullptr, *head_dense_w = nullptr;
+  const float *type_f = nullptr, *emb_g = nullptr, *emb_b = nullptr, *head_db = nullptr, *head_ow = nullptr, *head_ob = nullptr;
   int esz = 4;
   int chunk_tokens = 0;
   bool tc = false;  // tensor-core GEMM path
@@ -226,6 +236,10 @@ LayerDev layer_in_slot(const prism_handle* h, int s) {
 }
 
 LayerDev layer_resident(const prism_handle* h, int l) {
+  if (h->enc) {  // the two FFN maps take the places of gate and down
+    const prism_encoder_layer_weights& e = h->enc_layers[l];
+    return LayerDev{nullptr, e.w_qkv, nullptr, nullptr, e.w_o, nullptr, e.w_ffn1, e.w_ffn1, e.w_ffn2};
+  }
   const prism_layer_weights& w = h->layers[l];
   return LayerDev{w.g_attn, w.w_qkv, w.g_q, w.g_k, w.w_o, w.g_ffn, w.w_gate, w.w_up, w.w_down};
 }
@@ -283,13 +297,25 @@ int validate_cfg(const prism_model_cfg& c, std::string* why) {
   if (c.hidden_offload != 0 && c.hidden_offload != 1) return bad("hidden_offload must be 0 or 1");
   if (c.hidden_offload && c.activation_budget_bytes <= 0) return bad("hidden_offload needs an activation budget");
   if (c.shared_prefix != PRISM_PREFIX_AUTO && c.shared_prefix != PRISM_PREFIX_OFF) return bad("shared_prefix must be 0 or 1");
+  if (c.arch != PRISM_ARCH_DECODER && c.arch != PRISM_ARCH_ENCODER) return bad("unknown arch");
   auto unsup = [&](const char* m) { *why = m; return PRISM_ERR_UNSUPPORTED; };
+  const bool enc = c.arch == PRISM_ARCH_ENCODER;
+  if (enc) {
+    if (c.qk_norm) return bad("the encoder stack has no QK-norm");
+    if (c.pos_offset < 0 || c.max_positions < 1 || (long long)c.max_seq_len + c.pos_offset > c.max_positions)
+      return bad("max_seq_len + pos_offset exceeds max_positions");
+    if (c.weight_residency != PRISM_WEIGHTS_DEVICE) return unsup("the encoder stack keeps its weights on the device");
+    if (c.embed_cache_rows || c.hidden_offload) return unsup("embedding cache and hidden-state offload are decoder-only");
+    if (c.gemm_impl != PRISM_IMPL_AUTO && c.gemm_impl != PRISM_IMPL_SIMT) return unsup("encoder GEMMs: AUTO or SIMT");
+    if (c.attention_impl == PRISM_IMPL_MMA) return unsup("encoder attention: AUTO, SOLO or SIMT");
+  }
   if (c.head_dim % 2 || c.head_dim > 256) return unsup("head_dim must be even and <= 256");
   if (c.hidden % 4 || c.hidden > 8192) return unsup("hidden must be a multiple of 4 and <= 8192");
   if (c.dtype == PRISM_BF16) {
     if (c.hidden % 8 || c.ffn % 8 || c.head_dim % 8) return unsup("bf16 mode needs hidden, ffn, head_dim multiples of 8");
-    if (c.gemm_impl != PRISM_IMPL_SIMT && (c.ffn % 128)) return unsup("tensor-core SwiGLU needs ffn multiple of 128");
-    if (c.attention_impl != PRISM_IMPL_SIMT && c.head_dim != 128) return unsup("tensor-core attention needs head_dim 128");
+    if (!enc && c.gemm_impl != PRISM_IMPL_SIMT && (c.ffn % 128)) return unsup("tensor-core SwiGLU needs ffn multiple of 128");
+    if (c.attention_impl != PRISM_IMPL_SIMT && c.head_dim != 128 && !(enc && c.head_dim == 64))
+      return unsup("tensor-core attention needs head_dim 128 (encoder stack: 128 or 64)");
   }
   return PRISM_OK;
 }
@@ -364,9 +390,11 @@ void prism_destroy(prism_handle* h) {
   delete h;
 }
 
-static int create_impl(prism_handle* h, const prism_model_cfg* cfg, const prism_weights* w) {
+static int create_impl(prism_handle* h, const prism_model_cfg* cfg, const prism_weights* w,
+                       const prism_encoder_weights* ew) {
   const prism_model_cfg& c = *cfg;
   h->cfg = c;
+  h->enc = ew != nullptr;
   h->esz = c.dtype == PRISM_BF16 ? 2 : 4;
   h->tc = c.dtype == PRISM_BF16 && (c.gemm_impl == PRISM_IMPL_AUTO || c.gemm_impl == PRISM_IMPL_SOLO);
   h->pair = c.gemm_impl == PRISM_IMPL_AUTO;
@@ -375,13 +403,36 @@ static int create_impl(prism_handle* h, const prism_model_cfg* cfg, const prism_
           : c.attention_impl == PRISM_IMPL_AUTO ? ((((c.n_q_heads / c.n_kv_heads) & 1) == 0) ? 3 : 1)
           : c.attention_impl == PRISM_IMPL_SOLO ? 1
           : c.attention_impl == PRISM_IMPL_MMA  ? 2 : 0;
+  if (h->fa == 3 && c.head_dim != 128) h->fa = 1;  // the two-head kernel is written for head_dim 128
   const bool streamed = c.weight_residency == PRISM_WEIGHTS_HOST_STREAMED;
+  if (h->enc) {
+    const void* glob[] = {ew->embed, ew->pos_embed, ew->type_embed, ew->emb_ln_g, ew->emb_ln_b, ew->head_dense_w,
+                          ew->head_dense_b, ew->head_out_w, ew->head_out_b, ew->layers};
+    for (const void* p : glob)
+      if (!p) return fail(h, PRISM_ERR_INVALID_ARG, "null weight pointer");
+    if ((reinterpret_cast<uintptr_t>(ew->embed) & 15) || (reinterpret_cast<uintptr_t>(ew->pos_embed) & 15) ||
+        (reinterpret_cast<uintptr_t>(ew->head_dense_w) & 15))
+      return fail(h, PRISM_ERR_INVALID_ARG, "embedding tables and head matrix must be 16-byte aligned");
+    h->embed = ew->embed;
+    h->pos_embed = ew->pos_embed;
+    h->head_dense_w = ew->head_dense_w;
+    h->enc_layers.assign(ew->layers, ew->layers + c.n_layers);
+    for (const prism_encoder_layer_weights& lw : h->enc_layers) {
+      const void* mats[] = {lw.w_qkv, lw.w_o, lw.w_ffn1, lw.w_ffn2};
+      for (const void* p : mats)
+        if (!p || (reinterpret_cast<uintptr_t>(p) & 15)) return fail(h, PRISM_ERR_INVALID_ARG, "layer tensor null or not 16-byte aligned");
+      const void* vecs[] = {lw.b_qkv, lw.b_o, lw.ln1_g, lw.ln1_b, lw.b_ffn1, lw.b_ffn2, lw.ln2_g, lw.ln2_b};
+      for (const void* p : vecs)
+        if (!p) return fail(h, PRISM_ERR_INVALID_ARG, "layer vector null");
+    }
+  } else {
   if (!w->embed || !w->g_final || !w->score_head || !w->layers) return fail(h, PRISM_ERR_INVALID_ARG, "null weight pointer");
   h->embed = w->embed;
   h->g_final = w->g_final;
   h->score_head = w->score_head;
   h->layers.assign(w->layers, w->layers + c.n_layers);
-  for (int l = 0; l < c.n_layers; ++l) {
+  }
+  for (int l = 0; l < c.n_layers && !h->enc; ++l) {
     const prism_layer_weights& lw = h->layers[l];
     const void* req[] = {lw.g_attn, lw.w_qkv, lw.w_o, lw.g_ffn, lw.w_gate, lw.w_up, lw.w_down};
     for (const void* p : req)
@@ -520,22 +571,71 @@ static int create_impl(prism_handle* h, const prism_model_cfg* cfg, const prism_
     }
   }
 
-  PRISM_LAUNCH(h, launch_rope_table(h->rope_cos, h->rope_sin, c.max_seq_len, c.head_dim, c.rope_theta, 0));
-  if (h->rope_fused) PRISM_LAUNCH(h, launch_rope_table_fused(h->rope_fused, c.max_seq_len, c.rope_theta, 0));
-  PRISM_LAUNCH(h, launch_score_diff(h->score_head, c.dtype, c.hidden, h->w_diff, 0));
+  if (h->enc) {
+    // fp32 copies of every vector (biases, LayerNorm gain and shift, head vectors): one buffer, 16-byte aligned slices
+    const size_t F = (size_t)c.ffn;
+    const size_t per_layer = align_up(nqkv, 4) + 6 * align_up(D, 4) + align_up(F, 4);
+    const size_t glob = 5 * align_up(D, 4) + 4;
+    float* buf = nullptr;
+    PRISM_CUDA(h, dev_alloc(h, &buf, per_layer * c.n_layers + glob));
+    float* cur = buf;
+    auto widen = [&](const void* src, size_t n, const float** dst) -> cudaError_t {
+      *dst = cur;
+      cudaError_t e = launch_to_f32(src, c.dtype, (int)n, cur, 0);
+      cur += align_up(n, 4);
+      return e;
+    };
+    PRISM_CUDA(h, widen(ew->type_embed, D, &h->type_f));
+    PRISM_CUDA(h, widen(ew->emb_ln_g, D, &h->emb_g));
+    PRISM_CUDA(h, widen(ew->emb_ln_b, D, &h->emb_b));
+    PRISM_CUDA(h, widen(ew->head_dense_b, D, &h->head_db));
+    PRISM_CUDA(h, widen(ew->head_out_w, D, &h->head_ow));
+    PRISM_CUDA(h, widen(ew->head_out_b, 1, &h->head_ob));
+    h->enc_vec.resize(c.n_layers);
+    for (int l = 0; l < c.n_layers; ++l) {
+      const prism_encoder_layer_weights& lw = h->enc_layers[l];
+      EncVec& v = h->enc_vec[l];
+      PRISM_CUDA(h, widen(lw.b_qkv, nqkv, &v.b_qkv));
+      PRISM_CUDA(h, widen(lw.b_o, D, &v.b_o));
+      PRISM_CUDA(h, widen(lw.ln1_g, D, &v.ln1_g));
+      PRISM_CUDA(h, widen(lw.ln1_b, D, &v.ln1_b));
+      PRISM_CUDA(h, widen(lw.b_ffn1, F, &v.b_ffn1));
+      PRISM_CUDA(h, widen(lw.b_ffn2, D, &v.b_ffn2));
+      PRISM_CUDA(h, widen(lw.ln2_g, D, &v.ln2_g));
+      PRISM_CUDA(h, widen(lw.ln2_b, D, &v.ln2_b));
+    }
+  } else {
+    PRISM_LAUNCH(h, launch_rope_table(h->rope_cos, h->rope_sin, c.max_seq_len, c.head_dim, c.rope_theta, 0));
+    if (h->rope_fused) PRISM_LAUNCH(h, launch_rope_table_fused(h->rope_fused, c.max_seq_len, c.rope_theta, 0));
+    PRISM_LAUNCH(h, launch_score_diff(h->score_head, c.dtype, c.hidden, h->w_diff, 0));
+  }
   PRISM_CUDA(h, cudaDeviceSynchronize());
   return PRISM_OK;
 }
 
+static int create_any(const prism_model_cfg* cfg, const prism_weights* w, const prism_encoder_weights* ew,
+                      prism_handle** out);
+
 int prism_create(const prism_model_cfg* cfg, const prism_weights* w, prism_handle** out) {
   if (out) *out = nullptr;
-  if (!cfg || !w || !out) return PRISM_ERR_INVALID_ARG;
+  if (!cfg || !w || !out || cfg->arch != PRISM_ARCH_DECODER) return PRISM_ERR_INVALID_ARG;
+  return create_any(cfg, w, nullptr, out);
+}
+
+int prism_create_encoder(const prism_model_cfg* cfg, const prism_encoder_weights* w, prism_handle** out) {
+  if (out) *out = nullptr;
+  if (!cfg || !w || !out || cfg->arch != PRISM_ARCH_ENCODER) return PRISM_ERR_INVALID_ARG;
+  return create_any(cfg, nullptr, w, out);
+}
+
+static int create_any(const prism_model_cfg* cfg, const prism_weights* w, const prism_encoder_weights* ew,
+                      prism_handle** out) {
   std::string why;
   int rc = validate_cfg(*cfg, &why);
   if (rc != PRISM_OK) return rc;
   prism_handle* h = new (std::nothrow) prism_handle();
   if (!h) return PRISM_ERR_NOMEM;
-  rc = create_impl(h, cfg, w);
+  rc = create_impl(h, cfg, w, ew);
   if (rc != PRISM_OK) {
     prism_destroy(h);
     return rc;
@@ -584,9 +684,9 @@ bool next_dir(prism_handle* h, bool supported) {
 }
 
 cudaError_t gemm_tc_any(prism_handle* h, const TmaDesc& a, const TmaDesc& b0, const TmaDesc& b1, void* out, float* resid,
-                        int m, int n, int k, int epi, const QkvRopeArgs* qa, cudaStream_t st) {
+                        int m, int n, int k, int epi, const QkvRopeArgs* qa, cudaStream_t st, const float* bias = nullptr) {
   const bool rev = next_dir(h, h->pair);
-  return h->pair ? launch_gemm_tc2(a, b0, b1, out, resid, m, n, k, epi, qa, h->errword, st, rev)
+  return h->pair ? launch_gemm_tc2(a, b0, b1, out, resid, m, n, k, epi, qa, h->errword, st, rev, bias)
                  : launch_gemm_tc(a, b0, b1, out, resid, m, n, k, epi, qa, h->errword, st);
 }
 
@@ -659,6 +759,67 @@ int run_layer_chunk(prism_handle* h, const LayerDev& W, const LayerMaps* maps, f
   else
     PRISM_LAUNCH_P(h, st, PRISM_K_GEMM_DOWN, 2.0 * R * D * c.ffn,
                    launch_gemm_simt(h->hbuf, W.w_down, nullptr, nullptr, xr, rows, D, c.ffn, c.dtype, kEpiResidual, st));
+  return PRISM_OK;
+}
+
+// One post-norm encoder block over the same rows.  The block starts with the LayerNorm its predecessor left
+// pending (the embedding LayerNorm for block 0, else LN2 of block l - 1), so that, as in the decoder path, a
+// chunk's normed GEMM input is produced right before it is consumed; LN2 of the last executed block is applied by
+// the probe to the one row it reads.
+int run_layer_chunk_encoder(prism_handle* h, int l, const LayerDev& W, const LayerMaps* maps, float* x, const int* cu_dev,
+                            int s0, int s1, int r0, int rows, int max_len, cudaStream_t st) {
+  const prism_model_cfg& c = h->cfg;
+  const int D = c.hidden, dh = c.head_dim, F = c.ffn;
+  const int nqkv = (c.n_q_heads + 2 * c.n_kv_heads) * dh, hd = c.n_q_heads * dh;
+  float* xr = x + (size_t)r0 * D;
+  const EncVec& V = h->enc_vec[l];
+  const float* g0 = l == 0 ? h->emb_g : h->enc_vec[l - 1].ln2_g;
+  const float* b0 = l == 0 ? h->emb_b : h->enc_vec[l - 1].ln2_b;
+  const double R = rows, norm_bytes = R * D * (8.0 + h->esz);
+  double attn_flops = 0.0;
+  for (int s = s0; s < s1; ++s) {
+    const double L = h->h_cu[s + 1] - h->h_cu[s];
+    attn_flops += (c.causal ? 2.0 : 4.0) * L * L * c.n_q_heads * dh;
+  }
+  PRISM_LAUNCH_P(h, st, PRISM_K_RMSNORM, norm_bytes, launch_layernorm(xr, g0, b0, c.dtype, rows, D, c.rms_eps, h->a_norm, st, next_dir(h, true)));
+  if (h->tc)
+    PRISM_LAUNCH_P(h, st, PRISM_K_GEMM_QKV, 2.0 * R * nqkv * D,
+                   gemm_tc_any(h, h->map_a_norm, maps->qkv, maps->qkv, h->qkv, nullptr, rows, nqkv, D, kEpiStoreBias, nullptr, st, V.b_qkv));
+  else
+    PRISM_LAUNCH_P(h, st, PRISM_K_GEMM_QKV, 2.0 * R * nqkv * D,
+                   launch_gemm_simt(h->a_norm, W.w_qkv, nullptr, h->qkv, nullptr, rows, nqkv, D, c.dtype, kEpiStoreBias, st, V.b_qkv));
+  next_dir(h, false);
+  if (h->fa == 3)
+    PRISM_LAUNCH_P(h, st, PRISM_K_ATTENTION, attn_flops,
+                   launch_attention_tc2(h->qkv, h->attn, cu_dev, s0, s1 - s0, r0, rows, max_len, c.n_q_heads, c.n_kv_heads, c.causal,
+                                        h->errword, st, false));
+  else if (h->fa == 1)
+    PRISM_LAUNCH_P(h, st, PRISM_K_ATTENTION, attn_flops,
+                   launch_attention_tc(h->qkv, h->attn, cu_dev, s0, s1 - s0, r0, rows, max_len, c.n_q_heads, c.n_kv_heads, c.causal,
+                                       h->errword, st, dh));
+  else
+    PRISM_LAUNCH_P(h, st, PRISM_K_ATTENTION, attn_flops,
+                   launch_attention_simt(h->qkv, h->attn, cu_dev, s0, s1 - s0, r0, max_len, c.n_q_heads, c.n_kv_heads, dh,
+                                         c.causal, c.dtype, st));
+  if (h->tc)
+    PRISM_LAUNCH_P(h, st, PRISM_K_GEMM_O, 2.0 * R * D * hd,
+                   gemm_tc_any(h, h->map_attn, maps->o, maps->o, nullptr, xr, rows, D, hd, kEpiResidualBias, nullptr, st, V.b_o));
+  else
+    PRISM_LAUNCH_P(h, st, PRISM_K_GEMM_O, 2.0 * R * D * hd,
+                   launch_gemm_simt(h->attn, W.w_o, nullptr, nullptr, xr, rows, D, hd, c.dtype, kEpiResidualBias, st, V.b_o));
+  PRISM_LAUNCH_P(h, st, PRISM_K_RMSNORM, norm_bytes, launch_layernorm(xr, V.ln1_g, V.ln1_b, c.dtype, rows, D, c.rms_eps, h->a_norm, st, next_dir(h, true)));
+  if (h->tc)
+    PRISM_LAUNCH_P(h, st, PRISM_K_GEMM_GATEUP, 2.0 * R * F * D,
+                   gemm_tc_any(h, h->map_a_norm, maps->gate, maps->gate, h->hbuf, nullptr, rows, F, D, kEpiGeluBias, nullptr, st, V.b_ffn1));
+  else
+    PRISM_LAUNCH_P(h, st, PRISM_K_GEMM_GATEUP, 2.0 * R * F * D,
+                   launch_gemm_simt(h->a_norm, W.w_gate, nullptr, h->hbuf, nullptr, rows, F, D, c.dtype, kEpiGeluBias, st, V.b_ffn1));
+  if (h->tc)
+    PRISM_LAUNCH_P(h, st, PRISM_K_GEMM_DOWN, 2.0 * R * D * F,
+                   gemm_tc_any(h, h->map_hbuf, maps->down, maps->down, nullptr, xr, rows, D, F, kEpiResidualBias, nullptr, st, V.b_ffn2));
+  else
+    PRISM_LAUNCH_P(h, st, PRISM_K_GEMM_DOWN, 2.0 * R * D * F,
+                   launch_gemm_simt(h->hbuf, W.w_down, nullptr, nullptr, xr, rows, D, F, c.dtype, kEpiResidualBias, st, V.b_ffn2));
   return PRISM_OK;
 }
 
@@ -770,7 +931,7 @@ int select_impl(prism_handle* h, const int32_t* query, int32_t lq, const int32_t
     if (h->h_off[i + 1] < h->h_off[i]) return fail(h, PRISM_ERR_BAD_INPUT, "cand_offsets not monotone");
   // Shared query prefix: under causal attention the query's rows are the same in every sequence, so they are
   // stored and computed once in front of the documents (rows [0, lq)); cu then holds document rows only.
-  const int prefix = (c.shared_prefix == PRISM_PREFIX_AUTO && h->fa == 3 && c.causal && !h->offload && !shard && N >= 2 &&
+  const int prefix = (c.shared_prefix == PRISM_PREFIX_AUTO && !h->enc && h->fa == 3 && c.causal && !h->offload && !shard && N >= 2 &&
                       lq >= 8 && lq <= 120 && (lq & 7) == 0 && (long long)lq + h->h_off[N] <= h->chunk_tokens)
                          ? lq
                          : 0;
@@ -814,6 +975,11 @@ int select_impl(prism_handle* h, const int32_t* query, int32_t lq, const int32_t
   PRISM_LAUNCH_P(h, st, PRISM_K_PACK, 12.0 * total,
                  launch_pack_tokens(query, lq, cand, off, h->cu[cur], N, (int)total, c.vocab, h->tokens, h->pos, h->errword, st,
                                     prefix > 0));
+  if (h->enc)
+    PRISM_LAUNCH_P(h, st, PRISM_K_EMBED, (double)total * c.hidden * (4.0 + 2.0 * h->esz),
+                   launch_embed_encoder(h->embed, h->pos_embed, h->type_f, c.dtype, h->tokens, h->pos, c.pos_offset, (int)total,
+                                        c.hidden, h->x[cur], st));
+  else
   PRISM_LAUNCH_P(h, st, PRISM_K_EMBED, (double)total * c.hidden * (4.0 + h->esz),
                  launch_embed(h->cache_rows > 0 ? h->cache_dev : h->embed, c.dtype, h->tokens, (int)total, c.hidden, h->x[cur], st,
                               h->cache_rows > 0 ? h->tok2slot_dev : nullptr));
@@ -857,7 +1023,9 @@ int select_impl(prism_handle* h, const int32_t* query, int32_t lq, const int32_t
         ++s1;
       }
       const int r0 = h->h_cu[s0], rows = h->h_cu[s1] - r0;
-      if (!h->offload) {
+      if (h->enc) {
+        if ((rc = run_layer_chunk_encoder(h, l, W, maps, h->x[cur], h->cu[cur], s0, s1, r0, rows, max_len, st)) != PRISM_OK) return rc;
+      } else if (!h->offload) {
         if ((rc = run_layer_chunk(h, W, maps, h->x[cur], h->cu[cur], s0, s1, r0, rows, max_len, st)) != PRISM_OK) return rc;
       } else if (rows > 0) {
         // Chunk `chunks` goes through device buffer chunks % 3: fetched on in_stream once the buffer's previous
@@ -925,6 +1093,12 @@ int select_impl(prism_handle* h, const int32_t* query, int32_t lq, const int32_t
       p.prefix = prefix;
       const int nxt = cur ^ 1;
       float* score_buf = shard ? shard->exchange : h->scores;
+      if (h->enc) {
+        const EncVec& V = h->enc_vec[layers_run - 1];  // the last executed block's LN2 is still pending
+        PRISM_LAUNCH_P(h, st, PRISM_K_PROBE, (double)n * c.hidden * (4.0 + (double)c.hidden * h->esz),
+                       launch_probe_encoder(h->x[cur], h->cu[cur], n, c.hidden, V.ln2_g, V.ln2_b, c.rms_eps, h->head_dense_w,
+                                            c.dtype, h->head_db, h->head_ow, h->head_ob, score_buf, st));
+      } else
       PRISM_LAUNCH_P(h, st, PRISM_K_PROBE, 4.0 * n * c.hidden,
                      launch_probe(h->x[cur], h->cu[cur], n, c.hidden, h->g_final, c.dtype, h->w_diff, c.rms_eps, score_buf, st, prefix));
       if (shard && shard->reduce(shard->ctx, n, st) != 0) return fail(h, PRISM_ERR_CUDA, "the score exchange callback failed");

@@ -17,7 +17,8 @@ __device__ __forceinline__ void stf(__nv_bfloat16* p, float v) { *p = __float2bf
 template <typename T, int kEpi>
 __global__ void __launch_bounds__(256) k_gemm_simt(const T* __restrict__ a, const T* __restrict__ b,
                                                    const T* __restrict__ b2, T* __restrict__ out,
-                                                   float* __restrict__ resid, int m, int n, int k) {
+                                                   float* __restrict__ resid, int m, int n, int k,
+                                                   const float* __restrict__ bias) {
   constexpr int BM = 64, BN = 64, BK = 16;
   __shared__ float sa[BK][BM + 1];
   __shared__ float sb[BK][BN + 1];
@@ -68,6 +69,12 @@ __global__ void __launch_bounds__(256) k_gemm_simt(const T* __restrict__ a, cons
         const float g = acc[i][j];
         stf(out + o, g / (1.f + expf(-g)) * acc2[i][j]);
       }
+      if constexpr (kEpi == kEpiStoreBias) stf(out + o, acc[i][j] + bias[gn]);
+      if constexpr (kEpi == kEpiGeluBias) {
+        const float y = acc[i][j] + bias[gn];
+        stf(out + o, 0.5f * y * (1.f + erff(y * 0.70710678118654752f)));
+      }
+      if constexpr (kEpi == kEpiResidualBias) resid[o] += acc[i][j] + bias[gn];
     }
   }
 }
@@ -126,18 +133,25 @@ __global__ void __launch_bounds__(128) k_attention_simt(const T* __restrict__ qk
 }  // namespace
 
 cudaError_t launch_gemm_simt(const void* a, const void* b, const void* b2, void* out, float* resid, int m,
-                             int n, int k, int dtype, int epilogue, cudaStream_t st) {
+                             int n, int k, int dtype, int epilogue, cudaStream_t st, const float* bias) {
   if (m <= 0 || n <= 0) return cudaSuccess;
+  if (epilogue >= kEpiStoreBias && !bias) return cudaErrorInvalidValue;
   dim3 grid((n + 63) / 64, (m + 63) / 64);
 #define PRISM_SIMT(T, E) \
-  k_gemm_simt<T, E><<<grid, 256, 0, st>>>((const T*)a, (const T*)b, (const T*)b2, (T*)out, resid, m, n, k)
+  k_gemm_simt<T, E><<<grid, 256, 0, st>>>((const T*)a, (const T*)b, (const T*)b2, (T*)out, resid, m, n, k, bias)
   if (dtype == 1) {
     if (epilogue == kEpiStore) PRISM_SIMT(__nv_bfloat16, kEpiStore);
     else if (epilogue == kEpiResidual) PRISM_SIMT(__nv_bfloat16, kEpiResidual);
+    else if (epilogue == kEpiStoreBias) PRISM_SIMT(__nv_bfloat16, kEpiStoreBias);
+    else if (epilogue == kEpiGeluBias) PRISM_SIMT(__nv_bfloat16, kEpiGeluBias);
+    else if (epilogue == kEpiResidualBias) PRISM_SIMT(__nv_bfloat16, kEpiResidualBias);
     else PRISM_SIMT(__nv_bfloat16, kEpiSwiGLU);
   } else {
     if (epilogue == kEpiStore) PRISM_SIMT(float, kEpiStore);
     else if (epilogue == kEpiResidual) PRISM_SIMT(float, kEpiResidual);
+    else if (epilogue == kEpiStoreBias) PRISM_SIMT(float, kEpiStoreBias);
+    else if (epilogue == kEpiGeluBias) PRISM_SIMT(float, kEpiGeluBias);
+    else if (epilogue == kEpiResidualBias) PRISM_SIMT(float, kEpiResidualBias);
     else PRISM_SIMT(float, kEpiSwiGLU);
   }
 #undef PRISM_SIMT

@@ -31,6 +31,12 @@ def _L():
         L.prism_op_wait_selftest.argtypes = [C.c_uint64, vp, vp]
         L.prism_op_wait_selftest.restype = C.c_int
         L.prism_op_compact.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, vp]
+        L.prism_op_gemm_bias.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, vp, vp]
+        L.prism_op_layernorm.argtypes = [vp, vp, vp, i32, i32, i32, f32, vp, vp]
+        L.prism_op_embed_encoder.argtypes = [vp, vp, vp, i32, vp, vp, i32, i32, i32, vp, vp]
+        L.prism_op_probe_encoder.argtypes = [vp, vp, i32, i32, vp, vp, f32, vp, i32, vp, vp, vp, vp, vp]
+        for n in ("gemm_bias", "layernorm", "embed_encoder", "probe_encoder"):
+            getattr(L, "prism_op_" + n).restype = C.c_int
         for n in ("pack", "embed", "rmsnorm", "qknorm_rope", "gemm", "attention", "probe", "route", "compact"):
             getattr(L, "prism_op_" + n).restype = C.c_int
         _proto_done = True
@@ -71,6 +77,26 @@ def prism_op_qknorm_rope(qkv, dtype, pos, n_q_heads, n_kv_heads, head_dim, qk_no
 def prism_op_gemm(a, b, b2, out, resid, m, n, k, dtype, epilogue, impl, err_word):
     _check(_L().prism_op_gemm(_p(a), _p(b), _p(b2), _p(out), _p(resid), m, n, k, dtype, epilogue, impl, _p(err_word),
                               _stream()), "gemm")
+
+
+def prism_op_gemm_bias(a, b, bias, out, resid, m, n, k, dtype, epilogue, impl, err_word):
+    _check(_L().prism_op_gemm_bias(_p(a), _p(b), _p(bias), _p(out), _p(resid), m, n, k, dtype, epilogue, impl, _p(err_word),
+                                   _stream()), "gemm_bias")
+
+
+def prism_op_layernorm(x, gain, shift, dtype, eps, out):
+    _check(_L().prism_op_layernorm(_p(x), _p(gain), _p(shift), dtype, x.shape[0], x.shape[1], eps, _p(out), _stream()),
+           "layernorm")
+
+
+def prism_op_embed_encoder(table, pos_table, type_row, dtype, tokens, pos, pos_offset, x):
+    _check(_L().prism_op_embed_encoder(_p(table), _p(pos_table), _p(type_row), dtype, _p(tokens), _p(pos), pos_offset,
+                                       tokens.numel(), x.shape[1], _p(x), _stream()), "embed_encoder")
+
+
+def prism_op_probe_encoder(x, cu, n, gain, shift, eps, dense_w, dtype, dense_b, out_w, out_b, scores):
+    _check(_L().prism_op_probe_encoder(_p(x), _p(cu), n, x.shape[1], _p(gain), _p(shift), eps, _p(dense_w), dtype, _p(dense_b),
+                                       _p(out_w), _p(out_b), _p(scores), _stream()), "probe_encoder")
 
 
 def prism_op_gemm_qkv_rope(a, w_qkv, out, m, k, n_q_heads, n_kv_heads, qk_norm, g_q, g_k, eps, pos, theta, max_pos, err_word):

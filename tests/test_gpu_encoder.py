@@ -1,0 +1,234 @@
+"""-m gpu: the encoder-only reranker stack (Sec. 6.1, Table 1) through the C ABI against the encoder oracle: its
+kernels one by one (embedding sum, LayerNorm, biased GEMM epilogues with the exact GELU, head_dim-64 tensor-core
+attention, the first-token classifier probe) and prism_select end to end in fp32 (1e-4) and bf16 (3e-2)."""
+from dataclasses import replace
+
+import numpy as np
+import pytest
+
+import oracle
+import synth
+from synth.configs import (ARCH_ENCODER, DTYPE_BF16, DTYPE_FP32, MODE_CLUSTER, MODE_FIXED_KEEP, MODE_NONE, ModelCfg,
+                           Schedule, Workload)
+from synth.weights import round_to_bf16
+
+from parity import check_end_to_end, check_replay, check_scores
+from test_gpu_select import TOL_BF16, TOL_FP32, dev_i32, run
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+FP32, BF16, AUTO, SIMT, SOLO = 0, 1, 0, 1, 3
+
+
+@pytest.fixture(scope="module")
+def P():
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    import paper_2510_15620_b200 as pkg
+    return pkg
+
+
+def dev(a, dt=torch.float32):
+    return torch.from_numpy(np.ascontiguousarray(a)).to("cuda").to(dt)
+
+
+# ------------------------------------------------------------------------------------------ kernels
+@pytest.mark.parametrize("dtype", [FP32, BF16])
+@pytest.mark.parametrize("rows,d", [(1, 8), (37, 256), (300, 1024), (77, 2048), (19, 2560), (9, 8192)])
+def test_layernorm(P, dtype, rows, d):
+    """Warp-per-row (d <= 2048) and block-per-row kernels, in place plus the typed copy; rows with a large common
+    offset check that the variance is taken about the mean."""
+    rng = np.random.default_rng(rows + d)
+    x = (rng.normal(size=(rows, d)) * 3 + 100.0 * rng.normal(size=(rows, 1))).astype(np.float32)
+    g = (1 + 0.1 * rng.normal(size=d)).astype(np.float32)
+    b = (0.1 * rng.normal(size=d)).astype(np.float32)
+    tx = dev(x)
+    out = torch.zeros(rows, d, dtype=torch.bfloat16 if dtype == BF16 else torch.float32, device="cuda")
+    P.ops.prism_op_layernorm(tx, dev(g), dev(b), dtype, 1e-5, out)
+    ref = oracle.layernorm(x.astype(np.float64), g.astype(np.float64), b.astype(np.float64), 1e-5)
+    got = tx.cpu().numpy()
+    assert np.max(np.abs(got - ref)) < 2e-4                      # fp32 sums over rows offset by ~100
+    if dtype == BF16:
+        assert np.array_equal(out.float().cpu().numpy(), round_to_bf16(got))      # the copy is the rounded in-place value
+    else:
+        assert np.array_equal(out.cpu().numpy(), got)
+
+
+@pytest.mark.parametrize("dtype", [FP32, BF16])
+def test_embed_encoder(P, dtype):
+    rng = np.random.default_rng(3)
+    v, mp, d, n = 50, 40, 64, 33
+    tab, ptab, ty = (rng.normal(size=s).astype(np.float32) for s in ((v, d), (mp, d), (d,)))
+    if dtype == BF16:
+        tab, ptab = round_to_bf16(tab), round_to_bf16(ptab)
+    tok = rng.integers(0, v, size=n).astype(np.int32)
+    pos = rng.integers(0, mp - 2, size=n).astype(np.int32)
+    tdt = torch.bfloat16 if dtype == BF16 else torch.float32
+    x = torch.zeros(n, d, device="cuda")
+    P.ops.prism_op_embed_encoder(dev(tab, tdt), dev(ptab, tdt), dev(ty), dtype, dev_i32(tok), dev_i32(pos), 2, x)
+    ref = tab[tok].astype(np.float64) + ptab[pos + 2] + ty
+    assert np.max(np.abs(x.cpu().numpy() - ref)) < 1e-6
+
+
+def _gemm_bias_ref(a, b, bias, resid, epi):
+    c = a.astype(np.float64) @ b.astype(np.float64).T + bias.astype(np.float64)
+    return c if epi == 0 else resid.astype(np.float64) + c if epi == 1 else oracle.gelu(c)
+
+
+@pytest.mark.parametrize("epi", [0, 1, 2])
+@pytest.mark.parametrize("m,n,k", [(5, 64, 32), (130, 192, 100), (300, 512, 768)])
+def test_gemm_bias_fp32_simt(P, m, n, k, epi):
+    rng = np.random.default_rng(m + n + k + epi)
+    a = rng.normal(size=(m, k)).astype(np.float32)
+    b = (rng.normal(size=(n, k)) * 0.05).astype(np.float32)
+    bias = rng.normal(size=n).astype(np.float32)
+    resid = rng.normal(size=(m, n)).astype(np.float32)
+    out, rs = torch.zeros(m, n, device="cuda"), dev(resid)
+    P.ops.prism_op_gemm_bias(dev(a), dev(b), dev(bias), out, rs, m, n, k, FP32, epi, SIMT, None)
+    ref = _gemm_bias_ref(a, b, bias, resid, epi)
+    got = (rs if epi == 1 else out).cpu().numpy()
+    assert np.max(np.abs(got - ref)) < 1e-5 * max(1.0, np.max(np.abs(ref)))
+
+
+@pytest.mark.parametrize("impl", [AUTO, SIMT])
+@pytest.mark.parametrize("epi", [0, 1, 2])
+@pytest.mark.parametrize("m,n,k", [(1, 256, 64), (129, 256, 72), (300, 512, 320), (1000, 1024, 1024), (777, 384, 200),
+                                   (4100, 3072, 512), (513, 4096, 1024)])
+def test_gemm_bias_bf16(P, m, n, k, epi, impl):
+    """The pair tcgen05 kernel's bias / bias + GELU / bias + residual epilogues (and the CUDA-core ones) against an
+    fp64 matmul; a bias of order 1 makes a dropped or shifted bias fail by orders of magnitude."""
+    rng = np.random.default_rng(m * 7 + n + k + epi)
+    a = round_to_bf16(rng.normal(size=(m, k)).astype(np.float32))
+    b = round_to_bf16((rng.normal(size=(n, k)) * 0.05).astype(np.float32))
+    bias = rng.normal(size=n).astype(np.float32)
+    resid = rng.normal(size=(m, n)).astype(np.float32)
+    out = torch.zeros(m, n, dtype=torch.bfloat16, device="cuda")
+    rs = dev(resid)
+    err = torch.zeros(1, dtype=torch.int32, device="cuda")
+    P.ops.prism_op_gemm_bias(dev(a, torch.bfloat16), dev(b, torch.bfloat16), dev(bias), out, rs, m, n, k, BF16, epi, impl, err)
+    torch.cuda.synchronize()
+    assert int(err.item()) == 0
+    ref = _gemm_bias_ref(a, b, bias, resid, epi)
+    got = (rs if epi == 1 else out.float()).cpu().numpy()
+    scale = np.max(np.abs(ref))
+    tol = (2.0 ** -8) * scale + 1e-3 if epi != 1 else 1e-4 * scale + 1e-4
+    assert np.max(np.abs(got - ref)) < tol, np.max(np.abs(got - ref))
+
+
+@pytest.mark.parametrize("causal", [0, 1])
+@pytest.mark.parametrize("impl,hq,hkv", [(AUTO, 4, 4), (AUTO, 4, 2), (SOLO, 3, 1), (SIMT, 4, 4)])
+def test_attention_head_dim_64(P, impl, hq, hkv, causal):
+    from test_gpu_ops import _attn_ref
+    rng = np.random.default_rng(64 + causal + hq)
+    lens = np.array([1, 7, 64, 65, 130, 200, 63, 128, 129, 300, 513])
+    cu = np.zeros(len(lens) + 1, np.int32)
+    cu[1:] = np.cumsum(lens)
+    qkv = round_to_bf16(rng.normal(size=(cu[-1], (hq + 2 * hkv) * 64)).astype(np.float32))
+    out = torch.zeros(int(cu[-1]), hq * 64, dtype=torch.bfloat16, device="cuda")
+    err = torch.zeros(1, dtype=torch.int32, device="cuda")
+    P.ops.prism_op_attention(dev(qkv, torch.bfloat16), out, dev_i32(cu), len(lens), int(lens.max()), hq, hkv, 64, causal, BF16,
+                             impl, err)
+    torch.cuda.synchronize()
+    assert int(err.item()) == 0
+    ref = _attn_ref(qkv, cu, hq, hkv, 64, bool(causal))
+    assert np.max(np.abs(out.float().cpu().numpy() - ref)) < 2e-2
+
+
+@pytest.mark.parametrize("dtype", [FP32, BF16])
+def test_probe_encoder(P, dtype):
+    rng = np.random.default_rng(9)
+    d, lens = 256, np.array([5, 1, 40, 0, 17])
+    cu = np.zeros(len(lens) + 1, np.int32)
+    cu[1:] = np.cumsum(lens)
+    x = rng.normal(size=(int(cu[-1]), d)).astype(np.float32)
+    g, b = (1 + 0.1 * rng.normal(size=d)).astype(np.float32), (0.1 * rng.normal(size=d)).astype(np.float32)
+    dw = (rng.normal(size=(d, d)) * 0.08).astype(np.float32)
+    if dtype == BF16:
+        dw = round_to_bf16(dw)
+    db, ow, ob = rng.normal(size=d).astype(np.float32) * 0.1, rng.normal(size=d).astype(np.float32) * 0.1, np.array([0.3], np.float32)
+    sc = torch.zeros(len(lens), device="cuda")
+    P.ops.prism_op_probe_encoder(dev(x), dev_i32(cu), len(lens), dev(g), dev(b), 1e-5, dev(dw, torch.bfloat16 if dtype == BF16 else torch.float32),
+                                 dtype, dev(db), dev(ow), dev(ob), sc)
+    w = {"head_dense_w": dw, "head_dense_b": db, "head_out_w": ow, "head_out_b": ob}
+    ref = [oracle.head_score(oracle.layernorm(x[cu[i]].astype(np.float64), g.astype(np.float64), b.astype(np.float64), 1e-5), w)
+           if lens[i] else 0.0 for i in range(len(lens))]
+    assert np.max(np.abs(sc.cpu().numpy() - np.array(ref))) < 2e-5
+
+
+# ------------------------------------------------------------------------------------------ end to end
+ENC_TINY = ModelCfg(n_layers=3, hidden=128, n_q_heads=4, n_kv_heads=4, head_dim=32, ffn=256, vocab=997, rope_theta=1.0,
+                    rms_eps=1e-5, causal=0, qk_norm=0, dtype=DTYPE_FP32, arch=ARCH_ENCODER, max_positions=130, pos_offset=2)
+ENC_TINY_WL = Workload("enc_tiny_fp32", ENC_TINY, 16, 3, 8, ("uniform", 8, 100, 8, 100),
+                       Schedule(MODE_FIXED_KEEP, (1, 2), (9, 5)), cfg_index=11)
+ENC_MID = ModelCfg(n_layers=5, hidden=1024, n_q_heads=16, n_kv_heads=16, head_dim=64, ffn=4096, vocab=4096, rope_theta=1.0,
+                   rms_eps=1e-5, causal=0, qk_norm=0, dtype=DTYPE_BF16, arch=ARCH_ENCODER, max_positions=514, pos_offset=2)
+ENC_MID_WL = Workload("enc_mid_bf16", ENC_MID, 24, 4, 16, ("uniform", 20, 300, 20, 300),
+                      Schedule(MODE_CLUSTER, (2, 4), cv_threshold=0.3), cfg_index=12)
+
+
+def make_model(P, cfg, w, req, **kw):
+    lens = np.diff(req["cand_offsets"]) + len(req["query"])
+    return P.PrismModel(cfg, P.upload_weights(w, cfg.dtype), int(lens.max()), len(lens), int(lens.sum()), **kw)
+
+
+def test_encoder_fp32_end_to_end(P):
+    wl, cfg = ENC_TINY_WL, ENC_TINY
+    w = synth.make_weights(cfg, seed=2)
+    req = synth.make_request(wl, 0)
+    S = oracle.score_matrix(req["query"], req["cand_tokens"], req["cand_offsets"], w, cfg, [1, 2, 3])
+    m = make_model(P, cfg, w, req)
+    for sched in (Schedule(MODE_NONE), wl.schedule, Schedule(MODE_CLUSTER, (1, 2), cv_threshold=0.05)):
+        idx, sc, tr = run(P, m, req, wl.top_k, sched)
+        assert check_scores(tr, S, TOL_FP32) < TOL_FP32
+        check_replay(tr, idx, sc, wl.n_candidates, wl.top_k, cfg.n_layers, sched)
+        check_end_to_end(tr, idx, S, wl.n_candidates, wl.top_k, cfg.n_layers, sched, TOL_FP32)
+    # unpruned: the plain definition (score all, sort, take K)
+    idx, sc, _ = run(P, m, req, wl.top_k, Schedule(MODE_NONE))
+    ref = oracle.oracle_select(req["query"], req["cand_tokens"], req["cand_offsets"], wl.top_k, w, cfg, Schedule(MODE_NONE), S=S)
+    assert list(idx) == ref.topk_idx
+    m.close()
+
+
+@pytest.mark.parametrize("gemm_impl,attn_impl", [(AUTO, AUTO), (SIMT, SIMT), (AUTO, SIMT), (SIMT, AUTO)])
+def test_encoder_bf16_paths_match_oracle(P, gemm_impl, attn_impl):
+    wl, cfg = ENC_MID_WL, ENC_MID
+    w = synth.make_weights(cfg, seed=5)
+    req = synth.make_request(wl, 0)
+    S = oracle.score_matrix(req["query"], req["cand_tokens"], req["cand_offsets"], w, cfg, [2, 4, 5])
+    m = make_model(P, cfg, w, req, gemm_impl=gemm_impl, attention_impl=attn_impl)
+    for sched in (Schedule(MODE_NONE), wl.schedule, replace(wl.schedule, select_winners=0)):
+        idx, sc, tr = run(P, m, req, wl.top_k, sched)
+        check_scores(tr, S, TOL_BF16)
+        check_replay(tr, idx, sc, wl.n_candidates, wl.top_k, cfg.n_layers, sched)
+        check_end_to_end(tr, idx, S, wl.n_candidates, wl.top_k, cfg.n_layers, sched, TOL_BF16)
+    assert tr.shared_prefix_rows == 0                      # bidirectional attention: the query rows depend on the document
+    m.close()
+
+
+def test_encoder_chunked_execution_is_result_neutral(P):
+    wl, cfg = ENC_MID_WL, ENC_MID
+    w = synth.make_weights(cfg, seed=5)
+    req = synth.make_request(wl, 1)
+    lens = np.diff(req["cand_offsets"]) + wl.query_len
+    total = int(lens.sum())
+    base = run(P, make_model(P, cfg, w, req), req, wl.top_k, wl.schedule)
+    per_tok = 2 * (cfg.hidden + 3 * cfg.hidden + cfg.hidden + cfg.ffn)
+    budget = 2 * total * cfg.hidden * 4 + (total // 4) * per_tok
+    got = run(P, make_model(P, cfg, w, req, activation_budget_bytes=budget), req, wl.top_k, wl.schedule)
+    assert got[2].n_chunks_max >= 3
+    assert np.array_equal(base[0], got[0]) and np.array_equal(base[1].view(np.uint32), got[1].view(np.uint32))
+    for r1, r2 in zip(base[2].records, got[2].records):
+        assert np.array_equal(r1.scores.view(np.uint32), r2.scores.view(np.uint32)) and r1.active_ids == r2.active_ids
+
+
+def test_encoder_rejects_what_it_does_not_support(P):
+    cfg = ENC_TINY
+    w = synth.make_weights(cfg, seed=2)
+    req = synth.make_request(ENC_TINY_WL, 0)
+    for kw in (dict(stream_weights=True), dict(hidden_offload=True, activation_budget_bytes=1 << 30)):
+        with pytest.raises(P.PrismError) as e:
+            make_model(P, cfg, w, req, **kw)
+        assert e.value.status == -8, e.value                 # PRISM_ERR_UNSUPPORTED
+    with pytest.raises(P.PrismError) as e:
+        make_model(P, replace(cfg, max_positions=20), w, req)       # positions would run past the table
+    assert e.value.status == -1
