@@ -359,7 +359,8 @@ def run_prism(args):
                 rows_total = per[n]["work_per_step"] / (2.0 * nn * kk)          # sum of M over the class's launches
                 tb += NCU_TRAFFIC_M8192[n] * rows_total / 8192.0
             traffic = tb / g_n
-        line["roofline"] = {"kernel": "k_gemm_tc2 (tcgen05 cta_group::2 projection GEMMs: qkv, o, gate/up, down)", "bound": "tensor",
+        gemm_names = "qkv, o, ffn1 + GELU, ffn2; all with bias" if getattr(cfg, "arch", 0) == 1 else "qkv, o, gate/up, down"
+        line["roofline"] = {"kernel": f"k_gemm_tc2 (tcgen05 cta_group::2 projection GEMMs: {gemm_names})", "bound": "tensor",
                             "achieved": ach, "peak": peak, "unit": "TFLOP/s", "frac": ach / peak if peak else None,
                             "peak_source": f"bf16_tflops_sustained of {peaks['source']} (kernel timed inside a long step)",
                             "frac_of_burst_peak": ach / peaks["bf16_tflops"],

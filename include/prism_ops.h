@@ -96,7 +96,7 @@ PRISM_API int prism_op_embed_encoder(const void* table, const void* pos_table, c
 
 /* Encoder score probe: for each sequence, LayerNorm (gain, shift, eps) of its FIRST row, then
  * out_w . tanh(dense_w y + dense_b) + out_b[0].  dense_w [d, d] in element type `dtype`, all vectors fp32.
- * A sequence without rows scores 0. */
+ * A sequence without rows scores 0.  d a multiple of 4.  Allocates and frees a temporary scratch of 2 n d floats. */
 PRISM_API int prism_op_probe_encoder(const float* x, const int32_t* cu, int32_t n, int32_t d, const float* gain, const float* shift,
                            float eps, const void* dense_w, int32_t dtype, const float* dense_b, const float* out_w,
                            const float* out_b, float* scores, void* stream);

@@ -137,9 +137,10 @@ cudaError_t launch_layernorm(float* x, const float* gain, const float* shift, in
                              void* out, cudaStream_t st, bool reverse = false);
 // Score of sequence i from its FIRST row: LayerNorm (gain, shift) of the row, then
 // out_w . tanh(dense_w y + dense_b) + out_b.  dense_w [d, d] has element type `dtype`, the vectors are fp32.
+// scratch: 2 * n * d floats.  Three launches.
 cudaError_t launch_probe_encoder(const float* x, const int* cu, int n, int d, const float* gain, const float* shift,
                                  float eps, const void* dense_w, int dtype, const float* dense_b, const float* out_w,
-                                 const float* out_b, float* scores, cudaStream_t st);
+                                 const float* out_b, float* scores, float* scratch, cudaStream_t st);
 // n values of element type `dtype` widened to fp32
 cudaError_t launch_to_f32(const void* src, int dtype, int n, float* dst, cudaStream_t st);
 cudaError_t launch_score_diff(const void* score_head, int dtype, int d, float* w_diff, cudaStream_t st);

@@ -327,19 +327,20 @@ __global__ void __launch_bounds__(256) k_layernorm(float* __restrict__ x, const 
 
 // Score probe of the encoder stack (Sec. 4.1: the model's own classifier on an intermediate hidden state): the
 // FIRST row of sequence i goes through the pending LayerNorm of the block it leaves, then
-// score = out_w . tanh(dense_w y + dense_b) + out_b.  One block per sequence; the normed row sits in shared
-// memory, every warp takes output units w, w + 8, ... with the lanes striding the row (coalesced weight reads).
-template <typename WT>
-__global__ void __launch_bounds__(256) k_probe_encoder(const float* __restrict__ x, const int* __restrict__ cu, int d,
-                                                       const float* __restrict__ gain, const float* __restrict__ shift,
-                                                       float eps, const WT* __restrict__ dense_w,
-                                                       const float* __restrict__ dense_b, const float* __restrict__ out_w,
-                                                       const float* __restrict__ out_b, float* __restrict__ scores) {
-  extern __shared__ float y[];  // [d]
+// score = out_w . tanh(dense_w y + dense_b) + out_b.  Three small kernels over a scratch of 2 n d floats, every
+// sum in a fixed order (the scores are the same bit for bit whatever the chunking or the launch geometry):
+//   norm   one block per sequence: y[i,:] = LayerNorm(first row)
+//   units  one WARP per output unit j of the dense map: its weight row stays in registers while the warp walks
+//          the sequences, t[i,j] = out_w[j] * tanh(w_j . y[i,:] + dense_b[j])
+//   sum    one block per sequence: score[i] = sum_j t[i,j] + out_b
+__global__ void __launch_bounds__(256) k_probe_enc_norm(const float* __restrict__ x, const int* __restrict__ cu, int d,
+                                                        const float* __restrict__ gain, const float* __restrict__ shift,
+                                                        float eps, float* __restrict__ y) {
   __shared__ float red[32];
   const int i = blockIdx.x;
+  float* yr = y + (size_t)i * d;
   if (cu[i + 1] == cu[i]) {  // a sequence without rows (another rank's candidate)
-    if (threadIdx.x == 0) scores[i] = 0.f;
+    for (int c = threadIdx.x; c < d; c += 256) yr[c] = 0.f;
     return;
   }
   const float* row = x + (size_t)cu[i] * d;
@@ -352,19 +353,67 @@ __global__ void __launch_bounds__(256) k_probe_encoder(const float* __restrict__
     sq += t * t;
   }
   const float r = 1.0f / sqrtf(block_sum(sq, red) / (float)d + eps);
-  for (int c = threadIdx.x; c < d; c += 256) y[c] = (row[c] - mean) * r * gain[c] + shift[c];
-  __syncthreads();
-  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-  float acc = 0.f;  // lane 0 of each warp: sum over its units of out_w[j] * tanh(...)
-  for (int j = w; j < d; j += 8) {
-    const WT* wr = dense_w + (size_t)j * d;
-    float dot = 0.f;
-    for (int c = lane; c < d; c += 32) dot = fmaf(to_f(wr[c]), y[c], dot);
-    dot = warp_sum(dot);
-    if (lane == 0) acc += out_w[j] * tanhf(dot + dense_b[j]);
+  for (int c = threadIdx.x; c < d; c += 256) yr[c] = (row[c] - mean) * r * gain[c] + shift[c];
+}
+
+// kPer > 0: d = 128 * kPer and the unit's weight row sits in registers (4 * kPer floats per lane);
+// kPer = 0: any d that is a multiple of 4, the row is re-read (from L1) for every sequence.
+template <typename WT, int kPer>
+__global__ void __launch_bounds__(256) k_probe_enc_units(const float* __restrict__ y, int n, int d,
+                                                         const WT* __restrict__ dense_w, const float* __restrict__ dense_b,
+                                                         const float* __restrict__ out_w, float* __restrict__ t) {
+  const int lane = threadIdx.x & 31;
+  const int j = blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (j >= d) return;
+  const WT* wr = dense_w + (size_t)j * d;
+  const float bj = dense_b[j], oj = out_w[j];
+  auto load4 = [&](int c) {  // weights c .. c + 3 of the row as floats
+    if constexpr (sizeof(WT) == 2) {
+      const uint2 raw = *reinterpret_cast<const uint2*>(wr + c);
+      const __nv_bfloat16* b = reinterpret_cast<const __nv_bfloat16*>(&raw);
+      return make_float4(to_f(b[0]), to_f(b[1]), to_f(b[2]), to_f(b[3]));
+    } else {
+      return *reinterpret_cast<const float4*>(wr + c);
+    }
+  };
+  float4 w[kPer > 0 ? kPer : 1];
+  if constexpr (kPer > 0) {
+#pragma unroll
+    for (int q = 0; q < kPer; ++q) w[q] = load4((lane + 32 * q) * 4);
   }
-  const float total = block_sum(lane == 0 ? acc : 0.f, red);
-  if (threadIdx.x == 0) scores[i] = total + out_b[0];
+  for (int i = 0; i < n; ++i) {
+    const float4* yr = reinterpret_cast<const float4*>(y + (size_t)i * d);
+    float dot = 0.f;
+    if constexpr (kPer > 0) {
+#pragma unroll
+      for (int q = 0; q < kPer; ++q) {
+        const float4 v = yr[lane + 32 * q];
+        dot = fmaf(w[q].x, v.x, fmaf(w[q].y, v.y, fmaf(w[q].z, v.z, fmaf(w[q].w, v.w, dot))));
+      }
+    } else {
+      for (int c = lane; c < (d >> 2); c += 32) {
+        const float4 v = yr[c], ww = load4(c * 4);
+        dot = fmaf(ww.x, v.x, fmaf(ww.y, v.y, fmaf(ww.z, v.z, fmaf(ww.w, v.w, dot))));
+      }
+    }
+    dot = warp_sum(dot);
+    if (lane == 0) t[(size_t)i * d + j] = oj * tanhf(dot + bj);
+  }
+}
+
+__global__ void __launch_bounds__(256) k_probe_enc_sum(const float* __restrict__ t, const int* __restrict__ cu, int d,
+                                                       const float* __restrict__ out_b, float* __restrict__ scores) {
+  __shared__ float red[32];
+  const int i = blockIdx.x;
+  if (cu[i + 1] == cu[i]) {
+    if (threadIdx.x == 0) scores[i] = 0.f;
+    return;
+  }
+  const float* tr = t + (size_t)i * d;
+  float s = 0.f;
+  for (int c = threadIdx.x; c < d; c += 256) s += tr[c];
+  s = block_sum(s, red);
+  if (threadIdx.x == 0) scores[i] = s + out_b[0];
 }
 
 template <typename WT>
@@ -654,15 +703,24 @@ cudaError_t launch_layernorm(float* x, const float* gain, const float* shift, in
 
 cudaError_t launch_probe_encoder(const float* x, const int* cu, int n, int d, const float* gain, const float* shift,
                                  float eps, const void* dense_w, int dtype, const float* dense_b, const float* out_w,
-                                 const float* out_b, float* scores, cudaStream_t st) {
+                                 const float* out_b, float* scores, float* scratch, cudaStream_t st) {
   if (n <= 0) return cudaSuccess;
-  const size_t smem = (size_t)d * sizeof(float);
-  if (dtype == 1)
-    k_probe_encoder<__nv_bfloat16><<<n, 256, smem, st>>>(x, cu, d, gain, shift, eps, (const __nv_bfloat16*)dense_w, dense_b,
-                                                         out_w, out_b, scores);
-  else
-    k_probe_encoder<float><<<n, 256, smem, st>>>(x, cu, d, gain, shift, eps, (const float*)dense_w, dense_b, out_w, out_b,
-                                                 scores);
+  if (d & 3) return cudaErrorInvalidValue;
+  float *y = scratch, *t = scratch + (size_t)n * d;
+  k_probe_enc_norm<<<n, 256, 0, st>>>(x, cu, d, gain, shift, eps, y);
+  const int grid = (d + 7) / 8;
+#define PRISM_UNITS(WT, P) k_probe_enc_units<WT, P><<<grid, 256, 0, st>>>(y, n, d, (const WT*)dense_w, dense_b, out_w, t)
+  if (dtype == 1) {
+    if (d == 1024) PRISM_UNITS(__nv_bfloat16, 8);
+    else if (d == 768) PRISM_UNITS(__nv_bfloat16, 6);
+    else if (d == 2048) PRISM_UNITS(__nv_bfloat16, 16);
+    else PRISM_UNITS(__nv_bfloat16, 0);
+  } else {
+    if (d == 1024) PRISM_UNITS(float, 8);
+    else PRISM_UNITS(float, 0);
+  }
+#undef PRISM_UNITS
+  k_probe_enc_sum<<<n, 256, 0, st>>>(t, cu, d, out_b, scores);
   return cudaGetLastError();
 }
 

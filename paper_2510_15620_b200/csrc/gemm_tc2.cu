@@ -83,6 +83,22 @@ __device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
                ::"r"(bar), "h"((uint16_t)3) : "memory");
 }
 
+// gelu(x) = x Phi(x) without a branch: Phi from the rational-times-Gaussian form of erfc (Abramowitz & Stegun
+// 7.1.26, absolute error below 1.5e-7, far under the bf16 rounding of the result), two special-function
+// operations and a handful of FMAs per element, so that the epilogue keeps up with the MMAs.
+__device__ __forceinline__ float gelu_fast(float x) {
+  const float z = fabsf(x) * 0.70710678118654752f;
+  const float t = __fdividef(1.f, fmaf(0.3275911f, z, 1.f));
+  float p = fmaf(1.061405429f, t, -1.453152027f);
+  p = fmaf(p, t, 1.421413741f);
+  p = fmaf(p, t, -0.284496736f);
+  p = fmaf(p, t, 0.254829592f);
+  float e;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(-1.4426950408889634f * z * z));
+  const float tail = 0.5f * p * t * e;           // 0.5 erfc(|x| / sqrt 2) = Phi(-|x|)
+  return x * (x >= 0.f ? 1.f - tail : tail);
+}
+
 // kind::f16 instruction descriptor: D fp32, A/B bf16, both K-major, M=128, N=256.
 constexpr uint32_t kIdesc = idesc_bf16(2 * BM, BN, 0);  // the pair's instruction: M = 256
 
@@ -463,7 +479,7 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
                             __uint_as_float(r[4 * v + 2]) + bv.z, __uint_as_float(r[4 * v + 3]) + bv.w};
               if constexpr (kEpi == kEpiGeluBias) {
 #pragma unroll
-                for (int e = 0; e < 4; ++e) y[e] = 0.5f * y[e] * (1.f + erff(y[e] * 0.70710678118654752f));
+                for (int e = 0; e < 4; ++e) y[e] = gelu_fast(y[e]);
               }
 #pragma unroll
               for (int e = 0; e < 4; ++e) r[4 * v + e] = __float_as_uint(y[e]);

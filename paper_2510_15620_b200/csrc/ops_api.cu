@@ -111,7 +111,15 @@ int prism_op_probe_encoder(const float* x, const int32_t* cu, int32_t n, int32_t
                            const float* out_b, float* scores, void* stream) {
   if (!x || !cu || !gain || !shift || !dense_w || !dense_b || !out_w || !out_b || !scores || n < 0 || d < 1 || d > 8192)
     return PRISM_ERR_INVALID_ARG;
-  return st_of(launch_probe_encoder(x, cu, n, d, gain, shift, eps, dense_w, dtype, dense_b, out_w, out_b, scores, S(stream)));
+  if (n == 0) return PRISM_OK;
+  if (d % 4) return PRISM_ERR_INVALID_ARG;
+  float* scratch = nullptr;
+  cudaError_t e = cudaMalloc(&scratch, 2 * (size_t)n * d * sizeof(float));
+  if (e != cudaSuccess) return st_of(e);
+  e = launch_probe_encoder(x, cu, n, d, gain, shift, eps, dense_w, dtype, dense_b, out_w, out_b, scores, scratch, S(stream));
+  cudaStreamSynchronize(S(stream));
+  cudaFree(scratch);
+  return st_of(e);
 }
 
 int prism_op_gemm_qkv_rope(const void* a, const void* w_qkv, void* out, int32_t m, int32_t k, int32_t n_q_heads,

@@ -42,6 +42,7 @@ struct prism_handle {
   std::vector<prism_encoder_layer_weights> enc_layers;
   std::vector<EncVec> enc_vec;
   const void *pos_embed = nullptr, *head_dense_w = nullptr;
+  float* probe_scratch = nullptr;  // [2, max_candidates, D]
   const float *type_f = nullptr, *emb_g = nullptr, *emb_b = nullptr, *head_db = nullptr, *head_ow = nullptr, *head_ob = nullptr;
   int esz = 4;
   int chunk_tokens = 0;
@@ -591,6 +592,7 @@ static int create_impl(prism_handle* h, const prism_model_cfg* cfg, const prism_
     PRISM_CUDA(h, widen(ew->head_dense_b, D, &h->head_db));
     PRISM_CUDA(h, widen(ew->head_out_w, D, &h->head_ow));
     PRISM_CUDA(h, widen(ew->head_out_b, 1, &h->head_ob));
+    PRISM_CUDA(h, dev_alloc(h, &h->probe_scratch, 2 * N * D));
     h->enc_vec.resize(c.n_layers);
     for (int l = 0; l < c.n_layers; ++l) {
       const prism_encoder_layer_weights& lw = h->enc_layers[l];
@@ -1097,7 +1099,8 @@ int select_impl(prism_handle* h, const int32_t* query, int32_t lq, const int32_t
         const EncVec& V = h->enc_vec[layers_run - 1];  // the last executed block's LN2 is still pending
         PRISM_LAUNCH_P(h, st, PRISM_K_PROBE, (double)n * c.hidden * (4.0 + (double)c.hidden * h->esz),
                        launch_probe_encoder(h->x[cur], h->cu[cur], n, c.hidden, V.ln2_g, V.ln2_b, c.rms_eps, h->head_dense_w,
-                                            c.dtype, h->head_db, h->head_ow, h->head_ob, score_buf, st));
+                                            c.dtype, h->head_db, h->head_ow, h->head_ob, score_buf, h->probe_scratch, st));
+        h->launches += 2;  // the probe is three kernels
       } else
       PRISM_LAUNCH_P(h, st, PRISM_K_PROBE, 4.0 * n * c.hidden,
                      launch_probe(h->x[cur], h->cu[cur], n, c.hidden, h->g_final, c.dtype, h->w_diff, c.rms_eps, score_buf, st, prefix));

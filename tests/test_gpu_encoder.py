@@ -135,14 +135,16 @@ def test_attention_head_dim_64(P, impl, hq, hkv, causal):
 
 
 @pytest.mark.parametrize("dtype", [FP32, BF16])
-def test_probe_encoder(P, dtype):
+@pytest.mark.parametrize("d", [256, 768, 1024, 2048])
+def test_probe_encoder(P, dtype, d):
+    """Widths whose weight row sits in registers (768, 1024, 2048 in bf16; 1024 in fp32) and the generic path."""
     rng = np.random.default_rng(9)
-    d, lens = 256, np.array([5, 1, 40, 0, 17])
+    lens = np.array([5, 1, 40, 0, 17])
     cu = np.zeros(len(lens) + 1, np.int32)
     cu[1:] = np.cumsum(lens)
     x = rng.normal(size=(int(cu[-1]), d)).astype(np.float32)
     g, b = (1 + 0.1 * rng.normal(size=d)).astype(np.float32), (0.1 * rng.normal(size=d)).astype(np.float32)
-    dw = (rng.normal(size=(d, d)) * 0.08).astype(np.float32)
+    dw = (rng.normal(size=(d, d)) * (1.3 / np.sqrt(d))).astype(np.float32)
     if dtype == BF16:
         dw = round_to_bf16(dw)
     db, ow, ob = rng.normal(size=d).astype(np.float32) * 0.1, rng.normal(size=d).astype(np.float32) * 0.1, np.array([0.3], np.float32)
