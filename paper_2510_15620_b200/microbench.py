@@ -4,6 +4,9 @@ synthetic operands, one JSON line per run.  Also the small-case driver for profi
     python -m paper_2510_15620_b200.microbench --op gemm --m 35200 --n 4096 --k 1024 --epilogue 0
     python -m paper_2510_15620_b200.microbench --op attention --seqs 100 --len-lo 160 --len-hi 544
     python -m paper_2510_15620_b200.microbench --op rmsnorm|rope|compact --rows 35200 --d 1024
+    python -m paper_2510_15620_b200.microbench --op gemm_bias --m 35200 --n 4096 --k 1024 --epilogue 2   (encoder stack)
+    python -m paper_2510_15620_b200.microbench --op layernorm --rows 35200 --d 1024
+    python -m paper_2510_15620_b200.microbench --op attention --head-dim 64 --hq 16 --hkv 16 --causal 0
 """
 from __future__ import annotations
 
@@ -36,7 +39,8 @@ def _time(fn, iters, warmup, flush):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--op", required=True, choices=["gemm", "qkv_rope", "attention", "rmsnorm", "rope", "compact"])
+    ap.add_argument("--op", required=True, choices=["gemm", "qkv_rope", "attention", "rmsnorm", "rope", "compact", "gemm_bias", "layernorm"])
+    ap.add_argument("--head-dim", type=int, default=128)
     ap.add_argument("--m", type=int, default=35200)
     ap.add_argument("--n", type=int, default=4096)
     ap.add_argument("--k", type=int, default=1024)
@@ -72,6 +76,25 @@ def main():
         med, best = _time(fn, a.iters, a.warmup, flush)
         fl = 2.0 * m * n * k * (2 if a.epilogue == 2 else 1)
         out.update(m=m, n=n, k=k, epilogue=a.epilogue, ms=med, ms_min=best, tflops=fl / med / 1e9, err=int(err.item()))
+    elif a.op == "gemm_bias":
+        m, n, k = a.m, a.n, a.k
+        A = rnd(m, k).to(torch.bfloat16)
+        B = (rnd(n, k) * 0.05).to(torch.bfloat16)
+        bias = rnd(n)
+        O = torch.empty(m, n, dtype=torch.bfloat16, device=dev)
+        R = rnd(m, n)
+        err = torch.zeros(1, dtype=torch.int32, device=dev)
+        fn = lambda: ops.prism_op_gemm_bias(A, B, bias, O, R, m, n, k, PRISM_BF16, a.epilogue, a.impl, err)
+        med, best = _time(fn, a.iters, a.warmup, flush)
+        out.update(m=m, n=n, k=k, epilogue=a.epilogue, ms=med, ms_min=best, tflops=2.0 * m * n * k / med / 1e9, err=int(err.item()))
+    elif a.op == "layernorm":
+        x = rnd(a.rows, a.d)
+        gain, shift = torch.ones(a.d, device=dev), torch.zeros(a.d, device=dev)
+        o = torch.empty(a.rows, a.d, dtype=torch.bfloat16, device=dev)
+        fn = lambda: ops.prism_op_layernorm(x, gain, shift, PRISM_BF16, 1e-5, o)
+        med, best = _time(fn, a.iters, a.warmup, flush)
+        out.update(rows=a.rows, d=a.d, ms=med, ms_min=best, gbs=a.rows * a.d * 10.0 / med / 1e6,
+                   bytes_per_element="4 read + 4 written in place + 2 for the bf16 copy")
     elif a.op == "qkv_rope":
         m, k = a.m, a.k
         n = (a.hq + 2 * a.hkv) * 128
@@ -89,7 +112,7 @@ def main():
         lens = rng.integers(a.len_lo, a.len_hi + 1, size=a.seqs)
         cu = np.zeros(a.seqs + 1, np.int32)
         cu[1:] = np.cumsum(lens)
-        dh = 128
+        dh = a.head_dim
         qkv = rnd(int(cu[-1]), (a.hq + 2 * a.hkv) * dh).to(torch.bfloat16)
         o = torch.empty(int(cu[-1]), a.hq * dh, dtype=torch.bfloat16, device=dev)
         cud = torch.from_numpy(cu).to(dev)
@@ -97,7 +120,7 @@ def main():
         fn = lambda: ops.prism_op_attention(qkv, o, cud, a.seqs, int(lens.max()), a.hq, a.hkv, dh, a.causal, PRISM_BF16, a.impl, err)
         med, best = _time(fn, a.iters, a.warmup, flush)
         fl = float(np.sum((2.0 if a.causal else 4.0) * lens.astype(np.float64) ** 2 * a.hq * dh))
-        out.update(seqs=a.seqs, tokens=int(cu[-1]), causal=a.causal, ms=med, ms_min=best, tflops=fl / med / 1e9)
+        out.update(seqs=a.seqs, tokens=int(cu[-1]), causal=a.causal, head_dim=dh, ms=med, ms_min=best, tflops=fl / med / 1e9)
     elif a.op == "rmsnorm":
         x = rnd(a.rows, a.d)
         gain = torch.ones(a.d, dtype=torch.bfloat16, device=dev)
