@@ -11,6 +11,7 @@ from .reranker import (rmsnorm, rope_rotate, attention, layer_forward,  # noqa: 
                        candidate_scores, score_matrix)
 from .encoder import (layernorm, gelu, embed_tokens, encoder_layer_forward, head_score,  # noqa: F401
                       encoder_candidate_scores, encoder_score_matrix)
+from .quant import unpack_w4, dequantize_w4, dequantize_weights  # noqa: F401
 from .prune_rule import (coefficient_of_variation, rank_order, optimal_partition,  # noqa: F401
                          route_clusters, replay_select, MODE_NONE, MODE_FIXED_KEEP, MODE_CLUSTER)
 from .select import oracle_select  # noqa: F401

@@ -9,3 +9,4 @@ compute code.
 from .configs import ModelCfg, Schedule, Workload, WORKLOADS, workload  # noqa: F401
 from .weights import make_weights, round_to_bf16, bf16_bits  # noqa: F401
 from .requests import make_request  # noqa: F401
+from .quant import quantize_weights, quantize_matrix, pack_matrix, packed_sections  # noqa: F401
