@@ -29,7 +29,7 @@ if ROOT not in sys.path:
 METRIC = "candidate-tokens/s (p50/p99 top-K select latency in ms beside it)"
 UNIT = "candidate-tokens/s"
 KERNEL_CLASSES = ["pack", "embed", "rmsnorm", "gemm_qkv", "rope", "attention", "gemm_o", "gemm_gateup", "gemm_down",
-                  "probe", "route", "compact"]
+                  "probe", "route", "compact", "dequant"]
 GEMM_CLASSES = ("gemm_qkv", "gemm_o", "gemm_gateup", "gemm_down")
 # dram__bytes_read.sum + dram__bytes_write.sum of one k_gemm_tc2 launch at M = 8192 with the cfg1 weight
 # shapes, from the ncu captures summarised under profiles/gemm_tc2_*.md.
@@ -221,9 +221,13 @@ def run_prism(args):
         max_tot = int(max(l[o != 0].sum() for l, o in zip(lens_all, owned))) or 1
     reduce = (lambda t: P.all_reduce_scores(t)) if (by_cand and world > 1) else (lambda t: None)
     w_np = synth.make_weights(cfg, wl.weight_seed)
+    w4 = args.weight_format == "w4"
+    if w4:  # Sec. 6.1's quantised arm: 4-bit codes + bf16 scale and 4-bit zero point per 128 input channels
+        w_np = synth.quantize_weights(w_np, 128)
     tw = P.upload_weights(w_np, cfg.dtype, device=str(dev), layers_pinned_host=bool(wl.stream_weights))
     model = P.PrismModel(cfg, tw, max_seq, wl.n_candidates, max_tot, activation_budget_bytes=wl.activation_budget_bytes,
-                         stream_weights=bool(wl.stream_weights), shared_prefix=args.shared_prefix == "on")
+                         stream_weights=bool(wl.stream_weights), shared_prefix=args.shared_prefix == "on",
+                         weight_format=P.PRISM_WFMT_W4 if w4 else P.PRISM_WFMT_PLAIN, quant_group=128 if w4 else 0)
     d = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(dev)
     dreqs = [(d(r["query"]), d(r["cand_tokens"]), d(r["cand_offsets"])) for r in reqs]
     pin = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).pin_memory().numpy()
@@ -308,6 +312,7 @@ def run_prism(args):
                        "tokens_per_request": int(np.mean([l.sum() for l in lens_all])),
                        # causal attention: the query's rows are computed once per request instead of once per
                        # candidate (same scores bit for bit); the metric keeps counting query + document per candidate
+                       "weight_format": "w4a16 (round-to-nearest, group 128)" if w4 else "bf16" if cfg.dtype == 1 else "f32",
                        "shared_query_prefix_rows": prefix_rows,
                        "rows_computed_first_layer": int(np.mean([l.sum() - (len(l) - 1) * prefix_rows for l in lens_all])),
                        "schedule": {"mode": sched.mode, "probe_layers": list(sched.probe_layers),
@@ -376,7 +381,7 @@ def run_prism(args):
                                    (v["work_per_step"] / (v["ms_per_step"] * 1e-3) / (1e12 if n in GEMM_CLASSES or n == "attention" else 1e9)
                                     if v["ms_per_step"] > 0 else 0.0)}
                            for n, v in per.items()}
-        if not args.no_cpu_baseline:
+        if not args.no_cpu_baseline and not w4:   # the oracle leg times the unquantised model
             ids = oracle_sample_ids(wl, reqs[0], max_cand=8)
             n_c = len(ids)
             rate, dt, t = oracle_sample_rate(wl, w_np, reqs[0], ids)
@@ -404,6 +409,9 @@ def main():
     ap.add_argument("--shared-prefix", default="on", choices=["on", "off"],
                     help="on: the query's rows are stored and computed once per request where the path supports it "
                          "(causal attention; results are bit-identical); off: one query copy per candidate")
+    ap.add_argument("--weight-format", default="plain", choices=["plain", "w4"],
+                    help="w4: the layer matrices are stored (and, for the streamed workload, copied) as 4-bit codes and "
+                         "rebuilt as bf16 layer by layer on the device")
     ap.add_argument("--shard", default="requests", choices=["requests", "candidates"],
                     help="requests: every rank serves its own requests (weak scaling, the default); candidates: all "
                          "ranks share each request, one score all-reduce per probe (strong scaling)")

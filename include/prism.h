@@ -60,6 +60,20 @@ enum { PRISM_PRUNE_NONE = 0, PRISM_PRUNE_FIXED_KEEP = 1, PRISM_PRUNE_CLUSTER = 2
  * 128x256 tiles. */
 enum { PRISM_IMPL_AUTO = 0, PRISM_IMPL_SIMT = 1, PRISM_IMPL_MMA = 2, PRISM_IMPL_SOLO = 3 };
 
+/* weight_format of prism_model_cfg.  PLAIN: matrices in the element type of cfg.dtype.  W4: the quantised arm of
+ * the paper's evaluation (Sec. 6.1: the method composed with 4-bit weight-only quantisation, 16-bit activations).
+ * The five matrices of every layer (w_qkv, w_o, w_gate, w_up, w_down) are packed blobs; for an [N, K] matrix and
+ * group size G = quant_group, every section starting on a 16-byte boundary:
+ *     codes   N*K/2 bytes, row-major; byte (n, k/2) holds code(n,k) in its low nibble for even k, high nibble for odd k
+ *     scales  N*K/G bf16, row-major [N, K/G]
+ *     zeros   N*K/G bytes (0..15), row-major
+ *     value(n,k) = bf16( float(scale[n,k/G]) * (code(n,k) - zero[n,k/G]) )
+ * Before a layer runs, its matrices are rebuilt as bf16 into one layer-sized device scratch and the usual GEMMs read
+ * that; with PRISM_WEIGHTS_HOST_STREAMED the PACKED layer crosses the host link (a quarter of the bytes).  Results
+ * equal those of a PLAIN handle given the dequantised matrices, bit for bit.  Norm gains, embedding and score head
+ * stay plain. */
+enum { PRISM_WFMT_PLAIN = 0, PRISM_WFMT_W4 = 1 };
+
 /* arch of prism_model_cfg.  DECODER: the pre-norm blocks described at prism_model_cfg, created by prism_create.
  * ENCODER: the encoder-only reranker the paper evaluates next to them (BGE-M3's, an XLM-RoBERTa stack; Sec. 6.1,
  * Table 1), created by prism_create_encoder: token + learned position + token-type embedding, LayerNorm, then
@@ -129,6 +143,9 @@ typedef struct {
                       SIMT, attention_impl AUTO, SOLO or SIMT. */
   int32_t max_positions;    /* encoder: rows of the learned position table; max_seq_len + pos_offset <= max_positions */
   int32_t pos_offset;       /* encoder: token p of a sequence reads position row p + pos_offset (2 for XLM-RoBERTa) */
+  int32_t weight_format;    /* PRISM_WFMT_*; W4 needs dtype PRISM_BF16 and arch PRISM_ARCH_DECODER */
+  int32_t quant_group;      /* W4: input channels per scale / zero point: 32, 64 or 128, dividing hidden, ffn and
+                               n_q_heads * head_dim */
 } prism_model_cfg;
 
 typedef struct {
@@ -355,6 +372,7 @@ PRISM_API int64_t prism_launch_count(const prism_handle* h);
 enum {
   PRISM_K_PACK = 0, PRISM_K_EMBED, PRISM_K_RMSNORM, PRISM_K_GEMM_QKV, PRISM_K_ROPE, PRISM_K_ATTENTION,
   PRISM_K_GEMM_O, PRISM_K_GEMM_GATEUP, PRISM_K_GEMM_DOWN, PRISM_K_PROBE, PRISM_K_ROUTE, PRISM_K_COMPACT,
+  PRISM_K_DEQUANT, /* W4 -> bf16 of a layer's matrices (weight_format PRISM_WFMT_W4) */
   PRISM_N_KERNEL_CLASSES
 };
 typedef struct {

@@ -101,6 +101,11 @@ PRISM_API int prism_op_probe_encoder(const float* x, const int32_t* cu, int32_t 
                            float eps, const void* dense_w, int32_t dtype, const float* dense_b, const float* out_w,
                            const float* out_b, float* scores, void* stream);
 
+/* W4 -> bf16 (PRISM_WFMT_W4 in prism.h gives the packed layout): out[n, k] bf16 from the packed blob of an [n, k]
+ * matrix with `group` input channels per scale / zero point (group a multiple of 32, k a multiple of group; blob and
+ * out device pointers, 16-byte aligned). */
+PRISM_API int prism_op_dequant_w4(const void* blob, int32_t n, int32_t k, int32_t group, void* out, void* stream);
+
 /* Score probe (Sec. 4.1: the model's classifier on an intermediate hidden state): for each sequence,
  * final RMSNorm of its last row, then logit(score_head row 0) - logit(score_head row 1).
  * Allocates and frees a temporary [d] float vector. */

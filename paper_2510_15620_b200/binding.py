@@ -12,6 +12,7 @@ import torch
 PRISM_FP32, PRISM_BF16 = 0, 1
 PRISM_IMPL_AUTO, PRISM_IMPL_SIMT, PRISM_IMPL_MMA, PRISM_IMPL_SOLO = 0, 1, 2, 3
 PRISM_ARCH_DECODER, PRISM_ARCH_ENCODER = 0, 1
+PRISM_WFMT_PLAIN, PRISM_WFMT_W4 = 0, 1
 PRISM_MAX_CLUSTERS = 8
 
 # PRISM_LIBRARY overrides the in-tree library (e.g. an instrumented build of the same sources).
@@ -57,7 +58,7 @@ class _ModelCfg(C.Structure):
                 ("activation_budget_bytes", C.c_int64), ("weight_residency", C.c_int32), ("gemm_impl", C.c_int32),
                 ("attention_impl", C.c_int32), ("embed_cache_rows", C.c_int32), ("hidden_offload", C.c_int32),
                 ("shared_prefix", C.c_int32), ("arch", C.c_int32), ("max_positions", C.c_int32),
-                ("pos_offset", C.c_int32)]
+                ("pos_offset", C.c_int32), ("weight_format", C.c_int32), ("quant_group", C.c_int32)]
 
 
 class _LayerWeights(C.Structure):
@@ -180,6 +181,9 @@ def upload_weights(w: Dict[str, object], dtype: int, device: str = "cuda", layer
     bf16 mode) -> torch tensors of the library's element type.  Layer tensors go to pinned host memory
     when they are to be streamed, the embedding table when it is to be cached row by row."""
     def conv(a: np.ndarray, pinned: bool) -> torch.Tensor:
+        if a.dtype == np.uint8:             # a packed W4 matrix: bytes as they are
+            t = torch.from_numpy(np.ascontiguousarray(a))
+            return t.pin_memory() if pinned else t.to(device)
         t = torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32))
         if dtype == PRISM_BF16:
             t = t.to(torch.bfloat16)        # exact: the values are bf16-representable
@@ -197,7 +201,7 @@ class PrismModel:
     def __init__(self, cfg, weights: Dict[str, object], max_seq_len: int, max_candidates: int, max_total_tokens: int,
                  activation_budget_bytes: int = 0, stream_weights: bool = False, gemm_impl: int = PRISM_IMPL_AUTO,
                  attention_impl: int = PRISM_IMPL_AUTO, embed_cache_rows: int = 0, hidden_offload: bool = False,
-                 shared_prefix: bool = True):
+                 shared_prefix: bool = True, weight_format: int = 0, quant_group: int = 0):
         self._h = C.c_void_p()
         self.cfg = cfg
         self._weights = weights            # keep the tensors alive for the life of the handle
@@ -205,7 +209,8 @@ class PrismModel:
                       cfg.rope_theta, cfg.rms_eps, cfg.causal, cfg.qk_norm, cfg.dtype, max_seq_len, max_candidates,
                       max_total_tokens, activation_budget_bytes, 1 if stream_weights else 0, gemm_impl, attention_impl,
                       embed_cache_rows, 1 if hidden_offload else 0, 0 if shared_prefix else 1,
-                      getattr(cfg, "arch", 0), getattr(cfg, "max_positions", 0), getattr(cfg, "pos_offset", 0))
+                      getattr(cfg, "arch", 0), getattr(cfg, "max_positions", 0), getattr(cfg, "pos_offset", 0),
+                      weight_format, quant_group)
         if getattr(cfg, "arch", 0) == PRISM_ARCH_ENCODER:
             elayers = (_EncLayerWeights * cfg.n_layers)()
             for i, lw in enumerate(weights["layers"]):

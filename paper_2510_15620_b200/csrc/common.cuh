@@ -141,6 +141,16 @@ cudaError_t launch_layernorm(float* x, const float* gain, const float* shift, in
 cudaError_t launch_probe_encoder(const float* x, const int* cu, int n, int d, const float* gain, const float* shift,
                                  float eps, const void* dense_w, int dtype, const float* dense_b, const float* out_w,
                                  const float* out_b, float* scores, float* scratch, cudaStream_t st);
+// W4 weights: bytes of the packed blob of an [n, k] matrix, and the offsets of its scale and zero-point sections.
+inline size_t w4_align16(size_t v) { return (v + 15) / 16 * 16; }
+inline size_t w4_scales_offset(size_t n, size_t k) { return w4_align16(n * k / 2); }
+inline size_t w4_zeros_offset(size_t n, size_t k, size_t group) { return w4_align16(w4_scales_offset(n, k) + 2 * n * (k / group)); }
+inline size_t w4_blob_bytes(size_t n, size_t k, size_t group) { return w4_align16(w4_zeros_offset(n, k, group) + n * (k / group)); }
+// out[n, k] bf16 = scale * (code - zero) per group of `group` input channels
+cudaError_t launch_dequant_w4(const void* blob, int n, int k, int group, void* out, cudaStream_t st);
+// the same for up to five matrices in one launch (a layer)
+cudaError_t launch_dequant_w4_batch(const void* const* blobs, const int* n, const int* k, void* const* outs, int count,
+                                    int group, cudaStream_t st);
 // n values of element type `dtype` widened to fp32
 cudaError_t launch_to_f32(const void* src, int dtype, int n, float* dst, cudaStream_t st);
 cudaError_t launch_score_diff(const void* score_head, int dtype, int d, float* w_diff, cudaStream_t st);

@@ -416,6 +416,68 @@ __global__ void __launch_bounds__(256) k_probe_enc_sum(const float* __restrict__
   if (threadIdx.x == 0) scores[i] = s + out_b[0];
 }
 
+// W4A16 (Sec. 6.1, the quantised arm): rebuild a packed [n, k] matrix as bf16.  One thread per 8 consecutive
+// input channels of a row: 4 code bytes in, 16 bytes out; value = bf16(float(scale) * (code - zero)), the product
+// being exact in fp32.  HBM-bound: 0.53 bytes read and 2 written per weight.
+// Up to five matrices (one layer) per launch: blockIdx.y selects the matrix, the blocks of a matrix stride over its
+// 32-weight pieces (16 code bytes in, 64 bytes out, one scale and zero point: groups are multiples of 32 channels
+// and rows of 32 weights, so a piece never straddles a group); two independent pieces per thread in flight.
+struct W4Batch {
+  const unsigned char* blob[5];
+  __nv_bfloat16* out[5];
+  int n[5], k[5];
+  int count, group;
+};
+
+__global__ void __launch_bounds__(256) k_dequant_w4(const W4Batch b) {
+  const int mi = blockIdx.y;
+  const int k = b.k[mi], group = b.group;
+  const unsigned k32 = (unsigned)k >> 5, ng = (unsigned)(k / group), g32 = (unsigned)group >> 5;
+  const size_t n = (size_t)b.n[mi];
+  const unsigned n_pc = (unsigned)(n * k32);  // < 2^31 for every supported shape (checked by the launcher)
+  const unsigned char* codes = b.blob[mi];
+  const size_t off_s = (n * k / 2 + 15) / 16 * 16, off_z = (off_s + 2 * n * ng + 15) / 16 * 16;
+  const __nv_bfloat16* scales = reinterpret_cast<const __nv_bfloat16*>(codes + off_s);
+  const unsigned char* zeros = codes + off_z;
+  const uint4* code_words = reinterpret_cast<const uint4*>(codes);  // piece p = 16-byte word p (rows are k/2 bytes)
+  uint4* out = reinterpret_cast<uint4*>(b.out[mi]);                 // piece p = 16-byte words 4p .. 4p+3 of the output
+  constexpr int kU = 2;
+  const unsigned stride = gridDim.x * 256u;
+  for (unsigned base = blockIdx.x * 256u + threadIdx.x; base < n_pc; base += stride * kU) {
+    uint4 c[kU];
+    float sc[kU];
+    int z[kU];
+#pragma unroll
+    for (int u = 0; u < kU; ++u) {
+      const unsigned p = base + u * stride;
+      if (p < n_pc) {
+        const unsigned row = p / k32, g = row * ng + (p - row * k32) / g32;
+        c[u] = __ldg(code_words + p);
+        sc[u] = __bfloat162float(scales[g]);
+        z[u] = zeros[g];
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < kU; ++u) {
+      const unsigned p = base + u * stride;
+      if (p < n_pc) {
+        const uint32_t w[4] = {c[u].x, c[u].y, c[u].z, c[u].w};
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {  // 4 code bytes = 8 weights = one 16-byte store
+          uint32_t pk[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const int lo = (int)((w[q] >> (8 * e)) & 15u) - z[u], hi = (int)((w[q] >> (8 * e + 4)) & 15u) - z[u];  // even k, odd k
+            const __nv_bfloat162 v = __floats2bfloat162_rn(sc[u] * (float)lo, sc[u] * (float)hi);
+            pk[e] = *reinterpret_cast<const uint32_t*>(&v);
+          }
+          out[(size_t)p * 4 + q] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+        }
+      }
+    }
+  }
+}
+
 template <typename WT>
 __global__ void k_to_f32(const WT* __restrict__ src, int n, float* __restrict__ dst) {
   for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) dst[i] = to_f(src[i]);
@@ -722,6 +784,33 @@ cudaError_t launch_probe_encoder(const float* x, const int* cu, int n, int d, co
 #undef PRISM_UNITS
   k_probe_enc_sum<<<n, 256, 0, st>>>(t, cu, d, out_b, scores);
   return cudaGetLastError();
+}
+
+cudaError_t launch_dequant_w4_batch(const void* const* blobs, const int* n, const int* k, void* const* outs, int count,
+                                    int group, cudaStream_t st) {
+  if (count < 1 || count > 5 || group <= 0 || (group & 31)) return cudaErrorInvalidValue;
+  W4Batch b{};
+  b.count = count;
+  b.group = group;
+  long long most = 0;
+  for (int i = 0; i < count; ++i) {
+    const long long oct = (long long)n[i] * (k[i] >> 5);
+    if (n[i] <= 0 || k[i] <= 0 || (k[i] % group) || oct >= (1ll << 31)) return cudaErrorInvalidValue;
+    b.blob[i] = static_cast<const unsigned char*>(blobs[i]);
+    b.out[i] = static_cast<__nv_bfloat16*>(outs[i]);
+    b.n[i] = n[i];
+    b.k[i] = k[i];
+    most = oct > most ? oct : most;
+  }
+  // blocks per matrix: enough for the largest one at two pieces per thread, at most 8 per SM and matrix
+  const int gx = grid_for((most + 1) / 2, 256, 148 * 8);
+  k_dequant_w4<<<dim3(gx, count), 256, 0, st>>>(b);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_dequant_w4(const void* blob, int n, int k, int group, void* out, cudaStream_t st) {
+  if (n <= 0 || k <= 0) return cudaSuccess;
+  return launch_dequant_w4_batch(&blob, &n, &k, &out, 1, group, st);
 }
 
 cudaError_t launch_to_f32(const void* src, int dtype, int n, float* dst, cudaStream_t st) {

@@ -74,6 +74,12 @@ int prism_op_gemm(const void* a, const void* b, const void* b2, void* out, float
   return st_of(launch_gemm_simt(a, b, b2, out, resid, m, n, k, dtype, epilogue, S(stream)));
 }
 
+int prism_op_dequant_w4(const void* blob, int32_t n, int32_t k, int32_t group, void* out, void* stream) {
+  if (!blob || !out || n < 0 || k < 32 || group < 32 || (k % group) || (group % 32)) return PRISM_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(blob) & 15) || (reinterpret_cast<uintptr_t>(out) & 15)) return PRISM_ERR_INVALID_ARG;
+  return st_of(launch_dequant_w4(blob, n, k, group, out, S(stream)));
+}
+
 int prism_op_gemm_bias(const void* a, const void* b, const float* bias, void* out, float* resid, int32_t m, int32_t n,
                        int32_t k, int32_t dtype, int32_t epilogue, int32_t impl, int32_t* err_word, void* stream) {
   if (!a || !b || !bias || m < 0 || n < 1 || k < 1 || epilogue < 0 || epilogue > 2) return PRISM_ERR_INVALID_ARG;

@@ -43,6 +43,10 @@ struct prism_handle {
   std::vector<EncVec> enc_vec;
   const void *pos_embed = nullptr, *head_dense_w = nullptr;
   float* probe_scratch = nullptr;  // [2, max_candidates, D]
+  // W4 weights (cfg.weight_format == PRISM_WFMT_W4): the layer about to run is rebuilt as bf16 here
+  bool w4 = false;
+  void* wq[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};  // w_qkv, w_o, w_gate, w_up, w_down
+  LayerMaps maps_w4{};
   const float *type_f = nullptr, *emb_g = nullptr, *emb_b = nullptr, *head_db = nullptr, *head_ow = nullptr, *head_ob = nullptr;
   int esz = 4;
   int chunk_tokens = 0;
@@ -221,6 +225,11 @@ size_t per_token_bytes(const prism_model_cfg& c, int esz) {
   return ((size_t)c.hidden + nqkv + (size_t)c.n_q_heads * c.head_dim + (size_t)c.ffn) * esz;
 }
 
+// Bytes of an [n, k] layer matrix as the caller stores it (and as it crosses the host link when streamed).
+size_t matrix_bytes(const prism_handle* h, size_t n, size_t k) {
+  return h->w4 ? w4_blob_bytes(n, k, (size_t)h->cfg.quant_group) : n * k * (size_t)h->esz;
+}
+
 LayerDev layer_in_slot(const prism_handle* h, int s) {
   const unsigned char* b = h->slot[s];
   LayerDev d;
@@ -267,16 +276,16 @@ int enqueue_layer_copy(prism_handle* h, int l, int s) {
   unsigned char* b = h->slot[s];
   cudaStream_t cs = h->copy_stream;
   PRISM_CUDA(h, cudaMemcpyAsync(b + h->off_g_attn, w.g_attn, d * e, cudaMemcpyHostToDevice, cs));
-  PRISM_CUDA(h, cudaMemcpyAsync(b + h->off_qkv, w.w_qkv, nqkv * d * e, cudaMemcpyHostToDevice, cs));
+  PRISM_CUDA(h, cudaMemcpyAsync(b + h->off_qkv, w.w_qkv, matrix_bytes(h, nqkv, d), cudaMemcpyHostToDevice, cs));
   if (c.qk_norm) {
     PRISM_CUDA(h, cudaMemcpyAsync(b + h->off_gq, w.g_q, dh * e, cudaMemcpyHostToDevice, cs));
     PRISM_CUDA(h, cudaMemcpyAsync(b + h->off_gk, w.g_k, dh * e, cudaMemcpyHostToDevice, cs));
   }
-  PRISM_CUDA(h, cudaMemcpyAsync(b + h->off_o, w.w_o, d * hd * e, cudaMemcpyHostToDevice, cs));
+  PRISM_CUDA(h, cudaMemcpyAsync(b + h->off_o, w.w_o, matrix_bytes(h, d, hd), cudaMemcpyHostToDevice, cs));
   PRISM_CUDA(h, cudaMemcpyAsync(b + h->off_g_ffn, w.g_ffn, d * e, cudaMemcpyHostToDevice, cs));
-  PRISM_CUDA(h, cudaMemcpyAsync(b + h->off_gate, w.w_gate, (size_t)c.ffn * d * e, cudaMemcpyHostToDevice, cs));
-  PRISM_CUDA(h, cudaMemcpyAsync(b + h->off_up, w.w_up, (size_t)c.ffn * d * e, cudaMemcpyHostToDevice, cs));
-  PRISM_CUDA(h, cudaMemcpyAsync(b + h->off_down, w.w_down, d * (size_t)c.ffn * e, cudaMemcpyHostToDevice, cs));
+  PRISM_CUDA(h, cudaMemcpyAsync(b + h->off_gate, w.w_gate, matrix_bytes(h, c.ffn, d), cudaMemcpyHostToDevice, cs));
+  PRISM_CUDA(h, cudaMemcpyAsync(b + h->off_up, w.w_up, matrix_bytes(h, c.ffn, d), cudaMemcpyHostToDevice, cs));
+  PRISM_CUDA(h, cudaMemcpyAsync(b + h->off_down, w.w_down, matrix_bytes(h, d, c.ffn), cudaMemcpyHostToDevice, cs));
   PRISM_CUDA(h, cudaEventRecord(h->ev_copied[s], cs));
   return PRISM_OK;
 }
@@ -299,6 +308,13 @@ int validate_cfg(const prism_model_cfg& c, std::string* why) {
   if (c.hidden_offload && c.activation_budget_bytes <= 0) return bad("hidden_offload needs an activation budget");
   if (c.shared_prefix != PRISM_PREFIX_AUTO && c.shared_prefix != PRISM_PREFIX_OFF) return bad("shared_prefix must be 0 or 1");
   if (c.arch != PRISM_ARCH_DECODER && c.arch != PRISM_ARCH_ENCODER) return bad("unknown arch");
+  if (c.weight_format != PRISM_WFMT_PLAIN && c.weight_format != PRISM_WFMT_W4) return bad("unknown weight_format");
+  if (c.weight_format == PRISM_WFMT_W4) {
+    if (c.quant_group != 32 && c.quant_group != 64 && c.quant_group != 128) return bad("quant_group must be 32, 64 or 128");
+    if (c.dtype != PRISM_BF16 || c.arch != PRISM_ARCH_DECODER) { *why = "W4 weights need bf16 and the decoder stack"; return PRISM_ERR_UNSUPPORTED; }
+    if (c.hidden % c.quant_group || c.ffn % c.quant_group || (c.n_q_heads * c.head_dim) % c.quant_group)
+      return bad("quant_group must divide hidden, ffn and n_q_heads * head_dim");
+  }
   auto unsup = [&](const char* m) { *why = m; return PRISM_ERR_UNSUPPORTED; };
   const bool enc = c.arch == PRISM_ARCH_ENCODER;
   if (enc) {
@@ -396,6 +412,7 @@ static int create_impl(prism_handle* h, const prism_model_cfg* cfg, const prism_
   const prism_model_cfg& c = *cfg;
   h->cfg = c;
   h->enc = ew != nullptr;
+  h->w4 = c.weight_format == PRISM_WFMT_W4;
   h->esz = c.dtype == PRISM_BF16 ? 2 : 4;
   h->tc = c.dtype == PRISM_BF16 && (c.gemm_impl == PRISM_IMPL_AUTO || c.gemm_impl == PRISM_IMPL_SOLO);
   h->pair = c.gemm_impl == PRISM_IMPL_AUTO;
@@ -540,16 +557,17 @@ static int create_impl(prism_handle* h, const prism_model_cfg* cfg, const prism_
   if (streamed) {
     const size_t e = h->esz, dh = c.head_dim;
     size_t off = 0;
-    auto place = [&](size_t* o, size_t elems) { *o = off; off = align_up(off + elems * e, 256); };
+    auto place_b = [&](size_t* o, size_t bytes) { *o = off; off = align_up(off + bytes, 256); };
+    auto place = [&](size_t* o, size_t elems) { place_b(o, elems * e); };
     place(&h->off_g_attn, D);
-    place(&h->off_qkv, nqkv * D);
+    place_b(&h->off_qkv, matrix_bytes(h, nqkv, D));
     place(&h->off_gq, dh);
     place(&h->off_gk, dh);
-    place(&h->off_o, D * hd);
+    place_b(&h->off_o, matrix_bytes(h, D, hd));
     place(&h->off_g_ffn, D);
-    place(&h->off_gate, (size_t)c.ffn * D);
-    place(&h->off_up, (size_t)c.ffn * D);
-    place(&h->off_down, D * (size_t)c.ffn);
+    place_b(&h->off_gate, matrix_bytes(h, c.ffn, D));
+    place_b(&h->off_up, matrix_bytes(h, c.ffn, D));
+    place_b(&h->off_down, matrix_bytes(h, D, c.ffn));
     h->slot_bytes = off;
     for (int s = 0; s < 2; ++s) PRISM_CUDA(h, dev_alloc(h, &h->slot[s], off));
     PRISM_CUDA(h, cudaStreamCreateWithFlags(&h->copy_stream, cudaStreamNonBlocking));
@@ -559,11 +577,19 @@ static int create_impl(prism_handle* h, const prism_model_cfg* cfg, const prism_
     }
   }
 
+  if (h->w4) {
+    const size_t F = (size_t)c.ffn, elems[5] = {nqkv * D, D * hd, F * D, F * D, D * F};
+    for (int i = 0; i < 5; ++i) PRISM_CUDA(h, dev_alloc(h, (unsigned char**)&h->wq[i], elems[i] * 2));
+  }
   if (h->tc) {
     PRISM_CUDA(h, make_tma_2d_bf16(&h->map_a_norm, h->a_norm, chunk, D, 128, 64));
     PRISM_CUDA(h, make_tma_2d_bf16(&h->map_attn, h->attn, chunk, hd, 128, 64));
     PRISM_CUDA(h, make_tma_2d_bf16(&h->map_hbuf, h->hbuf, chunk, c.ffn, 128, 64));
-    if (streamed) {
+    if (h->w4) {
+      // the GEMMs always read the bf16 scratch: one set of weight maps
+      const LayerDev d{nullptr, h->wq[0], nullptr, nullptr, h->wq[1], nullptr, h->wq[2], h->wq[3], h->wq[4]};
+      PRISM_CUDA(h, build_maps(h, d, &h->maps_w4));
+    } else if (streamed) {
       h->maps.resize(2);
       for (int s = 0; s < 2; ++s) PRISM_CUDA(h, build_maps(h, layer_in_slot(h, s), &h->maps[s]));
     } else {
@@ -1006,8 +1032,22 @@ int select_impl(prism_handle* h, const int32_t* query, int32_t lq, const int32_t
   for (int l = 0; l < c.n_layers && !done; ++l) {
     const int s = l & 1;
     LayerDev W = streamed ? layer_in_slot(h, s) : layer_resident(h, l);
-    const LayerMaps* maps = h->tc ? &h->maps[streamed ? s : l] : nullptr;
+    const LayerMaps* maps = !h->tc ? nullptr : h->w4 ? &h->maps_w4 : &h->maps[streamed ? s : l];
     if (streamed) PRISM_CUDA(h, cudaStreamWaitEvent(st, h->ev_copied[s], 0));
+    if (h->w4) {
+      // rebuild the layer's five matrices as bf16; the stream orders this after the previous layer's last GEMM
+      const int D = c.hidden, F = c.ffn, nq = (c.n_q_heads + 2 * c.n_kv_heads) * c.head_dim, hd = c.n_q_heads * c.head_dim;
+      const void* src[5] = {W.w_qkv, W.w_o, W.w_gate, W.w_up, W.w_down};
+      const int rows[5] = {nq, D, F, F, D}, cols[5] = {D, hd, D, D, F};
+      double bytes = 0.0;  // 4 bits in, 16 bits out per weight, plus one scale and zero point per group
+      for (int i = 0; i < 5; ++i) bytes += (double)rows[i] * cols[i] * (2.5 + 3.0 / c.quant_group);
+      PRISM_LAUNCH_P(h, st, PRISM_K_DEQUANT, bytes, launch_dequant_w4_batch(src, rows, cols, h->wq, 5, c.quant_group, st));
+      W.w_qkv = h->wq[0];
+      W.w_o = h->wq[1];
+      W.w_gate = h->wq[2];
+      W.w_up = h->wq[3];
+      W.w_down = h->wq[4];
+    }
     // chunks on sequence boundaries: the longest prefix of the remaining sequences that fits
     int s0 = 0, chunks = 0;
     if (prefix) {  // one chunk: the prefix rows and every sequence's own rows

@@ -6,6 +6,7 @@ synthetic operands, one JSON line per run.  Also the small-case driver for profi
     python -m paper_2510_15620_b200.microbench --op rmsnorm|rope|compact --rows 35200 --d 1024
     python -m paper_2510_15620_b200.microbench --op gemm_bias --m 35200 --n 4096 --k 1024 --epilogue 2   (encoder stack)
     python -m paper_2510_15620_b200.microbench --op layernorm --rows 35200 --d 1024
+    python -m paper_2510_15620_b200.microbench --op dequant --n 12288 --k 4096          (W4 -> bf16, group 128)
     python -m paper_2510_15620_b200.microbench --op attention --head-dim 64 --hq 16 --hkv 16 --causal 0
 """
 from __future__ import annotations
@@ -39,7 +40,7 @@ def _time(fn, iters, warmup, flush):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--op", required=True, choices=["gemm", "qkv_rope", "attention", "rmsnorm", "rope", "compact", "gemm_bias", "layernorm"])
+    ap.add_argument("--op", required=True, choices=["gemm", "qkv_rope", "attention", "rmsnorm", "rope", "compact", "gemm_bias", "layernorm", "dequant"])
     ap.add_argument("--head-dim", type=int, default=128)
     ap.add_argument("--m", type=int, default=35200)
     ap.add_argument("--n", type=int, default=4096)
@@ -87,6 +88,19 @@ def main():
         fn = lambda: ops.prism_op_gemm_bias(A, B, bias, O, R, m, n, k, PRISM_BF16, a.epilogue, a.impl, err)
         med, best = _time(fn, a.iters, a.warmup, flush)
         out.update(m=m, n=n, k=k, epilogue=a.epilogue, ms=med, ms_min=best, tflops=2.0 * m * n * k / med / 1e9, err=int(err.item()))
+    elif a.op == "dequant":
+        n, k, grp = a.n, a.k, 128
+        ng = k // grp
+        up16 = lambda v: (v + 15) // 16 * 16
+        total = up16(up16(up16(n * k // 2) + 2 * n * ng) + n * ng)
+        blob = torch.randint(0, 256, (total,), dtype=torch.uint8, device=dev, generator=g)
+        off_s = up16(n * k // 2)
+        blob[off_s: off_s + 2 * n * ng] = torch.tensor([0x00, 0x3C], dtype=torch.uint8, device=dev).repeat(n * ng)  # scales 2^-7
+        o = torch.empty(n, k, dtype=torch.bfloat16, device=dev)
+        fn = lambda: ops.prism_op_dequant_w4(blob, n, k, grp, o)
+        med, best = _time(fn, a.iters, a.warmup, flush)
+        out.update(n=n, k=k, group=grp, ms=med, ms_min=best, gbs=n * k * (2.5 + 3.0 / grp) / med / 1e6,
+                   bytes_per_weight="0.5 code + 2 written + 3 / group for scale and zero point")
     elif a.op == "layernorm":
         x = rnd(a.rows, a.d)
         gain, shift = torch.ones(a.d, device=dev), torch.zeros(a.d, device=dev)

@@ -35,7 +35,8 @@ def _L():
         L.prism_op_layernorm.argtypes = [vp, vp, vp, i32, i32, i32, f32, vp, vp]
         L.prism_op_embed_encoder.argtypes = [vp, vp, vp, i32, vp, vp, i32, i32, i32, vp, vp]
         L.prism_op_probe_encoder.argtypes = [vp, vp, i32, i32, vp, vp, f32, vp, i32, vp, vp, vp, vp, vp]
-        for n in ("gemm_bias", "layernorm", "embed_encoder", "probe_encoder"):
+        L.prism_op_dequant_w4.argtypes = [vp, i32, i32, i32, vp, vp]
+        for n in ("gemm_bias", "layernorm", "embed_encoder", "probe_encoder", "dequant_w4"):
             getattr(L, "prism_op_" + n).restype = C.c_int
         for n in ("pack", "embed", "rmsnorm", "qknorm_rope", "gemm", "attention", "probe", "route", "compact"):
             getattr(L, "prism_op_" + n).restype = C.c_int
@@ -77,6 +78,10 @@ def prism_op_qknorm_rope(qkv, dtype, pos, n_q_heads, n_kv_heads, head_dim, qk_no
 def prism_op_gemm(a, b, b2, out, resid, m, n, k, dtype, epilogue, impl, err_word):
     _check(_L().prism_op_gemm(_p(a), _p(b), _p(b2), _p(out), _p(resid), m, n, k, dtype, epilogue, impl, _p(err_word),
                               _stream()), "gemm")
+
+
+def prism_op_dequant_w4(blob, n, k, group, out):
+    _check(_L().prism_op_dequant_w4(_p(blob), n, k, group, _p(out), _stream()), "dequant_w4")
 
 
 def prism_op_gemm_bias(a, b, bias, out, resid, m, n, k, dtype, epilogue, impl, err_word):
