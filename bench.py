@@ -126,12 +126,12 @@ def sum_over_ranks(value: float, world: int, device=None) -> float:
 # ----------------------------------------------------------------------------------------------- oracle legs
 def oracle_sample_ids(wl, req, budget_s: float = 25.0, max_cand: int = 2):
     """A bounded sample of the request for the CPU oracle: up to max_cand candidates, shortest first, as long
-    as the estimated time (2 * layer parameters flops per token at the ~1.6e11 flop/s the fp64 numpy forward
-    sustains on 16 cores) stays within budget_s; always at least one."""
+    as the estimated time (2 * layer parameters flops per token at the ~4e11 flop/s the fp64 numpy forward
+    sustains on 16 cores; 5e11 - 8e11 were measured) stays within budget_s; always at least one."""
     cfg = wl.model
     p_layer = cfg.hidden * (cfg.n_q_heads + 2 * cfg.n_kv_heads) * cfg.head_dim + cfg.n_q_heads * cfg.head_dim * cfg.hidden \
         + 3 * cfg.hidden * cfg.ffn
-    s_per_token = 2.0 * p_layer * cfg.n_layers / 1.6e11
+    s_per_token = 2.0 * p_layer * cfg.n_layers / 4e11
     lens = np.diff(req["cand_offsets"]) + len(req["query"])
     order = np.argsort(lens, kind="stable")
     ids, t = [], 0.0
@@ -382,7 +382,7 @@ def run_prism(args):
                                     if v["ms_per_step"] > 0 else 0.0)}
                            for n, v in per.items()}
         if not args.no_cpu_baseline and not w4:   # the oracle leg times the unquantised model
-            ids = oracle_sample_ids(wl, reqs[0], max_cand=8)
+            ids = oracle_sample_ids(wl, reqs[0], max_cand=32)
             n_c = len(ids)
             rate, dt, t = oracle_sample_rate(wl, w_np, reqs[0], ids)
             line["cpu_baseline"] = {"value": rate, "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle",

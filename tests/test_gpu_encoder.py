@@ -234,3 +234,23 @@ def test_encoder_rejects_what_it_does_not_support(P):
     with pytest.raises(P.PrismError) as e:
         make_model(P, replace(cfg, max_positions=20), w, req)       # positions would run past the table
     assert e.value.status == -1
+
+
+def test_encoder_candidate_sharded_equals_unsharded(P):
+    """The sharded entry point on an encoder handle: ranks as threads of this process (one GPU), host-side score sum."""
+    from test_gpu_sharded import run_sharded
+    wl, cfg = ENC_MID_WL, ENC_MID
+    w = synth.make_weights(cfg, seed=5)
+    req = synth.make_request(wl, 0)
+    lens = np.diff(req["cand_offsets"]) + wl.query_len
+    owner = P.shard_candidates(lens, 2)
+    base = make_model(P, cfg, w, req)
+    ref_idx, ref_sc, ref_tr = run(P, base, req, wl.top_k, wl.schedule)
+    out, calls = run_sharded(P, cfg, w, req, wl.top_k, wl.schedule, owner, 2)
+    assert calls == len(ref_tr.records)
+    for idx, sc, tr in out:
+        assert np.array_equal(idx, ref_idx) and np.array_equal(sc.view(np.uint32), ref_sc.view(np.uint32))
+        for a, b in zip(tr.records, ref_tr.records):
+            assert a.active_ids == b.active_ids
+            assert np.array_equal(np.asarray(a.scores).view(np.uint32), np.asarray(b.scores).view(np.uint32))
+    base.close()
