@@ -270,9 +270,17 @@ def run_prism(args):
         else:
             model.select(q, c, o, wl.top_k, s, want_trace=False)
 
-    prefix_rows = 0  # what the library reports for this workload (one untimed traced request)
+    prefix_rows, workspace_bytes = 0, None  # what the library reports for this workload (one untimed traced request)
     if not by_cand:
-        prefix_rows = model.select(*dreqs[0], wl.top_k, sched, want_trace=True)[2].shared_prefix_rows
+        tr0 = model.select(*dreqs[0], wl.top_k, sched, want_trace=True)[2]
+        prefix_rows, workspace_bytes = tr0.shared_prefix_rows, tr0.workspace_bytes
+
+    def tensor_bytes(t, on_device):
+        if isinstance(t, dict):
+            return sum(tensor_bytes(v, on_device) for v in t.values())
+        if isinstance(t, (list, tuple)):
+            return sum(tensor_bytes(v, on_device) for v in t)
+        return t.numel() * t.element_size() if (t.is_cuda == on_device) else 0
 
     def host_step(i):
         q, c, o = hreqs[i % n_req]
@@ -313,6 +321,10 @@ def run_prism(args):
                        # causal attention: the query's rows are computed once per request instead of once per
                        # candidate (same scores bit for bit); the metric keeps counting query + document per candidate
                        "weight_format": "w4a16 (round-to-nearest, group 128)" if w4 else "bf16" if cfg.dtype == 1 else "f32",
+                       # what the request holds: the caller's weight tensors on the device and in pinned host memory
+                       # (streamed layers), and everything the handle allocated on the device (activations, slots, scratch)
+                       "memory_bytes": {"weights_device": tensor_bytes(tw, True), "weights_pinned_host": tensor_bytes(tw, False),
+                                        "handle_device": workspace_bytes},
                        "shared_query_prefix_rows": prefix_rows,
                        "rows_computed_first_layer": int(np.mean([l.sum() - (len(l) - 1) * prefix_rows for l in lens_all])),
                        "schedule": {"mode": sched.mode, "probe_layers": list(sched.probe_layers),
