@@ -138,9 +138,10 @@ typedef struct {
                       PRISM_PREFIX_OFF (1), every sequence carries its own copy of the query. */
   int32_t arch;             /* PRISM_ARCH_*.  For PRISM_ARCH_ENCODER: rms_eps is the LayerNorm epsilon; rope_theta and
                       qk_norm are ignored (qk_norm must be 0); causal is normally 0; head_dim is 64 or 128 on the
-                      tensor-core path; ffn a multiple of 8; weight_residency must be PRISM_WEIGHTS_DEVICE,
-                      embed_cache_rows 0 and hidden_offload 0 (PRISM_ERR_UNSUPPORTED otherwise); gemm_impl AUTO or
-                      SIMT, attention_impl AUTO, SOLO or SIMT. */
+                      tensor-core path; ffn a multiple of 8; embed_cache_rows and hidden_offload must be 0
+                      (PRISM_ERR_UNSUPPORTED otherwise); gemm_impl AUTO or SIMT, attention_impl AUTO, SOLO or SIMT.
+                      With PRISM_WEIGHTS_HOST_STREAMED the four matrices of a block are streamed; its vectors are
+                      read once at creation. */
   int32_t max_positions;    /* encoder: rows of the learned position table; max_seq_len + pos_offset <= max_positions */
   int32_t pos_offset;       /* encoder: token p of a sequence reads position row p + pos_offset (2 for XLM-RoBERTa) */
   int32_t weight_format;    /* PRISM_WFMT_*; W4 needs dtype PRISM_BF16 and arch PRISM_ARCH_DECODER */
@@ -173,8 +174,9 @@ typedef struct {
 } prism_weights;
 
 /* Weights of one encoder block.  Matrices have the element type of cfg.dtype and are device pointers, 16-byte
- * aligned; the vectors (biases, LayerNorm gain and shift) have the same element type and are widened to fp32
- * copies inside prism_create_encoder. */
+ * aligned (pinned host pointers with PRISM_WEIGHTS_HOST_STREAMED); the vectors (biases, LayerNorm gain and shift)
+ * have the same element type, may live in device or pinned host memory, and are widened to fp32 device copies
+ * inside prism_create_encoder. */
 typedef struct {
   const void* w_qkv;  /* [(Hq+2Hkv)*dh, D]: all q heads, then k heads, then v heads */
   const void* b_qkv;  /* [(Hq+2Hkv)*dh] */

@@ -232,6 +232,9 @@ size_t matrix_bytes(const prism_handle* h, size_t n, size_t k) {
 
 LayerDev layer_in_slot(const prism_handle* h, int s) {
   const unsigned char* b = h->slot[s];
+  if (h->enc)  // the four matrices; the vectors were widened to fp32 device copies at creation
+    return LayerDev{nullptr, b + h->off_qkv, nullptr, nullptr, b + h->off_o, nullptr, b + h->off_gate, b + h->off_gate,
+                    b + h->off_down};
   LayerDev d;
   d.g_attn = b + h->off_g_attn;
   d.w_qkv = b + h->off_qkv;
@@ -270,11 +273,20 @@ cudaError_t build_maps(const prism_handle* h, const LayerDev& d, LayerMaps* m) {
 // Enqueue the host->device copy of layer l into slot s on the copy stream.
 int enqueue_layer_copy(prism_handle* h, int l, int s) {
   const prism_model_cfg& c = h->cfg;
-  const prism_layer_weights& w = h->layers[l];
   const size_t e = h->esz, d = c.hidden, dh = c.head_dim;
   const size_t nqkv = (size_t)(c.n_q_heads + 2 * c.n_kv_heads) * dh, hd = (size_t)c.n_q_heads * dh;
   unsigned char* b = h->slot[s];
   cudaStream_t cs = h->copy_stream;
+  if (h->enc) {
+    const prism_encoder_layer_weights& w = h->enc_layers[l];
+    PRISM_CUDA(h, cudaMemcpyAsync(b + h->off_qkv, w.w_qkv, nqkv * d * e, cudaMemcpyHostToDevice, cs));
+    PRISM_CUDA(h, cudaMemcpyAsync(b + h->off_o, w.w_o, d * hd * e, cudaMemcpyHostToDevice, cs));
+    PRISM_CUDA(h, cudaMemcpyAsync(b + h->off_gate, w.w_ffn1, (size_t)c.ffn * d * e, cudaMemcpyHostToDevice, cs));
+    PRISM_CUDA(h, cudaMemcpyAsync(b + h->off_down, w.w_ffn2, d * (size_t)c.ffn * e, cudaMemcpyHostToDevice, cs));
+    PRISM_CUDA(h, cudaEventRecord(h->ev_copied[s], cs));
+    return PRISM_OK;
+  }
+  const prism_layer_weights& w = h->layers[l];
   PRISM_CUDA(h, cudaMemcpyAsync(b + h->off_g_attn, w.g_attn, d * e, cudaMemcpyHostToDevice, cs));
   PRISM_CUDA(h, cudaMemcpyAsync(b + h->off_qkv, w.w_qkv, matrix_bytes(h, nqkv, d), cudaMemcpyHostToDevice, cs));
   if (c.qk_norm) {
@@ -321,7 +333,6 @@ int validate_cfg(const prism_model_cfg& c, std::string* why) {
     if (c.qk_norm) return bad("the encoder stack has no QK-norm");
     if (c.pos_offset < 0 || c.max_positions < 1 || (long long)c.max_seq_len + c.pos_offset > c.max_positions)
       return bad("max_seq_len + pos_offset exceeds max_positions");
-    if (c.weight_residency != PRISM_WEIGHTS_DEVICE) return unsup("the encoder stack keeps its weights on the device");
     if (c.embed_cache_rows || c.hidden_offload) return unsup("embedding cache and hidden-state offload are decoder-only");
     if (c.gemm_impl != PRISM_IMPL_AUTO && c.gemm_impl != PRISM_IMPL_SIMT) return unsup("encoder GEMMs: AUTO or SIMT");
     if (c.attention_impl == PRISM_IMPL_MMA) return unsup("encoder attention: AUTO, SOLO or SIMT");
@@ -559,14 +570,14 @@ static int create_impl(prism_handle* h, const prism_model_cfg* cfg, const prism_
     size_t off = 0;
     auto place_b = [&](size_t* o, size_t bytes) { *o = off; off = align_up(off + bytes, 256); };
     auto place = [&](size_t* o, size_t elems) { place_b(o, elems * e); };
-    place(&h->off_g_attn, D);
+    if (!h->enc) place(&h->off_g_attn, D);
     place_b(&h->off_qkv, matrix_bytes(h, nqkv, D));
-    place(&h->off_gq, dh);
-    place(&h->off_gk, dh);
+    if (!h->enc) place(&h->off_gq, dh);
+    if (!h->enc) place(&h->off_gk, dh);
     place_b(&h->off_o, matrix_bytes(h, D, hd));
-    place(&h->off_g_ffn, D);
+    if (!h->enc) place(&h->off_g_ffn, D);
     place_b(&h->off_gate, matrix_bytes(h, c.ffn, D));
-    place_b(&h->off_up, matrix_bytes(h, c.ffn, D));
+    if (!h->enc) place_b(&h->off_up, matrix_bytes(h, c.ffn, D));
     place_b(&h->off_down, matrix_bytes(h, D, c.ffn));
     h->slot_bytes = off;
     for (int s = 0; s < 2; ++s) PRISM_CUDA(h, dev_alloc(h, &h->slot[s], off));

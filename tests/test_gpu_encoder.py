@@ -170,7 +170,8 @@ ENC_MID_WL = Workload("enc_mid_bf16", ENC_MID, 24, 4, 16, ("uniform", 20, 300, 2
 
 def make_model(P, cfg, w, req, **kw):
     lens = np.diff(req["cand_offsets"]) + len(req["query"])
-    return P.PrismModel(cfg, P.upload_weights(w, cfg.dtype), int(lens.max()), len(lens), int(lens.sum()), **kw)
+    tw = P.upload_weights(w, cfg.dtype, layers_pinned_host=bool(kw.get("stream_weights", False)))
+    return P.PrismModel(cfg, tw, int(lens.max()), len(lens), int(lens.sum()), **kw)
 
 
 def test_encoder_fp32_end_to_end(P):
@@ -227,7 +228,7 @@ def test_encoder_rejects_what_it_does_not_support(P):
     cfg = ENC_TINY
     w = synth.make_weights(cfg, seed=2)
     req = synth.make_request(ENC_TINY_WL, 0)
-    for kw in (dict(stream_weights=True), dict(hidden_offload=True, activation_budget_bytes=1 << 30)):
+    for kw in (dict(hidden_offload=True, activation_budget_bytes=1 << 30),):
         with pytest.raises(P.PrismError) as e:
             make_model(P, cfg, w, req, **kw)
         assert e.value.status == -8, e.value                 # PRISM_ERR_UNSUPPORTED
@@ -254,3 +255,17 @@ def test_encoder_candidate_sharded_equals_unsharded(P):
             assert a.active_ids == b.active_ids
             assert np.array_equal(np.asarray(a.scores).view(np.uint32), np.asarray(b.scores).view(np.uint32))
     base.close()
+
+
+def test_encoder_layer_streaming_is_result_neutral(P):
+    """Overlapped layer streaming (Sec. 4.2) for the encoder stack: the four matrices of a block come from pinned
+    host memory through two device slots; nothing a caller sees may change."""
+    wl, cfg = ENC_MID_WL, ENC_MID
+    w = synth.make_weights(cfg, seed=5)
+    req = synth.make_request(wl, 2)
+    for sched in (Schedule(MODE_NONE), wl.schedule):
+        base = run(P, make_model(P, cfg, w, req), req, wl.top_k, sched)
+        got = run(P, make_model(P, cfg, w, req, stream_weights=True), req, wl.top_k, sched)
+        assert np.array_equal(base[0], got[0]) and np.array_equal(base[1].view(np.uint32), got[1].view(np.uint32))
+        for r1, r2 in zip(base[2].records, got[2].records):
+            assert np.array_equal(r1.scores.view(np.uint32), r2.scores.view(np.uint32)) and r1.active_ids == r2.active_ids
