@@ -333,7 +333,7 @@ int validate_cfg(const prism_model_cfg& c, std::string* why) {
     if (c.qk_norm) return bad("the encoder stack has no QK-norm");
     if (c.pos_offset < 0 || c.max_positions < 1 || (long long)c.max_seq_len + c.pos_offset > c.max_positions)
       return bad("max_seq_len + pos_offset exceeds max_positions");
-    if (c.embed_cache_rows || c.hidden_offload) return unsup("embedding cache and hidden-state offload are decoder-only");
+    if (c.embed_cache_rows) return unsup("the embedding-row cache is decoder-only");
     if (c.gemm_impl != PRISM_IMPL_AUTO && c.gemm_impl != PRISM_IMPL_SIMT) return unsup("encoder GEMMs: AUTO or SIMT");
     if (c.attention_impl == PRISM_IMPL_MMA) return unsup("encoder attention: AUTO, SOLO or SIMT");
   }
@@ -806,11 +806,11 @@ int run_layer_chunk(prism_handle* h, const LayerDev& W, const LayerMaps* maps, f
 // chunk's normed GEMM input is produced right before it is consumed; LN2 of the last executed block is applied by
 // the probe to the one row it reads.
 int run_layer_chunk_encoder(prism_handle* h, int l, const LayerDev& W, const LayerMaps* maps, float* x, const int* cu_dev,
-                            int s0, int s1, int r0, int rows, int max_len, cudaStream_t st) {
+                            int s0, int s1, int r0, int rows, int max_len, cudaStream_t st, bool x_is_chunk = false) {
   const prism_model_cfg& c = h->cfg;
   const int D = c.hidden, dh = c.head_dim, F = c.ffn;
   const int nqkv = (c.n_q_heads + 2 * c.n_kv_heads) * dh, hd = c.n_q_heads * dh;
-  float* xr = x + (size_t)r0 * D;
+  float* xr = x_is_chunk ? x : x + (size_t)r0 * D;
   const EncVec& V = h->enc_vec[l];
   const float* g0 = l == 0 ? h->emb_g : h->enc_vec[l - 1].ln2_g;
   const float* b0 = l == 0 ? h->emb_b : h->enc_vec[l - 1].ln2_b;
@@ -1076,7 +1076,7 @@ int select_impl(prism_handle* h, const int32_t* query, int32_t lq, const int32_t
         ++s1;
       }
       const int r0 = h->h_cu[s0], rows = h->h_cu[s1] - r0;
-      if (h->enc) {
+      if (h->enc && !h->offload) {
         if ((rc = run_layer_chunk_encoder(h, l, W, maps, h->x[cur], h->cu[cur], s0, s1, r0, rows, max_len, st)) != PRISM_OK) return rc;
       } else if (!h->offload) {
         if ((rc = run_layer_chunk(h, W, maps, h->x[cur], h->cu[cur], s0, s1, r0, rows, max_len, st)) != PRISM_OK) return rc;
@@ -1105,7 +1105,9 @@ int select_impl(prism_handle* h, const int32_t* query, int32_t lq, const int32_t
         PRISM_CUDA(h, cudaMemcpyAsync(h->xc[slot], hx, bytes, cudaMemcpyHostToDevice, h->in_stream));
         PRISM_CUDA(h, cudaEventRecord(h->ev_in[slot], h->in_stream));
         PRISM_CUDA(h, cudaStreamWaitEvent(st, h->ev_in[slot], 0));
-        if ((rc = run_layer_chunk(h, W, maps, h->xc[slot], h->cu[cur], s0, s1, r0, rows, max_len, st, true)) != PRISM_OK) return rc;
+        rc = h->enc ? run_layer_chunk_encoder(h, l, W, maps, h->xc[slot], h->cu[cur], s0, s1, r0, rows, max_len, st, true)
+                    : run_layer_chunk(h, W, maps, h->xc[slot], h->cu[cur], s0, s1, r0, rows, max_len, st, true);
+        if (rc != PRISM_OK) return rc;
         PRISM_CUDA(h, cudaEventRecord(h->ev_done[slot], st));
         PRISM_CUDA(h, cudaStreamWaitEvent(h->out_stream, h->ev_done[slot], 0));
         PRISM_CUDA(h, cudaMemcpyAsync(hx, h->xc[slot], bytes, cudaMemcpyDeviceToHost, h->out_stream));

@@ -228,10 +228,11 @@ def test_encoder_rejects_what_it_does_not_support(P):
     cfg = ENC_TINY
     w = synth.make_weights(cfg, seed=2)
     req = synth.make_request(ENC_TINY_WL, 0)
-    for kw in (dict(hidden_offload=True, activation_budget_bytes=1 << 30),):
-        with pytest.raises(P.PrismError) as e:
-            make_model(P, cfg, w, req, **kw)
-        assert e.value.status == -8, e.value                 # PRISM_ERR_UNSUPPORTED
+    with pytest.raises(P.PrismError) as e:
+        lens = np.diff(req["cand_offsets"]) + len(req["query"])
+        tw = P.upload_weights(w, cfg.dtype, embed_pinned_host=True)
+        P.PrismModel(cfg, tw, int(lens.max()), len(lens), int(lens.sum()), embed_cache_rows=100)
+    assert e.value.status == -8, e.value                     # PRISM_ERR_UNSUPPORTED
     with pytest.raises(P.PrismError) as e:
         make_model(P, replace(cfg, max_positions=20), w, req)       # positions would run past the table
     assert e.value.status == -1
@@ -266,6 +267,25 @@ def test_encoder_layer_streaming_is_result_neutral(P):
     for sched in (Schedule(MODE_NONE), wl.schedule):
         base = run(P, make_model(P, cfg, w, req), req, wl.top_k, sched)
         got = run(P, make_model(P, cfg, w, req, stream_weights=True), req, wl.top_k, sched)
+        assert np.array_equal(base[0], got[0]) and np.array_equal(base[1].view(np.uint32), got[1].view(np.uint32))
+        for r1, r2 in zip(base[2].records, got[2].records):
+            assert np.array_equal(r1.scores.view(np.uint32), r2.scores.view(np.uint32)) and r1.active_ids == r2.active_ids
+
+
+def test_encoder_hidden_state_offload_is_result_neutral(P):
+    """Dynamic offloading of the hidden states (Sec. 4.3) for the encoder stack: host-resident hidden states through
+    three device chunk buffers, alone and together with layer streaming."""
+    wl, cfg = ENC_MID_WL, ENC_MID
+    w = synth.make_weights(cfg, seed=5)
+    req = synth.make_request(wl, 1)
+    lens = np.diff(req["cand_offsets"]) + wl.query_len
+    chunk_rows = int(lens.sum()) // 4
+    per_tok = 2 * (cfg.hidden + 3 * cfg.hidden + cfg.hidden + cfg.ffn)
+    budget = chunk_rows * (3 * cfg.hidden * 4 + per_tok)
+    base = run(P, make_model(P, cfg, w, req), req, wl.top_k, wl.schedule)
+    for kw in (dict(), dict(stream_weights=True)):
+        got = run(P, make_model(P, cfg, w, req, hidden_offload=True, activation_budget_bytes=budget, **kw), req, wl.top_k, wl.schedule)
+        assert got[2].n_chunks_max >= 3
         assert np.array_equal(base[0], got[0]) and np.array_equal(base[1].view(np.uint32), got[1].view(np.uint32))
         for r1, r2 in zip(base[2].records, got[2].records):
             assert np.array_equal(r1.scores.view(np.uint32), r2.scores.view(np.uint32)) and r1.active_ids == r2.active_ids
