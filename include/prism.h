@@ -62,7 +62,8 @@ enum { PRISM_IMPL_AUTO = 0, PRISM_IMPL_SIMT = 1, PRISM_IMPL_MMA = 2, PRISM_IMPL_
 
 /* weight_format of prism_model_cfg.  PLAIN: matrices in the element type of cfg.dtype.  W4: the quantised arm of
  * the paper's evaluation (Sec. 6.1: the method composed with 4-bit weight-only quantisation, 16-bit activations).
- * The five matrices of every layer (w_qkv, w_o, w_gate, w_up, w_down) are packed blobs; for an [N, K] matrix and
+ * The five matrices of every layer (w_qkv, w_o, w_gate, w_up, w_down; for the encoder stack w_qkv, w_o, w_ffn1, w_ffn2)
+ * are packed blobs; for an [N, K] matrix and
  * group size G = quant_group, every section starting on a 16-byte boundary:
  *     codes   N*K/2 bytes, row-major; byte (n, k/2) holds code(n,k) in its low nibble for even k, high nibble for odd k
  *     scales  N*K/G bf16, row-major [N, K/G]
@@ -144,7 +145,7 @@ typedef struct {
                       read once at creation. */
   int32_t max_positions;    /* encoder: rows of the learned position table; max_seq_len + pos_offset <= max_positions */
   int32_t pos_offset;       /* encoder: token p of a sequence reads position row p + pos_offset (2 for XLM-RoBERTa) */
-  int32_t weight_format;    /* PRISM_WFMT_*; W4 needs dtype PRISM_BF16 and arch PRISM_ARCH_DECODER */
+  int32_t weight_format;    /* PRISM_WFMT_*; W4 needs dtype PRISM_BF16 */
   int32_t quant_group;      /* W4: input channels per scale / zero point: 32, 64 or 128, dividing hidden, ffn and
                                n_q_heads * head_dim */
 } prism_model_cfg;

@@ -26,6 +26,8 @@ MATRIX_SHAPES = {  # name -> (rows, cols) from the model configuration
     "w_gate": lambda c: (c.ffn, c.hidden),
     "w_up": lambda c: (c.ffn, c.hidden),
     "w_down": lambda c: (c.hidden, c.ffn),
+    "w_ffn1": lambda c: (c.ffn, c.hidden),   # encoder stack
+    "w_ffn2": lambda c: (c.hidden, c.ffn),
 }
 
 

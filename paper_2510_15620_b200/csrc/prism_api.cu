@@ -279,10 +279,10 @@ int enqueue_layer_copy(prism_handle* h, int l, int s) {
   cudaStream_t cs = h->copy_stream;
   if (h->enc) {
     const prism_encoder_layer_weights& w = h->enc_layers[l];
-    PRISM_CUDA(h, cudaMemcpyAsync(b + h->off_qkv, w.w_qkv, nqkv * d * e, cudaMemcpyHostToDevice, cs));
-    PRISM_CUDA(h, cudaMemcpyAsync(b + h->off_o, w.w_o, d * hd * e, cudaMemcpyHostToDevice, cs));
-    PRISM_CUDA(h, cudaMemcpyAsync(b + h->off_gate, w.w_ffn1, (size_t)c.ffn * d * e, cudaMemcpyHostToDevice, cs));
-    PRISM_CUDA(h, cudaMemcpyAsync(b + h->off_down, w.w_ffn2, d * (size_t)c.ffn * e, cudaMemcpyHostToDevice, cs));
+    PRISM_CUDA(h, cudaMemcpyAsync(b + h->off_qkv, w.w_qkv, matrix_bytes(h, nqkv, d), cudaMemcpyHostToDevice, cs));
+    PRISM_CUDA(h, cudaMemcpyAsync(b + h->off_o, w.w_o, matrix_bytes(h, d, hd), cudaMemcpyHostToDevice, cs));
+    PRISM_CUDA(h, cudaMemcpyAsync(b + h->off_gate, w.w_ffn1, matrix_bytes(h, c.ffn, d), cudaMemcpyHostToDevice, cs));
+    PRISM_CUDA(h, cudaMemcpyAsync(b + h->off_down, w.w_ffn2, matrix_bytes(h, d, c.ffn), cudaMemcpyHostToDevice, cs));
     PRISM_CUDA(h, cudaEventRecord(h->ev_copied[s], cs));
     return PRISM_OK;
   }
@@ -323,7 +323,7 @@ int validate_cfg(const prism_model_cfg& c, std::string* why) {
   if (c.weight_format != PRISM_WFMT_PLAIN && c.weight_format != PRISM_WFMT_W4) return bad("unknown weight_format");
   if (c.weight_format == PRISM_WFMT_W4) {
     if (c.quant_group != 32 && c.quant_group != 64 && c.quant_group != 128) return bad("quant_group must be 32, 64 or 128");
-    if (c.dtype != PRISM_BF16 || c.arch != PRISM_ARCH_DECODER) { *why = "W4 weights need bf16 and the decoder stack"; return PRISM_ERR_UNSUPPORTED; }
+    if (c.dtype != PRISM_BF16) { *why = "W4 weights need bf16"; return PRISM_ERR_UNSUPPORTED; }
     if (c.hidden % c.quant_group || c.ffn % c.quant_group || (c.n_q_heads * c.head_dim) % c.quant_group)
       return bad("quant_group must divide hidden, ffn and n_q_heads * head_dim");
   }
@@ -1048,15 +1048,18 @@ int select_impl(prism_handle* h, const int32_t* query, int32_t lq, const int32_t
     if (h->w4) {
       // rebuild the layer's five matrices as bf16; the stream orders this after the previous layer's last GEMM
       const int D = c.hidden, F = c.ffn, nq = (c.n_q_heads + 2 * c.n_kv_heads) * c.head_dim, hd = c.n_q_heads * c.head_dim;
-      const void* src[5] = {W.w_qkv, W.w_o, W.w_gate, W.w_up, W.w_down};
-      const int rows[5] = {nq, D, F, F, D}, cols[5] = {D, hd, D, D, F};
+      // decoder: qkv, o, gate, up, down; encoder: qkv, o, ffn1, ffn2 (the last into the "down" scratch)
+      const int nm = h->enc ? 4 : 5;
+      const void* src[5] = {W.w_qkv, W.w_o, W.w_gate, h->enc ? W.w_down : W.w_up, W.w_down};
+      void* dst[5] = {h->wq[0], h->wq[1], h->wq[2], h->enc ? h->wq[4] : h->wq[3], h->wq[4]};
+      const int rows[5] = {nq, D, F, h->enc ? D : F, D}, cols[5] = {D, hd, D, h->enc ? F : D, F};
       double bytes = 0.0;  // 4 bits in, 16 bits out per weight, plus one scale and zero point per group
-      for (int i = 0; i < 5; ++i) bytes += (double)rows[i] * cols[i] * (2.5 + 3.0 / c.quant_group);
-      PRISM_LAUNCH_P(h, st, PRISM_K_DEQUANT, bytes, launch_dequant_w4_batch(src, rows, cols, h->wq, 5, c.quant_group, st));
+      for (int i = 0; i < nm; ++i) bytes += (double)rows[i] * cols[i] * (2.5 + 3.0 / c.quant_group);
+      PRISM_LAUNCH_P(h, st, PRISM_K_DEQUANT, bytes, launch_dequant_w4_batch(src, rows, cols, dst, nm, c.quant_group, st));
       W.w_qkv = h->wq[0];
       W.w_o = h->wq[1];
       W.w_gate = h->wq[2];
-      W.w_up = h->wq[3];
+      W.w_up = h->enc ? h->wq[2] : h->wq[3];
       W.w_down = h->wq[4];
     }
     // chunks on sequence boundaries: the longest prefix of the remaining sequences that fits

@@ -20,7 +20,7 @@ import numpy as np
 
 from .weights import bf16_bits, round_to_bf16
 
-MATRICES = ("w_qkv", "w_o", "w_gate", "w_up", "w_down")
+MATRICES = ("w_qkv", "w_o", "w_gate", "w_up", "w_down", "w_ffn1", "w_ffn2")   # decoder and encoder layer matrices
 
 
 def _align16(v: int) -> int:

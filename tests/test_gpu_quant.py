@@ -99,3 +99,26 @@ def test_w4_rejects_bad_configurations(P, quantised):
     with pytest.raises(P.PrismError) as e:
         model(P, wq, req, weight_format=P.PRISM_WFMT_W4, quant_group=48)
     assert e.value.status == -1
+
+
+def test_w4_encoder_handle_equals_plain_handle_on_the_dequantised_matrices(P):
+    from test_gpu_encoder import ENC_MID, ENC_MID_WL
+    cfg, wl = ENC_MID, ENC_MID_WL
+    w = synth.make_weights(cfg, seed=5)
+    wq = synth.quantize_weights(w, group=64)
+    wd = oracle.dequantize_weights(wq, cfg, 64)
+    wd32 = {k: v for k, v in wd.items() if k != "layers"}
+    wd32["layers"] = [{k: np.asarray(v, np.float32) for k, v in l.items()} for l in wd["layers"]]
+    req = synth.make_request(wl, 0)
+    lens = np.diff(req["cand_offsets"]) + len(req["query"])
+    mk = lambda ww, **kw: P.PrismModel(cfg, P.upload_weights(ww, cfg.dtype, layers_pinned_host=bool(kw.get("stream_weights", False))),
+                                       int(lens.max()), len(lens), int(lens.sum()), **kw)
+    plain = mk(wd32)
+    ref = run(P, plain, req, wl.top_k, wl.schedule)
+    for kw in (dict(), dict(stream_weights=True)):
+        q4 = mk(wq, weight_format=P.PRISM_WFMT_W4, quant_group=64, **kw)
+        same(run(P, q4, req, wl.top_k, wl.schedule), ref)
+        q4.close()
+    S = oracle.score_matrix(req["query"], req["cand_tokens"], req["cand_offsets"], wd, cfg, [2, 4, 5])
+    check_scores(ref[2], S, TOL_BF16)
+    plain.close()
