@@ -139,8 +139,7 @@ typedef struct {
                       PRISM_PREFIX_OFF (1), every sequence carries its own copy of the query. */
   int32_t arch;             /* PRISM_ARCH_*.  For PRISM_ARCH_ENCODER: rms_eps is the LayerNorm epsilon; rope_theta and
                       qk_norm are ignored (qk_norm must be 0); causal is normally 0; head_dim is 64 or 128 on the
-                      tensor-core path; ffn a multiple of 8; embed_cache_rows must be 0
-                      (PRISM_ERR_UNSUPPORTED otherwise); gemm_impl AUTO or SIMT, attention_impl AUTO, SOLO or SIMT.
+                      tensor-core path; ffn a multiple of 8; gemm_impl AUTO or SIMT, attention_impl AUTO, SOLO or SIMT.
                       With PRISM_WEIGHTS_HOST_STREAMED the four matrices of a block are streamed; its vectors are
                       read once at creation. */
   int32_t max_positions;    /* encoder: rows of the learned position table; max_seq_len + pos_offset <= max_positions */

@@ -130,7 +130,7 @@ cudaError_t launch_probe(const float* x, const int* cu, int n, int d, const void
 // the first norm of the first block)
 cudaError_t launch_embed_encoder(const void* table, const void* pos_table, const float* type_row, int dtype,
                                  const int* tokens, const int* pos, int pos_offset, int total, int d, float* x,
-                                 cudaStream_t st);
+                                 cudaStream_t st, const int* tok2slot = nullptr);
 // In place: x[r,:] = (x[r,:] - mean) / sqrt(var + eps) * gain + shift (fp32), and the same values in element type
 // `dtype` to out (the next GEMM's input).
 cudaError_t launch_layernorm(float* x, const float* gain, const float* shift, int dtype, int rows, int d, float eps,

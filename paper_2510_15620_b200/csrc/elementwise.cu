@@ -243,10 +243,11 @@ __global__ void __launch_bounds__(256) k_rmsnorm_warp(const float* __restrict__ 
 template <typename WT>
 __global__ void __launch_bounds__(128) k_embed_encoder(const WT* __restrict__ table, const WT* __restrict__ pos_table,
                                                        const float* __restrict__ type_row, const int* __restrict__ tokens,
-                                                       const int* __restrict__ pos, int pos_offset, int d,
-                                                       float* __restrict__ x) {
+                                                       const int* __restrict__ tok2slot, const int* __restrict__ pos,
+                                                       int pos_offset, int d, float* __restrict__ x) {
   const int t = blockIdx.x;
-  const WT* a = table + (size_t)tokens[t] * d;
+  const int tok = tokens[t];
+  const WT* a = table + (size_t)(tok2slot ? tok2slot[tok] : tok) * d;  // with a row cache, `table` is the cache
   const WT* b = pos_table + (size_t)(pos[t] + pos_offset) * d;
   float* dst = x + (size_t)t * d;
   for (int c = threadIdx.x * 4; c < d; c += blockDim.x * 4) {
@@ -720,15 +721,15 @@ cudaError_t launch_rmsnorm(const float* x, const void* gain, int dtype, int rows
 
 cudaError_t launch_embed_encoder(const void* table, const void* pos_table, const float* type_row, int dtype,
                                  const int* tokens, const int* pos, int pos_offset, int total, int d, float* x,
-                                 cudaStream_t st) {
+                                 cudaStream_t st, const int* tok2slot) {
   if (total <= 0) return cudaSuccess;
   if (d % 4) return cudaErrorInvalidValue;
   if (dtype == 1)
     k_embed_encoder<__nv_bfloat16><<<total, 128, 0, st>>>((const __nv_bfloat16*)table, (const __nv_bfloat16*)pos_table,
-                                                          type_row, tokens, pos, pos_offset, d, x);
+                                                          type_row, tokens, tok2slot, pos, pos_offset, d, x);
   else
-    k_embed_encoder<float><<<total, 128, 0, st>>>((const float*)table, (const float*)pos_table, type_row, tokens, pos,
-                                                  pos_offset, d, x);
+    k_embed_encoder<float><<<total, 128, 0, st>>>((const float*)table, (const float*)pos_table, type_row, tokens, tok2slot,
+                                                  pos, pos_offset, d, x);
   return cudaGetLastError();
 }
 

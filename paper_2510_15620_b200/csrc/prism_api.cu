@@ -333,7 +333,6 @@ int validate_cfg(const prism_model_cfg& c, std::string* why) {
     if (c.qk_norm) return bad("the encoder stack has no QK-norm");
     if (c.pos_offset < 0 || c.max_positions < 1 || (long long)c.max_seq_len + c.pos_offset > c.max_positions)
       return bad("max_seq_len + pos_offset exceeds max_positions");
-    if (c.embed_cache_rows) return unsup("the embedding-row cache is decoder-only");
     if (c.gemm_impl != PRISM_IMPL_AUTO && c.gemm_impl != PRISM_IMPL_SIMT) return unsup("encoder GEMMs: AUTO or SIMT");
     if (c.attention_impl == PRISM_IMPL_MMA) return unsup("encoder attention: AUTO, SOLO or SIMT");
   }
@@ -532,10 +531,10 @@ static int create_impl(prism_handle* h, const prism_model_cfg* cfg, const prism_
   PRISM_CUDA(h, dev_alloc(h, &h->trace_ids, (size_t)c.n_layers * N));
   PRISM_CUDA(h, dev_alloc(h, &h->owned_dev, N));
   if (c.embed_cache_rows > 0) {
-    if ((reinterpret_cast<uintptr_t>(w->embed) & 15) || (D * h->esz) % 16)
+    if ((reinterpret_cast<uintptr_t>(h->embed) & 15) || (D * h->esz) % 16)
       return fail(h, PRISM_ERR_INVALID_ARG, "the host embedding table must be 16-byte aligned with rows of a multiple of 16 bytes");
     cudaPointerAttributes pa{};
-    if (cudaPointerGetAttributes(&pa, w->embed) != cudaSuccess || pa.type != cudaMemoryTypeHost) {
+    if (cudaPointerGetAttributes(&pa, h->embed) != cudaSuccess || pa.type != cudaMemoryTypeHost) {
       cudaGetLastError();
       return fail(h, PRISM_ERR_INVALID_ARG, "embed_cache_rows > 0 needs the embedding table in pinned host memory");
     }
@@ -1016,8 +1015,9 @@ int select_impl(prism_handle* h, const int32_t* query, int32_t lq, const int32_t
                                     prefix > 0));
   if (h->enc)
     PRISM_LAUNCH_P(h, st, PRISM_K_EMBED, (double)total * c.hidden * (4.0 + 2.0 * h->esz),
-                   launch_embed_encoder(h->embed, h->pos_embed, h->type_f, c.dtype, h->tokens, h->pos, c.pos_offset, (int)total,
-                                        c.hidden, h->x[cur], st));
+                   launch_embed_encoder(h->cache_rows > 0 ? h->cache_dev : h->embed, h->pos_embed, h->type_f, c.dtype, h->tokens,
+                                        h->pos, c.pos_offset, (int)total, c.hidden, h->x[cur], st,
+                                        h->cache_rows > 0 ? h->tok2slot_dev : nullptr));
   else
   PRISM_LAUNCH_P(h, st, PRISM_K_EMBED, (double)total * c.hidden * (4.0 + h->esz),
                  launch_embed(h->cache_rows > 0 ? h->cache_dev : h->embed, c.dtype, h->tokens, (int)total, c.hidden, h->x[cur], st,

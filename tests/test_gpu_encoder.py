@@ -229,9 +229,7 @@ def test_encoder_rejects_what_it_does_not_support(P):
     w = synth.make_weights(cfg, seed=2)
     req = synth.make_request(ENC_TINY_WL, 0)
     with pytest.raises(P.PrismError) as e:
-        lens = np.diff(req["cand_offsets"]) + len(req["query"])
-        tw = P.upload_weights(w, cfg.dtype, embed_pinned_host=True)
-        P.PrismModel(cfg, tw, int(lens.max()), len(lens), int(lens.sum()), embed_cache_rows=100)
+        make_model(P, cfg, w, req, gemm_impl=3)                     # the single-CTA GEMM has no bias epilogues
     assert e.value.status == -8, e.value                     # PRISM_ERR_UNSUPPORTED
     with pytest.raises(P.PrismError) as e:
         make_model(P, replace(cfg, max_positions=20), w, req)       # positions would run past the table
@@ -289,3 +287,21 @@ def test_encoder_hidden_state_offload_is_result_neutral(P):
         assert np.array_equal(base[0], got[0]) and np.array_equal(base[1].view(np.uint32), got[1].view(np.uint32))
         for r1, r2 in zip(base[2].records, got[2].records):
             assert np.array_equal(r1.scores.view(np.uint32), r2.scores.view(np.uint32)) and r1.active_ids == r2.active_ids
+
+
+def test_encoder_embedding_row_cache_is_result_neutral(P):
+    """Embedding table caching (Sec. 4.4) for the encoder stack: the token table stays in pinned host memory, the
+    device holds an LRU cache of its rows."""
+    wl, cfg = ENC_MID_WL, ENC_MID
+    w = synth.make_weights(cfg, seed=5)
+    reqs = [synth.make_request(wl, r) for r in range(2)]
+    lens = [np.diff(r["cand_offsets"]) + wl.query_len for r in reqs]
+    mx, tot = max(int(l.max()) for l in lens), max(int(l.sum()) for l in lens)
+    base = P.PrismModel(cfg, P.upload_weights(w, cfg.dtype), mx, wl.n_candidates, tot)
+    cached = P.PrismModel(cfg, P.upload_weights(w, cfg.dtype, embed_pinned_host=True), mx + 64, wl.n_candidates, tot + 4096,
+                          embed_cache_rows=cfg.vocab)
+    for r in reqs:
+        a, b = run(P, base, r, wl.top_k, wl.schedule), run(P, cached, r, wl.top_k, wl.schedule)
+        assert np.array_equal(a[0], b[0]) and np.array_equal(a[1].view(np.uint32), b[1].view(np.uint32))
+    hits, misses, evictions = cached.embed_cache_stats()
+    assert misses > 0 and hits > 0 and evictions == 0
