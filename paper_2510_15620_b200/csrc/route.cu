@@ -1,5 +1,7 @@
 // S11/S13: rank, dispersion (CV), optimal 1-D clustering, three-way routing, survivor offsets and
-// the final top-K, for one scored layer.  One thread block; n <= 4096 candidates.
+// the final top-K, for one scored layer.  One thread block decides; n <= 4096 candidates.  From 512 candidates on
+// the block is the first of a cluster of eight whose other blocks only help with the quadratic part, the rows of
+// the clustering's cost table (one warp per row, rows dealt round-robin over all warps of the cluster).
 //
 // The decision arithmetic is fp64 on fp32 scores in a fixed left-to-right order with explicitly
 // rounded operations (no FMA contraction), so that the integer outcome (cuts, survivor set, new
@@ -17,6 +19,7 @@ struct Shared {
   float score[kMaxCandidates];
   int id[kMaxCandidates];
   int rank[kMaxCandidates];
+  float by_rank[kMaxCandidates];  // the scores in rank order (read by the sequential fp64 sums)
   int warp_a[32], warp_b[32];
   int carry_a, carry_b;
   int lo_keep, hi_keep;  // ranks [lo_keep, hi_keep) survive
@@ -48,16 +51,61 @@ __device__ __forceinline__ double group_cost(const double* p1, const double* p2,
   return dsub(s2, ddiv(dmul(s1, s1), (double)(j - i)));
 }
 
+__device__ __forceinline__ uint32_t cluster_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
+// Row c of the cost table: D[c][j] = min over i of D[c-1][i] + cost(i, j), the smallest such i in arg.  One warp per
+// j; the lanes stride over i and keep their first strict minimum, the warp takes the smallest (cost, i) pair, which
+// is the i a left-to-right scan with `<` would keep.
+__device__ __forceinline__ void dp_row(int c, int n, const double* __restrict__ p1, const double* __restrict__ p2,
+                                       const int* __restrict__ valid, const double* __restrict__ dprev,
+                                       double* __restrict__ dcur, int* __restrict__ arg_row, int warp_id, int n_warps,
+                                       int lane) {
+  const double inf = __longlong_as_double(0x7ff0000000000000LL);
+  for (int j = warp_id; j <= n; j += n_warps) {
+    double best = inf;
+    int bi = 0;
+    if (j >= c && valid[j]) {
+      for (int i = c - 1 + lane; i < j; i += 32) {
+        const double dp = dprev[i];
+        if (dp == inf) continue;
+        const double tot = dadd(dp, group_cost(p1, p2, i, j));
+        if (tot < best) { best = tot; bi = i; }
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        const double ob = __shfl_xor_sync(0xffffffffu, best, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+        if (ob < best || (ob == best && ob != inf && oi < bi)) { best = ob; bi = oi; }
+      }
+      if (best == inf) bi = 0;
+    }
+    if (lane == 0) {
+      dcur[j] = best;
+      arg_row[j] = bi;
+    }
+  }
+}
+
 __global__ void __launch_bounds__(kThreads) k_route(const float* __restrict__ scores, const int* __restrict__ cu_old,
                                                     const int* __restrict__ seq2orig_old, int n, RouteParams p,
                                                     int* __restrict__ cu_new, int* __restrict__ seq2orig_new,
                                                     int* __restrict__ old_of_new, RouteState* __restrict__ state,
                                                     int* __restrict__ res_idx, float* __restrict__ res_score,
                                                     ProbeRecordDev* __restrict__ rec, float* __restrict__ trace_scores,
-                                                    int* __restrict__ trace_ids, unsigned char* __restrict__ scratch) {
+                                                    int* __restrict__ trace_ids, unsigned char* __restrict__ scratch,
+                                                    int n_cta) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   Shared& sh = *reinterpret_cast<Shared*>(smem_raw);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int crank = n_cta > 1 ? (int)cluster_rank() : 0;
+  const int n_warps = n_cta * (kThreads / 32), warp_id = warp * n_cta + crank;  // rows dealt round-robin over the cluster
   const int np1 = n + 1;
   double* p1 = reinterpret_cast<double*>(scratch);
   double* p2 = p1 + np1;
@@ -66,6 +114,50 @@ __global__ void __launch_bounds__(kThreads) k_route(const float* __restrict__ sc
   int* arg = reinterpret_cast<int*>(dbuf1 + np1);  // [kMaxClusters][np1]
   int* valid = arg + (size_t)kMaxClusters * np1;   // [np1]
   int* sorted = valid + np1;                       // [np1] batch position of each rank
+  volatile int* flags = sorted + np1;              // [2] in the scratch's tail: cluster? and with how many groups
+
+  int* rank_g = arg + (size_t)(kMaxClusters - 1) * np1;  // the table's last row is never a cost-table row (c - 2 <= 6)
+
+  // Every block of the cluster holds the scores and ids; the deciding block also records them for the trace.
+  for (int i = tid; i < n; i += kThreads) {
+    const float raw = scores[i];
+    sh.score[i] = (raw != raw) ? -INFINITY : raw;  // a NaN score ranks last instead of breaking the order
+    sh.id[i] = seq2orig_old[i];
+  }
+  __syncthreads();
+  // ---- rank by (score descending, original index ascending); with a cluster, candidate i is ranked by block i mod 8
+  for (int i = tid * n_cta + crank; i < n; i += kThreads * n_cta) {
+    const float si = sh.score[i];
+    const int ii = sh.id[i];
+    int r = 0;
+    for (int j = 0; j < n; ++j) {
+      const float sj = sh.score[j];
+      r += (sj > si) || (sj == si && sh.id[j] < ii);
+    }
+    if (n_cta > 1) rank_g[i] = r; else sh.rank[i] = r;
+    sorted[r] = i;
+  }
+  if (n_cta > 1) {
+    __syncthreads();
+    cluster_sync_all();  // all ranks are written
+  }
+
+  if (crank != 0) {
+    // Helper block: wait for the deciding block's verdict, then compute its share of every row of the cost table.
+    cluster_sync_all();
+    if (flags[0]) {
+      const int k = flags[1];
+      double* dprev = dbuf0;
+      double* dcur = dbuf1;
+      for (int c = 2; c <= k; ++c) {
+        dp_row(c, n, p1, p2, valid, dprev, dcur, arg + (size_t)(c - 2) * np1, warp_id, n_warps, lane);
+        cluster_sync_all();
+        double* t = dprev; dprev = dcur; dcur = t;
+      }
+    }
+    return;
+  }
+  bool verdict_out = false;  // has this block published flags and met the helpers?
 
   const int k_rem = state->k_rem;
   const int n_result = state->n_result;
@@ -73,12 +165,9 @@ __global__ void __launch_bounds__(kThreads) k_route(const float* __restrict__ sc
   const int tokens_before = p.prefix ? (cu_old[n] - p.prefix) + n * p.prefix : cu_old[n];
 
   for (int i = tid; i < n; i += kThreads) {
-    const float raw = scores[i];
-    sh.score[i] = (raw != raw) ? -INFINITY : raw;  // a NaN score ranks last instead of breaking the order
-    sh.id[i] = seq2orig_old[i];
-    sorted[i] = 0;
     if (trace_scores) trace_scores[i] = scores[i];
     if (trace_ids) trace_ids[i] = seq2orig_old[i];
+    if (n_cta > 1) sh.rank[i] = rank_g[i];
   }
   if (tid == 0) {
     sh.lo_keep = 0;
@@ -89,18 +178,7 @@ __global__ void __launch_bounds__(kThreads) k_route(const float* __restrict__ sc
   }
   __syncthreads();
 
-  // ---- rank by (score descending, original index ascending) --------------------------------
-  for (int i = tid; i < n; i += kThreads) {
-    const float si = sh.score[i];
-    const int ii = sh.id[i];
-    int r = 0;
-    for (int j = 0; j < n; ++j) {
-      const float sj = sh.score[j];
-      r += (sj > si) || (sj == si && sh.id[j] < ii);
-    }
-    sh.rank[i] = r;
-    sorted[r] = i;
-  }
+  for (int r = tid; r < n; r += kThreads) sh.by_rank[r] = sh.score[sorted[r]];
   __syncthreads();
 
   int fired = 0, n_selected = 0, n_dropped = 0, n_deferred = n, append_lo = 0, append_hi = 0;
@@ -128,7 +206,7 @@ __global__ void __launch_bounds__(kThreads) k_route(const float* __restrict__ sc
     if (tid == 0) {
       double acc = 0.0;
       for (int r = 0; r < n; ++r) {
-        const double s = (double)sh.score[sorted[r]];
+        const double s = (double)sh.by_rank[r];
         acc = (r == 0) ? s : dadd(acc, s);
       }
       const double mu = ddiv(acc, (double)n);
@@ -138,7 +216,7 @@ __global__ void __launch_bounds__(kThreads) k_route(const float* __restrict__ sc
       int distinct = 1;
       valid[0] = 0;
       for (int r = 0; r < n; ++r) {
-        const float sr = sh.score[sorted[r]];
+        const float sr = sh.by_rank[r];
         const double z = dsub((double)sr, mu);
         const double zz = dmul(z, z);
         a1 = (r == 0) ? z : dadd(a1, z);
@@ -146,7 +224,7 @@ __global__ void __launch_bounds__(kThreads) k_route(const float* __restrict__ sc
         p1[r + 1] = a1;
         p2[r + 1] = a2;
         if (r > 0) {
-          const int v = sh.score[sorted[r - 1]] != sr;
+          const int v = sh.by_rank[r - 1] != sr;
           valid[r] = v;
           distinct += v;
         }
@@ -174,25 +252,19 @@ __global__ void __launch_bounds__(kThreads) k_route(const float* __restrict__ sc
       // D[1][j]
       for (int j = tid; j <= n; j += kThreads)
         dbuf0[j] = (j >= 1 && valid[j]) ? group_cost(p1, p2, 0, j) : inf;
+      if (tid == 0) {
+        flags[0] = 1;
+        flags[1] = k;
+      }
       __syncthreads();
+      if (n_cta > 1) cluster_sync_all();  // the helpers see the prefix sums, the first row and the verdict
+      verdict_out = true;
       double* dprev = dbuf0;
       double* dcur = dbuf1;
       for (int c = 2; c <= k; ++c) {
-        for (int j = tid; j <= n; j += kThreads) {
-          double best = inf;
-          int bi = 0;
-          if (j >= c && valid[j]) {
-            for (int i = c - 1; i < j; ++i) {
-              const double dp = dprev[i];
-              if (dp == inf) continue;
-              const double tot = dadd(dp, group_cost(p1, p2, i, j));
-              if (tot < best) { best = tot; bi = i; }
-            }
-          }
-          dcur[j] = best;
-          arg[(size_t)(c - 2) * np1 + j] = bi;
-        }
+        dp_row(c, n, p1, p2, valid, dprev, dcur, arg + (size_t)(c - 2) * np1, warp_id, n_warps, lane);
         __syncthreads();
+        if (n_cta > 1) cluster_sync_all();  // every block's rows are written before the next row reads them
         double* t = dprev; dprev = dcur; dcur = t;
       }
       if (tid == 0) {
@@ -229,6 +301,11 @@ __global__ void __launch_bounds__(kThreads) k_route(const float* __restrict__ sc
     }
   }
   __syncthreads();
+  if (n_cta > 1 && !verdict_out) {  // nothing to cluster: release the helpers
+    if (tid == 0) flags[0] = 0;
+    __syncthreads();
+    cluster_sync_all();
+  }
 
   const int lo_keep = sh.lo_keep, hi_keep = sh.hi_keep;
   int n_new = hi_keep - lo_keep;
@@ -324,10 +401,25 @@ cudaError_t launch_route(const float* scores, const int* cu_old, const int* seq2
   static std::atomic<unsigned long long> smem_set{0};
   if (cudaError_t e = ensure_dynamic_smem(k_route, (int)sizeof(Shared), smem_set)) return e;
   if (n < 0 || n > kMaxCandidates) return cudaErrorInvalidValue;
-  k_route<<<1, kThreads, sizeof(Shared), st>>>(scores, cu_old, seq2orig_old, n, p, cu_new, seq2orig_new,
-                                               old_of_new, state, res_idx, res_score, rec, trace_scores,
-                                               trace_ids, (unsigned char*)scratch);
-  return cudaGetLastError();
+  // the quadratic part (n^2 / 2 group costs per cost-table row, an fp64 division each) is shared by a cluster of
+  // eight blocks once it dominates
+  const int n_cta = (n >= 512 && p.mode == 2 && !p.is_final) ? 8 : 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(n_cta);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = sizeof(Shared);
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = n_cta;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  unsigned char* scr = (unsigned char*)scratch;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, k_route, scores, cu_old, seq2orig_old, n, p, cu_new, seq2orig_new, old_of_new, state,
+                                     res_idx, res_score, rec, trace_scores, trace_ids, scr, n_cta);
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 }  // namespace prism

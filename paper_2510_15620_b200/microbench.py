@@ -7,6 +7,7 @@ synthetic operands, one JSON line per run.  Also the small-case driver for profi
     python -m paper_2510_15620_b200.microbench --op gemm_bias --m 35200 --n 4096 --k 1024 --epilogue 2   (encoder stack)
     python -m paper_2510_15620_b200.microbench --op layernorm --rows 35200 --d 1024
     python -m paper_2510_15620_b200.microbench --op dequant --n 12288 --k 4096          (W4 -> bf16, group 128)
+    python -m paper_2510_15620_b200.microbench --op probe|route --seqs 1000                (score probe; prune decision)
     python -m paper_2510_15620_b200.microbench --op attention --head-dim 64 --hq 16 --hkv 16 --causal 0
 """
 from __future__ import annotations
@@ -40,7 +41,7 @@ def _time(fn, iters, warmup, flush):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--op", required=True, choices=["gemm", "qkv_rope", "attention", "rmsnorm", "rope", "compact", "gemm_bias", "layernorm", "dequant"])
+    ap.add_argument("--op", required=True, choices=["gemm", "qkv_rope", "attention", "rmsnorm", "rope", "compact", "gemm_bias", "layernorm", "dequant", "probe", "route"])
     ap.add_argument("--head-dim", type=int, default=128)
     ap.add_argument("--m", type=int, default=35200)
     ap.add_argument("--n", type=int, default=4096)
@@ -88,6 +89,41 @@ def main():
         fn = lambda: ops.prism_op_gemm_bias(A, B, bias, O, R, m, n, k, PRISM_BF16, a.epilogue, a.impl, err)
         med, best = _time(fn, a.iters, a.warmup, flush)
         out.update(m=m, n=n, k=k, epilogue=a.epilogue, ms=med, ms_min=best, tflops=2.0 * m * n * k / med / 1e9, err=int(err.item()))
+    elif a.op == "probe":
+        rng = np.random.default_rng(0)
+        lens = rng.integers(a.len_lo, a.len_hi + 1, size=a.seqs)
+        cu = np.zeros(a.seqs + 1, np.int32)
+        cu[1:] = np.cumsum(lens)
+        x = rnd(int(cu[-1]), a.d)
+        gain = torch.ones(a.d, dtype=torch.bfloat16, device=dev)
+        head = (rnd(2, a.d) * 0.02).to(torch.bfloat16)
+        sc = torch.empty(a.seqs, device=dev)
+        cud = torch.from_numpy(cu).to(dev)
+        fn = lambda: ops.prism_op_probe(x, cud, a.seqs, gain, head, PRISM_BF16, 1e-6, sc)
+        med, best = _time(fn, a.iters, a.warmup, flush)
+        out.update(seqs=a.seqs, d=a.d, ms=med, ms_min=best, gbs=a.seqs * a.d * 4.0 / med / 1e6,
+                   note="the op wrapper also builds the head-difference vector, allocates and synchronises; the kernel alone is in the profile")
+    elif a.op == "route":
+        n = a.seqs
+        rng = np.random.default_rng(0)
+        lens = rng.integers(a.len_lo, a.len_hi + 1, size=n)
+        cu = np.zeros(n + 1, np.int32)
+        cu[1:] = np.cumsum(lens)
+        t = lambda v: torch.from_numpy(v).to(dev)
+        scores = t(rng.normal(size=n).astype(np.float32))
+        cud, ids = t(cu), t(np.arange(n, dtype=np.int32))
+        state0 = t(np.array([n, cu[-1], 10, 0, 0, 0, 0, 0], np.int32))
+        state = state0.clone()
+        cu_new, s2o, oon = (torch.empty(n + 1, dtype=torch.int32, device=dev) for _ in range(3))
+        ridx, rsc = torch.empty(n + 1, dtype=torch.int32, device=dev), torch.empty(n + 1, device=dev)
+        rec = torch.zeros(ops.RECORD_BYTES, dtype=torch.uint8, device=dev)
+
+        def fn():
+            state.copy_(state0)
+            ops.prism_op_route(scores, cud, ids, n, 2, 0, 0.5, 3, 0, 1, 0, 8, cu_new, s2o, oon, state, ridx, rsc, rec)
+        med, best = _time(fn, a.iters, a.warmup, flush)
+        out.update(candidates=n, ms=med, ms_min=best,
+                   note="includes the op wrapper's scratch allocation; the kernel alone is in the profile")
     elif a.op == "dequant":
         n, k, grp = a.n, a.k, 128
         ng = k // grp
