@@ -347,3 +347,24 @@ def test_cfg1_full_size_in_bench_configuration(P):
           f"tokens per layer {tr.tokens_per_layer}")
     assert any(r.fired for r in tr.records)
     model.close()
+
+
+def test_maximum_candidate_count_end_to_end(P):
+    """N = 4096 (PRISM_MAX_CANDIDATES) short candidates through a small bf16 model: every step that scales with N
+    (packing, probe, ranking and partition on a cluster of blocks, compaction) against the oracle."""
+    cfg = ModelCfg(n_layers=3, hidden=256, n_q_heads=2, n_kv_heads=1, head_dim=128, ffn=256, vocab=512, rope_theta=1e4,
+                   qk_norm=1, dtype=DTYPE_BF16, yes_id=3, no_id=4)
+    wl = Workload("max_n_bf16", cfg, 4096, 7, 8, ("uniform", 1, 40, 1, 40), Schedule(MODE_CLUSTER, (1, 2), cv_threshold=0.2),
+                  cfg_index=13)
+    w = synth.make_weights(cfg, seed=9)
+    req = synth.make_request(wl, 0)
+    S = oracle.score_matrix(req["query"], req["cand_tokens"], req["cand_offsets"], w, cfg, [1, 2, 3])
+    model = make_model(P, cfg, w, req)
+    for sched in (wl.schedule, Schedule(MODE_NONE)):
+        idx, sc, tr = run(P, model, req, wl.top_k, sched)
+        assert tr.records[0].n_active_before == 4096
+        check_scores(tr, S, TOL_BF16)
+        check_replay(tr, idx, sc, wl.n_candidates, wl.top_k, cfg.n_layers, sched)
+        check_end_to_end(tr, idx, S, wl.n_candidates, wl.top_k, cfg.n_layers, sched, TOL_BF16)
+    assert tr.shared_prefix_rows == 8
+    model.close()
