@@ -189,8 +189,12 @@ k_attention_tc2(const __grid_constant__ CUtensorMap map_qkv, const __grid_consta
           // Shared query prefix: rows 0 .. prefix-1 of the batch belong to every sequence, cu[s] is the first row
           // of the sequence's own part.  Row v of the sequence is batch row v (v < prefix) or beg + v - prefix.
           const int b = __ldg(cu + s);
-          it.len = prefix + __ldg(cu + s + 1) - b;
+          const int own = __ldg(cu + s + 1) - b;
+          it.len = prefix + own;
           if (it.qb * BM >= it.len) continue;
+          // a sequence without rows of its own (an empty document, or another rank's candidate) needs no item:
+          // the prefix rows it would compute are the ones the launch's first sequence writes
+          if (prefix > 0 && own == 0 && sl != 0) continue;
           it.beg = b - row0;
           it.first = sl == 0;
           const int kv_end = causal ? min(it.len, (it.qb + 1) * BM) : it.len;

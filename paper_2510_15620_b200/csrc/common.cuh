@@ -50,6 +50,7 @@ struct RouteParams {
   int is_final;  // 1: last layer, append the best k_rem and stop
   int layer;
   int prefix;    // shared query prefix: rows in front of the batch that belong to every sequence (0 = none)
+  const unsigned char* owned;  // candidate-sharded run with a prefix: which original candidates this rank runs (else null)
 };
 
 // Request state that lives on the device and is mirrored to the host after every scored layer.
@@ -60,7 +61,8 @@ struct RouteState {
   int n_result;
   int done;
   int err;
-  int pad0, pad1;
+  int pad0;  // written by the routing kernel: survivors that this rank runs (all of them unless candidate-sharded)
+  int pad1;
 };
 
 struct ProbeRecordDev {  // layout mirrors prism_probe_record
@@ -124,7 +126,8 @@ cudaError_t launch_qknorm_rope(void* qkv, int dtype, const int* pos, int rows, i
                                const void* g_k, float eps, const float* cos_t, const float* sin_t,
                                cudaStream_t st);
 cudaError_t launch_probe(const float* x, const int* cu, int n, int d, const void* g_final, int dtype,
-                         const float* w_diff, float eps, float* scores, cudaStream_t st, int prefix = 0);
+                         const float* w_diff, float eps, float* scores, cudaStream_t st, int prefix = 0,
+                         const unsigned char* owned = nullptr, const int* seq2orig = nullptr);
 // ---- encoder stack (post-norm blocks with LayerNorm, learned positions, first-token classification head) ----
 // x[t,:] = table[tokens[t],:] + pos_table[pos[t] + pos_offset,:] + type_row (fp32 sum; the embedding LayerNorm is
 // the first norm of the first block)

@@ -557,16 +557,19 @@ __global__ void __launch_bounds__(256) k_qknorm_rope(T* __restrict__ qkv, const 
 template <typename WT>
 __global__ void __launch_bounds__(256) k_probe(const float* __restrict__ x, const int* __restrict__ cu, int d,
                                                const WT* __restrict__ g_final, const float* __restrict__ w_diff,
-                                               float eps, int prefix, float* __restrict__ scores) {
+                                               float eps, int prefix, const unsigned char* __restrict__ owned,
+                                               const int* __restrict__ seq2orig, float* __restrict__ scores) {
   __shared__ float red[32];
   const int i = blockIdx.x;
   int last = cu[i + 1] - 1;
   if (cu[i + 1] == cu[i]) {
-    if (prefix == 0) {  // a sequence without rows (another rank's candidate): its score comes from there
+    // a sequence without rows: another rank's candidate (its score comes from there), or, with a shared query
+    // prefix, this rank's candidate with an empty document, which ends with the query
+    if (prefix == 0 || (owned && !owned[seq2orig[i]])) {
       if (threadIdx.x == 0) scores[i] = 0.f;
       return;
     }
-    last = prefix - 1;  // shared query prefix and an empty document: the sequence ends with the query
+    last = prefix - 1;
   }
   const float* row = x + (size_t)last * d;
   float ss = 0.f, dot = 0.f;
@@ -857,12 +860,15 @@ cudaError_t launch_qknorm_rope(void* qkv, int dtype, const int* pos, int rows, i
 }
 
 cudaError_t launch_probe(const float* x, const int* cu, int n, int d, const void* g_final, int dtype,
-                         const float* w_diff, float eps, float* scores, cudaStream_t st, int prefix) {
+                         const float* w_diff, float eps, float* scores, cudaStream_t st, int prefix,
+                         const unsigned char* owned, const int* seq2orig) {
   if (n <= 0) return cudaSuccess;
+  if (owned && !seq2orig) return cudaErrorInvalidValue;
   if (dtype == 1)
-    k_probe<__nv_bfloat16><<<n, 256, 0, st>>>(x, cu, d, (const __nv_bfloat16*)g_final, w_diff, eps, prefix, scores);
+    k_probe<__nv_bfloat16><<<n, 256, 0, st>>>(x, cu, d, (const __nv_bfloat16*)g_final, w_diff, eps, prefix, owned, seq2orig,
+                                              scores);
   else
-    k_probe<float><<<n, 256, 0, st>>>(x, cu, d, (const float*)g_final, w_diff, eps, prefix, scores);
+    k_probe<float><<<n, 256, 0, st>>>(x, cu, d, (const float*)g_final, w_diff, eps, prefix, owned, seq2orig, scores);
   return cudaGetLastError();
 }
 

@@ -969,8 +969,11 @@ int select_impl(prism_handle* h, const int32_t* query, int32_t lq, const int32_t
     if (h->h_off[i + 1] < h->h_off[i]) return fail(h, PRISM_ERR_BAD_INPUT, "cand_offsets not monotone");
   // Shared query prefix: under causal attention the query's rows are the same in every sequence, so they are
   // stored and computed once in front of the documents (rows [0, lq)); cu then holds document rows only.
-  const int prefix = (c.shared_prefix == PRISM_PREFIX_AUTO && !h->enc && h->fa == 3 && c.causal && !h->offload && !shard && N >= 2 &&
-                      lq >= 8 && lq <= 120 && (lq & 7) == 0 && (long long)lq + h->h_off[N] <= h->chunk_tokens)
+  long long own_docs = 0;  // document tokens of the candidates this rank runs
+  for (int i = 0; i < N; ++i)
+    if (!shard || shard->owned[i]) own_docs += (long long)h->h_off[i + 1] - h->h_off[i];
+  const int prefix = (c.shared_prefix == PRISM_PREFIX_AUTO && !h->enc && h->fa == 3 && c.causal && !h->offload && N >= 2 &&
+                      lq >= 8 && lq <= 120 && (lq & 7) == 0 && (long long)lq + own_docs <= h->chunk_tokens)
                          ? lq
                          : 0;
   if (prefix) {
@@ -1030,6 +1033,11 @@ int select_impl(prism_handle* h, const int32_t* query, int32_t lq, const int32_t
   }
 
   int n = N, T = (int)total, n_rec = 0, probe_j = 0, layers_run = 0, chunks_max = 0;
+  int n_mine = N;  // live candidates this rank runs
+  if (shard) {
+    n_mine = 0;
+    for (int i = 0; i < N; ++i) n_mine += shard->owned[i] ? 1 : 0;
+  }
   bool done = false;
   // hidden-state offload bookkeeping
   bool main_dirty = true, slot_used[3] = {false, false, false};
@@ -1124,7 +1132,7 @@ int select_impl(prism_handle* h, const int32_t* query, int32_t lq, const int32_t
     }
     if (h->offload) chunk_out_valid = chunks;  // the next layer's chunk c waits for this layer's write-back of chunk c
     chunks_max = std::max(chunks_max, chunks);
-    if (trace && trace->tokens_per_layer) trace->tokens_per_layer[l] = prefix ? T - prefix + n * prefix : T;
+    if (trace && trace->tokens_per_layer) trace->tokens_per_layer[l] = prefix ? T - prefix + n_mine * prefix : T;
     layers_run = l + 1;
     if (streamed) {
       PRISM_CUDA(h, cudaEventRecord(h->ev_freed[s], st));
@@ -1149,6 +1157,7 @@ int select_impl(prism_handle* h, const int32_t* query, int32_t lq, const int32_t
       p.is_final = is_final ? 1 : 0;
       p.layer = layers_run;
       p.prefix = prefix;
+      p.owned = (prefix && shard) ? h->owned_dev : nullptr;
       const int nxt = cur ^ 1;
       float* score_buf = shard ? shard->exchange : h->scores;
       if (h->enc) {
@@ -1159,7 +1168,8 @@ int select_impl(prism_handle* h, const int32_t* query, int32_t lq, const int32_t
         h->launches += 2;  // the probe is three kernels
       } else
       PRISM_LAUNCH_P(h, st, PRISM_K_PROBE, 4.0 * n * c.hidden,
-                     launch_probe(h->x[cur], h->cu[cur], n, c.hidden, h->g_final, c.dtype, h->w_diff, c.rms_eps, score_buf, st, prefix));
+                     launch_probe(h->x[cur], h->cu[cur], n, c.hidden, h->g_final, c.dtype, h->w_diff, c.rms_eps, score_buf, st, prefix,
+                                  (prefix && shard) ? h->owned_dev : nullptr, h->seq2orig[cur]));
       if (shard && shard->reduce(shard->ctx, n, st) != 0) return fail(h, PRISM_ERR_CUDA, "the score exchange callback failed");
       PRISM_LAUNCH_P(h, st, PRISM_K_ROUTE, 8.0 * n, launch_route(score_buf, h->cu[cur], h->seq2orig[cur], n, p, h->cu[nxt], h->seq2orig[nxt], h->old_of_new,
                                    h->state, h->res_idx, h->res_score, h->recs + n_rec,
@@ -1186,6 +1196,7 @@ int select_impl(prism_handle* h, const int32_t* query, int32_t lq, const int32_t
         cur = nxt;
         n = stt.n_active;
         T = stt.n_tokens;
+        n_mine = stt.pad0;
       }
     }
     if (streamed && !done && l + 2 < c.n_layers) {

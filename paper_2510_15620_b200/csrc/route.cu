@@ -27,6 +27,8 @@ struct Shared {
   int cuts[kMaxClusters];
   int k_eff;
   int do_cluster;
+  int n_owned;      // active candidates this rank runs (candidate-sharded runs with a shared prefix)
+  int n_owned_new;  // the same among the survivors
 };
 
 // Inclusive warp scan.
@@ -161,13 +163,13 @@ __global__ void __launch_bounds__(kThreads) k_route(const float* __restrict__ sc
 
   const int k_rem = state->k_rem;
   const int n_result = state->n_result;
-  // with a shared query prefix the batch holds the prefix rows once: report the sequences' own token count
-  const int tokens_before = p.prefix ? (cu_old[n] - p.prefix) + n * p.prefix : cu_old[n];
-
+  if (tid == 0) sh.n_owned = 0;
+  __syncthreads();
   for (int i = tid; i < n; i += kThreads) {
     if (trace_scores) trace_scores[i] = scores[i];
     if (trace_ids) trace_ids[i] = seq2orig_old[i];
     if (n_cta > 1) sh.rank[i] = rank_g[i];
+    if (p.prefix && p.owned && p.owned[sh.id[i]]) atomicAdd(&sh.n_owned, 1);
   }
   if (tid == 0) {
     sh.lo_keep = 0;
@@ -180,6 +182,9 @@ __global__ void __launch_bounds__(kThreads) k_route(const float* __restrict__ sc
 
   for (int r = tid; r < n; r += kThreads) sh.by_rank[r] = sh.score[sorted[r]];
   __syncthreads();
+  // with a shared query prefix the batch holds the prefix rows once: report query + document per sequence this
+  // rank runs (all of them, unless the candidates are sharded over ranks)
+  const int tokens_before = p.prefix ? (cu_old[n] - p.prefix) + (p.owned ? sh.n_owned : n) * p.prefix : cu_old[n];
 
   int fired = 0, n_selected = 0, n_dropped = 0, n_deferred = n, append_lo = 0, append_hi = 0;
   int k_after = k_rem, done = 0;
@@ -333,7 +338,7 @@ __global__ void __launch_bounds__(kThreads) k_route(const float* __restrict__ sc
   // ---- survivor offsets: stable compaction in batch order ---------------------------------
   int total_new = 0;
   if (!done) {
-    if (tid == 0) { sh.carry_a = 0; sh.carry_b = p.prefix; }  // the prefix rows stay in front
+    if (tid == 0) { sh.carry_a = 0; sh.carry_b = p.prefix; sh.n_owned_new = 0; }  // the prefix rows stay in front
     __syncthreads();
     for (int base = 0; base < n; base += kThreads) {
       const int i = base + tid;
@@ -358,6 +363,7 @@ __global__ void __launch_bounds__(kThreads) k_route(const float* __restrict__ sc
         cu_new[ea] = eb;
         seq2orig_new[ea] = sh.id[i];
         old_of_new[ea] = i;
+        if (p.owned && p.owned[sh.id[i]]) atomicAdd(&sh.n_owned_new, 1);
       }
       __syncthreads();
       if (tid == kThreads - 1) { sh.carry_a += sh.warp_a[31]; sh.carry_b += sh.warp_b[31]; }
@@ -376,6 +382,7 @@ __global__ void __launch_bounds__(kThreads) k_route(const float* __restrict__ sc
     state->k_rem = k_after;
     state->n_result = n_res_after;
     state->done = done;
+    state->pad0 = (!done && p.owned) ? sh.n_owned_new : n_new;  // survivors this rank runs
     if (rec) {
       rec->layer = p.layer;
       rec->n_active_before = n;

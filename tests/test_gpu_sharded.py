@@ -96,6 +96,11 @@ def test_sharded_equals_unsharded(P, mid_case, world):
         ref_idx, ref_sc, ref_tr = run(P, base, req, MID_WL.top_k, sched)
         out, calls = run_sharded(P, MID, w, req, MID_WL.top_k, sched, owner, world)
         assert calls == len(ref_tr.records)                        # one exchange per scored layer, nothing else
+        # the query's rows are shared on every rank too, and the ranks' token counts add up to the unsharded ones
+        assert ref_tr.shared_prefix_rows == len(req["query"]) and all(o[2].shared_prefix_rows == len(req["query"]) for o in out)
+        assert [sum(t) for t in zip(*[o[2].tokens_per_layer for o in out])] == ref_tr.tokens_per_layer
+        assert [sum(r.tokens_before for r in recs) for recs in zip(*[o[2].records for o in out])] == \
+               [r.tokens_before for r in ref_tr.records]
         for idx, sc, tr in out:
             assert np.array_equal(idx, ref_idx)
             assert np.array_equal(sc.view(np.uint32), ref_sc.view(np.uint32))
