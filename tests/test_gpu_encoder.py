@@ -305,3 +305,31 @@ def test_encoder_embedding_row_cache_is_result_neutral(P):
         assert np.array_equal(a[0], b[0]) and np.array_equal(a[1].view(np.uint32), b[1].view(np.uint32))
     hits, misses, evictions = cached.embed_cache_stats()
     assert misses > 0 and hits > 0 and evictions == 0
+
+
+@pytest.mark.parametrize("cfg,wl,tol", [(replace(ENC_TINY, causal=1), ENC_TINY_WL, TOL_FP32), (replace(ENC_MID, causal=1, n_layers=3), ENC_MID_WL, TOL_BF16)],
+                         ids=["fp32", "bf16"])
+def test_encoder_blocks_with_causal_attention(P, cfg, wl, tol):
+    """The causal flag on the encoder blocks (a post-norm decoder with learned positions): not one of the paper's
+    models, but the flag is honoured by every attention kernel and the oracle alike."""
+    w = synth.make_weights(cfg, seed=3)
+    if cfg.n_layers < len(w["layers"]):
+        w = dict(w, layers=w["layers"][:cfg.n_layers])
+    req = synth.make_request(wl, 3)
+    layers = list(range(1, cfg.n_layers + 1))
+    S = oracle.score_matrix(req["query"], req["cand_tokens"], req["cand_offsets"], w, cfg, layers)
+    S_bi = oracle.score_matrix(req["query"], req["cand_tokens"], req["cand_offsets"], w, replace(cfg, causal=0), layers[-1:],
+                               candidates=[0, 1])
+    assert np.max(np.abs(S_bi[layers[-1]] - S[layers[-1]][:2])) > 1e-3              # the flag matters
+    # under causal attention the first token sees only itself: every candidate of a request scores the same, which
+    # makes this a test of exact ties as well (equal scores bit for bit, order by candidate index)
+    assert np.ptp(S[layers[-1]]) < 1e-12
+    m = make_model(P, cfg, w, req)
+    sched = Schedule(MODE_FIXED_KEEP, tuple(layers[:-1]), tuple([wl.n_candidates] * (cfg.n_layers - 1)))
+    idx, sc, tr = run(P, m, req, wl.top_k, sched)
+    assert [r.layer for r in tr.records] == layers
+    check_scores(tr, S, tol)
+    check_replay(tr, idx, sc, wl.n_candidates, wl.top_k, cfg.n_layers, sched)
+    assert tr.shared_prefix_rows == 0
+    assert len(set(np.asarray(tr.records[-1].scores).view(np.uint32).tolist())) == 1 and list(idx) == list(range(wl.top_k))
+    m.close()
