@@ -309,6 +309,32 @@ def run_prism(args):
     h2d = int(np.mean([q.nbytes + c.nbytes + o.nbytes for q, c, o in hreqs]))
     d2h = int(hidx.nbytes + hsc.nbytes)
 
+    # document tokens only (the query is shared by all candidates of a request), beside the headline count
+    doc_toks = sum(int(lens_all[(W + i) % n_req].sum()) - lq * len(lens_all[(W + i) % n_req]) for i in range(K))
+    doc_toks_all = float(doc_toks) if by_cand else sum_over_ranks(float(doc_toks), world, dev)
+
+    # streamed workloads: what crosses the host link per request, and the time that alone would take
+    host_link = None
+    if wl.stream_weights and rank == 0 and not by_cand:
+        probe_host = torch.empty(1 << 30, dtype=torch.uint8).pin_memory()
+        probe_dev = torch.empty(1 << 30, dtype=torch.uint8, device=dev)
+        for _ in range(2):
+            probe_dev.copy_(probe_host, non_blocking=True)
+        ea, eb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ea.record()
+        for _ in range(3):
+            probe_dev.copy_(probe_host, non_blocking=True)
+        eb.record()
+        torch.cuda.synchronize()
+        h2d_gbs = 3 * (1 << 30) / (ea.elapsed_time(eb) * 1e-3) / 1e9
+        layer_bytes = tensor_bytes(tw["layers"], False) / cfg.n_layers
+        runs = [model.select(*dreqs[i], wl.top_k, sched, want_trace=True)[2].layers_run for i in range(n_req)]
+        per_req = float(np.mean(runs)) * layer_bytes
+        host_link = {"pinned_h2d_gbs": h2d_gbs, "layer_bytes": int(layer_bytes), "layers_streamed_per_request": float(np.mean(runs)),
+                     "bytes_per_request": int(per_req), "floor_ms": per_req / (h2d_gbs * 1e9) * 1e3,
+                     "note": "streaming stops when the forward terminates; the floor is bytes / measured pinned copy rate"}
+        del probe_host, probe_dev
+
     # the same kernels with pruning disabled -> what pruning buys on this workload
     off_ms, _, _ = timed(lambda i: dev_step(i, Schedule(MODE_NONE)), max(3, K // 4), 3)
     off_ms = max_over_ranks(off_ms / max(3, K // 4), world, dev)
@@ -333,6 +359,7 @@ def run_prism(args):
                        "parallelism": (f"{world} ranks share each request's candidates, one score all-reduce per probe"
                                        if by_cand else f"dp{world} over requests")},
             "latency_ms": {"p50": float(np.percentile(lat, 50)), "p99": float(np.percentile(lat, 99))},
+            "doc_tokens_per_s": doc_toks_all / (total_ms * 1e-3), "host_link": host_link,
             "pruning_off_ms_per_step": off_ms, "pruning_speedup": off_ms / (total_ms / K),
             "e2e": {"value": toks_all / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "p50_ms": float(np.percentile(e2e_lat, 50))},
@@ -387,6 +414,15 @@ def run_prism(args):
                             "traffic_note": "bytes per launch: ncu dram read+write of each GEMM shape at M = 8192 "
                                             "(profiles/gemm_tc2_*.md) scaled by the rows each launch processed",
                             "share_of_kernel_time": g_ms / tot_ms if tot_ms else None}
+        # the whole request against the tensor roofline: algorithmic flops of the live tokens (GEMMs and attention of
+        # the profiled steps, pruning included) over the request time, against the measured and the nominal peak
+        req_fl = g_fl + per["attention"]["work_per_step"]
+        req_tf = req_fl / (total_ms / K * 1e-3) / 1e12
+        line["request_roofline"] = {"flops_per_request": req_fl, "achieved_tflops": req_tf,
+                                    "frac_of_sustained_peak": req_tf / peak if peak else None,
+                                    "frac_of_burst_peak": req_tf / peaks["bf16_tflops"], "frac_of_nominal_2250": req_tf / 2250.0,
+                                    "note": "sum over layers of live tokens x 2 x layer parameters, plus attention flops, "
+                                            "divided by the request time (kernels of every kind, host round trips included)"}
         line["kernels"] = {n: {"ms_per_step": round(v["ms_per_step"], 4), "share": round(v["ms_per_step"] / tot_ms, 4),
                                "launches_per_step": v["launches_per_step"],
                                ("tflops" if n in GEMM_CLASSES or n == "attention" else "gbs"):
