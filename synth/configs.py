@@ -115,6 +115,12 @@ WORKLOADS: List[Workload] = [
     # beyond the five benchmark configurations: the encoder stack on cfg 1's request recipe
     Workload("cfg5_bge_m3_shaped", _BGE_M3, 100, 10, 32, ("uniform", 128, 512, 128, 512),
              Schedule(MODE_CLUSTER, (6, 9, 12, 15, 18, 21), cv_threshold=0.5), cfg_index=5),
+    # the request sizes of the paper's own measurements (Sec. 2.2 and Sec. 6: top-5 of 20 and top-10 of 60 candidates
+    # of at most 512 tokens, about 500 on average), on the 0.6B-shaped model: context beside the scaled-up workloads
+    Workload("cfg6_paper_20x500_0p6b", _QWEN3_06B, 20, 5, 32, ("uniform", 440, 480, 440, 480),
+             Schedule(MODE_CLUSTER, (8, 12, 16, 20, 24), cv_threshold=0.5), cfg_index=16),
+    Workload("cfg7_paper_60x500_0p6b", _QWEN3_06B, 60, 10, 32, ("uniform", 440, 480, 440, 480),
+             Schedule(MODE_CLUSTER, (8, 12, 16, 20, 24), cv_threshold=0.5), cfg_index=17),
 ]
 
 
