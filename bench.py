@@ -206,6 +206,12 @@ def run_prism(args):
         dist.init_process_group("nccl", device_id=dev)
 
     wl = synth.workload(args.workload)
+    # memory options of the handle (Sec. 4.2 - 4.4) on top of what the workload prescribes
+    from dataclasses import replace as _replace
+    if args.stream_weights:
+        wl = _replace(wl, stream_weights=1)
+    if args.activation_budget_mb:
+        wl = _replace(wl, activation_budget_bytes=int(args.activation_budget_mb) << 20)
     cfg = wl.model
     n_req = max(args.requests, 1)
     by_cand = args.shard == "candidates"
@@ -224,10 +230,12 @@ def run_prism(args):
     w4 = args.weight_format == "w4"
     if w4:  # Sec. 6.1's quantised arm: 4-bit codes + bf16 scale and 4-bit zero point per 128 input channels
         w_np = synth.quantize_weights(w_np, 128)
-    tw = P.upload_weights(w_np, cfg.dtype, device=str(dev), layers_pinned_host=bool(wl.stream_weights))
+    tw = P.upload_weights(w_np, cfg.dtype, device=str(dev), layers_pinned_host=bool(wl.stream_weights),
+                          embed_pinned_host=args.embed_cache_rows > 0)
     model = P.PrismModel(cfg, tw, max_seq, wl.n_candidates, max_tot, activation_budget_bytes=wl.activation_budget_bytes,
                          stream_weights=bool(wl.stream_weights), shared_prefix=args.shared_prefix == "on",
-                         weight_format=P.PRISM_WFMT_W4 if w4 else P.PRISM_WFMT_PLAIN, quant_group=128 if w4 else 0)
+                         weight_format=P.PRISM_WFMT_W4 if w4 else P.PRISM_WFMT_PLAIN, quant_group=128 if w4 else 0,
+                         embed_cache_rows=args.embed_cache_rows, hidden_offload=args.hidden_offload)
     d = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(dev)
     dreqs = [(d(r["query"]), d(r["cand_tokens"]), d(r["cand_offsets"])) for r in reqs]
     pin = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).pin_memory().numpy()
@@ -349,6 +357,8 @@ def run_prism(args):
                        "weight_format": "w4a16 (round-to-nearest, group 128)" if w4 else "bf16" if cfg.dtype == 1 else "f32",
                        # what the request holds: the caller's weight tensors on the device and in pinned host memory
                        # (streamed layers), and everything the handle allocated on the device (activations, slots, scratch)
+                       "handle_options": {"stream_weights": bool(wl.stream_weights), "activation_budget_bytes": wl.activation_budget_bytes,
+                                          "embed_cache_rows": args.embed_cache_rows, "hidden_offload": bool(args.hidden_offload)},
                        "memory_bytes": {"weights_device": tensor_bytes(tw, True), "weights_pinned_host": tensor_bytes(tw, False),
                                         "handle_device": workspace_bytes},
                        "shared_query_prefix_rows": prefix_rows,
@@ -457,6 +467,10 @@ def main():
     ap.add_argument("--shared-prefix", default="on", choices=["on", "off"],
                     help="on: the query's rows are stored and computed once per request where the path supports it "
                          "(causal attention; results are bit-identical); off: one query copy per candidate")
+    ap.add_argument("--stream-weights", action="store_true", help="layer weights in pinned host memory, two device slots (Sec. 4.2)")
+    ap.add_argument("--activation-budget-mb", type=int, default=0, help="chunked execution under this budget (Sec. 4.3)")
+    ap.add_argument("--embed-cache-rows", type=int, default=0, help="embedding table in pinned host memory, LRU row cache (Sec. 4.4)")
+    ap.add_argument("--hidden-offload", action="store_true", help="hidden states in pinned host memory, three device chunks (Sec. 4.3)")
     ap.add_argument("--weight-format", default="plain", choices=["plain", "w4"],
                     help="w4: the layer matrices are stored (and, for the streamed workload, copied) as 4-bit codes and "
                          "rebuilt as bf16 layer by layer on the device")
