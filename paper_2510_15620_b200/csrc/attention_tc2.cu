@@ -118,7 +118,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 k_attention_tc2(const __grid_constant__ CUtensorMap map_qkv, const __grid_constant__ CUtensorMap map_pre,
                 const __grid_constant__ CUtensorMap map_rest, __nv_bfloat16* __restrict__ out,
                 const int* __restrict__ cu, int seq0, int nseq, int row0, int nqb, int gsz, int hq, int hkv,
-                int causal, int reverse, int prefix, float scale_log2, int* __restrict__ sched,
+                int causal, int reverse, int prefix, int write_prefix, float scale_log2, int* __restrict__ sched,
                 int* __restrict__ err) {
   extern __shared__ unsigned char smem_raw[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -194,9 +194,9 @@ k_attention_tc2(const __grid_constant__ CUtensorMap map_qkv, const __grid_consta
           if (it.qb * BM >= it.len) continue;
           // a sequence without rows of its own (an empty document, or another rank's candidate) needs no item:
           // the prefix rows it would compute are the ones the launch's first sequence writes
-          if (prefix > 0 && own == 0 && sl != 0) continue;
+          if (prefix > 0 && own == 0 && !(write_prefix && sl == 0)) continue;
           it.beg = b - row0;
-          it.first = sl == 0;
+          it.first = write_prefix && sl == 0;
           const int kv_end = causal ? min(it.len, (it.qb + 1) * BM) : it.len;
           it.n_blocks = (kv_end + BN - 1) / BN;
           break;
@@ -558,7 +558,7 @@ __device__ int g_sched[kTickets][2];
 
 cudaError_t launch_attention_tc2(const void* qkv, void* out, const int* cu, int seq0, int nseq, int row0, int rows,
                                  int max_len, int n_q_heads, int n_kv_heads, int causal, int* err, cudaStream_t st,
-                                 bool reverse, int prefix) {
+                                 bool reverse, int prefix, const void* qkv_prefix, bool write_prefix) {
   if (nseq <= 0 || max_len <= 0 || rows <= 0) return cudaSuccess;
   if (n_kv_heads < 1 || n_q_heads % n_kv_heads || ((n_q_heads / n_kv_heads) & 1)) return cudaErrorInvalidValue;
   static std::atomic<unsigned long long> smem_set{0};
@@ -572,8 +572,12 @@ cudaError_t launch_attention_tc2(const void* qkv, void* out, const int* cu, int 
   mrest = mq;
   if (prefix) {
     // shared query prefix: max_len counts prefix + own rows; the first block of every tile is two boxes
-    if (prefix < 8 || prefix > 120 || (prefix & 7) || row0 != 0 || seq0 != 0 || !causal) return cudaErrorInvalidValue;
-    e = make_tma_2d_bf16(&mpre, qkv, (uint64_t)rows, ld, (uint32_t)prefix, 64);
+    // qkv_prefix: the q/k/v rows of the prefix (row 0 of that buffer is prefix row 0); null: they are the first rows
+    // of qkv.  write_prefix: this launch's first sequence stores the prefix rows of the output (rows 0.. of out).
+    if (prefix < 8 || prefix > 120 || (prefix & 7) || !causal) return cudaErrorInvalidValue;
+    if (!qkv_prefix && row0 != 0) return cudaErrorInvalidValue;
+    e = qkv_prefix ? make_tma_2d_bf16(&mpre, qkv_prefix, (uint64_t)prefix, ld, (uint32_t)prefix, 64)
+                   : make_tma_2d_bf16(&mpre, qkv, (uint64_t)rows, ld, (uint32_t)prefix, 64);
     if (e == cudaSuccess) e = make_tma_2d_bf16(&mrest, qkv, (uint64_t)rows, ld, (uint32_t)(128 - prefix), 64);
     if (e != cudaSuccess) return e;
   }
@@ -604,7 +608,7 @@ cudaError_t launch_attention_tc2(const void* qkv, void* out, const int* cu, int 
                                                       reinterpret_cast<const CUtensorMap&>(mpre),
                                                       reinterpret_cast<const CUtensorMap&>(mrest), (__nv_bfloat16*)out, cu,
                                                       seq0, nseq, row0, nqb, gsz, n_q_heads, n_kv_heads, causal, reverse ? 1 : 0,
-                                                      prefix, scale_log2,
+                                                      prefix, write_prefix ? 1 : 0, scale_log2,
                                                       sched, err);
   return cudaGetLastError();
 }

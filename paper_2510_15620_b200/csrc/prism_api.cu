@@ -43,6 +43,7 @@ struct prism_handle {
   std::vector<EncVec> enc_vec;
   const void *pos_embed = nullptr, *head_dense_w = nullptr;
   float* probe_scratch = nullptr;  // [2, max_candidates, D]
+  void* qkv_prefix = nullptr;      // q/k/v rows of a shared query prefix, kept for the later chunks of a layer
   // W4 weights (cfg.weight_format == PRISM_WFMT_W4): the layer about to run is rebuilt as bf16 here
   bool w4 = false;
   void* wq[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};  // w_qkv, w_o, w_gate, w_up, w_down
@@ -517,6 +518,7 @@ static int create_impl(prism_handle* h, const prism_model_cfg* cfg, const prism_
   PRISM_CUDA(h, dev_alloc(h, (unsigned char**)&h->qkv, chunk * nqkv * h->esz));
   PRISM_CUDA(h, dev_alloc(h, (unsigned char**)&h->attn, chunk * hd * h->esz));
   PRISM_CUDA(h, dev_alloc(h, (unsigned char**)&h->hbuf, chunk * (size_t)c.ffn * h->esz));
+  PRISM_CUDA(h, dev_alloc(h, (unsigned char**)&h->qkv_prefix, 128 * nqkv * h->esz));
   PRISM_CUDA(h, dev_alloc(h, &h->scores, N));
   PRISM_CUDA(h, dev_alloc(h, &h->res_idx, N));
   PRISM_CUDA(h, dev_alloc(h, &h->res_score, N));
@@ -732,8 +734,11 @@ cudaError_t gemm_tc_any(prism_handle* h, const TmaDesc& a, const TmaDesc& b0, co
 // x is the whole batch's hidden-state matrix, or (x_is_chunk) the buffer holding just this chunk's rows.
 // prefix > 0: rows [0, prefix) are the query shared by all sequences, cu holds the sequences' own rows, max_len
 // counts prefix + own rows (whole batch in one chunk, r0 = 0).
+// chunk_of_many: 0 = the batch is one chunk; 1 = first of several chunks (it holds the prefix rows: their q/k/v are
+// saved for the others); 2 = a later chunk (attention reads the saved prefix rows and writes none).
 int run_layer_chunk(prism_handle* h, const LayerDev& W, const LayerMaps* maps, float* x, const int* cu_dev, int s0, int s1,
-                    int r0, int rows, int max_len, cudaStream_t st, bool x_is_chunk = false, int prefix = 0) {
+                    int r0, int rows, int max_len, cudaStream_t st, bool x_is_chunk = false, int prefix = 0,
+                    int chunk_of_many = 0) {
   const prism_model_cfg& c = h->cfg;
   const int D = c.hidden, dh = c.head_dim;
   const int nqkv = (c.n_q_heads + 2 * c.n_kv_heads) * dh, hd = c.n_q_heads * dh;
@@ -763,10 +768,13 @@ int run_layer_chunk(prism_handle* h, const LayerDev& W, const LayerMaps* maps, f
                  launch_qknorm_rope(h->qkv, c.dtype, h->pos + r0, rows, c.n_q_heads, c.n_kv_heads, dh, c.qk_norm, W.g_q, W.g_k,
                                     c.rms_eps, h->rope_cos, h->rope_sin, st));
   if (h->fa != 3) next_dir(h, false);  // the other attention kernels walk forward
+  if (prefix && chunk_of_many == 1)
+    PRISM_CUDA(h, cudaMemcpyAsync(h->qkv_prefix, h->qkv, (size_t)prefix * nqkv * h->esz, cudaMemcpyDeviceToDevice, st));
   if (h->fa == 3)
     PRISM_LAUNCH_P(h, st, PRISM_K_ATTENTION, attn_flops,
                    launch_attention_tc2(h->qkv, h->attn, cu_dev, s0, s1 - s0, r0, rows, max_len, c.n_q_heads, c.n_kv_heads, c.causal,
-                                        h->errword, st, next_dir(h, true), prefix));
+                                        h->errword, st, next_dir(h, true), prefix,
+                                        (prefix && chunk_of_many) ? h->qkv_prefix : nullptr, chunk_of_many != 2));
   else if (h->fa == 1)
     PRISM_LAUNCH_P(h, st, PRISM_K_ATTENTION, attn_flops,
                    launch_attention_tc(h->qkv, h->attn, cu_dev, s0, s1 - s0, r0, rows, max_len, c.n_q_heads, c.n_kv_heads, c.causal,
@@ -972,8 +980,9 @@ int select_impl(prism_handle* h, const int32_t* query, int32_t lq, const int32_t
   long long own_docs = 0;  // document tokens of the candidates this rank runs
   for (int i = 0; i < N; ++i)
     if (!shard || shard->owned[i]) own_docs += (long long)h->h_off[i + 1] - h->h_off[i];
+  (void)own_docs;
   const int prefix = (c.shared_prefix == PRISM_PREFIX_AUTO && !h->enc && h->fa == 3 && c.causal && !h->offload && N >= 2 &&
-                      lq >= 8 && lq <= 120 && (lq & 7) == 0 && (long long)lq + own_docs <= h->chunk_tokens)
+                      lq >= 8 && lq <= 120 && (lq & 7) == 0)
                          ? lq
                          : 0;
   if (prefix) {
@@ -1072,22 +1081,21 @@ int select_impl(prism_handle* h, const int32_t* query, int32_t lq, const int32_t
     }
     // chunks on sequence boundaries: the longest prefix of the remaining sequences that fits
     int s0 = 0, chunks = 0;
-    if (prefix) {  // one chunk: the prefix rows and every sequence's own rows
-      int max_len = 0;
-      for (int i = 0; i < n; ++i) max_len = std::max(max_len, h->h_cu[i + 1] - h->h_cu[i]);
-      if ((rc = run_layer_chunk(h, W, maps, h->x[cur], h->cu[cur], 0, n, 0, h->h_cu[n], prefix + max_len, st, false, prefix)) != PRISM_OK)
-        return rc;
-      s0 = n;
-      chunks = 1;
-    }
+    const bool many = prefix && h->h_cu[n] > h->chunk_tokens;  // a shared prefix over several chunks
     while (s0 < n) {
+      // with a shared prefix the first chunk starts at row 0 and holds the prefix rows as well
+      const int base = (prefix && s0 == 0) ? 0 : h->h_cu[s0];
       int s1 = s0 + 1, max_len = h->h_cu[s1] - h->h_cu[s0];
-      while (s1 < n && h->h_cu[s1 + 1] - h->h_cu[s0] <= h->chunk_tokens) {
+      while (s1 < n && h->h_cu[s1 + 1] - base <= h->chunk_tokens) {
         max_len = std::max(max_len, h->h_cu[s1 + 1] - h->h_cu[s1]);
         ++s1;
       }
-      const int r0 = h->h_cu[s0], rows = h->h_cu[s1] - r0;
-      if (h->enc && !h->offload) {
+      const int r0 = base, rows = h->h_cu[s1] - r0;
+      if (prefix) {
+        if ((rc = run_layer_chunk(h, W, maps, h->x[cur], h->cu[cur], s0, s1, r0, rows, prefix + max_len, st, false, prefix,
+                                  !many ? 0 : s0 == 0 ? 1 : 2)) != PRISM_OK)
+          return rc;
+      } else if (h->enc && !h->offload) {
         if ((rc = run_layer_chunk_encoder(h, l, W, maps, h->x[cur], h->cu[cur], s0, s1, r0, rows, max_len, st)) != PRISM_OK) return rc;
       } else if (!h->offload) {
         if ((rc = run_layer_chunk(h, W, maps, h->x[cur], h->cu[cur], s0, s1, r0, rows, max_len, st)) != PRISM_OK) return rc;

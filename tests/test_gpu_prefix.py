@@ -106,8 +106,9 @@ def test_requests_the_prefix_path_does_not_take(P, weights, lq, n):
     same(a, b)
 
 
-def test_shared_prefix_with_streamed_weights_and_a_chunked_neighbour(P):
-    """Layer streaming keeps the prefix; a budget that splits the request into chunks drops it (one chunk only)."""
+def test_shared_prefix_with_streamed_weights_and_chunked_execution(P):
+    """Layer streaming and chunked execution keep the prefix: the first chunk of a layer holds the query's rows and
+    saves their q/k/v for the attention of the later chunks."""
     w = synth.make_weights(MID, seed=5)
     tw = P.upload_weights(w, MID.dtype, layers_pinned_host=True)
     req = synth.make_request(replace(MID_WL, query_len=32), 2)
@@ -117,10 +118,13 @@ def test_shared_prefix_with_streamed_weights_and_a_chunked_neighbour(P):
     total = int(req["cand_offsets"][-1]) + 32 * MID_WL.n_candidates
     per_tok = 2 * (MID.hidden + (MID.n_q_heads + 2 * MID.n_kv_heads) * MID.head_dim + MID.n_q_heads * MID.head_dim + MID.ffn)
     budget = 2 * total * MID.hidden * 4 + (total // 3) * per_tok
-    c = run(P, model(P, P.upload_weights(w, MID.dtype), req, activation_budget_bytes=budget), req, 4, SCHEDS[1])
-    if c[2].n_chunks_max > 1:
-        assert c[2].shared_prefix_rows == 0
-    same(c, b)
+    for sched in SCHEDS:
+        ref = run(P, model(P, P.upload_weights(w, MID.dtype), req, shared_prefix=False), req, 4, sched)
+        for div in (3, 7):
+            budget = 2 * total * MID.hidden * 4 + (total // div) * per_tok
+            c = run(P, model(P, P.upload_weights(w, MID.dtype), req, activation_budget_bytes=budget), req, 4, sched)
+            assert c[2].n_chunks_max >= div and c[2].shared_prefix_rows == 32
+            same(c, ref)
 
 
 def test_repeated_requests_of_different_shape_on_one_handle(P, weights):
