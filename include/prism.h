@@ -134,9 +134,9 @@ typedef struct {
                       N - 1 repeated copies of the query).  Scores, selections and traces are bit-identical to the
                       batch with one query copy per sequence; tokens_per_layer and tokens_before keep counting
                       query_len + document length per sequence.  Taken when: causal, bf16 tensor-core path with an
-                      even Hq / Hkv, 8 <= query_len <= 120 and query_len a multiple of 8, N >= 2, no hidden_offload
-                      (chunked execution included: the first chunk of a layer carries the query rows;
-                      prism_select_sharded included: every rank holds the query rows).  Otherwise, or with
+                      even Hq / Hkv, 8 <= query_len <= 120 and query_len a multiple of 8, N >= 2
+                      (under chunked execution and hidden_offload the first chunk of a layer carries the query
+                      rows; with prism_select_sharded every rank holds them).  Otherwise, or with
                       PRISM_PREFIX_OFF (1), every sequence carries its own copy of the query. */
   int32_t arch;             /* PRISM_ARCH_*.  For PRISM_ARCH_ENCODER: rms_eps is the LayerNorm epsilon; rope_theta and
                       qk_norm are ignored (qk_norm must be 0); causal is normally 0; head_dim is 64 or 128 on the

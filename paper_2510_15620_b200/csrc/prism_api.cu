@@ -981,7 +981,7 @@ int select_impl(prism_handle* h, const int32_t* query, int32_t lq, const int32_t
   for (int i = 0; i < N; ++i)
     if (!shard || shard->owned[i]) own_docs += (long long)h->h_off[i + 1] - h->h_off[i];
   (void)own_docs;
-  const int prefix = (c.shared_prefix == PRISM_PREFIX_AUTO && !h->enc && h->fa == 3 && c.causal && !h->offload && N >= 2 &&
+  const int prefix = (c.shared_prefix == PRISM_PREFIX_AUTO && !h->enc && h->fa == 3 && c.causal && N >= 2 &&
                       lq >= 8 && lq <= 120 && (lq & 7) == 0)
                          ? lq
                          : 0;
@@ -1091,9 +1091,10 @@ int select_impl(prism_handle* h, const int32_t* query, int32_t lq, const int32_t
         ++s1;
       }
       const int r0 = base, rows = h->h_cu[s1] - r0;
-      if (prefix) {
+      const int of_many = !many ? 0 : s0 == 0 ? 1 : 2;
+      if (prefix && !h->offload) {
         if ((rc = run_layer_chunk(h, W, maps, h->x[cur], h->cu[cur], s0, s1, r0, rows, prefix + max_len, st, false, prefix,
-                                  !many ? 0 : s0 == 0 ? 1 : 2)) != PRISM_OK)
+                                  of_many)) != PRISM_OK)
           return rc;
       } else if (h->enc && !h->offload) {
         if ((rc = run_layer_chunk_encoder(h, l, W, maps, h->x[cur], h->cu[cur], s0, s1, r0, rows, max_len, st)) != PRISM_OK) return rc;
@@ -1125,7 +1126,8 @@ int select_impl(prism_handle* h, const int32_t* query, int32_t lq, const int32_t
         PRISM_CUDA(h, cudaEventRecord(h->ev_in[slot], h->in_stream));
         PRISM_CUDA(h, cudaStreamWaitEvent(st, h->ev_in[slot], 0));
         rc = h->enc ? run_layer_chunk_encoder(h, l, W, maps, h->xc[slot], h->cu[cur], s0, s1, r0, rows, max_len, st, true)
-                    : run_layer_chunk(h, W, maps, h->xc[slot], h->cu[cur], s0, s1, r0, rows, max_len, st, true);
+                    : run_layer_chunk(h, W, maps, h->xc[slot], h->cu[cur], s0, s1, r0, rows, prefix + max_len, st, true, prefix,
+                                      of_many);
         if (rc != PRISM_OK) return rc;
         PRISM_CUDA(h, cudaEventRecord(h->ev_done[slot], st));
         PRISM_CUDA(h, cudaStreamWaitEvent(h->out_stream, h->ev_done[slot], 0));

@@ -47,6 +47,7 @@ def test_offload_is_result_neutral(P):
             got = run(P, m, reqs[i], MID_WL.top_k, MID_WL.schedule)
             same(got, ref[i])
         assert got[2].n_chunks_max >= 2
+        assert got[2].shared_prefix_rows == len(reqs[0]["query"]) == ref[0][2].shared_prefix_rows   # the query rows stay shared
         if not kw:                                                      # (streaming adds its two layer slots)
             assert got[2].workspace_bytes < ref[0][2].workspace_bytes
         m.close()
