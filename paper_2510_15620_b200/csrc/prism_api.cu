@@ -732,8 +732,8 @@ cudaError_t gemm_tc_any(prism_handle* h, const TmaDesc& a, const TmaDesc& b0, co
 
 // One decoder block over rows [r0, r0+rows) (sequences [s0, s1)) of the live batch.
 // x is the whole batch's hidden-state matrix, or (x_is_chunk) the buffer holding just this chunk's rows.
-// prefix > 0: rows [0, prefix) are the query shared by all sequences, cu holds the sequences' own rows, max_len
-// counts prefix + own rows (whole batch in one chunk, r0 = 0).
+// prefix > 0: rows [0, prefix) of the batch are the query shared by all sequences, cu holds the sequences' own rows,
+// max_len counts prefix + own rows; the chunk that starts at row 0 contains the prefix rows.
 // chunk_of_many: 0 = the batch is one chunk; 1 = first of several chunks (it holds the prefix rows: their q/k/v are
 // saved for the others); 2 = a later chunk (attention reads the saved prefix rows and writes none).
 int run_layer_chunk(prism_handle* h, const LayerDev& W, const LayerMaps* maps, float* x, const int* cu_dev, int s0, int s1,
