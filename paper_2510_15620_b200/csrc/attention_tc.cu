@@ -54,6 +54,7 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   constexpr int kQBytes = BM * DH * 2, kKBytes = BN * DH * 2, kVBytes = BN * DH * 2;
   constexpr int kTileBytes = tile_bytes_of(DH);
   extern __shared__ unsigned char smem_raw[];
+  pdl_sync();  // the offsets below are another kernel's output
   const int s = seq0 + blockIdx.z;
   const int beg = cu[s] - row0, len = cu[s + 1] - cu[s];
   const int qb = (int)gridDim.x - 1 - (int)blockIdx.x;  // heaviest query blocks first
@@ -327,14 +328,23 @@ cudaError_t launch_attention_tc(const void* qkv, void* out, const int* cu, int s
   if (e != cudaSuccess) return e;
   dim3 grid((max_len + BM - 1) / BM, n_q_heads, nseq);
   const float scale_log2 = 1.4426950408889634f / sqrtf((float)DH);
-  if (DH == 128)
-    k_attention_tc<128><<<grid, kThreads, smem_bytes_of(128), st>>>(
-        reinterpret_cast<const CUtensorMap&>(mq), reinterpret_cast<const CUtensorMap&>(mkv), (__nv_bfloat16*)out, cu, seq0,
-        row0, n_q_heads, n_kv_heads, causal, scale_log2, err);
-  else
-    k_attention_tc<64><<<grid, kThreads, smem_bytes_of(64), st>>>(
-        reinterpret_cast<const CUtensorMap&>(mq), reinterpret_cast<const CUtensorMap&>(mkv), (__nv_bfloat16*)out, cu, seq0,
-        row0, n_q_heads, n_kv_heads, causal, scale_log2, err);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = smem_bytes_of(DH);
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl_for(rows) ? 1 : 0;
+  const CUtensorMap& m0 = reinterpret_cast<const CUtensorMap&>(mq);
+  const CUtensorMap& m1 = reinterpret_cast<const CUtensorMap&>(mkv);
+  cudaError_t le = DH == 128 ? cudaLaunchKernelEx(&cfg, k_attention_tc<128>, m0, m1, (__nv_bfloat16*)out, cu, seq0, row0, n_q_heads,
+                                                  n_kv_heads, causal, scale_log2, err)
+                             : cudaLaunchKernelEx(&cfg, k_attention_tc<64>, m0, m1, (__nv_bfloat16*)out, cu, seq0, row0, n_q_heads,
+                                                  n_kv_heads, causal, scale_log2, err);
+  if (le != cudaSuccess) return le;
   return cudaGetLastError();
 }
 

@@ -165,6 +165,7 @@ k_attention_tc2(const __grid_constant__ CUtensorMap map_qkv, const __grid_consta
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  pdl_sync();  // set-up done: the kernel before this one (it may still own the work counters) has to be complete
   const uint32_t tmem = *tmem_slot;
   const int group = hq / hkv, npairs = hq / 2;
 
@@ -604,12 +605,23 @@ cudaError_t launch_attention_tc2(const void* qkv, void* out, const int* cu, int 
   }
   int* sched = sb + 2 * (ticket.fetch_add(1, std::memory_order_relaxed) % kTickets);
   const float scale_log2 = 1.4426950408889634f / sqrtf((float)DH);
-  k_attention_tc2<<<grid, kThreads, kSmemBytes, st>>>(reinterpret_cast<const CUtensorMap&>(mq),
-                                                      reinterpret_cast<const CUtensorMap&>(mpre),
-                                                      reinterpret_cast<const CUtensorMap&>(mrest), (__nv_bfloat16*)out, cu,
-                                                      seq0, nseq, row0, nqb, gsz, n_q_heads, n_kv_heads, causal, reverse ? 1 : 0,
-                                                      prefix, write_prefix ? 1 : 0, scale_log2,
-                                                      sched, err);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = kSmemBytes;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl_for(rows) ? 1 : 0;
+  const CUtensorMap& m0 = reinterpret_cast<const CUtensorMap&>(mq);
+  const CUtensorMap& m1 = reinterpret_cast<const CUtensorMap&>(mpre);
+  const CUtensorMap& m2 = reinterpret_cast<const CUtensorMap&>(mrest);
+  if (cudaError_t le = cudaLaunchKernelEx(&cfg, k_attention_tc2, m0, m1, m2, (__nv_bfloat16*)out, cu, seq0, nseq, row0, nqb, gsz,
+                                          n_q_heads, n_kv_heads, causal, reverse ? 1 : 0, prefix, write_prefix ? 1 : 0,
+                                          scale_log2, sched, err))
+    return le;
   return cudaGetLastError();
 }
 

@@ -101,6 +101,23 @@ struct alignas(64) TmaDesc {
   unsigned char bytes[128];
 };
 
+// Programmatic dependent launch: a kernel that starts with pdl_sync() may be launched with
+// cudaLaunchAttributeProgrammaticStreamSerialization.  Its blocks are then scheduled as soon as every block of the
+// kernel before it in the stream has started (that kernel's own pdl_sync() releases them), run their set-up
+// (barrier initialisation, tensor-memory allocation), and wait at this point until the predecessor has completed and
+// its writes are visible.  Nothing before the call may touch memory another kernel writes.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_sync() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+#endif
+// Whether a launcher sets the attribute for a kernel over `rows` rows: it pays where kernels are short (the
+// launch and set-up it hides are a few microseconds), and measured neutral to slightly negative on full batches, so it
+// is used up to 16 Ki rows.  PRISM_NO_PDL in the environment turns it off altogether.
+bool pdl_enabled();
+inline bool pdl_for(long long rows) { return rows <= 16384 && pdl_enabled(); }
+
 // ---- launchers (each returns the CUDA error of the launch; none synchronises) -----------------
 // owned (nullable, device, n bytes): candidates with owned[i] == 0 get length zero (candidate-sharded runs).
 cudaError_t launch_pack_offsets(const int* cand_offsets, int n, int query_len, int* cu, int* seq2orig,

@@ -1,6 +1,8 @@
 // HBM-bound kernels of the PRISM hot path: packing, embedding gather, RMSNorm, QK-norm + rotary
 // embedding, the score probe and the survivor row gather.  All accesses are 16-byte vectorised
 // and coalesced along the hidden dimension; reductions are fp32.
+#include <cstdlib>
+
 #include "common.cuh"
 
 namespace prism {
@@ -196,6 +198,7 @@ __global__ void __launch_bounds__(256) k_rmsnorm(const float* __restrict__ x, co
 template <typename OT, int kPer>
 __global__ void __launch_bounds__(256) k_rmsnorm_warp(const float* __restrict__ x, const OT* __restrict__ gain,
                                                       int rows, int d, float eps, OT* __restrict__ out, int reverse) {
+  pdl_sync();
   const int lane = threadIdx.x & 31;
   const long long blk = reverse ? (long long)gridDim.x - 1 - blockIdx.x : blockIdx.x;
   const long long row = blk * 8 + (threadIdx.x >> 5);
@@ -274,6 +277,7 @@ template <typename OT, int kPer, bool kWarp>
 __global__ void __launch_bounds__(256) k_layernorm(float* __restrict__ x, const float* __restrict__ gain,
                                                    const float* __restrict__ shift, int rows, int d, float eps,
                                                    OT* __restrict__ out, int reverse) {
+  pdl_sync();
   __shared__ float red[32];
   const int lane = kWarp ? (threadIdx.x & 31) : threadIdx.x;
   constexpr int kStride = kWarp ? 32 : 256;
@@ -621,6 +625,15 @@ __global__ void __launch_bounds__(256) k_compact_rows(const float* __restrict__ 
   }
 }
 
+}  // namespace
+
+bool pdl_enabled() {
+  static const bool on = std::getenv("PRISM_NO_PDL") == nullptr;
+  return on;
+}
+
+namespace {
+
 inline int grid_for(long long work, int block, int cap = 148 * 16) {
   long long g = (work + block - 1) / block;
   if (g < 1) g = 1;
@@ -691,7 +704,21 @@ cudaError_t launch_rmsnorm(const float* x, const void* gain, int dtype, int rows
   if (nv > 8 * 256) return cudaErrorInvalidValue;
   if (nv <= 16 * 32) {  // rows of up to 8 KB: one warp per row
     const unsigned grid = (unsigned)((rows + 7) / 8);
-#define PRISM_NORMW(OT, V) k_rmsnorm_warp<OT, V><<<grid, 256, 0, st>>>(x, (const OT*)gain, rows, d, eps, (OT*)out, reverse ? 1 : 0)
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(256);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl_for(rows) ? 1 : 0;
+    const int rev = reverse ? 1 : 0;
+#define PRISM_NORMW(OT, V)                                                                                                \
+  do {                                                                                                                    \
+    cudaError_t le = cudaLaunchKernelEx(&cfg, k_rmsnorm_warp<OT, V>, x, (const OT*)gain, rows, d, eps, (OT*)out, rev);      \
+    if (le != cudaSuccess) return le;                                                                                     \
+  } while (0)
     if (dtype == 1) {
       if (nv <= 128) PRISM_NORMW(__nv_bfloat16, 4);
       else if (nv <= 256) PRISM_NORMW(__nv_bfloat16, 8);
@@ -742,7 +769,20 @@ cudaError_t launch_layernorm(float* x, const float* gain, const float* shift, in
   const int nv = d >> 2;
   if ((d & 3) || nv > 8 * 256) return cudaErrorInvalidValue;
   const int rev = reverse ? 1 : 0;
-#define PRISM_LN(OT, P, W, G) k_layernorm<OT, P, W><<<(G), 256, 0, st>>>(x, gain, shift, rows, d, eps, (OT*)out, rev)
+  cudaLaunchConfig_t cfg = {};
+  cfg.blockDim = dim3(256);
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl_for(rows) ? 1 : 0;
+#define PRISM_LN(OT, P, W, G)                                                                                        \
+  do {                                                                                                               \
+    cfg.gridDim = dim3((unsigned)(G));                                                                                \
+    cudaError_t le = cudaLaunchKernelEx(&cfg, k_layernorm<OT, P, W>, x, gain, shift, rows, d, eps, (OT*)out, rev);     \
+    if (le != cudaSuccess) return le;                                                                                \
+  } while (0)
   if (nv <= 16 * 32) {  // rows of up to 8 KB: one warp per row
     const unsigned grid = (unsigned)((rows + 7) / 8);
     if (dtype == 1) {

@@ -84,23 +84,10 @@ __device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
 }
 
 // gelu(x) = x Phi(x) without a branch: Phi from the rational-times-Gaussian form of erfc (Abramowitz & Stegun
-// 7.1.26, absolute error below 1.5e-7, far under the bf16 rounding of the result), two special-function
-// operations and a handful of FMAs per element, so that the epilogue keeps up with the MMAs.
-__device__ __forceinline__ float gelu_fast(float x) {
-  const float z = fabsf(x) * 0.70710678118654752f;
-  const float t = __fdividef(1.f, fmaf(0.3275911f, z, 1.f));
-  float p = fmaf(1.061405429f, t, -1.453152027f);
-  p = fmaf(p, t, 1.421413741f);
-  p = fmaf(p, t, -0.284496736f);
-  p = fmaf(p, t, 0.254829592f);
-  float e;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(-1.4426950408889634f * z * z));
-  const float tail = 0.5f * p * t * e;           // 0.5 erfc(|x| / sqrt 2) = Phi(-|x|)
-  return x * (x >= 0.f ? 1.f - tail : tail);
-}
-
-// The same for two values at once with the polynomial in packed fp32 arithmetic (half the FMA issue slots); the
-// factor 0.5 of the tail is folded into the coefficients.
+// 7.1.26, absolute error below 5e-7, far under the bf16 rounding of the result): one reciprocal, one exp2 and a
+// handful of FMAs per element, so that the epilogue keeps up with the MMAs.  Two values at once, the polynomial and
+// the products in packed fp32 arithmetic (half the FMA issue slots); the factor 0.5 of the tail is folded into the
+// coefficients.
 __device__ __forceinline__ void gelu_fast2(float x0, float x1, float& y0, float& y1) {
   const float c = 0.70710678118654752f;
   const uint64_t z = f2_pack(fabsf(x0) * c, fabsf(x1) * c);
@@ -185,6 +172,7 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  pdl_sync();  // set-up done: the kernel before this one has to be complete from here on
   const uint32_t tmem_base = *tmem_slot;
   const uint32_t leader_full = map_to_cta(bar_full, 0);            // full[] of the leader, as seen from this CTA
   const uint32_t leader_acc_empty = map_to_cta(bar_acc_empty, 0);  // acc_empty[] of the leader
@@ -600,13 +588,15 @@ cudaError_t launch_gemm_tc2(const TmaDesc& a, const TmaDesc& b0, const TmaDesc& 
   cfg.blockDim = dim3(kThreads);
   cfg.dynamicSmemBytes = kSmemBytes;
   cfg.stream = st;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = 2;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = pdl_for(m) ? 2 : 1;
   cudaError_t le;
   if (epilogue == kEpiStore)
     le = cudaLaunchKernelEx(&cfg, k_gemm_tc2<kEpiStore>, ma, mb0, mb1, mr, o, m, n, k, q, reverse ? 1 : 0, err, bias);
