@@ -118,6 +118,7 @@ __global__ void k_pack_tokens(const int* __restrict__ query, int lq, const int* 
 }
 
 __global__ void k_positions(const int* __restrict__ cu, int n, int total, int prefix, int* __restrict__ pos) {
+  pdl_sync();
   for (int t = blockIdx.x * blockDim.x + threadIdx.x; t < total; t += gridDim.x * blockDim.x) {
     if (t < prefix) {
       pos[t] = t;
@@ -563,6 +564,7 @@ __global__ void __launch_bounds__(256) k_probe(const float* __restrict__ x, cons
                                                const WT* __restrict__ g_final, const float* __restrict__ w_diff,
                                                float eps, int prefix, const unsigned char* __restrict__ owned,
                                                const int* __restrict__ seq2orig, float* __restrict__ scores) {
+  pdl_sync();
   __shared__ float red[32];
   const int i = blockIdx.x;
   int last = cu[i + 1] - 1;
@@ -602,6 +604,7 @@ __global__ void __launch_bounds__(256) k_compact_rows(const float* __restrict__ 
                                                       const int* __restrict__ cu_new,
                                                       const int* __restrict__ old_of_new, int n_new,
                                                       int total_new, int d, int prefix) {
+  pdl_sync();
   const int nv = d >> 2;
   for (int t = blockIdx.x; t < total_new; t += gridDim.x) {
     int src = t;  // rows of a shared query prefix stay where they are
@@ -634,6 +637,21 @@ bool pdl_enabled() {
 
 namespace {
 
+// Launch with the programmatic-dependent-launch attribute (the kernel starts with pdl_sync()).
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), unsigned grid, unsigned block, cudaStream_t st, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(block);
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl_enabled() ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 inline int grid_for(long long work, int block, int cap = 148 * 16) {
   long long g = (work + block - 1) / block;
   if (g < 1) g = 1;
@@ -660,8 +678,7 @@ cudaError_t launch_pack_tokens(const int* query, int query_len, const int* cand_
 
 cudaError_t launch_positions(const int* cu, int n, int total, int* pos, cudaStream_t st, int prefix) {
   if (total <= 0) return cudaSuccess;
-  k_positions<<<grid_for(total, 256), 256, 0, st>>>(cu, n, total, prefix, pos);
-  return cudaGetLastError();
+  return launch_pdl(k_positions, (unsigned)grid_for(total, 256), 256, st, cu, n, total, prefix, pos);
 }
 
 cudaError_t launch_embed(const void* table, int dtype, const int* tokens, int total, int d, float* x,
@@ -905,11 +922,10 @@ cudaError_t launch_probe(const float* x, const int* cu, int n, int d, const void
   if (n <= 0) return cudaSuccess;
   if (owned && !seq2orig) return cudaErrorInvalidValue;
   if (dtype == 1)
-    k_probe<__nv_bfloat16><<<n, 256, 0, st>>>(x, cu, d, (const __nv_bfloat16*)g_final, w_diff, eps, prefix, owned, seq2orig,
-                                              scores);
-  else
-    k_probe<float><<<n, 256, 0, st>>>(x, cu, d, (const float*)g_final, w_diff, eps, prefix, owned, seq2orig, scores);
-  return cudaGetLastError();
+    return launch_pdl(k_probe<__nv_bfloat16>, (unsigned)n, 256, st, x, cu, d, (const __nv_bfloat16*)g_final, w_diff, eps, prefix,
+                      owned, seq2orig, scores);
+  return launch_pdl(k_probe<float>, (unsigned)n, 256, st, x, cu, d, (const float*)g_final, w_diff, eps, prefix, owned, seq2orig,
+                    scores);
 }
 
 cudaError_t launch_score_diff(const void* score_head, int dtype, int d, float* w_diff, cudaStream_t st) {
@@ -924,8 +940,7 @@ cudaError_t launch_compact_rows(const float* x_old, float* x_new, const int* cu_
                                 const int* old_of_new, int n_new, int total_new, int d, cudaStream_t st, int prefix) {
   if (total_new <= 0) return cudaSuccess;
   int grid = total_new < 148 * 8 ? total_new : 148 * 8;
-  k_compact_rows<<<grid, 256, 0, st>>>(x_old, x_new, cu_old, cu_new, old_of_new, n_new, total_new, d, prefix);
-  return cudaGetLastError();
+  return launch_pdl(k_compact_rows, (unsigned)grid, 256, st, x_old, x_new, cu_old, cu_new, old_of_new, n_new, total_new, d, prefix);
 }
 
 }  // namespace prism
