@@ -116,7 +116,13 @@ __device__ __forceinline__ void pdl_sync() {
 // launch and set-up it hides are a few microseconds), and measured neutral to slightly negative on full batches, so it
 // is used up to 16 Ki rows.  PRISM_NO_PDL in the environment turns it off altogether.
 bool pdl_enabled();
-inline bool pdl_for(long long rows) { return rows <= 16384 && pdl_enabled(); }
+// After a cross-stream dependency was enqueued (cudaStreamWaitEvent), the next launch of this thread goes out
+// without the attribute, so that nothing of it can be scheduled ahead of that dependency.
+void pdl_skip_next();
+inline bool pdl_for(long long rows) {
+  const bool on = pdl_enabled();  // consumes a pending pdl_skip_next()
+  return on && rows <= 16384;
+}
 
 // ---- launchers (each returns the CUDA error of the launch; none synchronises) -----------------
 // owned (nullable, device, n bytes): candidates with owned[i] == 0 get length zero (candidate-sharded runs).

@@ -630,8 +630,18 @@ __global__ void __launch_bounds__(256) k_compact_rows(const float* __restrict__ 
 
 }  // namespace
 
+namespace {
+thread_local bool t_pdl_skip = false;
+}
+
+void pdl_skip_next() { t_pdl_skip = true; }
+
 bool pdl_enabled() {
   static const bool on = std::getenv("PRISM_NO_PDL") == nullptr;
+  if (t_pdl_skip) {
+    t_pdl_skip = false;
+    return false;
+  }
   return on;
 }
 

@@ -1061,7 +1061,10 @@ int select_impl(prism_handle* h, const int32_t* query, int32_t lq, const int32_t
     const int s = l & 1;
     LayerDev W = streamed ? layer_in_slot(h, s) : layer_resident(h, l);
     const LayerMaps* maps = !h->tc ? nullptr : h->w4 ? &h->maps_w4 : &h->maps[streamed ? s : l];
-    if (streamed) PRISM_CUDA(h, cudaStreamWaitEvent(st, h->ev_copied[s], 0));
+    if (streamed) {
+      PRISM_CUDA(h, cudaStreamWaitEvent(st, h->ev_copied[s], 0));
+      pdl_skip_next();
+    }
     if (h->w4) {
       // rebuild the layer's five matrices as bf16; the stream orders this after the previous layer's last GEMM
       const int D = c.hidden, F = c.ffn, nq = (c.n_q_heads + 2 * c.n_kv_heads) * c.head_dim, hd = c.n_q_heads * c.head_dim;
@@ -1125,6 +1128,7 @@ int select_impl(prism_handle* h, const int32_t* query, int32_t lq, const int32_t
         PRISM_CUDA(h, cudaMemcpyAsync(h->xc[slot], hx, bytes, cudaMemcpyHostToDevice, h->in_stream));
         PRISM_CUDA(h, cudaEventRecord(h->ev_in[slot], h->in_stream));
         PRISM_CUDA(h, cudaStreamWaitEvent(st, h->ev_in[slot], 0));
+        pdl_skip_next();
         rc = h->enc ? run_layer_chunk_encoder(h, l, W, maps, h->xc[slot], h->cu[cur], s0, s1, r0, rows, max_len, st, true)
                     : run_layer_chunk(h, W, maps, h->xc[slot], h->cu[cur], s0, s1, r0, rows, prefix + max_len, st, true, prefix,
                                       of_many);
@@ -1154,6 +1158,7 @@ int select_impl(prism_handle* h, const int32_t* query, int32_t lq, const int32_t
       // probe and compaction read the host copy on the request's stream: every write-back must have landed
       // (out_stream is in order, so its latest event covers them all)
       PRISM_CUDA(h, cudaStreamWaitEvent(st, h->ev_chunk_out[last_out], 0));
+      pdl_skip_next();
       main_dirty = true;  // whatever the request stream does to the host copy now must precede later fetches
     }
     if (is_final || is_probe) {
