@@ -75,18 +75,35 @@ def attention(q: np.ndarray, k: np.ndarray, v: np.ndarray, causal: bool, round_p
     return out
 
 
+ROUNDING_POINTS = ("norm", "qk", "v", "p", "attn", "swiglu")
+
+
+def rounding_points(act: str):
+    """The set of stored tensors the mode `act` rounds to bfloat16."""
+    if act == "exact":
+        return frozenset()
+    if act == "bf16":
+        return frozenset(ROUNDING_POINTS)
+    on = frozenset(p for p in act.split(",") if p)
+    if not on <= set(ROUNDING_POINTS):
+        raise ValueError(f"unknown rounding point in {act!r}")
+    return on
+
+
 def layer_forward(x: np.ndarray, w: Dict[str, np.ndarray], cfg, act: str = "exact") -> np.ndarray:
     """One pre-norm decoder block on one sequence.  x: [L, D] fp64 -> [L, D].
 
     act = "exact": no rounding anywhere (the definition).  act = "bf16": the same steps with every
     stored activation rounded to bfloat16 where the bf16 precision contract stores it (normed inputs,
     q/k after the rotary embedding, v, attention probabilities, attention output, SwiGLU output); the
-    residual stream, norms, softmax and all sums stay exact."""
-    rnd = to_bf16 if act == "bf16" else (lambda t: t)
+    residual stream, norms, softmax and all sums stay exact.  A comma-separated subset of
+    ROUNDING_POINTS rounds at those points only (used to tell which stored tensor carries the noise)."""
+    on = rounding_points(act)
+    rnd = {p: (to_bf16 if p in on else (lambda t: t)) for p in ROUNDING_POINTS}
     L = x.shape[0]
     hq, hkv, dh = cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim
     W = {k: np.asarray(t, dtype=np.float64) for k, t in w.items()}
-    a = rnd(rmsnorm(x, W["g_attn"], cfg.rms_eps))
+    a = rnd["norm"](rmsnorm(x, W["g_attn"], cfg.rms_eps))
     qkv = a @ W["w_qkv"].T
     q = qkv[:, : hq * dh].reshape(L, hq, dh)
     k = qkv[:, hq * dh: (hq + hkv) * dh].reshape(L, hkv, dh)
@@ -95,15 +112,15 @@ def layer_forward(x: np.ndarray, w: Dict[str, np.ndarray], cfg, act: str = "exac
         q = rmsnorm(q, W["g_q"], cfg.rms_eps)
         k = rmsnorm(k, W["g_k"], cfg.rms_eps)
     pos = np.arange(L)
-    q = rnd(rope_rotate(q, pos, cfg.rope_theta))
-    k = rnd(rope_rotate(k, pos, cfg.rope_theta))
-    v = rnd(v)
-    o = rnd(attention(q, k, v, bool(cfg.causal), round_p=rnd if act == "bf16" else None)).reshape(L, hq * dh)
+    q = rnd["qk"](rope_rotate(q, pos, cfg.rope_theta))
+    k = rnd["qk"](rope_rotate(k, pos, cfg.rope_theta))
+    v = rnd["v"](v)
+    o = rnd["attn"](attention(q, k, v, bool(cfg.causal), round_p=to_bf16 if "p" in on else None)).reshape(L, hq * dh)
     x = x + o @ W["w_o"].T
-    b = rnd(rmsnorm(x, W["g_ffn"], cfg.rms_eps))
+    b = rnd["norm"](rmsnorm(x, W["g_ffn"], cfg.rms_eps))
     gate = b @ W["w_gate"].T
     up = b @ W["w_up"].T
-    h = rnd(gate / (1.0 + np.exp(-gate)) * up)     # silu(gate) * up
+    h = rnd["swiglu"](gate / (1.0 + np.exp(-gate)) * up)     # silu(gate) * up
     return x + h @ W["w_down"].T
 
 
