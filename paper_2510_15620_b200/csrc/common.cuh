@@ -81,6 +81,17 @@ constexpr size_t route_scratch_bytes(int n) {
          + 256;
 }
 
+// Arguments of the one-step routing entry points that the kernel itself cannot defend against: an unknown
+// mode, a FIXED_KEEP count below 1 (the survivor count would go negative and the new offsets would be written in
+// front of the caller's buffer) or a ddof other than 0 / 1.
+inline bool route_args_ok(int n, int mode, int keep_count, int n_clusters, int ddof, int max_n) {
+  if (n < 0 || n > max_n) return false;
+  if (mode != 0 && mode != 1 && mode != 2) return false;
+  if (mode == 1 && keep_count < 1) return false;
+  if (n_clusters < 2 || n_clusters > kMaxClusters) return false;
+  return ddof == 0 || ddof == 1;
+}
+
 // Raise a kernel's dynamic shared-memory limit once per device (the attribute is per device; `done` is a
 // bit mask over device ordinals, so concurrent callers at worst set it twice).
 template <typename Kernel>

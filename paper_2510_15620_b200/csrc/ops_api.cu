@@ -204,7 +204,7 @@ int prism_op_route(const float* scores, const int32_t* cu_old, const int32_t* se
                    void* stream) {
   if (!scores || !cu_old || !seq2orig_old || !cu_new || !seq2orig_new || !old_of_new || !state || !res_idx || !res_score)
     return PRISM_ERR_INVALID_ARG;
-  if (n < 0 || n > kMaxCandidates || n_clusters < 2 || n_clusters > kMaxClusters) return PRISM_ERR_INVALID_ARG;
+  if (!route_args_ok(n, mode, keep_count, n_clusters, std_ddof, kMaxCandidates)) return PRISM_ERR_INVALID_ARG;
   void* scratch = nullptr;
   cudaError_t e = cudaMalloc(&scratch, route_scratch_bytes(n));
   if (e != cudaSuccess) return st_of(e);

@@ -882,7 +882,7 @@ int cache_prepare(prism_handle* h, const int* query, int lq, const int* cand, in
     PRISM_CUDA(h, cudaMemcpyAsync(h->h_tokens + lq, cand, (size_t)n_cand * sizeof(int), cudaMemcpyDeviceToHost, st));
   PRISM_CUDA(h, cudaStreamSynchronize(st));
   const uint64_t now = ++h->request_no;
-  std::vector<int> missing;
+  std::vector<int> missing, hit_slots;
   int64_t distinct = 0;
   for (int i = 0; i < lq + n_cand; ++i) {
     const int t = h->h_tokens[i];
@@ -890,17 +890,20 @@ int cache_prepare(prism_handle* h, const int* query, int lq, const int* cand, in
     h->tok_seen[t] = now;
     ++distinct;
     const int s = h->slot_of_tok[t];
-    if (s >= 0) h->slot_stamp[s] = now;
+    if (s >= 0) hit_slots.push_back(s);
     else missing.push_back(t);
   }
   if (distinct > h->cache_rows) {
-    // undo the stamps of this request so that the cache state is as before
+    // a refused request leaves the cache as it found it: no row has been stamped yet, so the order in which rows
+    // will be evicted is unchanged; the marks and the request number are taken back
     for (int i = 0; i < lq + n_cand; ++i) {
       const int t = h->h_tokens[i];
       if (t >= 0 && t < c.vocab) h->tok_seen[t] = 0;
     }
+    --h->request_no;
     return fail(h, PRISM_ERR_SHAPE_LIMIT, "the request has more distinct tokens than the embedding cache has rows");
   }
+  for (int s : hit_slots) h->slot_stamp[s] = now;
   h->cache_hits += distinct - (int64_t)missing.size();
   h->cache_misses += (int64_t)missing.size();
   if (missing.empty()) return PRISM_OK;
@@ -975,6 +978,7 @@ int select_impl(prism_handle* h, const int32_t* query, int32_t lq, const int32_t
   h->h_cu[0] = 0;
   for (int i = 0; i < N; ++i)
     if (h->h_off[i + 1] < h->h_off[i]) return fail(h, PRISM_ERR_BAD_INPUT, "cand_offsets not monotone");
+  if (h->h_off[N] > 0 && !cand) return fail(h, PRISM_ERR_INVALID_ARG, "cand_tokens is null but cand_offsets[N] > 0");
   // Shared query prefix: under causal attention the query's rows are the same in every sequence, so they are
   // stored and computed once in front of the documents (rows [0, lq)); cu then holds document rows only.
   long long own_docs = 0;  // document tokens of the candidates this rank runs
@@ -1253,7 +1257,7 @@ int check_args(prism_handle* h, const void* q, int lq, const void* cand, const v
   if (N < 0 || K < 1 || lq < 0) return fail(h, PRISM_ERR_INVALID_ARG, "N < 0, K < 1 or query_len < 0");
   if (!off || !oi || !os || (lq > 0 && !q)) return fail(h, PRISM_ERR_INVALID_ARG, "null pointer argument");
   if (lq > h->cfg.max_seq_len) return fail(h, PRISM_ERR_SHAPE_LIMIT, "query_len exceeds max_seq_len");
-  (void)cand;
+  (void)cand;  // may be null when every document is empty: checked once the offsets are on the host
   return PRISM_OK;
 }
 

@@ -312,7 +312,8 @@ __global__ void __launch_bounds__(kThreads) k_route(const float* __restrict__ sc
     cluster_sync_all();
   }
 
-  const int lo_keep = sh.lo_keep, hi_keep = sh.hi_keep;
+  // ranks [lo_keep, hi_keep) survive; clamped so that no argument can make the survivor count negative
+  const int lo_keep = min(max(sh.lo_keep, 0), n), hi_keep = min(max(sh.hi_keep, lo_keep), n);
   int n_new = hi_keep - lo_keep;
   // Terminal condition: the survivors exactly fill the open slots.
   const bool terminal = !done && (n_new == k_after);
@@ -445,7 +446,7 @@ constexpr size_t kStaticRouteBytes = (prism::route_scratch_bytes(kStaticRouteMax
 static __device__ __align__(256) unsigned char g_route_static_scratch[kStaticRouteBytes];
 
 constexpr int kMaxDevices = 64;
-void* g_route_static_ptr[kMaxDevices] = {};  // device address of the array, per device, filled on first use
+std::atomic<void*> g_route_static_ptr[kMaxDevices] = {};  // device address of the array, per device, filled on first use
 
 }  // namespace
 
@@ -458,15 +459,16 @@ extern "C" int prism_op_route_static(const float* scores, const int32_t* cu_old,
   using namespace prism;
   if (!scores || !cu_old || !seq2orig_old || !cu_new || !seq2orig_new || !old_of_new || !state || !res_idx || !res_score)
     return PRISM_ERR_INVALID_ARG;
-  if (n < 0 || n_clusters < 2 || n_clusters > kMaxClusters) return PRISM_ERR_INVALID_ARG;
+  if (!route_args_ok(n, mode, keep_count, n_clusters, std_ddof, kMaxCandidates)) return PRISM_ERR_INVALID_ARG;
   if (n > kStaticRouteMaxN) return PRISM_ERR_SHAPE_LIMIT;  // the built-in scratch is sized for this many candidates
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return PRISM_ERR_CUDA;
-  if (!g_route_static_ptr[dev]) {
+  void* scratch = g_route_static_ptr[dev].load(std::memory_order_acquire);
+  if (!scratch) {
     // In host code the array's name is only a handle; the kernel needs the address it has on THIS device.
-    void* p = nullptr;
-    if (cudaGetSymbolAddress(&p, g_route_static_scratch) != cudaSuccess || !p) return PRISM_ERR_CUDA;
-    g_route_static_ptr[dev] = p;
+    // Two host threads may both get here: they look up, and store, the same address.
+    if (cudaGetSymbolAddress(&scratch, g_route_static_scratch) != cudaSuccess || !scratch) return PRISM_ERR_CUDA;
+    g_route_static_ptr[dev].store(scratch, std::memory_order_release);
   }
   RouteParams prm{};
   prm.mode = mode;
@@ -479,7 +481,7 @@ extern "C" int prism_op_route_static(const float* scores, const int32_t* cu_old,
   prm.layer = layer;
   cudaError_t e = launch_route(scores, cu_old, seq2orig_old, n, prm, cu_new, seq2orig_new, old_of_new,
                                reinterpret_cast<RouteState*>(state), res_idx, res_score,
-                               reinterpret_cast<ProbeRecordDev*>(rec), nullptr, nullptr, g_route_static_ptr[dev],
+                               reinterpret_cast<ProbeRecordDev*>(rec), nullptr, nullptr, scratch,
                                reinterpret_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? PRISM_OK : PRISM_ERR_CUDA;
 }

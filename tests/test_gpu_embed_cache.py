@@ -119,3 +119,41 @@ def test_cache_with_fp32_path_and_streamed_layers(P):
         same(run(P, m, req, MID_WL.top_k, MID_WL.schedule), ref)
     m.close()
     base.close()
+
+
+def _request_of(tokens_per_doc, query):
+    offs = np.zeros(len(tokens_per_doc) + 1, np.int32)
+    offs[1:] = np.cumsum([len(t) for t in tokens_per_doc])
+    return {"query": np.asarray(query, np.int32), "cand_tokens": np.concatenate(tokens_per_doc).astype(np.int32),
+            "cand_offsets": offs}
+
+
+def test_refused_request_leaves_the_eviction_order_alone(P):
+    """Requests A then B fill a cache of 64 rows; a request that holds all of A's tokens and too many others is
+    refused (SHAPE_LIMIT).  The refusal must not have refreshed A's rows: the next request's new tokens evict A's
+    rows (used longest ago), so B afterwards still finds all of its rows."""
+    wl = synth.workload(0)
+    w = synth.make_weights(wl.model)
+    q = [3, 4]
+    A = _request_of([np.arange(100, 116), np.arange(116, 130)], q)             # 30 + 2 distinct tokens
+    B = _request_of([np.arange(200, 216), np.arange(216, 230)], q)             # 30 new ones: 62 rows in use
+    X = _request_of([np.arange(100, 130), np.arange(300, 340)], q)             # 72 distinct tokens > 64 rows
+    C = _request_of([np.arange(400, 416), np.arange(416, 430)], q)             # 30 new ones: 28 evictions
+    big = _request_of([np.arange(0, 64), np.arange(64, 128)], q)
+    m = cached_model(P, wl.model, w, big, rows=64)
+    sched = None
+    run(P, m, A, 1, sched)
+    run(P, m, B, 1, sched)
+    assert m.embed_cache_stats() == (2, 62, 0)
+    with pytest.raises(P.PrismError) as e:
+        run(P, m, X, 1, sched)
+    assert e.value.status == -2
+    assert m.embed_cache_stats() == (2, 62, 0)
+    run(P, m, C, 1, sched)
+    h, mi, ev = m.embed_cache_stats()
+    assert (h, mi, ev) == (4, 92, 28)
+    run(P, m, B, 1, sched)                                                      # B's rows were younger than A's: all there
+    assert m.embed_cache_stats() == (h + 32, mi, ev)
+    run(P, m, A, 1, sched)                                                      # 28 of A's 30 rows went to C
+    assert m.embed_cache_stats()[1] == mi + 28
+    m.close()

@@ -152,6 +152,17 @@ def test_argument_and_input_errors(P, tiny):
     # N = 0 is an empty result, not an error
     idx, sc, _ = model.select(q, c, dev_i32(np.array([0])), 3)
     assert len(idx) == 0
+    # a null cand_tokens with document tokens announced by the offsets: refused on the host, nothing launched
+    before = model.launch_count
+    out_i, out_s = dev_i32(np.zeros(3)), torch.zeros(3, device="cuda")
+    with pytest.raises(P.PrismError) as e:
+        model._call(P.lib().prism_select, q.data_ptr(), q.numel(), None, o.data_ptr(), len(req["cand_offsets"]) - 1, 3,
+                    None, out_i.data_ptr(), out_s.data_ptr(), False, torch.cuda.current_stream().cuda_stream)
+    assert e.value.status == -1 and model.launch_count == before
+    # ... and allowed when every document is empty (each sequence is the query alone)
+    idx, sc, _ = model._call(P.lib().prism_select, q.data_ptr(), q.numel(), None, dev_i32(np.zeros(5)).data_ptr(), 4, 3,
+                             None, out_i.data_ptr(), out_s.data_ptr(), False, torch.cuda.current_stream().cuda_stream), None, None
+    assert idx[0] == 3 and out_i.cpu().tolist() == [0, 1, 2]           # four equal sequences: ties go to the lower index
     model.close()
 
 
