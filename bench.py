@@ -125,22 +125,22 @@ def sum_over_ranks(value: float, world: int, device=None) -> float:
 
 # ----------------------------------------------------------------------------------------------- oracle legs
 def oracle_sample_ids(wl, req, budget_s: float = 25.0, max_cand: int = 2):
-    """A bounded sample of the request for the CPU oracle: up to max_cand candidates, shortest first, as long
-    as the estimated time (2 * layer parameters flops per token at the ~4e11 flop/s the fp64 numpy forward
-    sustains on 16 cores; 5e11 - 8e11 were measured) stays within budget_s; always at least one."""
+    """A bounded, length-stratified sample of the request for the CPU oracle: m candidates evenly spaced in
+    length rank (the median first, then the extremes and the quantiles between them), with m the largest count
+    up to max_cand whose estimated time stays within budget_s (2 * layer parameters flops per token at the
+    ~4e11 flop/s the fp64 numpy forward sustains on 16 cores; 5e11 - 8e11 were measured); at least one."""
     cfg = wl.model
     p_layer = cfg.hidden * (cfg.n_q_heads + 2 * cfg.n_kv_heads) * cfg.head_dim + cfg.n_q_heads * cfg.head_dim * cfg.hidden \
         + 3 * cfg.hidden * cfg.ffn
     s_per_token = 2.0 * p_layer * cfg.n_layers / 4e11
     lens = np.diff(req["cand_offsets"]) + len(req["query"])
     order = np.argsort(lens, kind="stable")
-    ids, t = [], 0.0
-    for i in order[:max_cand]:
-        if ids and t + lens[i] * s_per_token > budget_s:
-            break
-        ids.append(int(i))
-        t += lens[i] * s_per_token
-    return sorted(ids)
+    n = len(order)
+    m = int(max(1, min(max_cand, n, budget_s / (float(np.mean(lens)) * s_per_token))))
+    ranks = [n // 2] if m == 1 else sorted(set(int(round(j * (n - 1) / (m - 1))) for j in range(m)))
+    if m == 1 and lens[order[n // 2]] * s_per_token > 1.5 * budget_s:
+        ranks = [0]         # even the median candidate is far beyond the budget (8B shape): the shortest one
+    return sorted(int(order[r]) for r in ranks)
 
 
 def oracle_sample_rate(wl, weights_np, req, ids):
@@ -165,18 +165,19 @@ def run_reference(args):
         return 0
     wl = synth.workload(args.workload)
     w = synth.make_weights(wl.model, wl.weight_seed)
-    n_cand = 1
+    n_cand = 3      # the shortest, the median and the longest candidate of each request (budget permitting)
     rates, times, toks = [], [], 0
     for step in range(args.warmup + args.steps):
         req = synth.make_request(wl, step)
-        rate, dt, t = oracle_sample_rate(wl, w, req, oracle_sample_ids(wl, req, max_cand=n_cand))
+        rate, dt, t = oracle_sample_rate(wl, w, req, oracle_sample_ids(wl, req, budget_s=20.0, max_cand=n_cand))
         if step >= args.warmup:
             rates.append(rate)
             times.append(dt)
             toks += t
     value = toks / sum(times)
     cores = os.cpu_count()
-    sample = f"the shortest of {wl.n_candidates} candidates per step, all {wl.model.n_layers} layers, unpruned fp64 numpy forward"
+    sample = (f"up to {n_cand} of {wl.n_candidates} candidates per step, evenly spaced in length rank, all "
+              f"{wl.model.n_layers} layers, unpruned fp64 numpy forward")
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": 1e3 * float(np.mean(times)), "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f64", "data": "synthetic",
@@ -185,6 +186,134 @@ def run_reference(args):
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
     return 0
+
+
+# ----------------------------------------------------------------------------------------------- side workloads
+def _tensor_bytes(t, on_device):
+    if isinstance(t, dict):
+        return sum(_tensor_bytes(v, on_device) for v in t.values())
+    if isinstance(t, (list, tuple)):
+        return sum(_tensor_bytes(v, on_device) for v in t)
+    return t.numel() * t.element_size() if (t.is_cuda == on_device) else 0
+
+
+def profile_classes(P, model, step_fn, n_steps):
+    """Per-kernel-class device time of n_steps requests (CUDA events the library records around every launch)."""
+    import ctypes as C
+    import torch
+
+    class Stat(C.Structure):
+        _fields_ = [("ms", C.c_double), ("work", C.c_double), ("launches", C.c_int64)]
+    lib = P.lib()
+    lib.prism_profile.argtypes = [C.c_void_p, C.c_int]
+    lib.prism_profile_read.argtypes = [C.c_void_p, C.POINTER(Stat), C.c_int]
+    stats = (Stat * len(KERNEL_CLASSES))()
+    lib.prism_profile(model._h, 1)
+    for i in range(n_steps):
+        step_fn(i)
+    torch.cuda.synchronize()
+    lib.prism_profile_read(model._h, stats, 1)
+    lib.prism_profile(model._h, 0)
+    return {n: {"ms_per_step": stats[j].ms / n_steps, "launches_per_step": stats[j].launches / n_steps,
+                "work_per_step": stats[j].work / n_steps} for j, n in enumerate(KERNEL_CLASSES)}
+
+
+def measure_side_workload(P, index: int, steps: int, warmup: int, dev, local: int):
+    """One of the other benchmark workloads, timed like the headline (device-resident inputs between CUDA events on
+    the launching stream, then host buffers through prism_select_host, then pruning off), with per-class rates,
+    clocks sampled during the timed region and the peak device memory.  No oracle leg."""
+    import gc
+    import torch
+    import synth
+    from synth.configs import MODE_NONE, Schedule
+
+    wl = synth.workload(index)
+    cfg = wl.model
+    n_req = 10
+    reqs = [synth.make_request(wl, s) for s in range(n_req)]
+    lq = wl.query_len
+    lens_all = [np.diff(r["cand_offsets"]) + lq for r in reqs]
+    torch.cuda.synchronize()
+    torch.cuda.reset_peak_memory_stats(dev)
+    base_bytes = torch.cuda.memory_allocated(dev)
+    w_np = synth.make_weights(cfg, wl.weight_seed)
+    tw = P.upload_weights(w_np, cfg.dtype, device=str(dev), layers_pinned_host=bool(wl.stream_weights))
+    del w_np
+    gc.collect()
+    model = P.PrismModel(cfg, tw, int(max(l.max() for l in lens_all)), wl.n_candidates, int(max(l.sum() for l in lens_all)),
+                         activation_budget_bytes=wl.activation_budget_bytes, stream_weights=bool(wl.stream_weights))
+    d = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(dev)
+    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).pin_memory().numpy()
+    dreqs = [(d(r["query"]), d(r["cand_tokens"]), d(r["cand_offsets"])) for r in reqs]
+    hreqs = [(pin(r["query"]), pin(r["cand_tokens"]), pin(r["cand_offsets"])) for r in reqs]
+    hidx = torch.empty(wl.top_k, dtype=torch.int32).pin_memory().numpy()
+    hsc = torch.empty(wl.top_k, dtype=torch.float32).pin_memory().numpy()
+    stream = torch.cuda.current_stream()
+    tr0 = model.select(*dreqs[0], wl.top_k, wl.schedule, want_trace=True)[2]
+
+    def timed(fn, k, w):
+        for i in range(w):
+            fn(i)
+        torch.cuda.synchronize()
+        n0 = model.launch_count
+        pairs = []
+        for i in range(k):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            fn(w + i)
+            b.record(stream)
+            pairs.append((a, b))
+        torch.cuda.synchronize()
+        lat = [a.elapsed_time(b) for a, b in pairs]
+        return pairs[0][0].elapsed_time(pairs[-1][1]), lat, model.launch_count - n0
+
+    dev_step = lambda i, s=wl.schedule: model.select(*dreqs[i % n_req], wl.top_k, s, want_trace=False)
+    host_step = lambda i: model.select_host(*hreqs[i % n_req], wl.top_k, wl.schedule, idx_out=hidx, sc_out=hsc)
+    sampler = ClockSampler(local)
+    sampler.start()
+    total_ms, lat, launches = timed(dev_step, steps, warmup)
+    clocks = sampler.stop()
+    toks = sum(int(lens_all[(warmup + i) % n_req].sum()) for i in range(steps))
+    e2e_steps = max(5, steps // 2)
+    e2e_ms, e2e_lat, _ = timed(host_step, e2e_steps, 2)
+    e2e_toks = sum(int(lens_all[(2 + i) % n_req].sum()) for i in range(e2e_steps))
+    off_steps = max(3, steps // 6)
+    off_ms, _, _ = timed(lambda i: dev_step(i, Schedule(MODE_NONE)), off_steps, 2)
+    per = profile_classes(P, model, lambda i: dev_step(warmup + i), max(3, min(steps, 5)))
+    peaks = measured_peaks()
+
+    def rate(names, scale):
+        ms = sum(per[n]["ms_per_step"] for n in names)
+        return (sum(per[n]["work_per_step"] for n in names) / (ms * 1e-3) / scale) if ms > 0 else 0.0
+    g_tf, a_tf = rate(GEMM_CLASSES, 1e12), rate(("attention",), 1e12)
+    req_fl = sum(per[n]["work_per_step"] for n in GEMM_CLASSES + ("attention",))
+    req_tf = req_fl / (total_ms / steps * 1e-3) / 1e12
+    out = {"workload": wl.name, "steps": steps, "warmup": warmup, "requests_cycled": n_req,
+           "tokens_per_request": int(np.mean([l.sum() for l in lens_all])), "candidates": wl.n_candidates, "top_k": wl.top_k,
+           "dtype": "bf16" if cfg.dtype == 1 else "f32",
+           "latency_ms": {"p50": float(np.percentile(lat, 50)), "p99": float(np.percentile(lat, 99))},
+           "ms_per_step": total_ms / steps, "candidate_tokens_per_s": toks / (total_ms * 1e-3),
+           "e2e": {"candidate_tokens_per_s": e2e_toks / (e2e_ms * 1e-3), "p50_ms": float(np.percentile(e2e_lat, 50)),
+                   "steps": e2e_steps,
+                   "h2d_bytes_per_step": int(np.mean([q.nbytes + c.nbytes + o.nbytes for q, c, o in hreqs])),
+                   "d2h_bytes_per_step": int(hidx.nbytes + hsc.nbytes)},
+           "pruning_off_ms_per_step": off_ms / off_steps, "pruning_speedup": (off_ms / off_steps) / (total_ms / steps),
+           "gemm": {"tflops": g_tf, "frac_of_sustained_peak": g_tf / peaks["bf16_tflops_sustained"],
+                    "frac_of_burst_peak": g_tf / peaks["bf16_tflops"], "frac_of_nominal_2250": g_tf / 2250.0},
+           "attention": {"tflops": a_tf, "frac_of_sustained_peak": a_tf / peaks["bf16_tflops_sustained"],
+                         "frac_of_burst_peak": a_tf / peaks["bf16_tflops"], "frac_of_nominal_2250": a_tf / 2250.0},
+           "rmsnorm_gbs": rate(("rmsnorm",), 1e9), "compact_gbs": rate(("compact",), 1e9), "embed_gbs": rate(("embed",), 1e9),
+           "route_us_per_launch": (1e3 * per["route"]["ms_per_step"] / per["route"]["launches_per_step"]
+                                   if per["route"]["launches_per_step"] else None),
+           "request_tflops": req_tf, "request_frac_of_sustained_peak": req_tf / peaks["bf16_tflops_sustained"],
+           "gpu_launches": int(launches), "clocks": clocks,
+           "handle_options": {"stream_weights": bool(wl.stream_weights), "activation_budget_bytes": wl.activation_budget_bytes,
+                              "chunks_per_layer_max": tr0.n_chunks_max, "shared_query_prefix_rows": tr0.shared_prefix_rows},
+           "device_bytes": {"handle": tr0.workspace_bytes, "weights_device": _tensor_bytes(tw, True),
+                            "weights_pinned_host": _tensor_bytes(tw, False),
+                            "torch_peak_allocated_above_start": int(torch.cuda.max_memory_allocated(dev) - base_bytes)}}
+    model.close()
+    return out
 
 
 # ----------------------------------------------------------------------------------------------- CUDA arm
@@ -440,12 +569,25 @@ def run_prism(args):
                                     if v["ms_per_step"] > 0 else 0.0)}
                            for n, v in per.items()}
         if not args.no_cpu_baseline and not w4:   # the oracle leg times the unquantised model
-            ids = oracle_sample_ids(wl, reqs[0], max_cand=32)
+            ids = oracle_sample_ids(wl, reqs[0], max_cand=20)
             n_c = len(ids)
             rate, dt, t = oracle_sample_rate(wl, w_np, reqs[0], ids)
             line["cpu_baseline"] = {"value": rate, "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle",
-                                    "sample": f"the {n_c} shortest of {wl.n_candidates} candidates of request 0 ({t} tokens), all "
+                                    "sample": f"{n_c} of {wl.n_candidates} candidates of request 0, evenly spaced in length rank "
+                                              f"(lengths {int(lens_all[0][ids].min())}..{int(lens_all[0][ids].max())} of "
+                                              f"{int(lens_all[0].min())}..{int(lens_all[0].max())}, {t} tokens), all "
                                               f"{cfg.n_layers} layers, unpruned fp64 numpy forward, {dt:.1f} s"}
+        plain = not (args.stream_weights or args.activation_budget_mb or args.embed_cache_rows or args.hidden_offload or w4)
+        if args.side_workloads == "on" and world == 1 and args.workload == 1 and plain and not by_cand:
+            # the other benchmark workloads (tiny fp32, 4B-, 8B-shaped, 1000-candidate stress) in the same run; the
+            # headline above stays the 0.6B-shaped workload.  Its handle is closed first: one handle at a time.
+            import gc
+            model.close()
+            line["workloads"] = {}
+            for index, k in ((0, 100), (2, 20), (3, 20), (4, 30)):
+                gc.collect()
+                torch.cuda.empty_cache()            # the previous workload's weights go back to the driver
+                line["workloads"][f"cfg{index}"] = measure_side_workload(P, index, k, 5, dev, local)
         print(json.dumps(line))
     model.close()
     if world > 1:
@@ -474,6 +616,9 @@ def main():
     ap.add_argument("--weight-format", default="plain", choices=["plain", "w4"],
                     help="w4: the layer matrices are stored (and, for the streamed workload, copied) as 4-bit codes and "
                          "rebuilt as bf16 layer by layer on the device")
+    ap.add_argument("--side-workloads", default="on", choices=["on", "off"],
+                    help="on (1 GPU, workload 1, no memory options): the line also carries a `workloads` block with the "
+                         "tiny fp32, 4B-shaped, 8B-shaped (streamed, chunked) and 1000-candidate workloads")
     ap.add_argument("--shard", default="requests", choices=["requests", "candidates"],
                     help="requests: every rank serves its own requests (weak scaling, the default); candidates: all "
                          "ranks share each request, one score all-reduce per probe (strong scaling)")
