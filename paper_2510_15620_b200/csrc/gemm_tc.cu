@@ -408,6 +408,46 @@ EncodeTiledFn get_encode() {
   return fn;
 }
 
+// A tensor map is a pure function of (kind, base, rows, cols, box); the layer loop asks for the same few maps
+// again and again (the handle's buffers are fixed and the row count changes only at a compaction), so each host
+// thread keeps the most recent ones.  Direct-mapped, 64 entries; a miss encodes and replaces.
+struct MapKey {
+  int kind;
+  const void* base;
+  uint64_t rows, cols;
+  uint32_t box_rows, box_cols;
+  bool operator==(const MapKey& o) const {
+    return kind == o.kind && base == o.base && rows == o.rows && cols == o.cols && box_rows == o.box_rows &&
+           box_cols == o.box_cols;
+  }
+};
+struct MapSlot {
+  MapKey key;
+  TmaDesc desc;
+  bool valid;
+};
+constexpr int kMapSlots = 64;
+
+template <typename Encode>
+cudaError_t cached_map(TmaDesc* out, const MapKey& key, Encode encode) {
+  thread_local MapSlot slots[kMapSlots] = {};
+  uint64_t h = reinterpret_cast<uintptr_t>(key.base) * 0x9E3779B97F4A7C15ull;
+  h ^= (key.rows + 0x632BE59BD9B4E019ull) * 0xC2B2AE3D27D4EB4Full;
+  h ^= (key.cols * 31 + key.box_rows * 7 + key.box_cols + (uint64_t)key.kind * 1315423911ull) * 0x165667B19E3779F9ull;
+  MapSlot& s = slots[(h >> 40) % kMapSlots];
+  if (s.valid && s.key == key) {
+    *out = s.desc;
+    return cudaSuccess;
+  }
+  const cudaError_t e = encode(out);
+  if (e == cudaSuccess) {
+    s.key = key;
+    s.desc = *out;
+    s.valid = true;
+  }
+  return e;
+}
+
 }  // namespace
 
 static_assert(sizeof(CUtensorMap) == sizeof(TmaDesc), "TmaDesc must mirror CUtensorMap");
@@ -418,14 +458,16 @@ cudaError_t make_tma_2d_bf16(TmaDesc* out, const void* base, uint64_t rows, uint
   if (!enc) return cudaErrorNotSupported;
   if ((reinterpret_cast<uintptr_t>(base) & 15) || (cols * 2) % 16 || box_cols * 2 != 128 || box_rows > 256)
     return cudaErrorInvalidValue;
-  cuuint64_t dims[2] = {cols, rows};
-  cuuint64_t strides[1] = {cols * 2};
-  cuuint32_t box[2] = {box_cols, box_rows};
-  cuuint32_t estr[2] = {1, 1};
-  CUresult r = enc(reinterpret_cast<CUtensorMap*>(out), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base),
-                   dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+  return cached_map(out, MapKey{0, base, rows, cols, box_rows, box_cols}, [&](TmaDesc* d) {
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {cols * 2};
+    cuuint32_t box[2] = {box_cols, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = enc(reinterpret_cast<CUtensorMap*>(d), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base),
+                     dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+  });
 }
 
 int gemm_tc_sm_count() {
@@ -445,28 +487,32 @@ cudaError_t make_tma_2d_f32_box32(TmaDesc* out, const void* base, uint64_t rows,
   EncodeTiledFn enc = get_encode();
   if (!enc) return cudaErrorNotSupported;
   if ((reinterpret_cast<uintptr_t>(base) & 15) || (cols * 4) % 16) return cudaErrorInvalidValue;
-  cuuint64_t dims[2] = {cols, rows};
-  cuuint64_t strides[1] = {cols * 4};
-  cuuint32_t box[2] = {32, 32};
-  cuuint32_t estr[2] = {1, 1};
-  CUresult r = enc(reinterpret_cast<CUtensorMap*>(out), CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base),
-                   dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                   CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+  return cached_map(out, MapKey{1, base, rows, cols, 32, 32}, [&](TmaDesc* d) {
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {cols * 4};
+    cuuint32_t box[2] = {32, 32};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = enc(reinterpret_cast<CUtensorMap*>(d), CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base),
+                     dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                     CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+  });
 }
 
 cudaError_t make_tma_2d_bf16_box32_sw64(TmaDesc* out, const void* base, uint64_t rows, uint64_t cols) {
   EncodeTiledFn enc = get_encode();
   if (!enc) return cudaErrorNotSupported;
   if ((reinterpret_cast<uintptr_t>(base) & 15) || (cols * 2) % 16) return cudaErrorInvalidValue;
-  cuuint64_t dims[2] = {cols, rows};
-  cuuint64_t strides[1] = {cols * 2};
-  cuuint32_t box[2] = {32, 32};
-  cuuint32_t estr[2] = {1, 1};
-  CUresult r = enc(reinterpret_cast<CUtensorMap*>(out), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base),
-                   dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B,
-                   CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+  return cached_map(out, MapKey{2, base, rows, cols, 32, 32}, [&](TmaDesc* d) {
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {cols * 2};
+    cuuint32_t box[2] = {32, 32};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = enc(reinterpret_cast<CUtensorMap*>(d), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base),
+                     dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B,
+                     CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+  });
 }
 
 cudaError_t launch_gemm_tc(const TmaDesc& a, const TmaDesc& b0, const TmaDesc& b1, void* out, float* resid, int m,
