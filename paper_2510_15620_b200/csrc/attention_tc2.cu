@@ -386,7 +386,7 @@ k_attention_tc2(const __grid_constant__ CUtensorMap map_qkv, const __grid_consta
         uint64_t rs2;
         // exponentials of one 32-key chunk into 16 packed bf16 pairs (key 2c in the low half) and the row sum
         auto chunk = [&](int ch, uint32_t* cur, uint32_t* out16) {
-          if (diag && ch > quarter) {  // every key of this chunk lies beyond every row of this warp
+          if ((diag && ch > quarter) || j * BN + ch * 32 >= it.len) {  // beyond every row of this warp, or beyond the end
 #pragma unroll
             for (int c = 0; c < 16; ++c) out16[c] = 0u;
             return;

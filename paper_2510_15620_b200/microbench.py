@@ -170,7 +170,12 @@ def main():
         fn = lambda: ops.prism_op_attention(qkv, o, cud, a.seqs, int(lens.max()), a.hq, a.hkv, dh, a.causal, PRISM_BF16, a.impl, err)
         med, best = _time(fn, a.iters, a.warmup, flush)
         fl = float(np.sum((2.0 if a.causal else 4.0) * lens.astype(np.float64) ** 2 * a.hq * dh))
-        out.update(seqs=a.seqs, tokens=int(cu[-1]), causal=a.causal, head_dim=dh, ms=med, ms_min=best, tflops=fl / med / 1e9)
+        # what the 128 x 128 (query block x key block) tiling executes: every block a sequence touches, whole
+        nb = (lens + 127) // 128
+        blocks = nb * (nb + 1) // 2 if a.causal else nb * nb
+        fl_exec = float(np.sum(blocks)) * 4.0 * 128 * 128 * dh * a.hq
+        out.update(seqs=a.seqs, tokens=int(cu[-1]), causal=a.causal, head_dim=dh, ms=med, ms_min=best, tflops=fl / med / 1e9,
+                   executed_tile_tflops=fl_exec / med / 1e9, useful_fraction_of_executed_tiles=fl / fl_exec)
     elif a.op == "rmsnorm":
         x = rnd(a.rows, a.d)
         gain = torch.ones(a.d, dtype=torch.bfloat16, device=dev)
