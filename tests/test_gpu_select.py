@@ -325,14 +325,15 @@ def _gold_scores(name, r):
     return S
 
 
-def test_cfg1_full_size_in_bench_configuration(P):
-    """Qwen3-0.6B-shaped, 100 candidates, the launch configuration bench.py times.  All candidates are
-    checked against stored oracle scores when the golden file is present; three sampled candidates are
-    always forwarded by the oracle on the spot."""
+@pytest.mark.parametrize("r", [0, 1, 2])
+def test_cfg1_full_size_in_bench_configuration(P, r):
+    """Qwen3-0.6B-shaped, 100 candidates, the launch configuration bench.py times, request seeds 0, 1 and 2.  All
+    candidates are checked against the stored oracle scores of the request (tests/golden/, written by
+    make_scores.py); three sampled candidates are also forwarded by the oracle on the spot."""
     wl = synth.workload(1)
     cfg = wl.model
     w = synth.make_weights(cfg, wl.weight_seed)
-    req = synth.make_request(wl, 0)
+    req = synth.make_request(wl, r)
     model = make_model(P, cfg, w, req)
     sched = wl.schedule
     # unpruned first: every candidate reaches the last layer
@@ -345,18 +346,25 @@ def test_cfg1_full_size_in_bench_configuration(P):
     Ss = oracle.score_matrix(req["query"], req["cand_tokens"], req["cand_offsets"], w, cfg, layers, candidates=sample)
     worst = check_scores(tr0, Ss, TOL_BF16, ids_known=sample)
     check_scores(tr, Ss, TOL_BF16, ids_known=sample)
-    S = _gold_scores(wl.name, 0)
+    S = _gold_scores(wl.name, r)
+    assert S is not None, "stored oracle scores of this request are missing"
     if S is not None:
         for j, c in enumerate(sample):                                  # the stored file is what the oracle computes
             for l in layers:
                 assert abs(S[l][c] - Ss[l][j]) < 1e-9
         worst = max(worst, check_scores(tr0, S, TOL_BF16))
         check_scores(tr, S, TOL_BF16)
-        check_end_to_end(tr, idx, S, wl.n_candidates, wl.top_k, cfg.n_layers, sched, TOL_BF16)
-        check_end_to_end(tr0, idx0, S, wl.n_candidates, wl.top_k, cfg.n_layers, Schedule(MODE_NONE), TOL_BF16)
-    print(f"cfg1 worst |score diff| vs oracle: {worst:.4g}; pruned run stopped after layer {tr.layers_run}; "
+        verdict = check_end_to_end(tr, idx, S, wl.n_candidates, wl.top_k, cfg.n_layers, sched, TOL_BF16)
+        ref = oracle.replay_select(lambda layer, a: np.asarray(S[layer])[np.asarray(a, np.int64)].astype(np.float32),
+                                   wl.n_candidates, wl.top_k, cfg.n_layers, sched)
+        print(f"cfg1 request {r}: pruned run vs the oracle's own decisions: {verdict}, overlap@{wl.top_k} "
+              f"{len(set(ref.topk_idx) & set(map(int, idx)))}/{len(idx)}")
+        # tr0 was traced under the never-firing schedule: the walk has to be given that schedule (its probes), not NONE
+        check_end_to_end(tr0, idx0, S, wl.n_candidates, wl.top_k, cfg.n_layers,
+                         Schedule(MODE_CLUSTER, sched.probe_layers, cv_threshold=1e30), TOL_BF16)
+    print(f"cfg1 request {r}: worst |score diff| vs oracle: {worst:.4g}; pruned run stopped after layer {tr.layers_run}; "
           f"tokens per layer {tr.tokens_per_layer}")
-    assert any(r.fired for r in tr.records)
+    assert any(rec.fired for rec in tr.records)
     model.close()
 
 
