@@ -205,3 +205,11 @@ def test_cfg3_qwen3_8b_streamed_and_chunked(P):
     assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1])
     for r1, r2 in zip(a[2].records, b[2].records):
         assert np.array_equal(r1.scores, r2.scores) and r1.active_ids == r2.active_ids
+
+
+@pytest.mark.parametrize("index", [2, 4])
+def test_second_request_of_the_4b_shaped_and_stress_workloads(P, index):
+    """Request seed 1 of the same workloads against its own stored oracle scores (every candidate): scores, replayed
+    decisions and the end-to-end check, as for request 0."""
+    _, _, res = _run_workload(P, index, r=1)
+    assert any(rec.fired for rec in res[0][2].records)
