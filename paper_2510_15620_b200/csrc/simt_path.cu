@@ -134,7 +134,9 @@ __global__ void __launch_bounds__(128) k_attention_simt(const T* __restrict__ qk
       const T* kr = base + (size_t)u * ld + koff;
       float acc = 0.f;
       if constexpr (sizeof(T) == 4) {
-        if ((dh & 3) == 0) {
+        // 16-byte loads where every key row starts on a 16-byte boundary (row pitch and head offsets are then
+        // multiples of 16 bytes too)
+        if ((dh & 3) == 0 && (reinterpret_cast<uintptr_t>(qkv) & 15) == 0) {
           const float4* k4 = reinterpret_cast<const float4*>(kr);
           const float4* q4 = reinterpret_cast<const float4*>(sq[w]);
           for (int c = 0; c < (dh >> 2); ++c) {
