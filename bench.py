@@ -568,7 +568,7 @@ def run_prism(args):
                                    (v["work_per_step"] / (v["ms_per_step"] * 1e-3) / (1e12 if n in GEMM_CLASSES or n == "attention" else 1e9)
                                     if v["ms_per_step"] > 0 else 0.0)}
                            for n, v in per.items()}
-        if not args.no_cpu_baseline and not w4:   # the oracle leg times the unquantised model
+        if not args.no_cpu_baseline and not w4 and world == 1:   # the oracle leg (N = 1 only) times the unquantised model
             ids = oracle_sample_ids(wl, reqs[0], max_cand=20)
             n_c = len(ids)
             rate, dt, t = oracle_sample_rate(wl, w_np, reqs[0], ids)
