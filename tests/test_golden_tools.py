@@ -42,6 +42,7 @@ def test_stored_score_files_cover_what_the_parity_tests_expect():
     expect = {"cfg1_qwen3_0p6b_scores_r0.txt": (1, 100), "cfg1_qwen3_0p6b_scores_r1.txt": (1, 100),
               "cfg1_qwen3_0p6b_scores_r2.txt": (1, 100), "cfg2_qwen3_4b_scores_r0.txt": (2, 200),
               "cfg2_qwen3_4b_scores_r1.txt": (2, 200), "cfg3_qwen3_8b_streamed_scores_r0.txt": (3, 100),
+              "cfg3_qwen3_8b_streamed_scores_r1.txt": (3, 100),
               "cfg4_stress_0p6b_scores_r0.txt": (4, 1000), "cfg4_stress_0p6b_scores_r1.txt": (4, 1000)}
     for name, (index, n) in expect.items():
         S, ids, head = make_scores.read_scores(os.path.join(GOLD, name))

@@ -147,7 +147,7 @@ def _run_workload(P, index, budgets=(None,), r=0):
             check_scores(tr_all, S, tol, ids_known=ids)
             rms, worst, n_sc = _score_stats(tr_all, S, ids)
             print(f"{wl.name}: all probes, nothing pruned: {n_sc} scores, rms {rms:.4f} (oracle's own bf16-storage noise "
-                  f"{sigma:.4f}), max {worst:.4f}, max relative to the layer's score rms "
+                  f"{sigma:.4f}), max {worst:.6f}, max relative to the layer's score rms "
                   f"{max(_relative(tr_all, S, ids)):.4f}")
             if tol > TOL_BF16:
                 assert rms <= RMS_RATIO_MAX * sigma, (rms, sigma)
@@ -207,8 +207,8 @@ def test_cfg3_qwen3_8b_streamed_and_chunked(P):
         assert np.array_equal(r1.scores, r2.scores) and r1.active_ids == r2.active_ids
 
 
-@pytest.mark.parametrize("index", [2, 4])
-def test_second_request_of_the_4b_shaped_and_stress_workloads(P, index):
+@pytest.mark.parametrize("index", [2, 3, 4])
+def test_second_request_of_the_large_workloads(P, index):
     """Request seed 1 of the same workloads against its own stored oracle scores (every candidate): scores, replayed
     decisions and the end-to-end check, as for request 0."""
     _, _, res = _run_workload(P, index, r=1)
