@@ -46,12 +46,14 @@ __device__ __forceinline__ float ex2(float x) {  // 2^x on the special-function 
 }
 
 // 2^x for a pair of exponents.  All softmax warps of the SM share its special-function unit, so kEmulated of
-// every 8 pairs take the FMA pipe instead (measured: 0, 2, 3 and 4 of 8 are within 4 % of each other, 2 is best):
-// x = n + f with n = round(x) (the 1.5 * 2^23 trick leaves n in the low bits of t), 2^f by a cubic whose relative
-// error (7.5e-5) is far below bf16 rounding, and n is added to the exponent field.  x is clamped to [-125, 126]:
-// masked scores (-inf) come out as 2^-125 instead of 0 (every row sum is at least 1), and exponents beyond
-// fp32 range still produce a sum that the range check catches.
-constexpr int kEmulated = 2;
+// every 8 pairs can take the FMA pipe instead: x = n + f with n = round(x) (the 1.5 * 2^23 trick leaves n in the low
+// bits of t), 2^f by a cubic whose relative error (7.5e-5) is far below bf16 rounding, and n is added to the exponent
+// field.  x is clamped to [-125, 126]: masked scores (-inf) come out as 2^-125 instead of 0 (every row sum is at least
+// 1), and exponents beyond fp32 range still produce a sum that the range check catches.
+// Measured in one call on the three benchmark shape sets: 0 of 8 -> 371 / 650 / 844 TFLOP/s, 1 -> 372 / 649 / 842,
+// 2 -> 371 / 641 / 834, 3 -> 362 / 625 / 815: the special-function pipe is about 20 % busy, so taking work off it
+// buys nothing and the extra instructions cost a little.  All exponentials therefore go to ex2.approx.
+constexpr int kEmulated = 0;
 __device__ __forceinline__ void exp2_pair(uint64_t xv, bool emulate, float& p0, float& p1) {
   float x0, x1;
   f2_unpack(xv, x0, x1);
