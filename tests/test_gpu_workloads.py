@@ -75,8 +75,10 @@ def _tolerance(index):
     candidates, 8 scored layers each) has an RMS of 0.03 - 0.04, so no bf16 evaluation can stay within 3e-2 on every
     score.  There the deviation is treated as what it is, noise: no score may be further from the oracle than
     SIGMAS_MAX times the oracle's own noise RMS, and the RMS deviation of the CUDA path over all stored candidates may
-    not exceed RMS_RATIO_MAX times it (the per-score bound is loose by construction: the largest of 800 - 1600
-    heavy-tailed deviations; the RMS bound is the one that would catch an arithmetic fault)."""
+    not exceed RMS_RATIO_MAX times it, nor their 99th percentile P99_SIGMAS_MAX times it (the per-score bound is loose
+    by construction: the largest of 800 - 1600 heavy-tailed deviations, which moved between 3.7 and 5.5 sigma when a
+    quarter of the attention kernel's exponentials changed from a cubic to ex2.approx; the RMS and percentile bounds
+    are the ones that would catch an arithmetic fault)."""
     exact, bf16 = GOLD_FILES[index]
     sigma, worst, n = _bf16_storage_noise(exact, bf16)
     return max(TOL_BF16, SIGMAS_MAX * sigma), sigma, worst, n
@@ -84,6 +86,7 @@ def _tolerance(index):
 
 SIGMAS_MAX = 6.0
 RMS_RATIO_MAX = 1.5
+P99_SIGMAS_MAX = 4.0
 GOLD_FILES = {
     2: ("cfg2_qwen3_4b_scores_r0.txt", "cfg2_qwen3_4b_scores_bf16act_r0_s16.txt"),
     3: ("cfg3_qwen3_8b_streamed_scores_r0.txt", "cfg3_qwen3_8b_streamed_scores_bf16act_r0_s32.txt"),
@@ -96,8 +99,8 @@ def _score_stats(tr, S, ids):
     col = {c: j for j, c in enumerate(ids)}
     d = [float(s) - float(S[rec.layer][col[int(i)]]) for rec in tr.records for i, s in zip(rec.active_ids, rec.scores)
          if int(i) in col]
-    d = np.asarray(d)
-    return float(np.sqrt(np.mean(d * d))), float(np.max(np.abs(d))), len(d)
+    d = np.abs(np.asarray(d))
+    return float(np.sqrt(np.mean(d * d))), float(np.max(d)), len(d), float(np.percentile(d, 99))
 
 
 def _run_workload(P, index, budgets=(None,), r=0):
@@ -134,7 +137,7 @@ def _run_workload(P, index, budgets=(None,), r=0):
             ref = oracle.replay_select(lambda layer, a: np.asarray(S[layer])[np.asarray(a, np.int64)].astype(np.float32),
                                        wl.n_candidates, wl.top_k, cfg.n_layers, wl.schedule)
             verdict += f", overlap@{wl.top_k} with the oracle's top-K {len(set(ref.topk_idx) & set(map(int, idx)))}/{len(idx)}"
-        rms, worst, n_sc = _score_stats(tr, S, ids)
+        rms, worst, n_sc, _ = _score_stats(tr, S, ids)
         print(f"{wl.name}: budget {b}, chunks/layer <= {tr.n_chunks_max}, stopped after layer {tr.layers_run}, "
               f"active per probe {[r.n_active_before for r in tr.records]}, pruned run: {n_sc} scores of stored candidates, "
               f"rms {rms:.4f}, max {worst:.4f}; end to end: {verdict}; workspace {tr.workspace_bytes / 2**30:.2f} GiB")
@@ -145,12 +148,13 @@ def _run_workload(P, index, budgets=(None,), r=0):
             never = Schedule(MODE_CLUSTER, wl.schedule.probe_layers, cv_threshold=1e30)
             _, _, tr_all = model.select(q, c, o, wl.top_k, never)
             check_scores(tr_all, S, tol, ids_known=ids)
-            rms, worst, n_sc = _score_stats(tr_all, S, ids)
+            rms, worst, n_sc, p99 = _score_stats(tr_all, S, ids)
             print(f"{wl.name}: all probes, nothing pruned: {n_sc} scores, rms {rms:.4f} (oracle's own bf16-storage noise "
-                  f"{sigma:.4f}), max {worst:.6f}, max relative to the layer's score rms "
-                  f"{max(_relative(tr_all, S, ids)):.4f}")
+                  f"{sigma:.4f}), 99th percentile {p99:.4f} = {p99 / sigma:.2f} sigma, max {worst:.4f} = {worst / sigma:.2f} sigma, "
+                  f"max relative to the layer's score rms {max(_relative(tr_all, S, ids)):.4f}")
             if tol > TOL_BF16:
                 assert rms <= RMS_RATIO_MAX * sigma, (rms, sigma)
+                assert p99 <= P99_SIGMAS_MAX * sigma, (p99, sigma)
         model.close()
     return wl, req, results
 
