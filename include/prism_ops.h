@@ -67,8 +67,9 @@ PRISM_API int prism_op_gemm_qkv_rope(const void* a, const void* w_qkv, void* out
 /* Attention over packed sequences: for sequence s (rows cu[s]..cu[s+1]) and query head h (kv head
  * h / (Hq/Hkv)): out = softmax(q k^T / sqrt(head_dim) [+ causal mask]) v.  qkv [total, (Hq+2Hkv)*dh],
  * out [total, Hq*dh].  total = cu[n_seq] rows; max_len >= the longest sequence.  impl: PRISM_IMPL_AUTO =
- * tcgen05 kernel (bf16; head_dim 128: two query heads of a KV group per CTA when Hq/Hkv is even, else one
- * head per CTA; head_dim 64: one head per CTA; reports an expired bounded wait in err_word bit 4), PRISM_IMPL_SOLO = the one-head tcgen05
+ * tcgen05 kernel (bf16; two query heads per CTA when Hq/Hkv is even (head_dim 128 or 64: the pair shares its KV
+ * head) or when Hq = Hkv is even at head_dim 64 (a KV head per query head); else one head per CTA; reports an
+ * expired bounded wait in err_word bit 4), PRISM_IMPL_SOLO = the one-head tcgen05
  * kernel, PRISM_IMPL_MMA = warp-level MMA kernel (bf16, head_dim 128), PRISM_IMPL_SIMT = CUDA cores. */
 PRISM_API int prism_op_attention(const void* qkv, void* out, const int32_t* cu, int32_t n_seq, int32_t total,
                                  int32_t max_len, int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim,

@@ -1,8 +1,10 @@
 // S5 on the 5th-generation tensor cores, two query heads per CTA: varlen flash attention over packed
-// sequences, bf16, head_dim 128, causal or bidirectional, for grouped-query models with an even group size.
+// sequences, bf16, causal or bidirectional; head_dim 128 for grouped-query models with an even group size, head_dim 64
+// for even group sizes and for one key/value head per query head (the encoder stack).
 //
-// A work item is (sequence, PAIR of query heads that share a key/value head, 128-query-row block): the
-// two heads' Q tiles ("A" and "B") use the same K_j / V_j tiles (128 keys each), which are fetched once.
+// A work item is (sequence, PAIR of query heads, 128-query-row block).  With an even group size the pair shares a
+// key/value head: the two heads' Q tiles ("A" and "B") use the same K_j / V_j tiles (128 keys each), which are
+// fetched once.  With one key/value head per query head (head_dim 64 only) a ring stage holds both heads' tiles.
 // One persistent CTA per SM walks the items, heaviest query blocks first; nothing but the item's end
 // separates consecutive items, so the loads and the first scores of the next item run under the tail of
 // the current one.  Warp-specialised, 576 threads:
@@ -29,12 +31,17 @@ namespace {
 
 using namespace tc;
 
-constexpr int BM = 128, BN = 128, DH = 128;
-constexpr int kTile = 128 * DH * 2;  // 32 KB: two [128 x 64] swizzled sub-tiles (Q, K and V tiles alike)
+constexpr int BM = 128, BN = 128;
 constexpr int NK = 2, NV = 2;
 constexpr int kStageBytes = 32 * 64;  // per softmax warp: 32 rows x 32 bf16 of output on their way to global memory
-constexpr int kSmemBytes = (2 + NK + NV) * kTile + 16 * kStageBytes + 1024 /*alignment slack*/ + 512 /*barriers, flags*/;
-static_assert(kSmemBytes <= 232448, "exceeds the shared memory one CTA may have");
+// One [128 x DH] tile (Q, K and V tiles alike): DH / 64 swizzled [128 x 64] sub-tiles, 32 KB at head_dim 128.
+__host__ __device__ constexpr int tile_bytes(int dh) { return 128 * dh * 2; }
+// kShare: the two query heads of an item read the same K / V head (a grouped-query pair), so a ring stage holds one
+// tile; otherwise (one K / V head per query head) it holds the two heads' tiles side by side.
+__host__ __device__ constexpr int smem_bytes(int dh, bool share) {
+  return (2 + (NK + NV) * (share ? 1 : 2)) * tile_bytes(dh) + 16 * kStageBytes + 1024 /*alignment slack*/ + 512 /*barriers, flags*/;
+}
+static_assert(smem_bytes(128, true) <= 232448 && smem_bytes(64, false) <= 232448, "exceeds the shared memory one CTA may have");
 constexpr float kBigSum = 1.2089258e24f;  // 2^80: row sums of one block beyond this move the reference
 constexpr int kThreads = 576;  // TMA warp, MMA warp, 2 x 8 softmax warps
 constexpr int kTmemCols = 512;
@@ -116,6 +123,7 @@ struct ItemReader {
   __device__ __forceinline__ void advance() { ++n; }
 };
 
+template <int DH, bool kShare>
 __global__ void __launch_bounds__(kThreads, 1)
 k_attention_tc2(const __grid_constant__ CUtensorMap map_qkv, const __grid_constant__ CUtensorMap map_pre,
                 const __grid_constant__ CUtensorMap map_rest, __nv_bfloat16* __restrict__ out,
@@ -127,8 +135,10 @@ k_attention_tc2(const __grid_constant__ CUtensorMap map_qkv, const __grid_consta
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
   unsigned char* gen = smem_raw + (base - raw);
-  const uint32_t s_q = base, s_k = base + 2 * kTile, s_v = s_k + NK * kTile, s_o = s_v + NV * kTile;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(gen + (2 + NK + NV) * kTile + 16 * kStageBytes);
+  constexpr int kTile = tile_bytes(DH), kSub = DH / 64;   // bytes per tile, [128 x 64] sub-tiles per tile
+  constexpr int kStage = (kShare ? 1 : 2) * kTile;         // one K (or V) ring stage
+  const uint32_t s_q = base, s_k = base + 2 * kTile, s_v = s_k + NK * kStage, s_o = s_v + NV * kStage;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(gen + 2 * kTile + (NK + NV) * kStage + 16 * kStageBytes);
   // q_full[2], q_empty[2], k_full[2], k_empty[2], v_full[2], v_empty[2], s_full[2], p_full[2], o_full[2]
   const uint32_t b_q_full = smem_u32(bars), b_q_empty = smem_u32(bars + 2);
   const uint32_t b_k_full = smem_u32(bars + 4), b_k_empty = smem_u32(bars + 6);
@@ -210,37 +220,42 @@ k_attention_tc2(const __grid_constant__ CUtensorMap map_qkv, const __grid_consta
         ring[slot] = it;
         mbar_arrive(b_item_full + 8 * slot);
         if (it.n_blocks == 0) break;
-        const int h0 = it.pair * 2, kvh = h0 / group;
-        const int kcol = (hq + kvh) * DH, vcol = (hq + hkv + kvh) * DH;
+        const int h0 = it.pair * 2;
         // 128 rows of the sequence starting at row 128 * blk, columns col .. col + 127, as two 64-column
         // sub-tiles.  The block that holds a shared prefix is put together from two row ranges (prefix rows, then
         // the sequence's own first 128 - prefix rows; prefix is a multiple of 8, so the second part starts on a
         // swizzle-atom boundary); the boxes add up to a full tile, so the byte count is the same.
         auto load_tile = [&](uint32_t dst, int col, int blk, uint32_t bar) {
-          mbar_expect_tx(bar, kTile);
           if (prefix > 0 && blk == 0) {
-            tma_load_2d(dst, &map_pre, col, 0, bar);
-            tma_load_2d(dst + kTile / 2, &map_pre, col + 64, 0, bar);
-            tma_load_2d(dst + prefix * 128, &map_rest, col, it.beg, bar);
-            tma_load_2d(dst + kTile / 2 + prefix * 128, &map_rest, col + 64, it.beg, bar);
+#pragma unroll
+            for (int sb = 0; sb < kSub; ++sb) {
+              tma_load_2d(dst + sb * (128 * 128), &map_pre, col + 64 * sb, 0, bar);
+              tma_load_2d(dst + sb * (128 * 128) + prefix * 128, &map_rest, col + 64 * sb, it.beg, bar);
+            }
           } else {
             const int row = it.beg + blk * 128 - prefix;
-            tma_load_2d(dst, &map_qkv, col, row, bar);
-            tma_load_2d(dst + kTile / 2, &map_qkv, col + 64, row, bar);
+#pragma unroll
+            for (int sb = 0; sb < kSub; ++sb) tma_load_2d(dst + sb * (128 * 128), &map_qkv, col + 64 * sb, row, bar);
           }
         };
         auto load_q = [&](int x) {
           if (!mbar_wait(b_q_empty + 8 * x, (ic & 1) ^ 1, err, abort_flag)) return false;
+          mbar_expect_tx(b_q_full + 8 * x, kTile);
           load_tile(s_q + x * kTile, (h0 + x) * DH, it.qb, b_q_full + 8 * x);
           return true;
         };
-        auto load_kv = [&](int col, int t, uint32_t ring, uint32_t b_full, uint32_t b_empty, uint32_t& cnt, int depth) {
+        // K (first = hq) or V (first = hq + hkv) of key block t into the next stage of its ring: one tile for a pair that
+        // shares its K / V head, else one tile per head, under one barrier
+        auto load_kv = [&](int first, int t, uint32_t ring, uint32_t b_full, uint32_t b_empty, uint32_t& cnt, int depth) {
           const uint32_t st = cnt % depth, u = cnt / depth;
           if (!mbar_wait(b_empty + 8 * st, (u & 1) ^ 1, err, abort_flag)) return false;
-          load_tile(ring + st * kTile, col, t, b_full + 8 * st);
+          mbar_expect_tx(b_full + 8 * st, kStage);
+          load_tile(ring + st * kStage, (first + h0 / group) * DH, t, b_full + 8 * st);
+          if (!kShare) load_tile(ring + st * kStage + kTile, (first + (h0 + 1) / group) * DH, t, b_full + 8 * st);
           ++cnt;
           return true;
         };
+        const int kcol = hq, vcol = hq + hkv;
         ok = load_q(0) && load_kv(kcol, 0, s_k, b_k_full, b_k_empty, kc, NK) && load_q(1);
         for (int t = 1; ok && t <= it.n_blocks; ++t) {
           if (t < it.n_blocks) ok = load_kv(kcol, t, s_k, b_k_full, b_k_empty, kc, NK);
@@ -259,6 +274,7 @@ k_attention_tc2(const __grid_constant__ CUtensorMap map_qkv, const __grid_consta
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       constexpr uint32_t kIdescS = idesc_bf16(BM, BN, 0), kIdescO = idesc_bf16(BM, DH, 1);
+      constexpr int kDepthSteps = DH / 16;  // MMA steps over head_dim for the scores
       ItemReader its, itp;  // the block whose scores are issued next; the block whose P V is issued next
       its.init(ring, b_item_full, b_item_empty);
       itp.init(ring, b_item_full, b_item_empty);
@@ -273,11 +289,11 @@ k_attention_tc2(const __grid_constant__ CUtensorMap map_qkv, const __grid_consta
         if (sj == 0 && !mbar_wait(b_q_full + 8 * x, sic & 1, err, abort_flag)) return false;
         if (x == 0 && !mbar_wait(b_k_full + 8 * st, (kc / NK) & 1, err, abort_flag)) return false;
         tc_fence_after();
-        const uint32_t sq = s_q + x * kTile, sk = s_k + st * kTile;
+        const uint32_t sq = s_q + x * kTile, sk = s_k + st * kStage + (kShare ? 0 : x * kTile);
 #pragma unroll
-        for (int kk = 0; kk < 8; ++kk) {  // 16 head-dim elements per step; sub-tile switches at kk = 4
-          const uint64_t da = smem_desc(sq + (kk >> 2) * (kTile / 2) + (kk & 3) * 32, 16, 1024);
-          const uint64_t db = smem_desc(sk + (kk >> 2) * (kTile / 2) + (kk & 3) * 32, 16, 1024);
+        for (int kk = 0; kk < kDepthSteps; ++kk) {  // 16 head-dim elements per step; the sub-tile switches at kk = 4
+          const uint64_t da = smem_desc(sq + (kk >> 2) * (128 * 128) + (kk & 3) * 32, 16, 1024);
+          const uint64_t db = smem_desc(sk + (kk >> 2) * (128 * 128) + (kk & 3) * 32, 16, 1024);
           umma_bf16(tmem + x * BN, da, db, kIdescS, kk != 0);
         }
         umma_commit(b_s_full + 8 * x);
@@ -299,10 +315,10 @@ k_attention_tc2(const __grid_constant__ CUtensorMap map_qkv, const __grid_consta
         if (!mbar_wait(b_p_full + 8 * x, pc & 1, err, abort_flag)) return false;
         if (x == 0 && !mbar_wait(b_v_full + 8 * st, (vc / NV) & 1, err, abort_flag)) return false;
         tc_fence_after();
-        const uint32_t sv = s_v + st * kTile;
+        const uint32_t sv = s_v + st * kStage + (kShare ? 0 : x * kTile);
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk) {  // 16 keys per step: 8 packed columns of P, 16 rows of V
-          const uint64_t db = smem_desc(sv + kk * 2048, kTile / 2, 1024);  // V: MN-major, two 64-wide dh atoms
+          const uint64_t db = smem_desc(sv + kk * 2048, 128 * 128, 1024);  // V: MN-major, DH / 64 dh atoms of 64
           umma_bf16_ts(tmem + 2 * BN + x * DH, tmem + x * BN + kk * 8, db, kIdescO, (pj | kk) != 0);
         }
         umma_commit(b_o_full + 8 * x);
@@ -332,7 +348,7 @@ k_attention_tc2(const __grid_constant__ CUtensorMap map_qkv, const __grid_consta
     const int quarter = warp & 3;         // the TMEM lane quarter this warp may access
     const int r = quarter * 32 + lane;    // row inside the tile = TMEM lane
     const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
-    const uint32_t t_s = tmem + lane_base + x * BN, t_o = tmem + lane_base + 2 * BN + x * DH + hf * 64;
+    const uint32_t t_s = tmem + lane_base + x * BN, t_o = tmem + lane_base + 2 * BN + x * DH + hf * (DH / 2);
     const uint32_t bar_s = b_s_full + 8 * x, bar_p = b_p_full + 8 * x, bar_o = b_o_full + 8 * x;
     // Meeting point of the two warps that share these 32 rows: an mbarrier with two arrivals (bounded wait, like
     // every other wait here) that also carries a vote.  Slot (u + 1) % 3 is cleared before the arrival at
@@ -451,7 +467,7 @@ k_attention_tc2(const __grid_constant__ CUtensorMap map_qkv, const __grid_consta
             if (!mbar_wait(bar_o, (gc - 1) & 1, err, abort_flag)) { ok = false; break; }  // complete already
             tc_fence_after();
 #pragma unroll 1
-            for (int c = 0; c < 2; ++c) {  // this thread's 64 columns of O
+            for (int c = 0; c < DH / 64; ++c) {  // this thread's DH / 2 columns of O
               uint32_t o[32];
               tmem_ld32(t_o + c * 32, o);
               tmem_ld_wait();
@@ -499,9 +515,9 @@ k_attention_tc2(const __grid_constant__ CUtensorMap map_qkv, const __grid_consta
       // This thread's 64 columns of O_x / l as bf16, 32 columns at a time through the warp's staging rows
       // (64 bytes each, 16-byte chunks XOR-swizzled), so that global stores are 64 contiguous bytes per row.
       const int row_w = it.qb * BM + quarter * 32;  // first row of this warp inside the sequence
-      __nv_bfloat16* ocol = out + (size_t)(it.pair * 2 + x) * DH + hf * 64;
+      __nv_bfloat16* ocol = out + (size_t)(it.pair * 2 + x) * DH + hf * (DH / 2);
 #pragma unroll 1
-      for (int part = 0; part < 2; ++part) {
+      for (int part = 0; part < DH / 64; ++part) {
         uint32_t o[32];
         tmem_ld32(t_o + part * 32, o);
         tmem_ld_wait();
@@ -561,11 +577,24 @@ __device__ int g_sched[kTickets][2];
 
 cudaError_t launch_attention_tc2(const void* qkv, void* out, const int* cu, int seq0, int nseq, int row0, int rows,
                                  int max_len, int n_q_heads, int n_kv_heads, int causal, int* err, cudaStream_t st,
-                                 bool reverse, int prefix, const void* qkv_prefix, bool write_prefix) {
+                                 bool reverse, int prefix, const void* qkv_prefix, bool write_prefix, int head_dim) {
   if (nseq <= 0 || max_len <= 0 || rows <= 0) return cudaSuccess;
-  if (n_kv_heads < 1 || n_q_heads % n_kv_heads || ((n_q_heads / n_kv_heads) & 1)) return cudaErrorInvalidValue;
-  static std::atomic<unsigned long long> smem_set{0};
-  if (cudaError_t e = ensure_dynamic_smem(k_attention_tc2, kSmemBytes, smem_set)) return e;
+  if (n_kv_heads < 1 || n_q_heads % n_kv_heads || (n_q_heads & 1)) return cudaErrorInvalidValue;
+  // Pairs of query heads: with an even group size both heads of a pair read one K / V head (tiles shared); with one
+  // K / V head per query head (head_dim 64 only: two tiles per stage fit) each head of the pair reads its own.
+  const int group = n_q_heads / n_kv_heads;
+  const bool share = (group & 1) == 0;
+  if (!share && group != 1) return cudaErrorInvalidValue;
+  if (!(head_dim == 128 && share) && head_dim != 64) return cudaErrorInvalidValue;
+  const int DH = head_dim;
+  const int kSmemBytes = smem_bytes(DH, share);
+  static std::atomic<unsigned long long> smem_set[3];
+  {
+    cudaError_t e = DH == 128 ? ensure_dynamic_smem(k_attention_tc2<128, true>, kSmemBytes, smem_set[0])
+                    : share   ? ensure_dynamic_smem(k_attention_tc2<64, true>, kSmemBytes, smem_set[1])
+                              : ensure_dynamic_smem(k_attention_tc2<64, false>, kSmemBytes, smem_set[2]);
+    if (e != cudaSuccess) return e;
+  }
   // Exactly `rows` rows are described, so tiles that run past the batch read zeros, never stale memory.
   const uint64_t ld = (uint64_t)(n_q_heads + 2 * n_kv_heads) * DH;
   TmaDesc mq, mpre, mrest;
@@ -620,10 +649,12 @@ cudaError_t launch_attention_tc2(const void* qkv, void* out, const int* cu, int 
   const CUtensorMap& m0 = reinterpret_cast<const CUtensorMap&>(mq);
   const CUtensorMap& m1 = reinterpret_cast<const CUtensorMap&>(mpre);
   const CUtensorMap& m2 = reinterpret_cast<const CUtensorMap&>(mrest);
-  if (cudaError_t le = cudaLaunchKernelEx(&cfg, k_attention_tc2, m0, m1, m2, (__nv_bfloat16*)out, cu, seq0, nseq, row0, nqb, gsz,
-                                          n_q_heads, n_kv_heads, causal, reverse ? 1 : 0, prefix, write_prefix ? 1 : 0,
-                                          scale_log2, sched, err))
-    return le;
+#define PRISM_ATTN2(D, S)                                                                                             \
+  cudaLaunchKernelEx(&cfg, k_attention_tc2<D, S>, m0, m1, m2, (__nv_bfloat16*)out, cu, seq0, nseq, row0, nqb, gsz,    \
+                     n_q_heads, n_kv_heads, causal, reverse ? 1 : 0, prefix, write_prefix ? 1 : 0, scale_log2, sched, err)
+  const cudaError_t le = DH == 128 ? PRISM_ATTN2(128, true) : share ? PRISM_ATTN2(64, true) : PRISM_ATTN2(64, false);
+#undef PRISM_ATTN2
+  if (le != cudaSuccess) return le;
   return cudaGetLastError();
 }
 

@@ -224,7 +224,7 @@ cudaError_t launch_attention_tc(const void* qkv, void* out, const int* cu, int s
 // Two query heads of a key/value group per CTA, persistent (needs an even group size n_q_heads / n_kv_heads).
 cudaError_t launch_attention_tc2(const void* qkv, void* out, const int* cu, int seq0, int nseq, int row0, int rows,
                                 int max_len, int n_q_heads, int n_kv_heads, int causal, int* err, cudaStream_t st, bool reverse = false, int prefix = 0,
-                                const void* qkv_prefix = nullptr, bool write_prefix = true);
+                                const void* qkv_prefix = nullptr, bool write_prefix = true, int head_dim = 128);
 cudaError_t launch_attention_mma(const void* qkv, void* out, const int* cu, int seq0, int nseq, int row0,
                                  int max_len, int n_q_heads, int n_kv_heads, int causal, cudaStream_t st);
 

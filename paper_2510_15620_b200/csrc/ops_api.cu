@@ -171,9 +171,11 @@ int prism_op_attention(const void* qkv, void* out, const int32_t* cu, int32_t n_
     if (head_dim != 128 && !(head_dim == 64 && impl != PRISM_IMPL_MMA)) return PRISM_ERR_UNSUPPORTED;
     if (impl == PRISM_IMPL_AUTO || impl == PRISM_IMPL_SOLO) {
       if (!err_word) return PRISM_ERR_INVALID_ARG;
-      if (impl == PRISM_IMPL_AUTO && head_dim == 128 && ((n_q_heads / n_kv_heads) & 1) == 0)
+      const int group = n_q_heads / n_kv_heads;
+      const bool two_heads = (group & 1) == 0 ? true : (group == 1 && head_dim == 64 && (n_q_heads & 1) == 0);
+      if (impl == PRISM_IMPL_AUTO && two_heads)
         return st_of(launch_attention_tc2(qkv, out, cu, 0, n_seq, 0, total, max_len, n_q_heads, n_kv_heads, causal,
-                                          err_word, S(stream)));
+                                          err_word, S(stream), false, 0, nullptr, true, head_dim));
       return st_of(launch_attention_tc(qkv, out, cu, 0, n_seq, 0, total, max_len, n_q_heads, n_kv_heads, causal, err_word,
                                        S(stream), head_dim));
     }

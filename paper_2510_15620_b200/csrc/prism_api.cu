@@ -427,12 +427,15 @@ static int create_impl(prism_handle* h, const prism_model_cfg* cfg, const prism_
   h->esz = c.dtype == PRISM_BF16 ? 2 : 4;
   h->tc = c.dtype == PRISM_BF16 && (c.gemm_impl == PRISM_IMPL_AUTO || c.gemm_impl == PRISM_IMPL_SOLO);
   h->pair = c.gemm_impl == PRISM_IMPL_AUTO;
-  // 0: CUDA cores, 1: tcgen05 one query head per CTA, 2: mma.sync, 3: tcgen05 two query heads per CTA (even groups)
+  // 0: CUDA cores, 1: tcgen05 one query head per CTA, 2: mma.sync, 3: tcgen05 two query heads per CTA: pairs that
+  // share a K / V head (even group sizes; head_dim 128 or 64) or, at head_dim 64, pairs of heads with a K / V head each
+  const int group_sz = c.n_q_heads / c.n_kv_heads;
+  const bool two_heads = (group_sz & 1) == 0 ? (c.head_dim == 128 || c.head_dim == 64)
+                                             : (group_sz == 1 && c.head_dim == 64 && (c.n_q_heads & 1) == 0);
   h->fa = c.dtype != PRISM_BF16 ? 0
-          : c.attention_impl == PRISM_IMPL_AUTO ? ((((c.n_q_heads / c.n_kv_heads) & 1) == 0) ? 3 : 1)
+          : c.attention_impl == PRISM_IMPL_AUTO ? (two_heads ? 3 : 1)
           : c.attention_impl == PRISM_IMPL_SOLO ? 1
           : c.attention_impl == PRISM_IMPL_MMA  ? 2 : 0;
-  if (h->fa == 3 && c.head_dim != 128) h->fa = 1;  // the two-head kernel is written for head_dim 128
   const bool streamed = c.weight_residency == PRISM_WEIGHTS_HOST_STREAMED;
   if (h->enc) {
     const void* glob[] = {ew->embed, ew->pos_embed, ew->type_embed, ew->emb_ln_g, ew->emb_ln_b, ew->head_dense_w,
@@ -774,7 +777,7 @@ int run_layer_chunk(prism_handle* h, const LayerDev& W, const LayerMaps* maps, f
     PRISM_LAUNCH_P(h, st, PRISM_K_ATTENTION, attn_flops,
                    launch_attention_tc2(h->qkv, h->attn, cu_dev, s0, s1 - s0, r0, rows, max_len, c.n_q_heads, c.n_kv_heads, c.causal,
                                         h->errword, st, next_dir(h, true), prefix,
-                                        (prefix && chunk_of_many) ? h->qkv_prefix : nullptr, chunk_of_many != 2));
+                                        (prefix && chunk_of_many) ? h->qkv_prefix : nullptr, chunk_of_many != 2, dh));
   else if (h->fa == 1)
     PRISM_LAUNCH_P(h, st, PRISM_K_ATTENTION, attn_flops,
                    launch_attention_tc(h->qkv, h->attn, cu_dev, s0, s1 - s0, r0, rows, max_len, c.n_q_heads, c.n_kv_heads, c.causal,
@@ -838,7 +841,7 @@ int run_layer_chunk_encoder(prism_handle* h, int l, const LayerDev& W, const Lay
   if (h->fa == 3)
     PRISM_LAUNCH_P(h, st, PRISM_K_ATTENTION, attn_flops,
                    launch_attention_tc2(h->qkv, h->attn, cu_dev, s0, s1 - s0, r0, rows, max_len, c.n_q_heads, c.n_kv_heads, c.causal,
-                                        h->errword, st, false));
+                                        h->errword, st, false, 0, nullptr, true, dh));
   else if (h->fa == 1)
     PRISM_LAUNCH_P(h, st, PRISM_K_ATTENTION, attn_flops,
                    launch_attention_tc(h->qkv, h->attn, cu_dev, s0, s1 - s0, r0, rows, max_len, c.n_q_heads, c.n_kv_heads, c.causal,
