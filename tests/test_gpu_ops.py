@@ -252,10 +252,12 @@ def _attn_ref(qkv, cu, hq, hkv, dh, causal):
 @pytest.mark.parametrize("causal", [1, 0])
 @pytest.mark.parametrize("dtype,impl,dh,hq,hkv", [(FP32, SIMT, 64, 4, 2), (BF16, SIMT, 128, 4, 2), (BF16, AUTO, 128, 4, 2),
                                                   (BF16, AUTO, 128, 8, 2), (BF16, AUTO, 128, 3, 1), (BF16, 2, 128, 4, 2),
-                                                  (BF16, SOLO, 128, 4, 2)])
+                                                  (BF16, SOLO, 128, 4, 2), (BF16, AUTO, 64, 4, 2), (BF16, AUTO, 64, 4, 4),
+                                                  (BF16, AUTO, 64, 3, 3), (BF16, SOLO, 64, 4, 4)])
 def test_attention(P, dtype, impl, dh, hq, hkv, causal):
-    """AUTO runs the two-heads-per-CTA tcgen05 kernel for even group sizes (2 and 4 here) and the one-head kernel
-    otherwise (group 3); SOLO forces the one-head kernel; 2 is the mma.sync kernel."""
+    """AUTO runs the two-heads-per-CTA tcgen05 kernel for even group sizes (2 and 4 here; at head_dim 64 also for an
+    even number of heads with a K/V head each) and the one-head kernel otherwise (group 3, or three heads of 64);
+    SOLO forces the one-head kernel; 2 is the mma.sync kernel."""
     rng = np.random.default_rng(dh + causal)
     lens = np.array([1, 7, 64, 65, 130, 200, 63, 128, 129, 300, 513])      # below, at and across the 64/128-row tiles
     cu = np.zeros(len(lens) + 1, np.int32)
