@@ -584,7 +584,7 @@ def run_prism(args):
             import gc
             model.close()
             line["workloads"] = {}
-            for index, k in ((0, 100), (2, 20), (3, 20), (4, 30)):
+            for index, k in ((0, 100), (2, 20), (3, 20), (4, 100)):
                 gc.collect()
                 torch.cuda.empty_cache()            # the previous workload's weights go back to the driver
                 line["workloads"][f"cfg{index}"] = measure_side_workload(P, index, k, 5, dev, local)
