@@ -264,3 +264,23 @@ def test_bf16_activation_mode_rounds_like_a_library_and_stays_close():
     rounded = oracle.candidate_scores(toks, w, cfg, [1, 2], act="bf16")
     for l in (1, 2):
         assert 0 < abs(exact[l] - rounded[l]) < 5e-2
+
+
+def test_rounding_points_of_the_bf16_mode_compose():
+    """The rounded-activation mode takes a subset of its six storage points: all six named one by one are the full
+    mode bit for bit, none is the exact forward, every single point moves the scores by less than all six together
+    can at most (the sum of the single moves bounds nothing, but each is non-zero and small), and an unknown name is
+    refused."""
+    from oracle.reranker import ROUNDING_POINTS, rounding_points
+    assert rounding_points("exact") == frozenset() and rounding_points("bf16") == frozenset(ROUNDING_POINTS)
+    wl, cfg, w = _tiny()
+    toks = np.random.default_rng(6).integers(0, cfg.vocab, size=48)
+    exact = oracle.candidate_scores(toks, w, cfg, [1, 2])
+    full = oracle.candidate_scores(toks, w, cfg, [1, 2], act="bf16")
+    named = oracle.candidate_scores(toks, w, cfg, [1, 2], act=",".join(ROUNDING_POINTS))
+    assert named == full
+    for p in ROUNDING_POINTS:
+        one = oracle.candidate_scores(toks, w, cfg, [1, 2], act=p)
+        assert all(0 < abs(one[l] - exact[l]) < 5e-2 for l in (1, 2)), p
+    with pytest.raises(ValueError):
+        oracle.candidate_scores(toks, w, cfg, [1], act="norm,softmax")
