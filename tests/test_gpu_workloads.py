@@ -71,7 +71,7 @@ def _exact_file(index, r):
 
 def _tolerance(index):
     """The score tolerance of a workload.  3e-2 is the stated bf16 tolerance and holds for the 0.6B-shaped workloads.
-    For the 36-layer 4B- and 8B-shaped models the oracle's own bf16-storage noise (measured on 16 length-stratified
+    For the 36-layer 4B- and 8B-shaped models the oracle's own bf16-storage noise (measured on 32 length-stratified
     candidates, 8 scored layers each) has an RMS of 0.03 - 0.04, so no bf16 evaluation can stay within 3e-2 on every
     score.  There the deviation is treated as what it is, noise: no score may be further from the oracle than
     SIGMAS_MAX times the oracle's own noise RMS, and the RMS deviation of the CUDA path over all stored candidates may
@@ -88,7 +88,7 @@ SIGMAS_MAX = 6.0
 RMS_RATIO_MAX = 1.5
 P99_SIGMAS_MAX = 4.0
 GOLD_FILES = {
-    2: ("cfg2_qwen3_4b_scores_r0.txt", "cfg2_qwen3_4b_scores_bf16act_r0_s16.txt"),
+    2: ("cfg2_qwen3_4b_scores_r0.txt", "cfg2_qwen3_4b_scores_bf16act_r0_s32.txt"),
     3: ("cfg3_qwen3_8b_streamed_scores_r0.txt", "cfg3_qwen3_8b_streamed_scores_bf16act_r0_s32.txt"),
     4: ("cfg4_stress_0p6b_scores_r0.txt", "cfg4_stress_0p6b_scores_bf16act_r0_s16.txt"),
 }
