@@ -7,6 +7,9 @@ candidates, query 32 tokens, documents uniform 128-512 tokens, K = 10, cluster p
 layers 8, 12, ..., 24).  `value` is candidate-tokens/s = submitted tokens of all requests / device
 time with the inputs already in HBM; `e2e` is the same through prism_select_host with host buffers.
 With --gpus N every rank serves its own stream of requests (no data-path collective; weak scaling).
+At N = 1 the default run also measures the other four benchmark workloads (tiny fp32, 4B-shaped, 8B-shaped streamed
+and chunked, 1000-candidate stress) and reports them in a `workloads` block of the same line; the headline keys stay
+those of workload 1.  `cpu_baseline` times the CPU oracle on a length-stratified sample of request 0.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload 1]
 """
